@@ -1,0 +1,345 @@
+/*
+ * lsmkv_oracle.c -- plain, slow, single-threaded CPU statement of the batch codec and the
+ * batched longest-cached-prefix probe of an LSM-backed KV-cache store.
+ *
+ * THIS IS TEST INFRASTRUCTURE. It exists so that the CUDA library can be checked against
+ * something obviously correct. It shares no code, header, table or constant generator with
+ * the CUDA library, is never linked into it, and must not be used as a product path.
+ *
+ * What it follows (paper section names; the paper fixes properties, this build fixes formats):
+ *   - Sec. 3.2 "Prefix-Preserving Storage Engine": the index maps a key that encodes a token
+ *     prefix to a compact record holding a file identifier and a byte offset; tensors live in
+ *     an append-only log (key-value separation).
+ *   - Sec. 3.4 "Batch Codec Operations": a batch's tensors are combined into one contiguous
+ *     payload on put and split again on get (identity codec here: a bit copy).
+ *   - App. B "Basic Operations": put_batch (keys + file_id/offset records + contiguous
+ *     tensors), probe (longest cached prefix by point lookups), get_batch (locations, then
+ *     batch tensor loading).
+ *   - Sec. 2.2 "Point Lookups": levels are checked in order and the first match is returned.
+ *
+ * Formats (this build's reading; the paper is silent on all of them):
+ *   key     = 4 x u64 {w0,w1,w2,w3}, compared lexicographically as unsigned words
+ *             w0 = (namespace << 32) | chunk index j
+ *             w1 = digest A of the token prefix S[0 : (j+1)*C)
+ *             w2 = digest B of the same prefix
+ *             w3 = (first token of chunk j << 32) | last token of chunk j
+ *   digest  = h <- 0; for every token t in order: h <- (h * BASE + (t + 1)) mod (2^61 - 1),
+ *             always the canonical representative in [0, 2^61 - 1)
+ *   record  = {u32 file_id, u32 reserved = 0, u64 offset}, offset = base + i * chunk_bytes
+ *   blob    = for l in 0..L-1: K page slab of layer l, then V page slab of layer l
+ *   pool    = 2L buffers (K of layers 0..L-1, then V of layers 0..L-1), each
+ *             [num_pages][page_tokens][kv_heads][head_dim] elements, page slab contiguous
+ *
+ * Every function reports an error by return value; nothing here aborts.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_EINVAL (-1)
+#define ORC_ECAPACITY (-2)
+#define ORC_EBADPAGE (-3)
+#define ORC_EBADREC (-4)
+
+static const uint64_t ORC_P = 0x1FFFFFFFFFFFFFFFULL; /* 2^61 - 1 */
+static const uint64_t ORC_BASE[2] = {0x0B4E0EF37BC32127ULL, 0x16A09E667F3BCC90ULL};
+
+typedef struct { uint64_t w[4]; } orc_key;
+typedef struct { uint32_t file_id, reserved; uint64_t offset; } orc_val;
+typedef struct {
+    uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
+    uint32_t page_tokens, chunk_tokens, ns, flags;
+} orc_geom;
+typedef struct { const orc_key *keys; const orc_val *vals; uint64_t n; } orc_run;
+
+/* ---- geometry ---------------------------------------------------------------------- */
+
+uint64_t orc_page_bytes(const orc_geom *g)
+{
+    return (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
+}
+
+uint64_t orc_chunk_bytes(const orc_geom *g)
+{
+    return 2ull * g->n_layers * orc_page_bytes(g);
+}
+
+static int geom_ok(const orc_geom *g)
+{
+    return g && g->n_layers && g->n_kv_heads && g->head_dim && g->elem_bytes &&
+           g->page_tokens && g->chunk_tokens == g->page_tokens;
+}
+
+/* ---- digest: one Horner step of the polynomial hash over the Mersenne prime 2^61-1 -- */
+
+uint64_t orc_digest_step(uint64_t h, uint32_t token, int lane)
+{
+    unsigned __int128 x = (unsigned __int128)h * ORC_BASE[lane] + ((uint64_t)token + 1ull);
+    return (uint64_t)(x % ORC_P);
+}
+
+/* digest of a whole token string (used by the pins) */
+uint64_t orc_digest(const uint32_t *tokens, uint64_t n, int lane)
+{
+    uint64_t h = 0;
+    for (uint64_t i = 0; i < n; ++i) h = orc_digest_step(h, tokens[i], lane);
+    return h;
+}
+
+/* ---- keys -------------------------------------------------------------------------- */
+
+int orc_key_cmp(const orc_key *a, const orc_key *b)
+{
+    for (int i = 0; i < 4; ++i) {
+        if (a->w[i] < b->w[i]) return -1;
+        if (a->w[i] > b->w[i]) return 1;
+    }
+    return 0;
+}
+
+/*
+ * Keys of chunks j = j_begin .. floor(len / C) - 1 of one sequence, written to keys_out in
+ * ascending j. The digest always runs from token 0: a key names the whole prefix, also when
+ * earlier chunks are not emitted. Returns the number of keys written.
+ */
+uint64_t orc_chunk_keys(const orc_geom *g, const uint32_t *tokens, uint64_t len,
+                        uint64_t j_begin, orc_key *keys_out)
+{
+    const uint64_t C = g->chunk_tokens;
+    const uint64_t nch = len / C;
+    uint64_t hA = 0, hB = 0, written = 0;
+    for (uint64_t j = 0; j < nch; ++j) {
+        for (uint64_t i = 0; i < C; ++i) {
+            const uint32_t t = tokens[j * C + i];
+            hA = orc_digest_step(hA, t, 0);
+            hB = orc_digest_step(hB, t, 1);
+        }
+        if (j >= j_begin) {
+            orc_key *k = &keys_out[written++];
+            k->w[0] = ((uint64_t)g->ns << 32) | (uint64_t)(uint32_t)j;
+            k->w[1] = hA;
+            k->w[2] = hB;
+            k->w[3] = ((uint64_t)tokens[j * C] << 32) | (uint64_t)tokens[j * C + C - 1];
+        }
+    }
+    return written;
+}
+
+/* ---- put_batch, device half: keys + records + packed blobs -------------------------- */
+
+/*
+ * kv_ptrs: 2L host pointers, K of layer 0..L-1 then V of layer 0..L-1.
+ * blob_out may be NULL (index-only encode: keys and records, no payload).
+ */
+int orc_encode_batch(const orc_geom *g, uint32_t n_req, const uint32_t *tokens,
+                     const uint64_t *seq_off, const uint32_t *start_chunk,
+                     const uint64_t *chunk_off, uint64_t n_chunks, const uint32_t *page_table,
+                     const uint8_t *const *kv_ptrs, uint64_t num_pages, uint32_t file_id,
+                     uint64_t base_offset, orc_key *keys_out, orc_val *vals_out,
+                     uint8_t *blob_out, uint64_t blob_capacity)
+{
+    if (!geom_ok(g)) return ORC_EINVAL;
+    const uint64_t C = g->chunk_tokens, L = g->n_layers;
+    const uint64_t pb = orc_page_bytes(g), cb = orc_chunk_bytes(g);
+    if (blob_out && blob_capacity < n_chunks * cb) return ORC_ECAPACITY;
+    if (n_req && chunk_off[n_req] != n_chunks) return ORC_EINVAL;
+
+    for (uint32_t r = 0; r < n_req; ++r) {
+        const uint64_t len = seq_off[r + 1] - seq_off[r];
+        const uint64_t nch = len / C;
+        const uint64_t start = start_chunk ? start_chunk[r] : 0;
+        const uint64_t cnt = nch > start ? nch - start : 0;
+        if (chunk_off[r + 1] - chunk_off[r] != cnt) return ORC_EINVAL;
+        if (cnt == 0) continue;
+        const uint64_t i0 = chunk_off[r];
+        if (orc_chunk_keys(g, tokens + seq_off[r], len, start, keys_out + i0) != cnt)
+            return ORC_EINVAL;
+        for (uint64_t c = 0; c < cnt; ++c) {
+            const uint64_t i = i0 + c;
+            vals_out[i].file_id = file_id;
+            vals_out[i].reserved = 0;
+            vals_out[i].offset = base_offset + i * cb;
+            if (!blob_out) continue;
+            const uint64_t page = page_table[i];
+            if (page >= num_pages) return ORC_EBADPAGE;
+            uint8_t *dst = blob_out + i * cb;
+            for (uint64_t l = 0; l < L; ++l) {
+                memcpy(dst + (2 * l) * pb, kv_ptrs[l] + page * pb, pb);         /* K, layer l */
+                memcpy(dst + (2 * l + 1) * pb, kv_ptrs[L + l] + page * pb, pb); /* V, layer l */
+            }
+        }
+    }
+    return ORC_OK;
+}
+
+/* ---- the index: immutable sorted runs, newest first --------------------------------- */
+
+/* first position in run whose key is >= key (plain binary search on a sorted array) */
+static uint64_t run_lower_bound(const orc_run *run, const orc_key *key)
+{
+    uint64_t lo = 0, hi = run->n;
+    while (lo < hi) {
+        const uint64_t mid = lo + (hi - lo) / 2;
+        if (orc_key_cmp(&run->keys[mid], key) < 0) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+/*
+ * Point lookup: runs are checked from newest (index 0) to oldest and the first run that holds
+ * the key decides. Returns 1 and fills *val on a hit, 0 on a miss. *run_idx (optional) gets
+ * the deciding run.
+ */
+int orc_lookup(const orc_run *runs, uint32_t n_runs, const orc_key *key, orc_val *val,
+               uint32_t *run_idx)
+{
+    for (uint32_t r = 0; r < n_runs; ++r) {
+        const uint64_t pos = run_lower_bound(&runs[r], key);
+        if (pos < runs[r].n && orc_key_cmp(&runs[r].keys[pos], key) == 0) {
+            if (val) *val = runs[r].vals[pos];
+            if (run_idx) *run_idx = r;
+            return 1;
+        }
+    }
+    return 0;
+}
+
+/*
+ * Flush: turn a write batch (keys in arrival order, duplicates allowed) into one sorted run
+ * with unique keys; of equal keys the LAST arrival survives (out-of-place update semantics).
+ * Returns the run length. keys_out/vals_out need room for n entries.
+ */
+typedef struct { orc_key k; orc_val v; uint64_t seq; } flush_ent;
+
+static int flush_cmp(const void *a, const void *b)
+{
+    const flush_ent *x = (const flush_ent *)a, *y = (const flush_ent *)b;
+    const int c = orc_key_cmp(&x->k, &y->k);
+    if (c) return c;
+    return (x->seq < y->seq) ? -1 : (x->seq > y->seq);
+}
+
+int64_t orc_flush(const orc_key *keys, const orc_val *vals, uint64_t n, orc_key *keys_out,
+                  orc_val *vals_out)
+{
+    if (n == 0) return 0;
+    flush_ent *e = (flush_ent *)malloc(n * sizeof(flush_ent));
+    if (!e) return ORC_ECAPACITY;
+    for (uint64_t i = 0; i < n; ++i) { e[i].k = keys[i]; e[i].v = vals[i]; e[i].seq = i; }
+    qsort(e, n, sizeof(flush_ent), flush_cmp);
+    uint64_t m = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        /* equal keys are adjacent and ordered by arrival: keep the last of each group */
+        if (i + 1 < n && orc_key_cmp(&e[i].k, &e[i + 1].k) == 0) continue;
+        keys_out[m] = e[i].k;
+        vals_out[m] = e[i].v;
+        ++m;
+    }
+    free(e);
+    return (int64_t)m;
+}
+
+/*
+ * Compaction of several runs (newest first) into one: the union of their keys, each key with
+ * the record of the newest run that holds it. Written as "concatenate oldest..newest, then
+ * flush", which is the definition of newest-wins. Returns the merged length.
+ */
+int64_t orc_merge_runs(const orc_run *runs, uint32_t n_runs, orc_key *keys_out,
+                       orc_val *vals_out)
+{
+    uint64_t total = 0;
+    for (uint32_t r = 0; r < n_runs; ++r) total += runs[r].n;
+    if (total == 0) return 0;
+    orc_key *k = (orc_key *)malloc(total * sizeof(orc_key));
+    orc_val *v = (orc_val *)malloc(total * sizeof(orc_val));
+    if (!k || !v) { free(k); free(v); return ORC_ECAPACITY; }
+    uint64_t at = 0;
+    for (uint32_t r = n_runs; r-- > 0;) { /* oldest first, so the newest arrives last */
+        memcpy(k + at, runs[r].keys, runs[r].n * sizeof(orc_key));
+        memcpy(v + at, runs[r].vals, runs[r].n * sizeof(orc_val));
+        at += runs[r].n;
+    }
+    const int64_t m = orc_flush(k, v, total, keys_out, vals_out);
+    free(k);
+    free(v);
+    return m;
+}
+
+/* ---- probe: longest cached prefix, first-miss rule ---------------------------------- */
+
+/*
+ * For query q with n_q = floor(len_q / C) chunks: hit_q = the largest h <= n_q such that the
+ * key of every chunk j < h is found by orc_lookup. recs_out[qchunk_off[q] + j] = the record
+ * found for j < hit_q and all-zero for j >= hit_q. keys_out (optional) receives every chunk
+ * key of every query. lookups_out (optional) counts point lookups performed.
+ */
+int orc_probe_batch(const orc_geom *g, uint32_t n_query, const uint32_t *tokens,
+                    const uint64_t *seq_off, const uint64_t *qchunk_off, const orc_run *runs,
+                    uint32_t n_runs, uint32_t *hit_out, orc_val *recs_out, orc_key *keys_out,
+                    uint64_t *lookups_out)
+{
+    if (!geom_ok(g)) return ORC_EINVAL;
+    const uint64_t C = g->chunk_tokens;
+    uint64_t lookups = 0;
+    for (uint32_t q = 0; q < n_query; ++q) {
+        const uint64_t len = seq_off[q + 1] - seq_off[q];
+        const uint64_t nch = len / C;
+        if (qchunk_off[q + 1] - qchunk_off[q] != nch) return ORC_EINVAL;
+        orc_key *keys = keys_out ? keys_out + qchunk_off[q]
+                                 : (orc_key *)malloc((nch ? nch : 1) * sizeof(orc_key));
+        if (!keys) return ORC_ECAPACITY;
+        orc_chunk_keys(g, tokens + seq_off[q], len, 0, keys);
+        orc_val *recs = recs_out + qchunk_off[q];
+        memset(recs, 0, nch * sizeof(orc_val));
+        uint64_t h = 0;
+        while (h < nch) {
+            orc_val v;
+            ++lookups;
+            if (!orc_lookup(runs, n_runs, &keys[h], &v, NULL)) break;
+            recs[h] = v;
+            ++h;
+        }
+        hit_out[q] = (uint32_t)h;
+        if (!keys_out) free(keys);
+    }
+    if (lookups_out) *lookups_out = lookups;
+    return ORC_OK;
+}
+
+/* ---- get_batch, tensor half: split hit blobs back into pool pages ------------------- */
+
+/*
+ * For every query q and chunk j < hit[q]: the blob at arenas[rec.file_id] + rec.offset is cut
+ * into 2L page slabs (K0,V0,K1,V1,...) which are written to page dst_page_table[idx] of the
+ * matching pool buffer. Nothing else in the pool is touched.
+ */
+int orc_decode_batch(const orc_geom *g, uint32_t n_query, const uint64_t *qchunk_off,
+                     const uint32_t *hit, const orc_val *recs, const uint8_t *const *arenas,
+                     const uint64_t *arena_bytes, uint32_t n_arenas,
+                     const uint32_t *dst_page_table, uint8_t *const *kv_ptrs,
+                     uint64_t num_pages)
+{
+    if (!geom_ok(g)) return ORC_EINVAL;
+    const uint64_t L = g->n_layers;
+    const uint64_t pb = orc_page_bytes(g), cb = orc_chunk_bytes(g);
+    for (uint32_t q = 0; q < n_query; ++q) {
+        const uint64_t nch = qchunk_off[q + 1] - qchunk_off[q];
+        if (hit[q] > nch) return ORC_EINVAL;
+        for (uint64_t j = 0; j < hit[q]; ++j) {
+            const uint64_t idx = qchunk_off[q] + j;
+            const orc_val rec = recs[idx];
+            if (rec.file_id >= n_arenas) return ORC_EBADREC;
+            if (rec.offset > arena_bytes[rec.file_id] ||
+                arena_bytes[rec.file_id] - rec.offset < cb) return ORC_EBADREC;
+            const uint64_t page = dst_page_table[idx];
+            if (page >= num_pages) return ORC_EBADPAGE;
+            const uint8_t *src = arenas[rec.file_id] + rec.offset;
+            for (uint64_t l = 0; l < L; ++l) {
+                memcpy(kv_ptrs[l] + page * pb, src + (2 * l) * pb, pb);
+                memcpy(kv_ptrs[L + l] + page * pb, src + (2 * l + 1) * pb, pb);
+            }
+        }
+    }
+    return ORC_OK;
+}
