@@ -1,0 +1,206 @@
+/*
+ * lsmkv.h -- C ABI of the B200 batch codec and longest-cached-prefix probe for an LSM-backed
+ * KV-cache store (device half of the put_batch / probe / get_batch operations of
+ * "On 10X Better Scalability: KV Stores Scale Up KV Cache", Sec. 3.2 and App. B, with the
+ * batch codec of Sec. 3.4).
+ *
+ * General rules
+ *   - Pointers marked [dev] are device pointers on the context's GPU, [host] are host pointers.
+ *     The caller owns every buffer; the library keeps no reference after a call returns,
+ *     except that device work enqueued by the call reads/writes the [dev] buffers until the
+ *     stream reaches the point following the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Every
+ *     batch call only enqueues work and returns; none of them synchronises.
+ *   - Return value: 0 = enqueued, negative = LSMKV_E* and nothing was enqueued.
+ *   - Problems only the GPU can see (a page id beyond the pool, a record that points outside
+ *     its arena, a misaligned buffer, a wait that ran out) never fault: the offending item is
+ *     skipped and recorded in a device status block read back by lsmkv_last_status().
+ *   - No call allocates device memory except lsmkv_create(), lsmkv_reserve() and a batch call
+ *     whose batch is larger than any before it (the internal workspace grows; call
+ *     lsmkv_reserve() up front to rule that out).
+ *
+ * Formats (version 1). The paper states properties (key order follows token-prefix order;
+ * index values are a file identifier plus a byte offset; a batch's tensors are stored
+ * contiguously); the concrete layouts are this library's:
+ *   key     4 x u64, ordered lexicographically as unsigned words:
+ *             w0 = (namespace << 32) | chunk index j
+ *             w1, w2 = two digests of the token prefix S[0 : (j+1)*C)
+ *             w3 = (first token of chunk j << 32) | last token of chunk j
+ *   digest  h <- 0; per token t: h <- (h*BASE + t + 1) mod (2^61 - 1), canonical in [0, 2^61-1)
+ *             BASE_A = 0x0B4E0EF37BC32127, BASE_B = 0x16A09E667F3BCC90
+ *   record  {u32 file_id, u32 reserved = 0, u64 offset}; the blob length is chunk_bytes
+ *   pool    2L buffers: K of layers 0..L-1, then V of layers 0..L-1, each
+ *             [num_pages][page_tokens][n_kv_heads][head_dim] elements (a page slab of
+ *             page_bytes = page_tokens*n_kv_heads*head_dim*elem_bytes is contiguous)
+ *   blob    for l in 0..L-1: K slab of layer l, V slab of layer l  (chunk_bytes = 2L*page_bytes)
+ *   A chunk is C = chunk_tokens tokens; a sequence of len tokens has floor(len / C) chunks and
+ *   a trailing partial chunk is never encoded, probed or decoded.
+ */
+#ifndef LSMKV_H
+#define LSMKV_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LSMKV_FORMAT_VERSION 1
+#define LSMKV_MAX_RUNS 64
+
+/* return codes */
+#define LSMKV_OK 0
+#define LSMKV_EINVAL (-1)     /* null / misaligned pointer, unsupported geometry, bad count */
+#define LSMKV_ECAPACITY (-2)  /* an output buffer is too small */
+#define LSMKV_ECUDA (-3)      /* a CUDA call failed; see lsmkv_last_cuda_error() */
+#define LSMKV_ENOMEM (-4)     /* host or device allocation failed */
+
+/* bits of lsmkv_status_t.flags */
+#define LSMKV_ST_BAD_PAGE 0x1u     /* a page id >= num_pages (item skipped) */
+#define LSMKV_ST_BAD_RECORD 0x2u   /* file_id >= n_arenas, or offset outside / misaligned (skipped) */
+#define LSMKV_ST_BAD_COUNT 0x4u    /* chunk_off / qchunk_off / hit disagree with the sequence lengths */
+#define LSMKV_ST_MISALIGNED 0x8u   /* a pool buffer is not 16-byte aligned (skipped) */
+#define LSMKV_ST_WAIT_EXPIRED 0x10u /* a bounded wait inside a kernel gave up */
+
+typedef struct lsmkv_ctx lsmkv_ctx;
+
+typedef struct { uint64_t w[4]; } lsmkv_key_t;                               /* 32 bytes */
+typedef struct { uint32_t file_id, reserved; uint64_t offset; } lsmkv_val_t; /* 16 bytes */
+
+typedef struct {
+    uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
+    uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens must equal page_tokens; flags = 0 */
+} lsmkv_geom_t;
+
+/* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i]. */
+typedef struct {
+    const lsmkv_key_t *keys; /* [dev] */
+    const lsmkv_val_t *vals; /* [dev] */
+    uint64_t n;
+} lsmkv_run_t;
+
+/* The paged KV pool. */
+typedef struct {
+    void *const *kv_ptrs; /* [dev] array of 2L [dev] pointers, each 16-byte aligned */
+    uint64_t num_pages;
+} lsmkv_pool_t;
+
+typedef struct {
+    uint32_t flags;        /* OR of LSMKV_ST_* since the last lsmkv_last_status() */
+    uint32_t reserved;
+    uint64_t first_bad;    /* smallest item index that set a flag (chunk / query index), or ~0 */
+    uint64_t chunks_encoded; /* counters since the last lsmkv_last_status() */
+    uint64_t lookups;        /* point lookups performed by probes */
+    uint64_t chunks_hit;     /* sum of hit lengths */
+    uint64_t empty_probes;   /* queries with hit length 0 */
+    uint64_t chunks_decoded;
+} lsmkv_status_t;
+
+/*
+ * Create a context on `device` for one KV geometry. Allocates the context, a small device
+ * status block and the workspace. Errors: LSMKV_EINVAL for a zero field, chunk_tokens !=
+ * page_tokens, or page_bytes not a multiple of 16; LSMKV_ECUDA / LSMKV_ENOMEM.
+ */
+int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *geom, int device);
+
+/* Free everything the context owns. Synchronises the device. NULL is accepted. */
+int lsmkv_destroy(lsmkv_ctx *ctx);
+
+/* Make the workspace large enough for batches of up to n_seq sequences and n_chunks chunks
+ * (n_chunks < 2^32 - 1), so that later batch calls of that size allocate nothing. May
+ * synchronise (it frees the old workspace). */
+int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks);
+
+/*
+ * put_batch, device half (App. B "Put Batch"; Sec. 3.4 "Batch Codec Operations").
+ * For request r with tokens[seq_off[r] .. seq_off[r+1]) and n_r = floor(len_r / C) chunks,
+ * chunks j = start_r .. n_r-1 are encoded (start_r = start_chunk[r], or 0 when start_chunk is
+ * NULL; the digest always covers the whole prefix from token 0). Encoded chunk number c of
+ * request r has output index i = chunk_off[r] + c and produces
+ *   keys_out[i]  the chunk key,
+ *   vals_out[i]  {file_id, 0, base_offset + i*chunk_bytes},
+ *   blob_out[i*chunk_bytes ..)  the 2L page slabs of pool page page_table[i].
+ *   tokens      [dev] u32, all sequences back to back
+ *   seq_off     [dev] u64[n_req+1], ascending
+ *   start_chunk [dev] u32[n_req] or NULL
+ *   chunk_off   [dev] u64[n_req+1], exclusive prefix sums of max(0, n_r - start_r);
+ *               chunk_off[n_req] must equal n_chunks (a mismatch sets LSMKV_ST_BAD_COUNT and
+ *               the request is skipped)
+ *   page_table  [dev] u32[n_chunks]; may be NULL together with pool and blob_out for an
+ *               index-only encode (keys and records, no payload)
+ *   blob_out    [dev], 16-byte aligned, blob_capacity >= n_chunks*chunk_bytes else
+ *               LSMKV_ECAPACITY
+ * Ordering (the paper's two-phase write, Sec. 3.2): keys, records and blobs of one call are
+ * complete at the same point of the stream; publish the records only after that point.
+ */
+int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint32_t *tokens,
+                       const uint64_t *seq_off, const uint32_t *start_chunk,
+                       const uint64_t *chunk_off, uint64_t n_chunks, const uint32_t *page_table,
+                       const lsmkv_pool_t *pool, uint32_t file_id, uint64_t base_offset,
+                       lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, void *blob_out,
+                       uint64_t blob_capacity);
+
+/*
+ * probe + the index half of get_batch (App. B "Probe", "Get Batch"; Sec. 2.2 "Point Lookups").
+ * For query q with n_q = floor(len_q / C) chunks, each chunk key is looked up in runs[0]
+ * (newest) .. runs[n_runs-1] (oldest) and the first run that holds it decides.
+ *   hit_chunks_out[q] = largest h <= n_q such that chunks 0..h-1 were all found,
+ *   recs_out[qchunk_off[q] + j] = the record found for j < h, all-zero bytes for j >= h.
+ *   runs       [host] array of n_runs <= LSMKV_MAX_RUNS descriptors (copied by the call)
+ *   qchunk_off [dev] u64[n_query+1], exclusive prefix sums of n_q; n_qchunks = qchunk_off[n_query]
+ *   keys_out   [dev] optional [n_qchunks]: every chunk key of every query (NULL to skip; the
+ *              probe then stops hashing a query at its first miss)
+ */
+int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint32_t *tokens,
+                      const uint64_t *seq_off, const uint64_t *qchunk_off, uint64_t n_qchunks,
+                      const lsmkv_run_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,
+                      lsmkv_val_t *recs_out, lsmkv_key_t *keys_out);
+
+/*
+ * get_batch, tensor half (App. B "Get Batch"; Sec. 3.4). For every query q and j < hit_chunks[q]
+ * the blob at arenas[rec.file_id] + rec.offset (rec = recs[qchunk_off[q] + j]) is split into
+ * its 2L page slabs, which are written to page dst_page_table[qchunk_off[q] + j] of the pool.
+ * No other byte of the pool changes. Destination pages must be distinct within the call.
+ *   arenas      [host] array of n_arenas [dev] base pointers (16-byte aligned), indexed by file_id
+ *   arena_bytes [host] size of each arena; records must satisfy offset + chunk_bytes <= size
+ *               and offset % 16 == 0 (else LSMKV_ST_BAD_RECORD, chunk skipped)
+ *   n_arenas    <= 64
+ */
+int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
+                       const uint64_t *qchunk_off, uint64_t n_qchunks,
+                       const uint32_t *hit_chunks, const lsmkv_val_t *recs,
+                       const void *const *arenas, const uint64_t *arena_bytes,
+                       uint32_t n_arenas, const uint32_t *dst_page_table,
+                       const lsmkv_pool_t *pool);
+
+/* Synchronise `stream`, copy the device status block to *out [host] and clear it. */
+int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out);
+
+/* The cudaError_t behind the last LSMKV_ECUDA of this context (0 if none). */
+int lsmkv_last_cuda_error(const lsmkv_ctx *ctx);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
+
+/*
+ * Tuning knobs (launch shapes only; results never depend on them). Returns LSMKV_EINVAL for an
+ * unknown name or a value outside its documented range.
+ *   "copy_mode"         0 = bulk-async copy engine (cp.async.bulk), 1 = 16-byte vector loads/stores
+ *   "copy_stage_bytes"  bytes per bulk copy, multiple of 16, 16..131072 (clamped to page_bytes)
+ *   "copy_stages"       bulk copies in flight per CTA, 1..32 (reduced to fit shared memory)
+ *   "copy_ctas_per_sm"  1..8        "copy_l2_hint"  0/1 = evict-first L2 policy on the copies
+ *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..32
+ */
+int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value);
+int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name);
+
+/* Static text for a return code. */
+const char *lsmkv_strerror(int code);
+
+/* LSMKV_FORMAT_VERSION the library was built with. */
+int lsmkv_format_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSMKV_H */

@@ -1,0 +1,446 @@
+// liblsmkv: host side of the C ABI declared in include/lsmkv.h. Validates arguments, keeps the
+// per-context workspace, and enqueues the kernels on the caller's stream. Nothing here touches
+// payload bytes on the host.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "lsmkv.h"
+#include "lsmkv_common.cuh"
+#include "lsmkv_copy.cuh"
+#include "lsmkv_keys.cuh"
+#include "lsmkv_probe.cuh"
+
+using namespace lsmkv;
+
+struct lsmkv_ctx {
+    lsmkv_geom_t geom;
+    int device;
+    int sm_count;
+    int max_smem_optin;
+    uint64_t page_bytes, chunk_bytes;
+    KeyConsts kc;
+    DevStatus *d_status;
+    // workspace: hit_off u64[ws_seq + 1] followed by plan u32[ws_chunks]
+    void *d_ws;
+    uint64_t ws_seq, ws_chunks;
+    int last_cuda;
+    uint64_t launches;
+    // tuning
+    int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
+    int64_t probe_warps_per_cta, simt_ctas_per_sm;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int cuda_fail(lsmkv_ctx *ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda = (int)e;
+    cudaGetLastError();   // clear the sticky-less error state
+    return LSMKV_ECUDA;
+}
+
+#define CU(ctx, call)                                            \
+    do {                                                         \
+        cudaError_t e__ = (call);                                \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);    \
+    } while (0)
+
+// (a * b) mod (2^61 - 1) on the host, for the power tables only
+uint64_t host_mulmod(uint64_t a, uint64_t b)
+{
+    const unsigned __int128 x = (unsigned __int128)a * b;
+    uint64_t s = (uint64_t)(x & kP) + (uint64_t)(x >> 61);
+    s = (s & kP) + (s >> 61);
+    return s >= kP ? s - kP : s;
+}
+
+uint64_t host_powmod(uint64_t b, uint64_t e)
+{
+    uint64_t r = 1;
+    while (e) {
+        if (e & 1) r = host_mulmod(r, b);
+        b = host_mulmod(b, b);
+        e >>= 1;
+    }
+    return r;
+}
+
+void fill_key_consts(KeyConsts &kc, uint32_t C)
+{
+    const uint64_t mA = host_powmod(kBaseA, C), mB = host_powmod(kBaseB, C);
+    uint64_t a = mA, b = mB;
+    for (int i = 0; i < 32; ++i) {
+        kc.pwA[i] = a;
+        kc.pwB[i] = b;
+        a = host_mulmod(a, mA);
+        b = host_mulmod(b, mB);
+    }
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int ensure_workspace(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
+{
+    if (n_seq <= ctx->ws_seq && n_chunks <= ctx->ws_chunks && ctx->d_ws) return LSMKV_OK;
+    const uint64_t ns = n_seq > ctx->ws_seq ? n_seq : ctx->ws_seq;
+    const uint64_t nc = n_chunks > ctx->ws_chunks ? n_chunks : ctx->ws_chunks;
+    void *p = nullptr;
+    const size_t bytes = (size_t)(ns + 2) * 8 + (size_t)(nc + 4) * 4;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
+    if (ctx->d_ws) cudaFree(ctx->d_ws);   // waits for work that may still use the old one
+    ctx->d_ws = p;
+    ctx->ws_seq = ns;
+    ctx->ws_chunks = nc;
+    return LSMKV_OK;
+}
+
+uint64_t *ws_hit_off(lsmkv_ctx *ctx) { return static_cast<uint64_t *>(ctx->d_ws); }
+uint32_t *ws_plan(lsmkv_ctx *ctx)
+{
+    return reinterpret_cast<uint32_t *>(static_cast<uint64_t *>(ctx->d_ws) + ctx->ws_seq + 2);
+}
+
+int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &ar,
+                uint64_t max_items)
+{
+    const uint64_t slabs = 2ull * ctx->geom.n_layers;
+    if (ctx->copy_mode == 1) {
+        job.piece_bytes = (uint32_t)ctx->page_bytes;
+        job.pieces_per_slab = 1;
+        uint64_t grid = (uint64_t)ctx->sm_count * (uint64_t)ctx->simt_ctas_per_sm;
+        const uint64_t units = max_items * slabs;
+        if (grid > units) grid = units;
+        if (grid == 0) return LSMKV_OK;
+        k_copy_slabs_simt<<<(unsigned)grid, 256, 0, s>>>(job, ar);
+    } else {
+        uint64_t piece = (uint64_t)ctx->copy_stage_bytes;
+        if (piece > ctx->page_bytes) piece = ctx->page_bytes;
+        job.piece_bytes = (uint32_t)piece;
+        job.pieces_per_slab = (uint32_t)((ctx->page_bytes + piece - 1) / piece);
+        const uint64_t stride = (piece + 127) & ~127ull;
+        int stages = (int)ctx->copy_stages;
+        const size_t per_cta_budget = (size_t)ctx->max_smem_optin / (size_t)ctx->copy_ctas_per_sm;
+        while (stages > 1 && (size_t)stages * stride + (size_t)stages * 8 + 1024 > per_cta_budget)
+            --stages;
+        const size_t smem = (size_t)stages * stride + (size_t)stages * 8;
+        if (smem > (size_t)ctx->max_smem_optin) return LSMKV_EINVAL;
+        uint64_t grid = (uint64_t)ctx->sm_count * (uint64_t)ctx->copy_ctas_per_sm;
+        const uint64_t pieces = max_items * slabs * job.pieces_per_slab;
+        const uint64_t need = (pieces + stages - 1) / stages;
+        if (grid > need) grid = need;
+        if (grid == 0) return LSMKV_OK;
+        if (ctx->copy_l2_hint) {
+            CU(ctx, cudaFuncSetAttribute(k_copy_slabs_bulk<true>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            k_copy_slabs_bulk<true><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
+        } else {
+            CU(ctx, cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            k_copy_slabs_bulk<false><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
+        }
+    }
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
+unsigned warp_grid(const lsmkv_ctx *ctx, uint64_t n_warps_wanted, unsigned threads,
+                   unsigned ctas_per_sm)
+{
+    const uint64_t wpc = threads / 32;
+    uint64_t grid = (n_warps_wanted + wpc - 1) / wpc;
+    const uint64_t cap = (uint64_t)ctx->sm_count * ctas_per_sm;
+    if (grid > cap) grid = cap;
+    return grid ? (unsigned)grid : 1u;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
+{
+    if (!out || !g) return LSMKV_EINVAL;
+    *out = nullptr;
+    if (!g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes || !g->page_tokens ||
+        g->chunk_tokens != g->page_tokens || g->flags != 0)
+        return LSMKV_EINVAL;
+    const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
+    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
+    lsmkv_ctx *ctx = new (std::nothrow) lsmkv_ctx();
+    if (!ctx) return LSMKV_ENOMEM;
+    std::memset(ctx, 0, sizeof(*ctx));
+    ctx->geom = *g;
+    ctx->device = device;
+    ctx->page_bytes = pb;
+    ctx->chunk_bytes = 2ull * g->n_layers * pb;
+    fill_key_consts(ctx->kc, g->chunk_tokens);
+    ctx->copy_mode = 0;
+    ctx->copy_stage_bytes = 32768;
+    ctx->copy_stages = 6;
+    ctx->copy_ctas_per_sm = 1;
+    ctx->copy_l2_hint = 0;
+    ctx->probe_warps_per_cta = 8;
+    ctx->simt_ctas_per_sm = 8;
+
+    DeviceGuard guard(device);
+    cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(DevStatus));
+    if (e == cudaSuccess) {
+        DevStatus z;
+        std::memset(&z, 0, sizeof(z));
+        z.first_bad = ~0ull;
+        e = cudaMemcpy(ctx->d_status, &z, sizeof(z), cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        delete ctx;
+        return LSMKV_ECUDA;
+    }
+    int rc = ensure_workspace(ctx, 1024, 65536);
+    if (rc != LSMKV_OK) {
+        cudaFree(ctx->d_status);
+        delete ctx;
+        return rc;
+    }
+    *out = ctx;
+    return LSMKV_OK;
+}
+
+int lsmkv_destroy(lsmkv_ctx *ctx)
+{
+    if (!ctx) return LSMKV_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->d_ws) cudaFree(ctx->d_ws);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    cudaGetLastError();
+    delete ctx;
+    return LSMKV_OK;
+}
+
+int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
+{
+    if (!ctx || n_chunks >= 0xFFFFFFFFull) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    return ensure_workspace(ctx, n_seq, n_chunks);
+}
+
+int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint32_t *tokens,
+                       const uint64_t *seq_off, const uint32_t *start_chunk,
+                       const uint64_t *chunk_off, uint64_t n_chunks, const uint32_t *page_table,
+                       const lsmkv_pool_t *pool, uint32_t file_id, uint64_t base_offset,
+                       lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, void *blob_out,
+                       uint64_t blob_capacity)
+{
+    if (!ctx) return LSMKV_EINVAL;
+    if (n_req == 0 || n_chunks == 0) return n_chunks == 0 ? LSMKV_OK : LSMKV_EINVAL;
+    if (!seq_off || !chunk_off || !tokens || !keys_out || !vals_out) return LSMKV_EINVAL;
+    if (!aligned16(keys_out) || !aligned16(vals_out)) return LSMKV_EINVAL;
+    const bool with_blob = blob_out != nullptr;
+    if (with_blob) {
+        if (!page_table || !pool || !pool->kv_ptrs || !aligned16(blob_out)) return LSMKV_EINVAL;
+        if (n_chunks > UINT64_MAX / ctx->chunk_bytes) return LSMKV_EINVAL;
+        if (blob_capacity < n_chunks * ctx->chunk_bytes) return LSMKV_ECAPACITY;
+    } else if (page_table || pool) {
+        return LSMKV_EINVAL;
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    const unsigned grid = warp_grid(ctx, n_req, 128, 16);
+    k_encode_keys<<<grid, 128, 0, s>>>(ctx->kc, ctx->geom.chunk_tokens, ctx->geom.ns, n_req, tokens,
+                                       seq_off, start_chunk, chunk_off, n_chunks, file_id,
+                                       base_offset, ctx->chunk_bytes, keys_out, vals_out,
+                                       ctx->d_status);
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    if (!with_blob) return LSMKV_OK;
+
+    CopyJob job;
+    std::memset(&job, 0, sizeof(job));
+    job.unpack = 0;
+    job.n_layers = ctx->geom.n_layers;
+    job.page_bytes = (uint32_t)ctx->page_bytes;
+    job.num_pages = pool->num_pages;
+    job.kv_ptrs = pool->kv_ptrs;
+    job.page_table = page_table;
+    job.blob = static_cast<unsigned char *>(blob_out);
+    job.n_items = n_chunks;
+    job.st = ctx->d_status;
+    ArenaTable ar;
+    std::memset(&ar, 0, sizeof(ar));
+    return launch_copy(ctx, s, job, ar, n_chunks);
+}
+
+int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint32_t *tokens,
+                      const uint64_t *seq_off, const uint64_t *qchunk_off, uint64_t n_qchunks,
+                      const lsmkv_run_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,
+                      lsmkv_val_t *recs_out, lsmkv_key_t *keys_out)
+{
+    if (!ctx) return LSMKV_EINVAL;
+    if (n_query == 0) return LSMKV_OK;
+    if (!seq_off || !qchunk_off || !hit_chunks_out) return LSMKV_EINVAL;
+    if (n_qchunks && (!tokens || !recs_out || !aligned16(recs_out))) return LSMKV_EINVAL;
+    if (keys_out && !aligned16(keys_out)) return LSMKV_EINVAL;
+    if (n_runs > LSMKV_MAX_RUNS || (n_runs && !runs)) return LSMKV_EINVAL;
+    RunTable rt;
+    std::memset(&rt, 0, sizeof(rt));
+    for (uint32_t r = 0; r < n_runs; ++r) {
+        if (runs[r].n && (!runs[r].keys || !runs[r].vals || !aligned16(runs[r].keys) ||
+                          !aligned16(runs[r].vals)))
+            return LSMKV_EINVAL;
+        rt.keys[r] = runs[r].keys;
+        rt.vals[r] = runs[r].vals;
+        rt.n[r] = runs[r].n;
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const unsigned threads = (unsigned)ctx->probe_warps_per_cta * 32u;
+    const unsigned grid = warp_grid(ctx, n_query, threads, 2048 / threads);
+    k_probe<<<grid, threads, 0, s>>>(ctx->kc, rt, n_runs, ctx->geom.chunk_tokens, ctx->geom.ns,
+                                     n_query, tokens, seq_off, qchunk_off, n_qchunks,
+                                     hit_chunks_out, recs_out, keys_out, ctx->d_status);
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
+int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
+                       const uint64_t *qchunk_off, uint64_t n_qchunks,
+                       const uint32_t *hit_chunks, const lsmkv_val_t *recs,
+                       const void *const *arenas, const uint64_t *arena_bytes,
+                       uint32_t n_arenas, const uint32_t *dst_page_table,
+                       const lsmkv_pool_t *pool)
+{
+    if (!ctx) return LSMKV_EINVAL;
+    if (n_query == 0 || n_qchunks == 0) return LSMKV_OK;
+    if (!qchunk_off || !hit_chunks || !recs || !dst_page_table || !pool || !pool->kv_ptrs)
+        return LSMKV_EINVAL;
+    if (n_arenas == 0 || n_arenas > (uint32_t)kMaxArenas || !arenas || !arena_bytes)
+        return LSMKV_EINVAL;
+    if (n_qchunks >= 0xFFFFFFFFull || !aligned16(recs)) return LSMKV_EINVAL;
+    ArenaTable ar;
+    std::memset(&ar, 0, sizeof(ar));
+    for (uint32_t a = 0; a < n_arenas; ++a) {
+        if (arena_bytes[a] && (!arenas[a] || !aligned16(arenas[a]))) return LSMKV_EINVAL;
+        ar.base[a] = static_cast<const unsigned char *>(arenas[a]);
+        ar.bytes[a] = arena_bytes[a];
+    }
+    DeviceGuard guard(ctx->device);
+    int rc = ensure_workspace(ctx, n_query, n_qchunks);
+    if (rc != LSMKV_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    uint64_t *hit_off = ws_hit_off(ctx);
+    uint32_t *plan = ws_plan(ctx);
+    k_plan_scan<<<1, 1024, 0, s>>>(n_query, qchunk_off, n_qchunks, hit_chunks, hit_off,
+                                   ctx->d_status);
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    k_plan_fill<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
+        n_query, qchunk_off, hit_off, recs, ar, n_arenas, ctx->chunk_bytes, plan, ctx->d_status);
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+
+    CopyJob job;
+    std::memset(&job, 0, sizeof(job));
+    job.unpack = 1;
+    job.n_layers = ctx->geom.n_layers;
+    job.page_bytes = (uint32_t)ctx->page_bytes;
+    job.num_pages = pool->num_pages;
+    job.kv_ptrs = pool->kv_ptrs;
+    job.page_table = dst_page_table;
+    job.n_items_dev = hit_off + n_query;
+    job.plan = plan;
+    job.recs = recs;
+    job.st = ctx->d_status;
+    return launch_copy(ctx, s, job, ar, n_qchunks);
+}
+
+int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out)
+{
+    if (!ctx || !out) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(ctx, cudaMemcpyAsync(out, ctx->d_status, sizeof(DevStatus), cudaMemcpyDeviceToHost, s));
+    CU(ctx, cudaStreamSynchronize(s));
+    DevStatus z;
+    std::memset(&z, 0, sizeof(z));
+    z.first_bad = ~0ull;
+    CU(ctx, cudaMemcpyAsync(ctx->d_status, &z, sizeof(z), cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaStreamSynchronize(s));
+    return LSMKV_OK;
+}
+
+int lsmkv_last_cuda_error(const lsmkv_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64_t *hi)
+{
+    struct { const char *n; int64_t *p; int64_t lo, hi; } tab[] = {
+        {"copy_mode", &ctx->copy_mode, 0, 1},
+        {"copy_stage_bytes", &ctx->copy_stage_bytes, 16, 1 << 17},
+        {"copy_stages", &ctx->copy_stages, 1, 32},
+        {"copy_ctas_per_sm", &ctx->copy_ctas_per_sm, 1, 8},
+        {"copy_l2_hint", &ctx->copy_l2_hint, 0, 1},
+        {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 32},
+        {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
+    };
+    for (auto &t : tab)
+        if (std::strcmp(t.n, name) == 0) { *lo = t.lo; *hi = t.hi; return t.p; }
+    return nullptr;
+}
+
+int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value)
+{
+    if (!ctx || !name) return LSMKV_EINVAL;
+    int64_t lo, hi;
+    int64_t *p = tuning_slot(ctx, name, &lo, &hi);
+    if (!p || value < lo || value > hi) return LSMKV_EINVAL;
+    if (std::strcmp(name, "copy_stage_bytes") == 0 && value % 16 != 0) return LSMKV_EINVAL;
+    *p = value;
+    return LSMKV_OK;
+}
+
+int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name)
+{
+    if (!ctx || !name) return LSMKV_EINVAL;
+    int64_t lo, hi;
+    int64_t *p = tuning_slot(const_cast<lsmkv_ctx *>(ctx), name, &lo, &hi);
+    return p ? *p : LSMKV_EINVAL;
+}
+
+const char *lsmkv_strerror(int code)
+{
+    switch (code) {
+    case LSMKV_OK: return "ok";
+    case LSMKV_EINVAL: return "invalid argument";
+    case LSMKV_ECAPACITY: return "output buffer too small";
+    case LSMKV_ECUDA: return "CUDA error";
+    case LSMKV_ENOMEM: return "out of memory";
+    default: return "unknown error";
+    }
+}
+
+int lsmkv_format_version(void) { return LSMKV_FORMAT_VERSION; }
+
+}  // extern "C"

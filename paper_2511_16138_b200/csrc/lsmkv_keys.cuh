@@ -1,0 +1,156 @@
+// Chunk keys: two polynomial digests over the Mersenne prime 2^61-1 of every chunk-aligned
+// token prefix, evaluated warp-cooperatively.
+//
+// The digest is defined sequentially (h <- h*B + t + 1 mod p per token). Because
+// H(XY) = H(X) * B^|Y| + H(Y), a warp hashes 32 consecutive chunks at once: every lane runs
+// the recurrence over its own chunk from h = 0, then an inclusive warp scan with the fixed
+// multiplier M = B^C stitches the chunk hashes into prefix hashes, and the running prefix of
+// the previous 32 chunks enters through M^(lane+1). All arithmetic is exact, so the result is
+// bit-identical to the sequential definition.
+#pragma once
+#include "lsmkv_common.cuh"
+
+namespace lsmkv {
+
+constexpr uint64_t kP = 0x1FFFFFFFFFFFFFFFull;  // 2^61 - 1
+constexpr uint64_t kBaseA = 0x0B4E0EF37BC32127ull;
+constexpr uint64_t kBaseB = 0x16A09E667F3BCC90ull;
+
+// pw[x][i] = (BASE_x ^ C) ^ (i+1) mod p for i = 0..31; entries 0,1,3,7,15 are the scan
+// multipliers M^1, M^2, M^4, M^8, M^16.
+struct KeyConsts {
+    uint64_t pwA[32];
+    uint64_t pwB[32];
+};
+
+// a, b < 2^61  ->  a*b mod p, canonical
+__host__ __device__ __forceinline__ uint64_t fold61(uint64_t s)  // s < 2^62
+{
+    s = (s & kP) + (s >> 61);
+    return s >= kP ? s - kP : s;
+}
+
+__device__ __forceinline__ uint64_t mulmod61(uint64_t a, uint64_t b)
+{
+    const uint64_t lo = a * b;
+    const uint64_t hi = __umul64hi(a, b);               // product < 2^122, hi < 2^58
+    // 2^61 = 1 (mod p):  hi*2^64 + lo = (lo & p) + (lo >> 61) + hi*8
+    return fold61((lo & kP) + ((lo >> 61) | (hi << 3)));
+}
+
+__device__ __forceinline__ uint64_t addmod61(uint64_t a, uint64_t b)  // a, b < p
+{
+    const uint64_t s = a + b;
+    return s >= kP ? s - kP : s;
+}
+
+__device__ __forceinline__ uint64_t horner61(uint64_t h, uint64_t base, uint32_t token)
+{
+    return fold61(mulmod61(h, base) + (uint64_t)token + 1ull);   // < p + 2^32 < 2^62
+}
+
+__device__ __forceinline__ uint64_t shfl_up64(uint64_t v, unsigned d)
+{
+    return __shfl_up_sync(0xFFFFFFFFu, v, d);
+}
+
+struct ChunkKey { uint64_t w0, w1, w2, w3; };
+
+// One warp, 32 consecutive chunks j = base_j + lane of the sequence starting at `seq`.
+// carryA/carryB: digests of the prefix that ends just before chunk base_j (0 at base_j = 0);
+// updated to the prefix that ends after chunk base_j + 31. Lanes with j >= nch contribute
+// nothing meaningful and their key must be ignored. Must be called by all 32 lanes.
+__device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
+                                                    uint32_t C, uint32_t ns, uint64_t base_j,
+                                                    uint64_t nch, uint64_t &carryA,
+                                                    uint64_t &carryB)
+{
+    const unsigned lane = lane_id();
+    const uint64_t j = base_j + lane;
+    uint64_t hA = 0, hB = 0;
+    uint32_t first = 0, last = 0;
+    if (j < nch) {
+        const uint32_t *t = seq + j * C;
+        first = __ldg(t);
+        last = first;
+        hA = (uint64_t)first + 1ull;
+        hB = hA;
+#pragma unroll 4
+        for (uint32_t i = 1; i < C; ++i) {
+            last = __ldg(t + i);
+            hA = horner61(hA, kBaseA, last);
+            hB = horner61(hB, kBaseB, last);
+        }
+    }
+    // inclusive scan: x_i <- x_{i-d} * M^d + x_i
+#pragma unroll
+    for (unsigned d = 1; d < 32; d <<= 1) {
+        const uint64_t uA = shfl_up64(hA, d), uB = shfl_up64(hB, d);
+        if (lane >= d) {
+            hA = addmod61(mulmod61(uA, kc.pwA[d - 1]), hA);
+            hB = addmod61(mulmod61(uB, kc.pwB[d - 1]), hB);
+        }
+    }
+    hA = addmod61(mulmod61(carryA, kc.pwA[lane]), hA);
+    hB = addmod61(mulmod61(carryB, kc.pwB[lane]), hB);
+    carryA = __shfl_sync(0xFFFFFFFFu, hA, 31);
+    carryB = __shfl_sync(0xFFFFFFFFu, hB, 31);
+    ChunkKey k;
+    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)j;
+    k.w1 = hA;
+    k.w2 = hB;
+    k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
+    return k;
+}
+
+__device__ __forceinline__ void store_key(lsmkv_key_t *dst, const ChunkKey &k)
+{
+    ulonglong2 *p = reinterpret_cast<ulonglong2 *>(dst);
+    p[0] = make_ulonglong2(k.w0, k.w1);
+    p[1] = make_ulonglong2(k.w2, k.w3);
+}
+
+// put_batch keys + records: one warp per request.
+__global__ void __launch_bounds__(128)
+k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uint32_t n_req,
+              const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
+              const uint32_t *__restrict__ start_chunk, const uint64_t *__restrict__ chunk_off,
+              uint64_t n_chunks, uint32_t file_id, uint64_t base_offset, uint64_t chunk_bytes,
+              lsmkv_key_t *__restrict__ keys_out, lsmkv_val_t *__restrict__ vals_out,
+              DevStatus *st)
+{
+    const unsigned lane = lane_id();
+    const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    for (uint64_t r = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_req;
+         r += warps) {
+        const uint64_t s0 = seq_off[r], s1 = seq_off[r + 1];
+        const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
+        const uint64_t start = start_chunk ? start_chunk[r] : 0;
+        const uint64_t cnt = nch > start ? nch - start : 0;
+        const uint64_t o0 = chunk_off[r], o1 = chunk_off[r + 1];
+        if (s1 < s0 || o1 < o0 || o1 - o0 != cnt || o1 > n_chunks || nch > 0xFFFFFFFFull) {
+            if (lane == 0) st_flag(st, LSMKV_ST_BAD_COUNT, r);
+            continue;
+        }
+        if (cnt == 0) continue;
+        uint64_t cA = 0, cB = 0;
+        for (uint64_t base = 0; base < nch; base += 32) {
+            const ChunkKey k = warp_chunk_keys(kc, tokens + s0, C, ns, base, nch, cA, cB);
+            const uint64_t j = base + lane;
+            if (j >= start && j < nch) {
+                const uint64_t i = o0 + (j - start);
+                store_key(keys_out + i, k);
+                uint4 v;
+                const uint64_t off = base_offset + i * chunk_bytes;
+                v.x = file_id;
+                v.y = 0;
+                v.z = (uint32_t)off;
+                v.w = (uint32_t)(off >> 32);
+                *reinterpret_cast<uint4 *>(vals_out + i) = v;
+            }
+        }
+        if (lane == 0) atomicAdd(&st->chunks_encoded, (unsigned long long)cnt);
+    }
+}
+
+}  // namespace lsmkv

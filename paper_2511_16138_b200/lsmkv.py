@@ -1,0 +1,309 @@
+"""ctypes binding of liblsmkv.so -- the same entry points as include/lsmkv.h.
+
+Argument marshalling only: tensors (anything with ``data_ptr()``), raw integer addresses or
+``None`` become pointers; every step of the path runs inside the CUDA library. There is no CPU
+fallback: if the shared library is missing or fails to load, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblsmkv.so")
+
+OK, EINVAL, ECAPACITY, ECUDA, ENOMEM = 0, -1, -2, -3, -4
+ST_BAD_PAGE, ST_BAD_RECORD, ST_BAD_COUNT, ST_MISALIGNED, ST_WAIT_EXPIRED = 1, 2, 4, 8, 16
+MAX_RUNS = 64
+KEY_BYTES, VAL_BYTES = 32, 16
+
+EXPORTS = (
+    "lsmkv_create", "lsmkv_destroy", "lsmkv_reserve", "lsmkv_encode_batch",
+    "lsmkv_probe_batch", "lsmkv_decode_batch", "lsmkv_last_status", "lsmkv_last_cuda_error",
+    "lsmkv_launch_count", "lsmkv_set_tuning", "lsmkv_get_tuning", "lsmkv_strerror",
+    "lsmkv_format_version",
+)
+
+
+class LsmkvError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        msg = f"{where}: {strerror(code)} ({code})"
+        if cuda:
+            msg += f", cudaError {cuda}"
+        super().__init__(msg)
+        self.code = code
+        self.cuda = cuda
+
+
+class GeomStruct(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("n_layers", "n_kv_heads", "head_dim", "elem_bytes",
+                                          "page_tokens", "chunk_tokens", "ns", "flags")]
+
+
+class RunStruct(C.Structure):
+    _fields_ = [("keys", C.c_void_p), ("vals", C.c_void_p), ("n", C.c_uint64)]
+
+
+class PoolStruct(C.Structure):
+    _fields_ = [("kv_ptrs", C.c_void_p), ("num_pages", C.c_uint64)]
+
+
+class StatusStruct(C.Structure):
+    _fields_ = [("flags", C.c_uint32), ("reserved", C.c_uint32), ("first_bad", C.c_uint64),
+                ("chunks_encoded", C.c_uint64), ("lookups", C.c_uint64),
+                ("chunks_hit", C.c_uint64), ("empty_probes", C.c_uint64),
+                ("chunks_decoded", C.c_uint64)]
+
+
+@dataclass(frozen=True)
+class Geom:
+    n_layers: int
+    n_kv_heads: int
+    head_dim: int
+    elem_bytes: int = 2
+    page_tokens: int = 16
+    chunk_tokens: int = 16
+    ns: int = 0
+    flags: int = 0
+
+    @property
+    def page_bytes(self) -> int:
+        return self.page_tokens * self.n_kv_heads * self.head_dim * self.elem_bytes
+
+    @property
+    def chunk_bytes(self) -> int:
+        return 2 * self.n_layers * self.page_bytes
+
+    def c(self) -> GeomStruct:
+        return GeomStruct(self.n_layers, self.n_kv_heads, self.head_dim, self.elem_bytes,
+                          self.page_tokens, self.chunk_tokens, self.ns, self.flags)
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load liblsmkv.so (built in-tree by ``paper_2511_16138_b200.build``). Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with "
+                          "`python -m paper_2511_16138_b200.build` (needs nvcc)")
+    L = C.CDLL(LIB_PATH)
+    vp, u32, u64, i64 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int64
+    L.lsmkv_create.restype = C.c_int
+    L.lsmkv_create.argtypes = [C.POINTER(vp), C.POINTER(GeomStruct), C.c_int]
+    L.lsmkv_destroy.restype = C.c_int
+    L.lsmkv_destroy.argtypes = [vp]
+    L.lsmkv_reserve.restype = C.c_int
+    L.lsmkv_reserve.argtypes = [vp, u64, u64]
+    L.lsmkv_encode_batch.restype = C.c_int
+    L.lsmkv_encode_batch.argtypes = [vp, vp, u32, vp, vp, vp, vp, u64, vp,
+                                     C.POINTER(PoolStruct), u32, u64, vp, vp, vp, u64]
+    L.lsmkv_probe_batch.restype = C.c_int
+    L.lsmkv_probe_batch.argtypes = [vp, vp, u32, vp, vp, vp, u64, C.POINTER(RunStruct), u32,
+                                    vp, vp, vp]
+    L.lsmkv_decode_batch.restype = C.c_int
+    L.lsmkv_decode_batch.argtypes = [vp, vp, u32, vp, u64, vp, vp, C.POINTER(vp),
+                                     C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
+    L.lsmkv_last_status.restype = C.c_int
+    L.lsmkv_last_status.argtypes = [vp, vp, C.POINTER(StatusStruct)]
+    L.lsmkv_last_cuda_error.restype = C.c_int
+    L.lsmkv_last_cuda_error.argtypes = [vp]
+    L.lsmkv_launch_count.restype = u64
+    L.lsmkv_launch_count.argtypes = [vp]
+    L.lsmkv_set_tuning.restype = C.c_int
+    L.lsmkv_set_tuning.argtypes = [vp, C.c_char_p, i64]
+    L.lsmkv_get_tuning.restype = i64
+    L.lsmkv_get_tuning.argtypes = [vp, C.c_char_p]
+    L.lsmkv_strerror.restype = C.c_char_p
+    L.lsmkv_strerror.argtypes = [C.c_int]
+    L.lsmkv_format_version.restype = C.c_int
+    L.lsmkv_format_version.argtypes = []
+    _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    try:
+        return lib().lsmkv_strerror(code).decode()
+    except Exception:
+        return "error"
+
+
+def _ptr(x):
+    """tensor / int / None -> address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(ctx, rc: int, where: str):
+    if rc != OK:
+        raise LsmkvError(rc, where, lib().lsmkv_last_cuda_error(ctx) if ctx else 0)
+
+
+# ---- the C entry points, one to one ------------------------------------------------------
+
+def lsmkv_create(geom: Geom, device: int = 0) -> int:
+    h = C.c_void_p()
+    g = geom.c()
+    _check(None, lib().lsmkv_create(C.byref(h), C.byref(g), device), "lsmkv_create")
+    return h.value
+
+
+def lsmkv_destroy(ctx) -> None:
+    _check(None, lib().lsmkv_destroy(ctx), "lsmkv_destroy")
+
+
+def lsmkv_reserve(ctx, n_seq: int, n_chunks: int) -> None:
+    _check(ctx, lib().lsmkv_reserve(ctx, n_seq, n_chunks), "lsmkv_reserve")
+
+
+def _pool(pool):
+    if pool is None:
+        return None
+    kv_ptrs, num_pages = pool
+    return PoolStruct(_ptr(kv_ptrs), num_pages)
+
+
+def lsmkv_encode_batch(ctx, stream, n_req, tokens, seq_off, start_chunk, chunk_off, n_chunks,
+                       page_table, pool, file_id, base_offset, keys_out, vals_out, blob_out,
+                       blob_capacity) -> None:
+    p = _pool(pool)
+    rc = lib().lsmkv_encode_batch(ctx, _stream(stream), n_req, _ptr(tokens), _ptr(seq_off),
+                                  _ptr(start_chunk), _ptr(chunk_off), n_chunks,
+                                  _ptr(page_table), C.byref(p) if p is not None else None,
+                                  file_id, base_offset, _ptr(keys_out), _ptr(vals_out),
+                                  _ptr(blob_out), blob_capacity)
+    _check(ctx, rc, "lsmkv_encode_batch")
+
+
+def lsmkv_probe_batch(ctx, stream, n_query, tokens, seq_off, qchunk_off, n_qchunks, runs,
+                      hit_chunks_out, recs_out, keys_out=None) -> None:
+    """runs: sequence of (keys, vals, n), newest first."""
+    n_runs = len(runs)
+    arr = (RunStruct * max(1, n_runs))()
+    for i, (k, v, n) in enumerate(runs):
+        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    rc = lib().lsmkv_probe_batch(ctx, _stream(stream), n_query, _ptr(tokens), _ptr(seq_off),
+                                 _ptr(qchunk_off), n_qchunks, arr, n_runs,
+                                 _ptr(hit_chunks_out), _ptr(recs_out), _ptr(keys_out))
+    _check(ctx, rc, "lsmkv_probe_batch")
+
+
+def lsmkv_decode_batch(ctx, stream, n_query, qchunk_off, n_qchunks, hit_chunks, recs, arenas,
+                       dst_page_table, pool) -> None:
+    """arenas: sequence of (base, n_bytes) indexed by file_id."""
+    n = len(arenas)
+    bases = (C.c_void_p * max(1, n))(*[_ptr(a) for a, _ in arenas])
+    sizes = (C.c_uint64 * max(1, n))(*[b for _, b in arenas])
+    p = _pool(pool)
+    rc = lib().lsmkv_decode_batch(ctx, _stream(stream), n_query, _ptr(qchunk_off), n_qchunks,
+                                  _ptr(hit_chunks), _ptr(recs), bases, sizes, n,
+                                  _ptr(dst_page_table), C.byref(p) if p is not None else None)
+    _check(ctx, rc, "lsmkv_decode_batch")
+
+
+def lsmkv_last_status(ctx, stream=None) -> dict:
+    st = StatusStruct()
+    _check(ctx, lib().lsmkv_last_status(ctx, _stream(stream), C.byref(st)), "lsmkv_last_status")
+    return {n: getattr(st, n) for n, _ in StatusStruct._fields_ if n != "reserved"}
+
+
+def lsmkv_launch_count(ctx) -> int:
+    return int(lib().lsmkv_launch_count(ctx))
+
+
+def lsmkv_set_tuning(ctx, name: str, value: int) -> None:
+    _check(ctx, lib().lsmkv_set_tuning(ctx, name.encode(), value), f"lsmkv_set_tuning({name})")
+
+
+def lsmkv_get_tuning(ctx, name: str) -> int:
+    return int(lib().lsmkv_get_tuning(ctx, name.encode()))
+
+
+def lsmkv_format_version() -> int:
+    return int(lib().lsmkv_format_version())
+
+
+# ---- convenience: a context object and a pool pointer table ------------------------------
+
+class Context:
+    """Owns one lsmkv_ctx. Methods forward to the functions above with ``self.handle``."""
+
+    def __init__(self, geom: Geom, device: int = 0):
+        self.geom = geom
+        self.device = device
+        self.handle = lsmkv_create(geom, device)
+
+    def close(self):
+        if self.handle:
+            lsmkv_destroy(self.handle)
+            self.handle = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def reserve(self, n_seq, n_chunks):
+        lsmkv_reserve(self.handle, n_seq, n_chunks)
+
+    def encode_batch(self, n_req, tokens, seq_off, start_chunk, chunk_off, n_chunks, page_table,
+                     pool, file_id, base_offset, keys_out, vals_out, blob_out, blob_capacity,
+                     stream=None):
+        lsmkv_encode_batch(self.handle, stream, n_req, tokens, seq_off, start_chunk, chunk_off,
+                           n_chunks, page_table, pool, file_id, base_offset, keys_out, vals_out,
+                           blob_out, blob_capacity)
+
+    def probe_batch(self, n_query, tokens, seq_off, qchunk_off, n_qchunks, runs, hit_chunks_out,
+                    recs_out, keys_out=None, stream=None):
+        lsmkv_probe_batch(self.handle, stream, n_query, tokens, seq_off, qchunk_off, n_qchunks,
+                          runs, hit_chunks_out, recs_out, keys_out)
+
+    def decode_batch(self, n_query, qchunk_off, n_qchunks, hit_chunks, recs, arenas,
+                     dst_page_table, pool, stream=None):
+        lsmkv_decode_batch(self.handle, stream, n_query, qchunk_off, n_qchunks, hit_chunks, recs,
+                           arenas, dst_page_table, pool)
+
+    def last_status(self, stream=None) -> dict:
+        return lsmkv_last_status(self.handle, stream)
+
+    def launch_count(self) -> int:
+        return lsmkv_launch_count(self.handle)
+
+    def set_tuning(self, name, value):
+        lsmkv_set_tuning(self.handle, name, value)
+
+    def get_tuning(self, name):
+        return lsmkv_get_tuning(self.handle, name)
+
+
+def pool_table(buffers):
+    """Device pointer table for 2L pool buffers (K layers, then V layers). Returns
+    ``(kv_ptrs tensor, num_pages)``; keep the tensor alive while kernels use it."""
+    import torch
+    ptrs = torch.tensor([b.data_ptr() for b in buffers], dtype=torch.int64,
+                        device=buffers[0].device)
+    return ptrs, int(buffers[0].shape[0])

@@ -1,0 +1,161 @@
+"""Helpers for the GPU parity tests: move numpy inputs to the device, run the CUDA library
+through its C ABI, run the oracle on the same inputs, and compare byte for byte."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from oracle import VAL_DTYPE
+from paper_2511_16138_b200 import hostindex, lsmkv, synth
+
+DEV = "cuda:0"
+
+
+def dev(a: np.ndarray) -> torch.Tensor:
+    """numpy array -> device byte tensor holding the same bytes (at least 16 bytes long)."""
+    b = np.ascontiguousarray(a).view(np.uint8).reshape(-1)
+    t = torch.zeros(max(16, b.size), dtype=torch.uint8, device=DEV)
+    if b.size:
+        t[:b.size] = torch.from_numpy(b.copy())
+    return t
+
+
+def host(t: torch.Tensor, dtype, n_bytes=None) -> np.ndarray:
+    a = t.detach().cpu().numpy().reshape(-1)
+    if n_bytes is not None:
+        a = a[:n_bytes]
+    return a.view(dtype)
+
+
+def ogeom(g: lsmkv.Geom) -> oracle.Geom:
+    return oracle.Geom(g.n_layers, g.n_kv_heads, g.head_dim, g.elem_bytes, g.page_tokens,
+                       g.chunk_tokens, g.ns, g.flags)
+
+
+class DevPool:
+    def __init__(self, g: lsmkv.Geom, num_pages: int, init: np.ndarray | None = None):
+        self.g, self.num_pages = g, num_pages
+        self.t = torch.zeros((2 * g.n_layers, num_pages, g.page_bytes), dtype=torch.uint8,
+                             device=DEV)
+        if init is not None:
+            self.t.copy_(torch.from_numpy(init))
+        self.table = lsmkv.pool_table([self.t[i] for i in range(2 * g.n_layers)])
+
+    def numpy(self) -> np.ndarray:
+        return self.t.cpu().numpy()
+
+
+def gpu_encode(ctx, g, batch, start_chunk, chunk_off, page_table, pool: DevPool | None,
+               file_id=0, base_offset=0):
+    n = int(chunk_off[-1])
+    d_tok, d_off, d_coff = dev(batch.tokens), dev(batch.seq_off), dev(chunk_off)
+    d_start = None if start_chunk is None else dev(np.asarray(start_chunk, np.uint32))
+    d_keys = torch.zeros(max(1, n) * 32, dtype=torch.uint8, device=DEV)
+    d_vals = torch.zeros(max(1, n) * 16, dtype=torch.uint8, device=DEV)
+    d_blob = d_pt = None
+    if pool is not None:
+        d_pt = dev(np.asarray(page_table, np.uint32))
+        d_blob = torch.zeros(max(16, n * g.chunk_bytes), dtype=torch.uint8, device=DEV)
+    ctx.encode_batch(batch.n, d_tok, d_off, d_start, d_coff, n, d_pt,
+                     pool.table if pool is not None else None, file_id, base_offset, d_keys,
+                     d_vals, d_blob, 0 if d_blob is None else n * g.chunk_bytes)
+    torch.cuda.synchronize()
+    keys = host(d_keys, np.uint64, n * 32).reshape(-1, 4)
+    vals = host(d_vals, VAL_DTYPE, n * 16)
+    blob = None if d_blob is None else host(d_blob, np.uint8, n * g.chunk_bytes)
+    return keys, vals, blob, d_blob
+
+
+def dev_runs(runs):
+    keep, out = [], []
+    for k, v in runs:
+        dk, dv = dev(k), dev(v)
+        keep.append((dk, dv))
+        out.append((dk, dv, len(k)))
+    return out, keep
+
+
+def gpu_probe(ctx, batch, qoff, runs, want_keys=True):
+    nq, total = batch.n, int(qoff[-1])
+    d_tok, d_off, d_qoff = dev(batch.tokens), dev(batch.seq_off), dev(qoff)
+    d_hit = torch.full((max(4, nq),), 0x7FFFFFFF, dtype=torch.int32, device=DEV)
+    d_recs = torch.full((max(1, total) * 16,), 0xAB, dtype=torch.uint8, device=DEV)
+    d_keys = torch.zeros(max(1, total) * 32, dtype=torch.uint8, device=DEV) if want_keys else None
+    druns, keep = dev_runs(runs)
+    ctx.probe_batch(nq, d_tok, d_off, d_qoff, total, druns, d_hit, d_recs, d_keys)
+    torch.cuda.synchronize()
+    hit = d_hit.cpu().numpy().view(np.uint32)[:nq]
+    recs = host(d_recs, VAL_DTYPE, total * 16)
+    keys = host(d_keys, np.uint64, total * 32).reshape(-1, 4) if want_keys else None
+    return hit, recs, keys, (d_qoff, d_hit, d_recs)
+
+
+def assert_status_clean(ctx):
+    st = ctx.last_status()
+    assert st["flags"] == 0, st
+    return st
+
+
+def roundtrip(g: lsmkv.Geom, store, query, start_chunk=None, n_runs=1, num_pages=None,
+              tuning=None, seed=0, base_offset=0):
+    """Encode `store`, flush into n_runs runs, probe `query`, decode the hits into a zeroed pool;
+    every output is compared with the oracle's. Returns a dict of the interesting outputs."""
+    og = ogeom(g)
+    rng = np.random.default_rng(seed)
+    C = g.chunk_tokens
+    nch = synth.chunk_counts(store.seq_off, C)
+    st = np.zeros(store.n, np.uint32) if start_chunk is None else np.asarray(start_chunk, np.uint32)
+    coff = synth.offsets(np.maximum(nch - st.astype(np.int64), 0))
+    n = int(coff[-1])
+    qoff = synth.offsets(synth.chunk_counts(query.seq_off, C))
+    nq_chunks = int(qoff[-1])
+    num_pages = num_pages or max(n, nq_chunks, 1) + 3
+    pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
+    src_pages = synth.random_pages(rng, num_pages, n)
+    dst_pages = synth.random_pages(rng, num_pages, nq_chunks)
+
+    # ---- oracle
+    o_keys, o_vals, o_blob = oracle.encode_batch(og, store.tokens, store.seq_off,
+                                                 None if start_chunk is None else st, coff,
+                                                 src_pages, pool_np, 0, base_offset)
+    owner = rng.integers(0, n_runs, n)
+    o_runs = [oracle.flush(o_keys[owner == r], o_vals[owner == r]) for r in range(n_runs)]
+    o_hit, o_recs, o_qkeys, _ = oracle.probe_batch(og, query.tokens, query.seq_off, qoff, o_runs,
+                                                   want_keys=True)
+    o_dst = np.zeros_like(pool_np)
+    arena_np = np.concatenate([np.zeros(base_offset, np.uint8), o_blob])
+    oracle.decode_batch(og, qoff, o_hit, o_recs, [arena_np], dst_pages, o_dst)
+
+    # ---- CUDA library
+    with lsmkv.Context(g, 0) as ctx:
+        for k, v in (tuning or {}).items():
+            ctx.set_tuning(k, v)
+        pool = DevPool(g, num_pages, pool_np)
+        keys, vals, blob, d_blob = gpu_encode(ctx, g, store, None if start_chunk is None else st,
+                                              coff, src_pages, pool, 0, base_offset)
+        assert np.array_equal(keys, o_keys), "chunk keys differ"
+        assert np.array_equal(vals, o_vals), "records differ"
+        assert np.array_equal(blob, o_blob), "blobs differ"
+        assert np.array_equal(pool.numpy(), pool_np), "encode modified the pool"
+        runs = [hostindex.flush(keys[owner == r], vals[owner == r]) for r in range(n_runs)]
+        for (k, v), (ok, ov) in zip(runs, o_runs):
+            assert np.array_equal(k, ok) and np.array_equal(v, ov)
+        hit, recs, qkeys, (d_qoff, d_hit, d_recs) = gpu_probe(ctx, query, qoff, runs)
+        assert np.array_equal(hit, o_hit), "hit lengths differ"
+        assert np.array_equal(qkeys, o_qkeys), "query keys differ"
+        assert np.array_equal(recs, o_recs), "hit records differ"
+        hit2, recs2, _, _ = gpu_probe(ctx, query, qoff, runs, want_keys=False)
+        assert np.array_equal(hit2, o_hit) and np.array_equal(recs2, o_recs)
+        dst = DevPool(g, num_pages)
+        d_arena = torch.zeros(max(16, base_offset + blob.size), dtype=torch.uint8, device=DEV)
+        d_arena[base_offset:base_offset + blob.size] = d_blob[:blob.size]
+        ctx.decode_batch(query.n, d_qoff, nq_chunks, d_hit, d_recs,
+                         [(d_arena, base_offset + blob.size)], dev(dst_pages), dst.table)
+        torch.cuda.synchronize()
+        assert np.array_equal(dst.numpy(), o_dst), "restored pool differs"
+        status = assert_status_clean(ctx)
+        assert status["chunks_encoded"] == n
+        assert status["chunks_hit"] == int(o_hit.sum()) * 2       # two probes
+        assert status["chunks_decoded"] == int(o_hit.sum())
+    return dict(hit=o_hit, n=n, status=status)

@@ -1,0 +1,138 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle -- byte
+equality of keys, records, blobs, hit lengths, hit records and the whole restored pool."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import VAL_DTYPE
+from paper_2511_16138_b200 import hostindex, lsmkv, synth
+
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+TINY = lsmkv.Geom(n_layers=4, n_kv_heads=8, head_dim=128, page_tokens=16, chunk_tokens=16)
+
+
+@pytest.mark.parametrize("n_runs", [1, 2])
+@pytest.mark.parametrize("tuning", [
+    {},                                                     # bulk copies, 32 KiB stages
+    {"copy_stage_bytes": 4096, "copy_stages": 12},
+    {"copy_stage_bytes": 12288, "copy_l2_hint": 1},         # ragged last piece of a 32 KiB slab
+    {"copy_mode": 1},
+])
+def test_config1_tiny_codec_full_compare(n_runs, tuning):
+    """Config 1: 4x8x128 bf16, page 16, 32 requests x 512 tokens sharing 0-256 tokens, probes
+    with the last 64 tokens re-drawn."""
+    w = synth.tiny_codec()
+    out = H.roundtrip(TINY, w.store, w.query, n_runs=n_runs, tuning=tuning, seed=1)
+    assert np.array_equal(out["hit"], w.expected_hit_tokens // 16)
+    assert out["n"] == 1024
+
+
+def test_start_chunk_and_base_offset():
+    w = synth.tiny_codec(n_req=12, seq_len=300)
+    g = lsmkv.Geom(2, 2, 64, page_tokens=16, chunk_tokens=16, ns=7)
+    rng = np.random.default_rng(3)
+    start = rng.integers(0, 22, 12).astype(np.uint32)      # some beyond the 18 chunks
+    start[0] = 0
+    H.roundtrip(g, w.store, w.query, start_chunk=start, n_runs=3, seed=2, base_offset=4096)
+
+
+@pytest.mark.parametrize("g", [
+    lsmkv.Geom(3, 4, 128, page_tokens=64, chunk_tokens=64),              # 64 KiB pages
+    lsmkv.Geom(2, 1, 24, elem_bytes=2, page_tokens=3, chunk_tokens=3),   # 144-byte pages
+    lsmkv.Geom(1, 1, 8, elem_bytes=1, page_tokens=2, chunk_tokens=2),    # 16-byte pages
+    lsmkv.Geom(5, 2, 40, elem_bytes=2, page_tokens=1, chunk_tokens=1),   # one token per chunk
+])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_geometries_and_ragged_lengths(g, mode):
+    rng = np.random.default_rng(5)
+    C = g.chunk_tokens
+    lens = [0, 1, C - 1, C, C + 1, 33 * C + 2, 70 * C, 5 * C, 32 * C, 31 * C + C // 2]
+    base = rng.integers(0, 5, 80 * C, dtype=np.uint32)
+    seqs = []
+    for n in lens:
+        s = base[:n].copy()
+        cut = int(rng.integers(0, n + 1))
+        s[cut:] = rng.integers(5, 10, n - cut)
+        seqs.append(s)
+    store = synth.make_batch(seqs)
+    qs = [s.copy() for s in seqs] + [base[:64 * C].copy(), rng.integers(5, 10, 9 * C, dtype=np.uint32)]
+    qs[5][20 * C + 1] ^= 1
+    query = synth.make_batch(qs)
+    H.roundtrip(g, store, query, n_runs=2, seed=6,
+                tuning={"copy_mode": mode, "copy_stage_bytes": 64})
+
+
+def test_long_sequences_cross_many_warp_batches():
+    g = lsmkv.Geom(1, 1, 8, elem_bytes=2, page_tokens=16, chunk_tokens=16)
+    w = synth.long_context(n_req=4, seq_len=16 * 700 + 5, shared=16 * 300, n_mutate=16 * 100)
+    out = H.roundtrip(g, w.store, w.query, n_runs=2, seed=7)
+    assert list(out["hit"]) == [600] * 4
+
+
+def test_empty_batches_and_no_runs():
+    g = TINY
+    with lsmkv.Context(g, 0) as ctx:
+        z = torch.zeros(64, dtype=torch.uint8, device=H.DEV)
+        ctx.encode_batch(0, z, z, None, z, 0, None, None, 0, 0, z, z, None, 0)
+        ctx.probe_batch(0, z, z, z, 0, [], z, z, None)
+        pool = H.DevPool(g, 2)
+        ctx.decode_batch(0, z, 0, z, z, [(z, 64)], z, pool.table)
+        # queries against an empty index: nothing is found
+        b = synth.make_batch([np.arange(40, dtype=np.uint32), np.arange(3, dtype=np.uint32)])
+        qoff = synth.offsets(synth.chunk_counts(b.seq_off, 16))
+        hit, recs, keys, _ = H.gpu_probe(ctx, b, qoff, [])
+        assert list(hit) == [0, 0] and not recs.view(np.uint8).any()
+        assert np.array_equal(keys, oracle.chunk_keys(H.ogeom(g), b.seq(0)))
+        H.assert_status_clean(ctx)
+
+
+def test_bad_inputs_are_flagged_and_skipped_without_faulting():
+    g = lsmkv.Geom(1, 1, 64, page_tokens=4, chunk_tokens=4)
+    og = H.ogeom(g)
+    b = synth.make_batch([np.arange(16, dtype=np.uint32)])
+    coff = synth.offsets([4])
+    rng = np.random.default_rng(8)
+    pool_np = synth.random_pool_bytes(rng, 2, 6, g.page_bytes)
+    with lsmkv.Context(g, 0) as ctx:
+        pool = H.DevPool(g, 6, pool_np)
+        pages = np.array([0, 9, 2, 3], dtype=np.uint32)                  # 9 is out of range
+        keys, vals, blob, d_blob = H.gpu_encode(ctx, g, b, None, coff, pages, pool)
+        st = ctx.last_status()
+        assert st["flags"] == lsmkv.ST_BAD_PAGE and st["first_bad"] == 1
+        good = np.array([0, 1, 2, 3], dtype=np.uint32)
+        _, _, want, = oracle.encode_batch(og, b.tokens, b.seq_off, None, coff, good, pool_np, 0, 0)
+        cb = g.chunk_bytes
+        assert np.array_equal(blob[:cb], want[:cb]) and np.array_equal(blob[2 * cb:], want[2 * cb:])
+        assert not blob[cb:2 * cb].any()                                 # skipped, left untouched
+        # chunk_off that disagrees with the sequence lengths
+        H.gpu_encode(ctx, g, b, None, synth.offsets([3]), good[:3], pool)
+        assert ctx.last_status()["flags"] == lsmkv.ST_BAD_COUNT
+        # records pointing outside the arena / unknown file / misaligned
+        recs = np.zeros(4, dtype=VAL_DTYPE)
+        recs["offset"] = [0, cb * 4, 8, cb]
+        recs["file_id"] = [0, 0, 0, 3]
+        dst = H.DevPool(g, 6)
+        arena = torch.from_numpy(want.copy()).to(H.DEV)
+        hit = np.array([4], dtype=np.uint32)
+        ctx.decode_batch(1, H.dev(coff), 4, H.dev(hit), H.dev(recs), [(arena, want.size)],
+                         H.dev(good), dst.table)
+        st = ctx.last_status()
+        assert st["flags"] == lsmkv.ST_BAD_RECORD and st["first_bad"] == 1
+        out = dst.numpy()
+        assert np.array_equal(out[:, 0], pool_np[:, 0]) and not out[:, 1:].any()
+        # hit length larger than the query's chunk count
+        ctx.decode_batch(1, H.dev(coff), 4, H.dev(np.array([5], np.uint32)), H.dev(recs),
+                         [(arena, want.size)], H.dev(good), dst.table)
+        assert ctx.last_status()["flags"] == lsmkv.ST_BAD_COUNT
+        # host-side rejections
+        with pytest.raises(lsmkv.LsmkvError) as e:
+            ctx.encode_batch(1, H.dev(b.tokens), H.dev(b.seq_off), None, H.dev(coff), 4,
+                             H.dev(good), pool.table, 0, 0, H.dev(keys), H.dev(vals), d_blob,
+                             4 * cb - 1)
+        assert e.value.code == lsmkv.ECAPACITY
+        with pytest.raises(lsmkv.LsmkvError):
+            ctx.set_tuning("no_such_knob", 1)
