@@ -1,0 +1,531 @@
+#!/usr/bin/env python
+"""Benchmark of the whole hot path: encode (chunk keys + records + pack) -> probe -> decode
+(unpack/scatter) over one batch of Llama-3-8B-shaped requests, on N GPUs of one node.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the whole path over the whole batch (256 requests of 1k-8k tokens,
+32 layers x 8 KV heads x 128, bf16, page 16: ~75k chunks of 2 MiB, ~147 GiB per direction),
+processed in waves that fit HBM (source pool + blob arena + destination pool per wave).
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_16138_b200 import synth  # noqa: E402
+
+METRIC = "codec_GBps_pack_plus_unpack"
+UNIT = "GB/s"
+WORKLOAD = ("configs[1]: Llama-3-8B KV shape, 32 layers x 8 KV heads x 128 head_dim bf16, page 16; "
+            "256 requests, lengths U[1k,8k], Zipf(1.1) tree of 64 shared prefixes; "
+            "full encode, probe, decode")
+GEOM = dict(n_layers=32, n_kv_heads=8, head_dim=128, elem_bytes=2, page_tokens=16, chunk_tokens=16)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--requests", type=int, default=256, help="requests in the batch (256 = the named workload)")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU baseline budget (0 = skip)")
+    ap.add_argument("--tuning", default="", help="name=value,... launch-shape knobs")
+    return ap.parse_args()
+
+
+# ---- workload --------------------------------------------------------------------------------
+
+def split_waves(nch: np.ndarray, n_waves: int):
+    """Contiguous groups of requests with roughly equal chunk counts."""
+    total = int(nch.sum())
+    bounds, acc, target = [0], 0, total / n_waves
+    for r, c in enumerate(nch):
+        acc += int(c)
+        if acc >= target * len(bounds) and len(bounds) < n_waves:
+            bounds.append(r + 1)
+    bounds.append(len(nch))
+    out = [(bounds[i], bounds[i + 1]) for i in range(len(bounds) - 1)]
+    return [w for w in out if w[1] > w[0]]
+
+
+def wave_batch(batch: synth.Batch, a: int, b: int) -> synth.Batch:
+    t0, t1 = int(batch.seq_off[a]), int(batch.seq_off[b])
+    return synth.Batch(batch.tokens[t0:t1], (batch.seq_off[a:b + 1] - batch.seq_off[a]).astype(np.uint64))
+
+
+def meminfo_available_bytes() -> int:
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 8 << 30
+
+
+# ---- clocks ----------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm),
+                "power_w_max": max(power), "reasons": sorted(reasons)}
+
+
+# ---- the CPU baseline (the oracle, as it stands, on a bounded sample) -------------------------
+
+def oracle_sample_pass(og, sample):
+    """One pass of the whole path on the CPU: encode, probe, decode. Returns bytes moved."""
+    import oracle
+    b, coff, pages, pool, runs, dst_pages, dst_pool = sample
+    keys, vals, blob = oracle.encode_batch(og, b.tokens, b.seq_off, None, coff, pages, pool, 0, 0)
+    hit, recs, _, _ = oracle.probe_batch(og, b.tokens, b.seq_off, coff, runs)
+    oracle.decode_batch(og, coff, hit, recs, [blob], dst_pages, dst_pool)
+    return blob.size + int(hit.sum()) * og.chunk_bytes
+
+
+def make_oracle_sample(batch, max_chunks, pool_pages_fn):
+    """The first requests of the batch up to max_chunks chunks, with a compact host pool."""
+    import oracle
+    og = oracle.Geom(**GEOM)
+    nch = synth.chunk_counts(batch.seq_off, og.chunk_tokens)
+    n_req = int(np.searchsorted(np.cumsum(nch), max_chunks, side="right"))
+    n_req = max(1, n_req)
+    b = wave_batch(batch, 0, n_req)
+    coff = synth.offsets(nch[:n_req])
+    n = int(coff[-1])
+    rng = synth.rng_for(2, 99)
+    pages = synth.random_pages(rng, n, n)
+    dst_pages = synth.random_pages(rng, n, n)
+    pool = pool_pages_fn(n, og)
+    keys, vals, _ = oracle.encode_batch(og, b.tokens, b.seq_off, None, coff, None, None, 0, 0,
+                                        with_blob=False)
+    runs = [oracle.flush(keys, vals)]
+    dst_pool = np.zeros_like(pool)
+    return og, (b, coff, pages, pool, runs, dst_pages, dst_pool), n_req, n
+
+
+def time_oracle(og, sample, budget_s):
+    t0 = time.perf_counter()
+    moved, passes = 0, 0
+    while True:
+        moved += oracle_sample_pass(og, sample)
+        passes += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or passes >= 50:
+            return moved / el / 1e9, passes, el
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on the host cores; one step = one pass
+    over a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.llama_requests(n_req=args.requests)
+    avail = meminfo_available_bytes()
+    cb = 2 * GEOM["n_layers"] * GEOM["page_tokens"] * GEOM["n_kv_heads"] * GEOM["head_dim"] * GEOM["elem_bytes"]
+    max_chunks = int(min(1024, max(8, avail * 0.4 / (3 * cb))))
+
+    def host_pool(n, og):
+        rng = synth.rng_for(2, 7)
+        return synth.random_pool_bytes(rng, 2 * og.n_layers, n, og.page_bytes)
+
+    og, sample, n_req, n = make_oracle_sample(w.batch, max_chunks, host_pool)
+    for _ in range(args.warmup):
+        oracle_sample_pass(og, sample)
+    t0 = time.perf_counter()
+    moved = 0
+    for _ in range(args.steps):
+        moved += oracle_sample_pass(og, sample)
+    el = time.perf_counter() - t0
+    val = moved / el / 1e9
+    desc = f"first {n_req} requests = {n} chunks ({n * cb / 2**30:.2f} GiB per direction) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": el / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---- our arm ---------------------------------------------------------------------------------
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2511_16138_b200 import hostindex, lsmkv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    g = lsmkv.Geom(**GEOM)
+    cb, pb, L2 = g.chunk_bytes, g.page_bytes, 2 * g.n_layers
+    # every rank gets its own batch of the same shape (weak scaling, no data-path collective)
+    w = synth.llama_requests(n_req=args.requests, config_id=2 + 100 * rank)
+    batch = w.batch
+    nch = synth.chunk_counts(batch.seq_off, g.chunk_tokens)
+    total_chunks = int(nch.sum())
+    payload = total_chunks * cb
+
+    free, _ = torch.cuda.mem_get_info()
+    budget = int(free * 0.80)
+    n_waves = 1
+    while 3 * -(-total_chunks // n_waves) * cb > budget:
+        n_waves += 1
+    waves = split_waves(nch, n_waves)
+    cap = max(int(nch[a:b].sum()) for a, b in waves)
+
+    ctx = lsmkv.Context(g, local_rank)
+    for kv in filter(None, args.tuning.split(",")):
+        k, v = kv.split("=")
+        ctx.set_tuning(k, int(v))
+    ctx.reserve(max(b - a for a, b in waves), cap)
+
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(synth.SEED0 + 2 + rank)
+
+    def new_pool(fill: bool):
+        bufs = []
+        for _ in range(L2):
+            if fill:
+                t = torch.randn(cap * pb // 2, dtype=torch.bfloat16, device=dev, generator=gen)
+                bufs.append(t.view(torch.uint8).view(cap, pb))
+            else:
+                bufs.append(torch.zeros((cap, pb), dtype=torch.uint8, device=dev))
+        return bufs, lsmkv.pool_table(bufs)
+
+    src_bufs, src_pool = new_pool(True)
+    dst_bufs, dst_pool = new_pool(False)
+    arena = torch.empty(cap * cb, dtype=torch.uint8, device=dev)
+
+    def up(a: np.ndarray):
+        b = np.ascontiguousarray(a).view(np.uint8).reshape(-1)
+        t = torch.empty(max(16, b.size), dtype=torch.uint8, device=dev)
+        t[:b.size] = torch.from_numpy(b.copy())
+        return t
+
+    rng = synth.rng_for(2, 1000 + rank)
+    W = []
+    for (a, b) in waves:
+        wb = wave_batch(batch, a, b)
+        coff = synth.offsets(nch[a:b])
+        n = int(coff[-1])
+        host = dict(tokens=wb.tokens, seq_off=wb.seq_off, coff=coff,
+                    src_pages=synth.random_pages(rng, cap, n),
+                    dst_pages=synth.random_pages(rng, cap, n))
+        d = dict(n_req=b - a, n=n, host=host, nch=nch[a:b],
+                 tokens=up(wb.tokens), seq_off=up(wb.seq_off), coff=up(coff),
+                 src_pages=up(host["src_pages"]), dst_pages=up(host["dst_pages"]),
+                 keys=torch.empty(n * 32, dtype=torch.uint8, device=dev),
+                 vals=torch.empty(n * 16, dtype=torch.uint8, device=dev),
+                 hit=torch.zeros(b - a, dtype=torch.int32, device=dev),
+                 recs=torch.empty(n * 16, dtype=torch.uint8, device=dev))
+        W.append(d)
+
+    def encode(d):
+        ctx.encode_batch(d["n_req"], d["tokens"], d["seq_off"], None, d["coff"], d["n"],
+                         d["src_pages"], src_pool, 0, 0, d["keys"], d["vals"], arena, d["n"] * cb,
+                         stream=stream)
+
+    def probe(d):
+        ctx.probe_batch(d["n_req"], d["tokens"], d["seq_off"], d["coff"], d["n"], d["runs"],
+                        d["hit"], d["recs"], None, stream=stream)
+
+    def decode(d):
+        ctx.decode_batch(d["n_req"], d["coff"], d["n"], d["hit"], d["recs"],
+                         [(arena, d["n"] * cb)], d["dst_pages"], dst_pool, stream=stream)
+
+    # ---- untimed preparation: the index (one sorted run per wave) from the encoder's own keys
+    for d in W:
+        encode(d)
+        torch.cuda.synchronize()
+        keys = d["keys"].cpu().numpy().view(np.uint64).reshape(-1, 4)
+        vals = d["vals"].cpu().numpy().reshape(-1, 16)
+        rk, rv = hostindex.flush(keys, vals)
+        d["run_t"] = (up(rk), up(rv))
+        d["runs"] = [(d["run_t"][0], d["run_t"][1], len(rk))]
+        probe(d)
+        decode(d)
+        torch.cuda.synchronize()
+        # self-check of this wave (device side): every chunk is a hit; sampled pages restored
+        assert np.array_equal(d["hit"].cpu().numpy(), d["nch"].astype(np.int32)), "probe missed"
+    st = ctx.last_status()
+    assert st["flags"] == 0, st
+
+    def step():
+        for d in W:
+            encode(d)
+            probe(d)
+            decode(d)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    ctx.last_status()
+    ctx.profile_enable(True)
+    ctx.profile_read()
+    launches0 = ctx.launch_count()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_total = e0.elapsed_time(e1)
+    launches = ctx.launch_count() - launches0
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    status = ctx.last_status()
+    assert status["flags"] == 0, status
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    moved_step = 2 * payload                      # bytes packed + bytes unpacked, per rank
+    value = world * moved_step / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, host buffers out, through the same C-ABI calls
+    e2e = None
+    if args.e2e_steps > 0:
+        e2e = run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream,
+                      barrier, world)
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, single GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and args.cpu_seconds > 0:
+        def gpu_pages(n, og):
+            idx = torch.arange(n, device=dev)
+            return torch.stack([b_[idx] for b_ in src_bufs]).cpu().numpy()
+        max_chunks = int(min(1024, max(8, meminfo_available_bytes() * 0.4 / (3 * cb))))
+        og, sample, s_req, s_n = make_oracle_sample(batch, max_chunks, gpu_pages)
+        v, passes, el = time_oracle(og, sample, args.cpu_seconds)
+        cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {s_req} requests = {s_n} chunks ({s_n * cb / 2**30:.2f} GiB per "
+                         f"direction), {passes} passes in {el:.1f} s; host cpus={os.cpu_count()}"}
+
+    if rank == 0:
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            with open(peaks_path) as f:
+                peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        else:
+            peak, peak_src = 6650.0, "fallback"
+        copy_ms = prof["pack"][0] + prof["unpack"][0]
+        copy_launches = prof["pack"][1] + prof["unpack"][1]
+        algo_bytes_per_launch = 2.0 * (2 * payload * args.steps) / max(1, copy_launches)
+        achieved = algo_bytes_per_launch / (copy_ms / max(1, copy_launches) * 1e-3) / 1e9
+        qchunks = total_chunks
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "requests": args.requests, "chunks": total_chunks,
+                       "payload_GiB_per_direction": payload / 2**30, "waves": len(W),
+                       "l2": "inputs larger than L2 (each wave moves >30 GiB)",
+                       "payload_dtype": "bf16 bit patterns (opaque)", "key_arithmetic": "u64",
+                       "tuning": {k: ctx.get_tuning(k) for k in
+                                  ("copy_mode", "copy_stage_bytes", "copy_stages",
+                                   "copy_ctas_per_sm", "copy_l2_hint")}},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "k_copy_slabs (pack + unpack launches)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_source": peak_src,
+                         "frac_of_8TBps_nominal": achieved / 8000.0, "traffic": None,
+                         "algorithmic_bytes_per_launch": algo_bytes_per_launch,
+                         "avg_launch_ms": copy_ms / max(1, copy_launches)},
+            "cpu_baseline": cpu,
+            "phases": {
+                "pack_GBps_payload": payload * args.steps / (prof["pack"][0] * 1e-3) / 1e9,
+                "unpack_GBps_payload": payload * args.steps / (prof["unpack"][0] * 1e-3) / 1e9,
+                "pack_hbm_frac_of_peak": 2 * payload * args.steps / (prof["pack"][0] * 1e-3) / 1e9 / peak,
+                "unpack_hbm_frac_of_peak": 2 * payload * args.steps / (prof["unpack"][0] * 1e-3) / 1e9 / peak,
+                "probe_keys_per_s": qchunks * args.steps / (prof["probe"][0] * 1e-3),
+                "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
+                "kernel_launches": {k: v[1] for k, v in prof.items()},
+                "lookups_per_step": status["lookups"] / args.steps,
+            },
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream, barrier, world):
+    """Same path with HOST buffers: per sub-batch the request descriptors go host->device, the
+    packed blobs, keys and records come back to (pinned) host memory as a tensor-log writer
+    would want them, then the blobs go host->device again and are scattered into the pool; hit
+    lengths come back to the host. The KV pool itself lives on the GPU by nature."""
+    cb = g.chunk_bytes
+    sub_cap = 2048                                   # chunks per sub-batch (4 GiB of blobs)
+    subs = []
+    for d in W:
+        nchw, a, acc = d["nch"], 0, 0
+        for r in range(len(nchw)):
+            if acc + int(nchw[r]) > sub_cap and r > a:
+                subs.append((d, a, r)); a, acc = r, 0
+            acc += int(nchw[r])
+        subs.append((d, a, len(nchw)))
+    max_n = max(int(d["nch"][a:b].sum()) for d, a, b in subs)
+    pin_blob = torch.empty(max_n * cb, dtype=torch.uint8, pin_memory=True)
+    pin_keys = torch.empty(max_n * 32, dtype=torch.uint8, pin_memory=True)
+    pin_vals = torch.empty(max_n * 16, dtype=torch.uint8, pin_memory=True)
+    pin_hit = torch.empty(4096, dtype=torch.int32, pin_memory=True)
+    prepared = []
+    for d, a, b in subs:
+        h = d["host"]
+        t0, t1 = int(h["seq_off"][a]), int(h["seq_off"][b])
+        c0, c1 = int(h["coff"][a]), int(h["coff"][b])
+        arrs = dict(tokens=h["tokens"][t0:t1], seq_off=(h["seq_off"][a:b + 1] - h["seq_off"][a]),
+                    coff=(h["coff"][a:b + 1] - h["coff"][a]), src=h["src_pages"][c0:c1],
+                    dst=h["dst_pages"][c0:c1])
+        pins = {k: torch.from_numpy(np.ascontiguousarray(v).view(np.uint8).copy()).pin_memory()
+                for k, v in arrs.items()}
+        devs = {k: torch.empty(max(16, v.numel()), dtype=torch.uint8, device=dev) for k, v in pins.items()}
+        prepared.append([d, b - a, c1 - c0, pins, devs, None])
+    # untimed: the index of each sub-batch (its records point into this sub-batch's blobs)
+    from paper_2511_16138_b200 import hostindex
+    keep = []
+    for p in prepared:
+        d, n_req, n, pins, devs, _ = p
+        for k in pins:
+            devs[k][:pins[k].numel()].copy_(pins[k])
+        ctx.encode_batch(n_req, devs["tokens"], devs["seq_off"], None, devs["coff"], n, None, None,
+                         0, 0, d["keys"], d["vals"], None, 0, stream=stream)
+        torch.cuda.synchronize()
+        rk, rv = hostindex.flush(d["keys"][:n * 32].cpu().numpy().view(np.uint64).reshape(-1, 4),
+                                 d["vals"][:n * 16].cpu().numpy().reshape(-1, 16))
+        tk = torch.from_numpy(rk.view(np.uint8).reshape(-1).copy()).to(dev)
+        tv = torch.from_numpy(rv.reshape(-1).copy()).to(dev)
+        keep.append((tk, tv))
+        p[5] = [(tk, tv, len(rk))]
+    h2d = d2h = 0
+    moved = 0
+
+    def one_step():
+        nonlocal h2d, d2h, moved
+        for d, n_req, n, pins, devs, runs in prepared:
+            for k in pins:
+                devs[k][:pins[k].numel()].copy_(pins[k], non_blocking=True)
+                h2d += pins[k].numel()
+            ctx.encode_batch(n_req, devs["tokens"], devs["seq_off"], None, devs["coff"], n,
+                             devs["src"], src_pool, 0, 0, d["keys"], d["vals"], arena, n * cb,
+                             stream=stream)
+            pin_blob[:n * cb].copy_(arena[:n * cb], non_blocking=True)
+            pin_keys[:n * 32].copy_(d["keys"][:n * 32], non_blocking=True)
+            pin_vals[:n * 16].copy_(d["vals"][:n * 16], non_blocking=True)
+            d2h += n * (cb + 48)
+            ctx.probe_batch(n_req, devs["tokens"], devs["seq_off"], devs["coff"], n, runs,
+                            d["hit"], d["recs"], None, stream=stream)
+            pin_hit[:n_req].copy_(d["hit"][:n_req], non_blocking=True)
+            d2h += n_req * 4
+            arena[:n * cb].copy_(pin_blob[:n * cb], non_blocking=True)
+            h2d += n * cb
+            ctx.decode_batch(n_req, devs["coff"], n, d["hit"], d["recs"], [(arena, n * cb)],
+                             devs["dst"], dst_pool, stream=stream)
+            moved += 2 * n * cb
+
+    one_step()                                      # warm-up (also faults in the pinned pages)
+    barrier()
+    st = ctx.last_status()
+    assert st["flags"] == 0 and st["chunks_decoded"] == sum(p[2] for p in prepared), st
+    h2d = d2h = moved = 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(max(1, args.e2e_steps)):
+        one_step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    steps = max(1, args.e2e_steps)
+    ctx.last_status()
+    return {"value": world * moved / (ms * 1e-3) / 1e9, "unit": UNIT,
+            "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
+            "steps": steps, "ms_per_step": ms / steps,
+            "note": "blobs, keys and records copied to pinned host memory and blobs copied back "
+                    "before the scatter; PCIe-bound"}
+
+
+if __name__ == "__main__":
+    main()

@@ -176,6 +176,26 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
 /* Synchronise `stream`, copy the device status block to *out [host] and clear it. */
 int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out);
 
+/*
+ * Optional per-kernel timing. While enabled, every kernel launch of this context is bracketed
+ * by CUDA events on the launching stream (no synchronisation). lsmkv_profile_read() waits for
+ * the recorded events, returns the summed device time and launch count per kernel class since
+ * the previous read, and clears them. Class LSMKV_K_PLAN covers the two small kernels that
+ * turn hit lengths into the list of chunks to copy.
+ */
+#define LSMKV_K_KEYS 0
+#define LSMKV_K_PACK 1
+#define LSMKV_K_PROBE 2
+#define LSMKV_K_PLAN 3
+#define LSMKV_K_UNPACK 4
+#define LSMKV_K_CLASSES 8
+typedef struct {
+    double ms[LSMKV_K_CLASSES];
+    uint64_t launches[LSMKV_K_CLASSES];
+} lsmkv_profile_t;
+int lsmkv_profile_enable(lsmkv_ctx *ctx, int on);
+int lsmkv_profile_read(lsmkv_ctx *ctx, lsmkv_profile_t *out /* [host] */);
+
 /* The cudaError_t behind the last LSMKV_ECUDA of this context (0 if none). */
 int lsmkv_last_cuda_error(const lsmkv_ctx *ctx);
 

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "lsmkv.h"
 #include "lsmkv_common.cuh"
@@ -30,6 +31,11 @@ struct lsmkv_ctx {
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm;
+    // optional per-kernel timing with CUDA events on the launching stream
+    bool profiling;
+    struct Timed { cudaEvent_t a, b; int cls; };
+    std::vector<Timed> pending;
+    std::vector<cudaEvent_t> free_events;
 };
 
 namespace {
@@ -90,6 +96,36 @@ void fill_key_consts(KeyConsts &kc, uint32_t C)
     }
 }
 
+// Brackets one kernel launch with events when profiling is on.
+struct LaunchTimer {
+    lsmkv_ctx *ctx;
+    cudaStream_t s;
+    lsmkv_ctx::Timed t{};
+    bool on;
+    static cudaEvent_t get(lsmkv_ctx *c)
+    {
+        cudaEvent_t e = nullptr;
+        if (!c->free_events.empty()) { e = c->free_events.back(); c->free_events.pop_back(); }
+        else if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); e = nullptr; }
+        return e;
+    }
+    LaunchTimer(lsmkv_ctx *c, cudaStream_t st, int cls) : ctx(c), s(st), on(c->profiling)
+    {
+        if (!on) return;
+        t.a = get(c);
+        t.b = get(c);
+        t.cls = cls;
+        if (!t.a || !t.b) { on = false; return; }
+        cudaEventRecord(t.a, s);
+    }
+    ~LaunchTimer()
+    {
+        if (!on) return;
+        cudaEventRecord(t.b, s);
+        ctx->pending.push_back(t);
+    }
+};
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int ensure_workspace(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
@@ -117,6 +153,7 @@ uint32_t *ws_plan(lsmkv_ctx *ctx)
 int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &ar,
                 uint64_t max_items)
 {
+    LaunchTimer timer(ctx, s, job.unpack ? LSMKV_K_UNPACK : LSMKV_K_PACK);
     const uint64_t slabs = 2ull * ctx->geom.n_layers;
     if (ctx->copy_mode == 1) {
         job.piece_bytes = (uint32_t)ctx->page_bytes;
@@ -181,9 +218,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
         return LSMKV_EINVAL;
     const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
     if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
-    lsmkv_ctx *ctx = new (std::nothrow) lsmkv_ctx();
+    lsmkv_ctx *ctx = new (std::nothrow) lsmkv_ctx();   // value-initialised: all fields zero
     if (!ctx) return LSMKV_ENOMEM;
-    std::memset(ctx, 0, sizeof(*ctx));
     ctx->geom = *g;
     ctx->device = device;
     ctx->page_bytes = pb;
@@ -231,6 +267,8 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     cudaDeviceSynchronize();
     if (ctx->d_ws) cudaFree(ctx->d_ws);
     if (ctx->d_status) cudaFree(ctx->d_status);
+    for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+    for (auto e : ctx->free_events) cudaEventDestroy(e);
     cudaGetLastError();
     delete ctx;
     return LSMKV_OK;
@@ -265,11 +303,14 @@ int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint3
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    const unsigned grid = warp_grid(ctx, n_req, 128, 16);
-    k_encode_keys<<<grid, 128, 0, s>>>(ctx->kc, ctx->geom.chunk_tokens, ctx->geom.ns, n_req, tokens,
-                                       seq_off, start_chunk, chunk_off, n_chunks, file_id,
-                                       base_offset, ctx->chunk_bytes, keys_out, vals_out,
-                                       ctx->d_status);
+    {
+        LaunchTimer timer(ctx, s, LSMKV_K_KEYS);
+        const unsigned grid = warp_grid(ctx, n_req, 128, 16);
+        k_encode_keys<<<grid, 128, 0, s>>>(ctx->kc, ctx->geom.chunk_tokens, ctx->geom.ns, n_req,
+                                           tokens, seq_off, start_chunk, chunk_off, n_chunks,
+                                           file_id, base_offset, ctx->chunk_bytes, keys_out,
+                                           vals_out, ctx->d_status);
+    }
     ++ctx->launches;
     CU(ctx, cudaGetLastError());
     if (!with_blob) return LSMKV_OK;
@@ -313,11 +354,15 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const unsigned threads = (unsigned)ctx->probe_warps_per_cta * 32u;
-    const unsigned grid = warp_grid(ctx, n_query, threads, 2048 / threads);
-    k_probe<<<grid, threads, 0, s>>>(ctx->kc, rt, n_runs, ctx->geom.chunk_tokens, ctx->geom.ns,
-                                     n_query, tokens, seq_off, qchunk_off, n_qchunks,
-                                     hit_chunks_out, recs_out, keys_out, ctx->d_status);
+    {
+        LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
+        const unsigned threads = (unsigned)ctx->probe_warps_per_cta * 32u;
+        const unsigned grid = warp_grid(ctx, n_query, threads, 2048 / threads);
+        k_probe<<<grid, threads, 0, s>>>(ctx->kc, rt, n_runs, ctx->geom.chunk_tokens,
+                                         ctx->geom.ns, n_query, tokens, seq_off, qchunk_off,
+                                         n_qchunks, hit_chunks_out, recs_out, keys_out,
+                                         ctx->d_status);
+    }
     ++ctx->launches;
     CU(ctx, cudaGetLastError());
     return LSMKV_OK;
@@ -351,14 +396,18 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
 
     uint64_t *hit_off = ws_hit_off(ctx);
     uint32_t *plan = ws_plan(ctx);
-    k_plan_scan<<<1, 1024, 0, s>>>(n_query, qchunk_off, n_qchunks, hit_chunks, hit_off,
-                                   ctx->d_status);
-    ++ctx->launches;
-    CU(ctx, cudaGetLastError());
-    k_plan_fill<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
-        n_query, qchunk_off, hit_off, recs, ar, n_arenas, ctx->chunk_bytes, plan, ctx->d_status);
-    ++ctx->launches;
-    CU(ctx, cudaGetLastError());
+    {
+        LaunchTimer timer(ctx, s, LSMKV_K_PLAN);
+        k_plan_scan<<<1, 1024, 0, s>>>(n_query, qchunk_off, n_qchunks, hit_chunks, hit_off,
+                                       ctx->d_status);
+        ++ctx->launches;
+        CU(ctx, cudaGetLastError());
+        k_plan_fill<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
+            n_query, qchunk_off, hit_off, recs, ar, n_arenas, ctx->chunk_bytes, plan,
+            ctx->d_status);
+        ++ctx->launches;
+        CU(ctx, cudaGetLastError());
+    }
 
     CopyJob job;
     std::memset(&job, 0, sizeof(job));
@@ -388,6 +437,36 @@ int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out)
     CU(ctx, cudaMemcpyAsync(ctx->d_status, &z, sizeof(z), cudaMemcpyHostToDevice, s));
     CU(ctx, cudaStreamSynchronize(s));
     return LSMKV_OK;
+}
+
+int lsmkv_profile_enable(lsmkv_ctx *ctx, int on)
+{
+    if (!ctx) return LSMKV_EINVAL;
+    ctx->profiling = on != 0;
+    return LSMKV_OK;
+}
+
+int lsmkv_profile_read(lsmkv_ctx *ctx, lsmkv_profile_t *out)
+{
+    if (!ctx || !out) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    std::memset(out, 0, sizeof(*out));
+    int rc = LSMKV_OK;
+    for (auto &t : ctx->pending) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(t.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.a, t.b);
+        if (e == cudaSuccess) {
+            out->ms[t.cls] += ms;
+            out->launches[t.cls] += 1;
+        } else {
+            rc = cuda_fail(ctx, e);
+        }
+        ctx->free_events.push_back(t.a);
+        ctx->free_events.push_back(t.b);
+    }
+    ctx->pending.clear();
+    return rc;
 }
 
 int lsmkv_last_cuda_error(const lsmkv_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }

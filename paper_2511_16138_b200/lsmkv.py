@@ -22,8 +22,10 @@ EXPORTS = (
     "lsmkv_create", "lsmkv_destroy", "lsmkv_reserve", "lsmkv_encode_batch",
     "lsmkv_probe_batch", "lsmkv_decode_batch", "lsmkv_last_status", "lsmkv_last_cuda_error",
     "lsmkv_launch_count", "lsmkv_set_tuning", "lsmkv_get_tuning", "lsmkv_strerror",
-    "lsmkv_format_version",
+    "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
 )
+K_KEYS, K_PACK, K_PROBE, K_PLAN, K_UNPACK, K_CLASSES = 0, 1, 2, 3, 4, 8
+K_NAMES = ("keys", "pack", "probe", "plan", "unpack")
 
 
 class LsmkvError(RuntimeError):
@@ -54,6 +56,10 @@ class StatusStruct(C.Structure):
                 ("chunks_encoded", C.c_uint64), ("lookups", C.c_uint64),
                 ("chunks_hit", C.c_uint64), ("empty_probes", C.c_uint64),
                 ("chunks_decoded", C.c_uint64)]
+
+
+class ProfileStruct(C.Structure):
+    _fields_ = [("ms", C.c_double * 8), ("launches", C.c_uint64 * 8)]
 
 
 @dataclass(frozen=True)
@@ -122,6 +128,10 @@ def lib() -> C.CDLL:
     L.lsmkv_strerror.argtypes = [C.c_int]
     L.lsmkv_format_version.restype = C.c_int
     L.lsmkv_format_version.argtypes = []
+    L.lsmkv_profile_enable.restype = C.c_int
+    L.lsmkv_profile_enable.argtypes = [vp, C.c_int]
+    L.lsmkv_profile_read.restype = C.c_int
+    L.lsmkv_profile_read.argtypes = [vp, C.POINTER(ProfileStruct)]
     _lib = L
     return L
 
@@ -236,6 +246,17 @@ def lsmkv_get_tuning(ctx, name: str) -> int:
     return int(lib().lsmkv_get_tuning(ctx, name.encode()))
 
 
+def lsmkv_profile_enable(ctx, on: bool) -> None:
+    _check(ctx, lib().lsmkv_profile_enable(ctx, int(on)), "lsmkv_profile_enable")
+
+
+def lsmkv_profile_read(ctx) -> dict:
+    """{kernel class name: (device ms, launches)} since the previous read."""
+    p = ProfileStruct()
+    _check(ctx, lib().lsmkv_profile_read(ctx, C.byref(p)), "lsmkv_profile_read")
+    return {n: (p.ms[i], int(p.launches[i])) for i, n in enumerate(K_NAMES)}
+
+
 def lsmkv_format_version() -> int:
     return int(lib().lsmkv_format_version())
 
@@ -289,6 +310,12 @@ class Context:
 
     def last_status(self, stream=None) -> dict:
         return lsmkv_last_status(self.handle, stream)
+
+    def profile_enable(self, on=True):
+        lsmkv_profile_enable(self.handle, on)
+
+    def profile_read(self) -> dict:
+        return lsmkv_profile_read(self.handle)
 
     def launch_count(self) -> int:
         return lsmkv_launch_count(self.handle)
