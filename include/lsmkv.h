@@ -54,6 +54,7 @@ extern "C" {
 #define LSMKV_ECAPACITY (-2)  /* an output buffer is too small */
 #define LSMKV_ECUDA (-3)      /* a CUDA call failed; see lsmkv_last_cuda_error() */
 #define LSMKV_ENOMEM (-4)     /* host or device allocation failed */
+#define LSMKV_ETOOBIG (-5)    /* lsmkv_decode_batch_static(): batch larger than the built-in scratch */
 
 /* bits of lsmkv_status_t.flags */
 #define LSMKV_ST_BAD_PAGE 0x1u     /* a page id >= num_pages (item skipped) */
@@ -172,6 +173,44 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
                        const void *const *arenas, const uint64_t *arena_bytes,
                        uint32_t n_arenas, const uint32_t *dst_page_table,
                        const lsmkv_pool_t *pool);
+
+/*
+ * Allocation-free decode (an addition of this library; the paper has no counterpart).
+ *
+ * Same result as lsmkv_decode_batch(), for callers that are not allowed to allocate device
+ * memory at all -- typically a plugin inside a serving process whose engine has claimed the
+ * whole of HBM for its own pools at start-up and forbids driver allocations afterwards, where
+ * a cudaMalloc can fail outright or stall every stream of the process while it runs. Such a
+ * caller cannot even create an lsmkv_ctx (lsmkv_create allocates), so this call takes the
+ * geometry and the device instead of a context and makes no cudaMalloc, cudaFree or other
+ * allocating call.
+ *
+ * The scratch the decode needs (prefix sums of the hit lengths, the list of chunks to copy, a
+ * status block) lives in a fixed array inside the library image, about 1.03 MiB per GPU that
+ * loads the library, held until the process exits. Consequences:
+ *   - limits: n_query <= LSMKV_STATIC_MAX_QUERIES and n_qchunks <= LSMKV_STATIC_MAX_CHUNKS;
+ *     anything larger returns LSMKV_ETOOBIG and enqueues nothing (split the batch);
+ *   - every call on a device uses the same array. The call resets what has to start from zero
+ *     (the status block); the rest is rewritten before it is read, so stale contents of an
+ *     earlier call never show. Two calls that overlap on the GPU (different streams without an
+ *     ordering between them) race on the array and give undefined results: serialise them;
+ *   - the first call on each device looks up the device address of the array (one-time
+ *     set-up, done with that device current). Make that first call before any stream capture
+ *     is started.
+ * Arguments as for lsmkv_decode_batch(), plus
+ *   geom, device   what lsmkv_create() would have been given
+ *   status_out     [dev] optional: receives the status block of this call (flags, first_bad,
+ *                  chunks_decoded) at the end of the enqueued work
+ * Launch shape is fixed (bulk-async copies, 32 KiB pieces); tuning knobs do not apply.
+ */
+#define LSMKV_STATIC_MAX_QUERIES 4096u
+#define LSMKV_STATIC_MAX_CHUNKS 262144u
+int lsmkv_decode_batch_static(const lsmkv_geom_t *geom, int device, void *stream,
+                              uint32_t n_query, const uint64_t *qchunk_off, uint64_t n_qchunks,
+                              const uint32_t *hit_chunks, const lsmkv_val_t *recs,
+                              const void *const *arenas, const uint64_t *arena_bytes,
+                              uint32_t n_arenas, const uint32_t *dst_page_table,
+                              const lsmkv_pool_t *pool, lsmkv_status_t *status_out);
 
 /* Synchronise `stream`, copy the device status block to *out [host] and clear it. */
 int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out);

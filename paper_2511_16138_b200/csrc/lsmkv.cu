@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -516,6 +517,7 @@ const char *lsmkv_strerror(int code)
     case LSMKV_ECAPACITY: return "output buffer too small";
     case LSMKV_ECUDA: return "CUDA error";
     case LSMKV_ENOMEM: return "out of memory";
+    case LSMKV_ETOOBIG: return "batch exceeds the built-in scratch of the allocation-free entry point";
     default: return "unknown error";
     }
 }
@@ -523,3 +525,158 @@ const char *lsmkv_strerror(int code)
 int lsmkv_format_version(void) { return LSMKV_FORMAT_VERSION; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free decode.
+//
+// lsmkv_decode_batch() needs a little global memory of its own: the exclusive prefix sums of the
+// hit lengths, the compact list of chunks to copy, and a status block. The regular entry point
+// keeps them in a cudaMalloc'ed per-context workspace. The variant below keeps them in a
+// fixed-size array that is part of the library image, so it runs without a context and without
+// any allocation. Layout of the array: [status block | hit_off u64[kStaticMaxQueries + 2] |
+// plan u32[kStaticMaxChunks]].
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint64_t kStaticMaxQueries = LSMKV_STATIC_MAX_QUERIES;
+constexpr uint64_t kStaticMaxChunks = LSMKV_STATIC_MAX_CHUNKS;
+constexpr size_t kStaticStatusBytes = 256;
+constexpr size_t kStaticHitOffBytes = (kStaticMaxQueries + 2) * sizeof(uint64_t);
+constexpr size_t kStaticBytes =
+    kStaticStatusBytes + kStaticHitOffBytes + kStaticMaxChunks * sizeof(uint32_t);
+
+// Lives in every GPU context that loads this library, until the process exits (~1.03 MiB).
+// NOTE: in host code `g_static_scratch` is only a handle for cudaGetSymbolAddress(); it is not
+// a device address and must never be handed to a kernel directly.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+// Device code may name the array directly: reset the status block at the start of a call
+// (everything else in the array is fully rewritten by the plan kernels before it is read).
+__global__ void k_static_reset()
+{
+    DevStatus *st = reinterpret_cast<DevStatus *>(g_static_scratch);
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        st->flags = 0;
+        st->reserved = 0;
+        st->first_bad = ~0ull;
+        st->chunks_encoded = st->lookups = st->chunks_hit = st->empty_probes = 0;
+        st->chunks_decoded = 0;
+    }
+}
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticDev {
+    bool ready;
+    unsigned char *scratch;   // device address of g_static_scratch on this device
+    int sm_count;
+    int max_smem_optin;
+};
+StaticDev g_static_dev[kStaticMaxDevices];
+std::mutex g_static_mu;
+
+// Once per device, with that device current: resolve the device address of the scratch array.
+int static_setup(int device, StaticDev **out)
+{
+    if (device < 0 || device >= kStaticMaxDevices) return LSMKV_EINVAL;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticDev &d = g_static_dev[device];
+    if (!d.ready) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        if (e != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return LSMKV_ECUDA;
+        }
+        d.scratch = static_cast<unsigned char *>(ptr);
+        d.ready = true;
+    }
+    *out = &d;
+    return LSMKV_OK;
+}
+
+}  // namespace
+
+extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void *stream,
+                                         uint32_t n_query, const uint64_t *qchunk_off,
+                                         uint64_t n_qchunks, const uint32_t *hit_chunks,
+                                         const lsmkv_val_t *recs, const void *const *arenas,
+                                         const uint64_t *arena_bytes, uint32_t n_arenas,
+                                         const uint32_t *dst_page_table,
+                                         const lsmkv_pool_t *pool, lsmkv_status_t *status_out)
+{
+    if (!g || !g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes ||
+        !g->page_tokens || g->chunk_tokens != g->page_tokens || g->flags != 0)
+        return LSMKV_EINVAL;
+    const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
+    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
+    const uint64_t cb = 2ull * g->n_layers * pb;
+    if (n_query > kStaticMaxQueries || n_qchunks > kStaticMaxChunks) return LSMKV_ETOOBIG;
+    if (!qchunk_off || !hit_chunks || !recs || !dst_page_table || !pool || !pool->kv_ptrs)
+        return LSMKV_EINVAL;
+    if (n_arenas == 0 || n_arenas > (uint32_t)kMaxArenas || !arenas || !arena_bytes ||
+        !aligned16(recs))
+        return LSMKV_EINVAL;
+    ArenaTable ar;
+    std::memset(&ar, 0, sizeof(ar));
+    for (uint32_t a = 0; a < n_arenas; ++a) {
+        if (arena_bytes[a] && (!arenas[a] || !aligned16(arenas[a]))) return LSMKV_EINVAL;
+        ar.base[a] = static_cast<const unsigned char *>(arenas[a]);
+        ar.bytes[a] = arena_bytes[a];
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return LSMKV_ECUDA;
+    StaticDev *sd = nullptr;
+    int rc = static_setup(device, &sd);
+    if (rc != LSMKV_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    DevStatus *st = reinterpret_cast<DevStatus *>(sd->scratch);
+    uint64_t *hit_off = reinterpret_cast<uint64_t *>(sd->scratch + kStaticStatusBytes);
+    uint32_t *plan = reinterpret_cast<uint32_t *>(sd->scratch + kStaticStatusBytes + kStaticHitOffBytes);
+
+    k_static_reset<<<1, 32, 0, s>>>();
+    if (n_query && n_qchunks) {
+        k_plan_scan<<<1, 1024, 0, s>>>(n_query, qchunk_off, n_qchunks, hit_chunks, hit_off, st);
+        uint64_t fill_grid = ((uint64_t)n_query + 7) / 8;
+        const uint64_t fill_cap = (uint64_t)sd->sm_count * 8;
+        if (fill_grid > fill_cap) fill_grid = fill_cap;
+        k_plan_fill<<<(unsigned)fill_grid, 256, 0, s>>>(n_query, qchunk_off, hit_off, recs, ar,
+                                                        n_arenas, cb, plan, st);
+        CopyJob job;
+        std::memset(&job, 0, sizeof(job));
+        job.unpack = 1;
+        job.n_layers = g->n_layers;
+        job.page_bytes = (uint32_t)pb;
+        job.num_pages = pool->num_pages;
+        job.kv_ptrs = pool->kv_ptrs;
+        job.page_table = dst_page_table;
+        job.n_items_dev = hit_off + n_query;
+        job.plan = plan;
+        job.recs = recs;
+        job.st = st;
+        const uint64_t piece = pb < 32768 ? pb : 32768;
+        job.piece_bytes = (uint32_t)piece;
+        job.pieces_per_slab = (uint32_t)((pb + piece - 1) / piece);
+        const uint64_t stride = (piece + 127) & ~127ull;
+        int stages = 6;
+        while (stages > 1 && (size_t)stages * stride + (size_t)stages * 8 + 1024 > (size_t)sd->max_smem_optin)
+            --stages;
+        const size_t smem = (size_t)stages * stride + (size_t)stages * 8;
+        const uint64_t pieces = n_qchunks * 2ull * g->n_layers * job.pieces_per_slab;
+        uint64_t grid = (uint64_t)sd->sm_count;
+        const uint64_t need = (pieces + stages - 1) / stages;
+        if (grid > need) grid = need;
+        cudaError_t e = cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) { cudaGetLastError(); return LSMKV_ECUDA; }
+        k_copy_slabs_bulk<false><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
+    }
+    if (status_out) {
+        cudaError_t e = cudaMemcpyAsync(status_out, st, sizeof(DevStatus), cudaMemcpyDeviceToDevice, s);
+        if (e != cudaSuccess) { cudaGetLastError(); return LSMKV_ECUDA; }
+    }
+    if (cudaGetLastError() != cudaSuccess) return LSMKV_ECUDA;
+    return LSMKV_OK;
+}

@@ -23,7 +23,10 @@ EXPORTS = (
     "lsmkv_probe_batch", "lsmkv_decode_batch", "lsmkv_last_status", "lsmkv_last_cuda_error",
     "lsmkv_launch_count", "lsmkv_set_tuning", "lsmkv_get_tuning", "lsmkv_strerror",
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
+    "lsmkv_decode_batch_static",
 )
+ETOOBIG = -5
+STATIC_MAX_QUERIES, STATIC_MAX_CHUNKS = 4096, 262144
 K_KEYS, K_PACK, K_PROBE, K_PLAN, K_UNPACK, K_CLASSES = 0, 1, 2, 3, 4, 8
 K_NAMES = ("keys", "pack", "probe", "plan", "unpack")
 
@@ -114,6 +117,10 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch.restype = C.c_int
     L.lsmkv_decode_batch.argtypes = [vp, vp, u32, vp, u64, vp, vp, C.POINTER(vp),
                                      C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
+    L.lsmkv_decode_batch_static.restype = C.c_int
+    L.lsmkv_decode_batch_static.argtypes = [C.POINTER(GeomStruct), C.c_int, vp, u32, vp, u64, vp,
+                                            vp, C.POINTER(vp), C.POINTER(u64), u32, vp,
+                                            C.POINTER(PoolStruct), vp]
     L.lsmkv_last_status.restype = C.c_int
     L.lsmkv_last_status.argtypes = [vp, vp, C.POINTER(StatusStruct)]
     L.lsmkv_last_cuda_error.restype = C.c_int
@@ -226,6 +233,26 @@ def lsmkv_decode_batch(ctx, stream, n_query, qchunk_off, n_qchunks, hit_chunks, 
                                   _ptr(hit_chunks), _ptr(recs), bases, sizes, n,
                                   _ptr(dst_page_table), C.byref(p) if p is not None else None)
     _check(ctx, rc, "lsmkv_decode_batch")
+
+
+def lsmkv_decode_batch_static(geom: Geom, device, stream, n_query, qchunk_off, n_qchunks,
+                              hit_chunks, recs, arenas, dst_page_table, pool,
+                              status_out=None) -> None:
+    """Decode without a context and without any device allocation: the scratch it needs is a
+    fixed array inside the library (see include/lsmkv.h for the limits and the sharing rules).
+    ``status_out``: optional device buffer of 56 bytes that receives this call's status block."""
+    n = len(arenas)
+    bases = (C.c_void_p * max(1, n))(*[_ptr(a) for a, _ in arenas])
+    sizes = (C.c_uint64 * max(1, n))(*[b for _, b in arenas])
+    p = _pool(pool)
+    g = geom.c()
+    rc = lib().lsmkv_decode_batch_static(C.byref(g), device, _stream(stream), n_query,
+                                         _ptr(qchunk_off), n_qchunks, _ptr(hit_chunks),
+                                         _ptr(recs), bases, sizes, n, _ptr(dst_page_table),
+                                         C.byref(p) if p is not None else None,
+                                         _ptr(status_out))
+    if rc != OK:
+        raise LsmkvError(rc, "lsmkv_decode_batch_static")
 
 
 def lsmkv_last_status(ctx, stream=None) -> dict:
