@@ -159,3 +159,82 @@ def roundtrip(g: lsmkv.Geom, store, query, start_chunk=None, n_runs=1, num_pages
         assert status["chunks_hit"] == int(o_hit.sum()) * 2       # two probes
         assert status["chunks_decoded"] == int(o_hit.sum())
     return dict(hit=o_hit, n=n, status=status)
+
+
+# ---- full-size helpers: pools as one tensor per buffer, checks on sampled pieces ---------------
+
+class BigPool:
+    """2L separate device buffers [num_pages, page_bytes], optionally filled with bf16 N(0,1)."""
+
+    def __init__(self, g: lsmkv.Geom, num_pages: int, fill: bool, seed: int = 0):
+        self.g, self.num_pages = g, num_pages
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(seed)
+        self.bufs = []
+        for _ in range(2 * g.n_layers):
+            if fill:
+                t = torch.randn(num_pages * g.page_bytes // 2, dtype=torch.bfloat16, device=DEV,
+                                generator=gen)
+                self.bufs.append(t.view(torch.uint8).view(num_pages, g.page_bytes))
+            else:
+                self.bufs.append(torch.zeros((num_pages, g.page_bytes), dtype=torch.uint8,
+                                             device=DEV))
+        self.table = lsmkv.pool_table(self.bufs)
+
+    def gather(self, pages) -> np.ndarray:
+        """Host copy [2L, n, page_bytes] of the given pages."""
+        idx = torch.as_tensor(np.asarray(pages, dtype=np.int64), device=DEV)
+        return torch.stack([b[idx] for b in self.bufs]).cpu().numpy()
+
+    def zero_(self):
+        for b in self.bufs:
+            b.zero_()
+
+
+def pages_equal_on_gpu(src: BigPool, src_pages, dst: BigPool, dst_pages, slice_pages=8192) -> bool:
+    """dst page dst_pages[i] == src page src_pages[i] in every buffer (device-side compare)."""
+    sp = torch.as_tensor(np.asarray(src_pages, dtype=np.int64), device=DEV)
+    dp = torch.as_tensor(np.asarray(dst_pages, dtype=np.int64), device=DEV)
+    for sb, db in zip(src.bufs, dst.bufs):
+        for a in range(0, len(sp), slice_pages):
+            if not torch.equal(sb[sp[a:a + slice_pages]], db[dp[a:a + slice_pages]]):
+                return False
+    return True
+
+
+def untouched_pages_zero(dst: BigPool, touched_pages) -> bool:
+    mask = torch.ones(dst.num_pages, dtype=torch.bool, device=DEV)
+    if len(touched_pages):
+        mask[torch.as_tensor(np.asarray(touched_pages, dtype=np.int64), device=DEV)] = False
+    idx = torch.nonzero(mask).flatten()
+    for b in dst.bufs:
+        for a in range(0, len(idx), 8192):
+            if b[idx[a:a + 8192]].any():
+                return False
+    return True
+
+
+def oracle_blob_range(g, seq_tokens, a, b, pool: BigPool, pages_ab, file_id, rec_offset_of_a):
+    """Oracle encode of chunks [a, b) of one sequence whose pool pages are pages_ab: returns
+    (keys, vals, blob) computed on the CPU from a compact host copy of those pages."""
+    og = ogeom(g)
+    C = g.chunk_tokens
+    host_pool = pool.gather(pages_ab)
+    toks = np.ascontiguousarray(seq_tokens[:b * C])
+    return oracle.encode_batch(og, toks, np.array([0, len(toks)], np.uint64),
+                               np.array([a], np.uint32), np.array([0, b - a], np.uint64),
+                               np.arange(b - a, dtype=np.uint32), host_pool, file_id,
+                               rec_offset_of_a)
+
+
+def oracle_decode_one(g, rec, blob_bytes):
+    """Oracle decode of one record whose blob is ``blob_bytes``: compact pool [2L, 1, page_bytes]."""
+    og = ogeom(g)
+    r = np.zeros(1, dtype=VAL_DTYPE)
+    r["file_id"] = 0
+    r["offset"] = 0
+    assert int(rec["reserved"]) == 0
+    out = np.zeros((2 * g.n_layers, 1, g.page_bytes), dtype=np.uint8)
+    oracle.decode_batch(og, np.array([0, 1], np.uint64), np.array([1], np.uint32), r,
+                        [np.ascontiguousarray(blob_bytes)], np.array([0], np.uint32), out)
+    return out
