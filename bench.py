@@ -213,11 +213,9 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2511_16138_b200 import hostindex, lsmkv
+    from paper_2511_16138_b200 import hostindex, lsmkv, ranks
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = ranks.rank_env()
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -234,7 +232,7 @@ def main():
     g = lsmkv.Geom(**GEOM)
     cb, pb, L2 = g.chunk_bytes, g.page_bytes, 2 * g.n_layers
     # every rank gets its own batch of the same shape (weak scaling, no data-path collective)
-    w = synth.llama_requests(n_req=args.requests, config_id=2 + 100 * rank)
+    w = synth.llama_requests(n_req=args.requests, config_id=ranks.workload_config_id(2, rank))
     batch = w.batch
     nch = synth.chunk_counts(batch.seq_off, g.chunk_tokens)
     total_chunks = int(nch.sum())
@@ -353,13 +351,10 @@ def main():
     ctx.profile_enable(False)
     status = ctx.last_status()
     assert status["flags"] == 0, status
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = ranks.max_over_ranks(ms_total, dev)
     ms_step = ms_total / args.steps
-    moved_step = 2 * payload                      # bytes packed + bytes unpacked, per rank
-    value = world * moved_step / (ms_step * 1e-3) / 1e9
+    moved_all = ranks.sum_over_ranks(2 * payload, dev)   # bytes packed + unpacked, all ranks
+    value = ranks.whole_job_rate(moved_all, ms_step) / 1e9
 
     # ---- end to end: host buffers in, host buffers out, through the same C-ABI calls
     e2e = None
@@ -512,15 +507,12 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
         one_step()
     e1.record(stream)
     barrier()
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2511_16138_b200 import ranks
+    ms = ranks.max_over_ranks(e0.elapsed_time(e1), dev)
+    moved = ranks.sum_over_ranks(moved, dev)
     steps = max(1, args.e2e_steps)
     ctx.last_status()
-    return {"value": world * moved / (ms * 1e-3) / 1e9, "unit": UNIT,
+    return {"value": ranks.whole_job_rate(moved, ms) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
             "steps": steps, "ms_per_step": ms / steps,
             "note": "blobs, keys and records copied to pinned host memory and blobs copied back "
