@@ -248,7 +248,7 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "copy_stage_bytes"  bytes per bulk copy, multiple of 16, 16..131072 (clamped to page_bytes)
  *   "copy_stages"       bulk copies in flight per CTA, 1..32 (reduced to fit shared memory)
  *   "copy_ctas_per_sm"  1..8        "copy_l2_hint"  0/1 = evict-first L2 policy on the copies
- *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..32
+ *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..16
  */
 int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value);
 int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name);

@@ -27,6 +27,9 @@ struct lsmkv_ctx {
     // workspace: hit_off u64[ws_seq + 1] followed by plan u32[ws_chunks]
     void *d_ws;
     uint64_t ws_seq, ws_chunks;
+    // fence-pointer directory of the probe: u64[n_runs * (jcap + 1)]
+    uint64_t *d_dir;
+    uint64_t dir_cap;
     int last_cuda;
     uint64_t launches;
     // tuning
@@ -145,6 +148,20 @@ int ensure_workspace(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
     return LSMKV_OK;
 }
 
+int ensure_dir(lsmkv_ctx *ctx, uint64_t entries)
+{
+    if (entries <= ctx->dir_cap && ctx->d_dir) return LSMKV_OK;
+    void *p = nullptr;
+    cudaError_t e = cudaMalloc(&p, (size_t)entries * sizeof(uint64_t));
+    if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
+    if (ctx->d_dir) cudaFree(ctx->d_dir);   // waits for work that may still use the old one
+    ctx->d_dir = static_cast<uint64_t *>(p);
+    ctx->dir_cap = entries;
+    return LSMKV_OK;
+}
+
+constexpr uint64_t kDirMaxJ = 65536;   // chunk indices covered by the probe's directory
+
 uint64_t *ws_hit_off(lsmkv_ctx *ctx) { return static_cast<uint64_t *>(ctx->d_ws); }
 uint32_t *ws_plan(lsmkv_ctx *ctx)
 {
@@ -231,7 +248,7 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->copy_stages = 6;
     ctx->copy_ctas_per_sm = 1;
     ctx->copy_l2_hint = 0;
-    ctx->probe_warps_per_cta = 8;
+    ctx->probe_warps_per_cta = 4;
     ctx->simt_ctas_per_sm = 8;
 
     DeviceGuard guard(device);
@@ -252,7 +269,9 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
         return LSMKV_ECUDA;
     }
     int rc = ensure_workspace(ctx, 1024, 65536);
+    if (rc == LSMKV_OK) rc = ensure_dir(ctx, 2 + 8 * (kDirMaxJ + 1));
     if (rc != LSMKV_OK) {
+        if (ctx->d_ws) cudaFree(ctx->d_ws);
         cudaFree(ctx->d_status);
         delete ctx;
         return rc;
@@ -267,6 +286,7 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     DeviceGuard guard(ctx->device);
     cudaDeviceSynchronize();
     if (ctx->d_ws) cudaFree(ctx->d_ws);
+    if (ctx->d_dir) cudaFree(ctx->d_dir);
     if (ctx->d_status) cudaFree(ctx->d_status);
     for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : ctx->free_events) cudaEventDestroy(e);
@@ -279,7 +299,9 @@ int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
 {
     if (!ctx || n_chunks >= 0xFFFFFFFFull) return LSMKV_EINVAL;
     DeviceGuard guard(ctx->device);
-    return ensure_workspace(ctx, n_seq, n_chunks);
+    int rc = ensure_workspace(ctx, n_seq, n_chunks);
+    if (rc != LSMKV_OK) return rc;
+    return ensure_dir(ctx, 2 + 8 * ((n_chunks < kDirMaxJ ? n_chunks : kDirMaxJ) + 1));
 }
 
 int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint32_t *tokens,
@@ -355,16 +377,38 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint32_t jcap = (uint32_t)(n_qchunks < kDirMaxJ ? n_qchunks : kDirMaxJ);
+    // d_dir: [0] = the probe's work counter, [2..] = the directory
+    {
+        int rc = ensure_dir(ctx, 2 + (uint64_t)n_runs * ((uint64_t)jcap + 1));
+        if (rc != LSMKV_OK) return rc;
+    }
+    unsigned long long *next_query = reinterpret_cast<unsigned long long *>(ctx->d_dir);
+    uint64_t *dir = ctx->d_dir + 2;
     {
         LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
-        const unsigned threads = (unsigned)ctx->probe_warps_per_cta * 32u;
-        const unsigned grid = warp_grid(ctx, n_query, threads, 2048 / threads);
-        k_probe<<<grid, threads, 0, s>>>(ctx->kc, rt, n_runs, ctx->geom.chunk_tokens,
-                                         ctx->geom.ns, n_query, tokens, seq_off, qchunk_off,
-                                         n_qchunks, hit_chunks_out, recs_out, keys_out,
-                                         ctx->d_status);
+        {
+            const uint64_t entries = (uint64_t)n_runs * ((uint64_t)jcap + 1);
+            uint64_t dgrid = (entries + 255) / 256;
+            const uint64_t dcap = (uint64_t)ctx->sm_count * 8;
+            if (dgrid > dcap) dgrid = dcap;
+            if (dgrid == 0) dgrid = 1;
+            k_run_dir<<<(unsigned)dgrid, 256, 0, s>>>(rt, n_runs, ctx->geom.ns, jcap, dir,
+                                                      next_query);
+            ++ctx->launches;
+        }
+        const unsigned warps = (unsigned)ctx->probe_warps_per_cta;
+        const unsigned threads = warps * 32u;
+        uint64_t grid = n_query;
+        const uint64_t cap = (uint64_t)ctx->sm_count * (2048u / threads);
+        if (grid > cap) grid = cap;
+        k_probe<<<(unsigned)grid, threads, 0, s>>>(ctx->kc, rt, n_runs, dir, jcap,
+                                                   ctx->geom.chunk_tokens, ctx->geom.ns, n_query,
+                                                   tokens, seq_off, qchunk_off, n_qchunks,
+                                                   hit_chunks_out, recs_out, keys_out,
+                                                   ctx->d_status, next_query);
+        ++ctx->launches;
     }
-    ++ctx->launches;
     CU(ctx, cudaGetLastError());
     return LSMKV_OK;
 }
@@ -482,7 +526,7 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"copy_stages", &ctx->copy_stages, 1, 32},
         {"copy_ctas_per_sm", &ctx->copy_ctas_per_sm, 1, 8},
         {"copy_l2_hint", &ctx->copy_l2_hint, 0, 1},
-        {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 32},
+        {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 16},
         {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
     };
     for (auto &t : tab)

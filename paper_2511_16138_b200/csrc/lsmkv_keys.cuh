@@ -56,21 +56,32 @@ __device__ __forceinline__ uint64_t shfl_up64(uint64_t v, unsigned d)
 
 struct ChunkKey { uint64_t w0, w1, w2, w3; };
 
-// One warp, 32 consecutive chunks j = base_j + lane of the sequence starting at `seq`.
-// carryA/carryB: digests of the prefix that ends just before chunk base_j (0 at base_j = 0);
-// updated to the prefix that ends after chunk base_j + 31. Lanes with j >= nch contribute
-// nothing meaningful and their key must be ignored. Must be called by all 32 lanes.
-__device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
-                                                    uint32_t C, uint32_t ns, uint64_t base_j,
-                                                    uint64_t nch, uint64_t &carryA,
-                                                    uint64_t &carryB)
+// Hash of one chunk from h = 0 (both lanes), plus its first and last token. 16-byte loads when
+// the chunk start is 16-byte aligned.
+__device__ __forceinline__ void chunk_hash(const uint32_t *t, uint32_t C, bool vec_ok,
+                                           uint64_t &hA, uint64_t &hB, uint32_t &first,
+                                           uint32_t &last)
 {
-    const unsigned lane = lane_id();
-    const uint64_t j = base_j + lane;
-    uint64_t hA = 0, hB = 0;
-    uint32_t first = 0, last = 0;
-    if (j < nch) {
-        const uint32_t *t = seq + j * C;
+    if (vec_ok) {
+        const uint4 *t4 = reinterpret_cast<const uint4 *>(t);
+        uint4 v = __ldg(t4);
+        first = v.x;
+        hA = (uint64_t)v.x + 1ull;
+        hB = hA;
+        hA = horner61(hA, kBaseA, v.y); hB = horner61(hB, kBaseB, v.y);
+        hA = horner61(hA, kBaseA, v.z); hB = horner61(hB, kBaseB, v.z);
+        hA = horner61(hA, kBaseA, v.w); hB = horner61(hB, kBaseB, v.w);
+        last = v.w;
+#pragma unroll 3
+        for (uint32_t i = 1; i < (C >> 2); ++i) {
+            v = __ldg(t4 + i);
+            hA = horner61(hA, kBaseA, v.x); hB = horner61(hB, kBaseB, v.x);
+            hA = horner61(hA, kBaseA, v.y); hB = horner61(hB, kBaseB, v.y);
+            hA = horner61(hA, kBaseA, v.z); hB = horner61(hB, kBaseB, v.z);
+            hA = horner61(hA, kBaseA, v.w); hB = horner61(hB, kBaseB, v.w);
+            last = v.w;
+        }
+    } else {
         first = __ldg(t);
         last = first;
         hA = (uint64_t)first + 1ull;
@@ -82,6 +93,23 @@ __device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const u
             hB = horner61(hB, kBaseB, last);
         }
     }
+}
+
+// One warp, 32 consecutive chunks j = base_j + lane of the sequence starting at `seq`: every
+// lane gets the digests of tokens [base_j*C, (j+1)*C), i.e. relative to the start of this
+// 32-chunk block (no carry yet). Lanes with j >= nch hold garbage. All 32 lanes must call.
+__device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint32_t *seq,
+                                                uint32_t C, uint64_t base_j, uint64_t nch,
+                                                uint64_t &hA, uint64_t &hB, uint32_t &first,
+                                                uint32_t &last)
+{
+    const unsigned lane = lane_id();
+    const uint64_t j = base_j + lane;
+    hA = 0; hB = 0; first = 0; last = 0;
+    if (j < nch) {
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
+        chunk_hash(seq + j * C, C, vec_ok, hA, hB, first, last);
+    }
     // inclusive scan: x_i <- x_{i-d} * M^d + x_i
 #pragma unroll
     for (unsigned d = 1; d < 32; d <<= 1) {
@@ -91,12 +119,25 @@ __device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const u
             hB = addmod61(mulmod61(uB, kc.pwB[d - 1]), hB);
         }
     }
+}
+
+// Same, with the running prefix: carryA/carryB are the digests of the prefix that ends just
+// before chunk base_j (0 at base_j = 0) and are advanced past chunk base_j + 31.
+__device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
+                                                    uint32_t C, uint32_t ns, uint64_t base_j,
+                                                    uint64_t nch, uint64_t &carryA,
+                                                    uint64_t &carryB)
+{
+    const unsigned lane = lane_id();
+    uint64_t hA, hB;
+    uint32_t first, last;
+    warp_block_scan(kc, seq, C, base_j, nch, hA, hB, first, last);
     hA = addmod61(mulmod61(carryA, kc.pwA[lane]), hA);
     hB = addmod61(mulmod61(carryB, kc.pwB[lane]), hB);
     carryA = __shfl_sync(0xFFFFFFFFu, hA, 31);
     carryB = __shfl_sync(0xFFFFFFFFu, hB, 31);
     ChunkKey k;
-    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)j;
+    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)(base_j + lane);
     k.w1 = hA;
     k.w2 = hB;
     k.w3 = ((uint64_t)first << 32) | (uint64_t)last;

@@ -1,6 +1,18 @@
-// Batched longest-cached-prefix probe: chunk keys of each query are looked up in the sorted
-// runs from newest to oldest; the hit length is the number of leading chunks that were all
-// found (first-miss rule), resolved per 32 chunks with one warp ballot.
+// Batched longest-cached-prefix probe.
+//
+// A CTA takes one query at a time. Its W warps hash 32*W consecutive chunks per round (each
+// warp one 32-chunk block; the block digests are chained through shared memory), every lane
+// looks its key up in the runs newest -> oldest, a warp ballot finds each warp's first miss and
+// a shared-memory minimum gives the query's. The hit length is the number of leading chunks
+// that were all found (first-miss rule); hashing stops at the round of the first miss unless
+// the caller asked for all keys.
+//
+// Lookups use fence pointers: the chunk index j is the most significant key field, so in every
+// run the keys of one j form a contiguous bucket. k_run_dir finds all bucket boundaries of all
+// runs up front (one binary search per boundary). Inside a bucket keys are ordered by the
+// digest w1, which is uniform on [0, 2^61), so the position is interpolated and pinned by a
+// branch-free binary search over a small window around the guess: ~6 dependent 8-byte loads
+// per run instead of ~20 32-byte ones, with identical control flow across the lanes of a warp.
 #pragma once
 #include "lsmkv_keys.cuh"
 
@@ -12,97 +24,226 @@ struct RunTable {
     uint64_t n[LSMKV_MAX_RUNS];
 };
 
-__device__ __forceinline__ int key_cmp_at(const lsmkv_key_t *e, const ChunkKey &k)
+__device__ __forceinline__ uint64_t key_w(const lsmkv_key_t *e, int i)
 {
-    const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(e);
-    const ulonglong2 a = __ldg(p);
-    if (a.x != k.w0) return a.x < k.w0 ? -1 : 1;
-    if (a.y != k.w1) return a.y < k.w1 ? -1 : 1;
-    const ulonglong2 b = __ldg(p + 1);
-    if (b.x != k.w2) return b.x < k.w2 ? -1 : 1;
-    if (b.y != k.w3) return b.y < k.w3 ? -1 : 1;
+    return __ldg(reinterpret_cast<const unsigned long long *>(e) + i);
+}
+
+// first index whose w0 >= w0_target
+__device__ __forceinline__ uint64_t lower_bound_w0(const lsmkv_key_t *keys, uint64_t n,
+                                                   uint64_t w0_target)
+{
+    uint64_t lo = 0, hi = n;
+    while (lo < hi) {
+        const uint64_t mid = lo + ((hi - lo) >> 1);
+        if (key_w(keys + mid, 0) < w0_target) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// dir[r * stride + j] = first index of run r whose chunk index is >= j (same namespace),
+// for j = 0..jcap (stride = jcap + 1).
+// Also resets the probe's work counter (*next_query) for the launch that follows.
+__global__ void __launch_bounds__(256)
+k_run_dir(const __grid_constant__ RunTable rt, uint32_t n_runs, uint32_t ns, uint32_t jcap,
+          uint64_t *__restrict__ dir, unsigned long long *next_query)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0) *next_query = 0;
+    const uint64_t stride = (uint64_t)jcap + 1;
+    const uint64_t total = (uint64_t)n_runs * stride;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        const uint32_t r = (uint32_t)(i / stride);
+        const uint64_t j = i - (uint64_t)r * stride;
+        dir[i] = lower_bound_w0(rt.keys[r], rt.n[r], ((uint64_t)ns << 32) + j);
+    }
+}
+
+// compare (w1,w2,w3) of entry e with the key; w0 is known to be equal inside a bucket
+__device__ __forceinline__ int bucket_cmp(const lsmkv_key_t *e, const ChunkKey &k)
+{
+    const uint64_t w1 = key_w(e, 1);
+    if (w1 != k.w1) return w1 < k.w1 ? -1 : 1;
+    const uint64_t w2 = key_w(e, 2);
+    if (w2 != k.w2) return w2 < k.w2 ? -1 : 1;
+    const uint64_t w3 = key_w(e, 3);
+    if (w3 != k.w3) return w3 < k.w3 ? -1 : 1;
     return 0;
+}
+
+// Plain exact binary search over [a, b) of a bucket with the full key (slow path).
+__device__ __noinline__ uint64_t bucket_find_exact(const lsmkv_key_t *keys, uint64_t a, uint64_t b,
+                                                   const ChunkKey &k)
+{
+    while (a < b) {
+        const uint64_t mid = a + ((b - a) >> 1);
+        const int c = bucket_cmp(keys + mid, k);
+        if (c == 0) return mid;
+        if (c < 0) a = mid + 1; else b = mid;
+    }
+    return ~0ull;
+}
+
+// Exact search of the key in bucket [lo, hi) of one run. Returns its index or ~0.
+//
+// Fast path: the digest w1 is uniform, so the key's rank inside the bucket is close to
+// w1 * cnt / 2^61 (standard deviation <= sqrt(cnt) / 2). A branch-free binary search on w1 over
+// a window of about +-2.5 standard deviations around that guess pins it with ~log2(window)
+// loads, the same number for every lane of a warp. Whenever the window cannot prove presence or
+// absence (the answer falls on a window edge, or digests tie) the slow path searches the whole
+// bucket with the full key, so the result is exact in every case.
+__device__ __forceinline__ uint64_t bucket_find(const lsmkv_key_t *keys, uint64_t lo, uint64_t hi,
+                                                const ChunkKey &k)
+{
+    const uint64_t cnt64 = hi - lo;
+    if (cnt64 == 0) return ~0ull;
+    if (cnt64 >= 0x40000000ull) return bucket_find_exact(keys, lo, hi, k);
+    const uint32_t cnt = (uint32_t)cnt64;
+    const unsigned long long *w1p = reinterpret_cast<const unsigned long long *>(keys + lo) + 1;
+    uint32_t a = 0, n = cnt;
+    if (cnt > 16) {
+        const uint32_t g = (uint32_t)__umul64hi(k.w1 << 3, cnt64);    // w1 * cnt / 2^61
+        const uint32_t R = 4u + (uint32_t)(1.25f * sqrtf((float)cnt));
+        a = g > R ? g - R : 0u;
+        const uint32_t e = min(cnt, g + R + 1u);
+        n = e - a;
+    }
+    const uint32_t a0 = a, e0 = a + n;
+    uint32_t pos = a;                              // last index in the window with w1 <= target
+    while (n > 1) {
+        const uint32_t half = n >> 1;
+        const uint64_t v = __ldg(w1p + 4ull * (pos + half));
+        pos = v <= k.w1 ? pos + half : pos;
+        n -= half;
+    }
+    const uint64_t v = __ldg(w1p + 4ull * pos);
+    if (v == k.w1) {
+        const lsmkv_key_t *e = keys + lo + pos;
+        if (key_w(e, 2) == k.w2 && key_w(e, 3) == k.w3) return lo + pos;
+        return bucket_find_exact(keys, lo, hi, k);             // digest tie: be exact
+    }
+    if (v > k.w1) {                                // only possible at pos == a0
+        return a0 > 0 ? bucket_find_exact(keys, lo, lo + a0, k) : ~0ull;
+    }
+    // v < target: absent unless the window ended before the bucket did
+    if (pos + 1 == e0 && e0 < cnt) return bucket_find_exact(keys, lo + e0, hi, k);
+    return ~0ull;
 }
 
 // Point lookup, newest run first; the first run that holds the key decides.
 __device__ __forceinline__ bool lookup_runs(const RunTable &rt, uint32_t n_runs,
+                                            const uint64_t *__restrict__ dir, uint32_t jcap,
                                             const ChunkKey &k, uint4 &val)
 {
+    const uint64_t j = k.w0 & 0xFFFFFFFFull;
+    const uint64_t stride = (uint64_t)jcap + 1;
     for (uint32_t r = 0; r < n_runs; ++r) {
         const lsmkv_key_t *keys = rt.keys[r];
-        uint64_t lo = 0, hi = rt.n[r];
-        while (lo < hi) {
-            const uint64_t mid = lo + ((hi - lo) >> 1);
-            const int c = key_cmp_at(keys + mid, k);
-            if (c == 0) {
-                val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + mid));
-                return true;
-            }
-            if (c < 0) lo = mid + 1; else hi = mid;
+        uint64_t lo, hi;
+        if (j < jcap) {
+            lo = __ldg(dir + r * stride + j);
+            hi = __ldg(dir + r * stride + j + 1);
+        } else {                                   // beyond the directory: find the bucket
+            lo = lower_bound_w0(keys, rt.n[r], k.w0);
+            hi = lower_bound_w0(keys, rt.n[r], k.w0 + 1);
+        }
+        const uint64_t pos = bucket_find(keys, lo, hi, k);
+        if (pos != ~0ull) {
+            val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + pos));
+            return true;
         }
     }
     return false;
 }
 
-__global__ void __launch_bounds__(256)
+constexpr int kProbeMaxWarps = 16;
+
+__global__ void __launch_bounds__(512)
 k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable rt,
-        uint32_t n_runs, uint32_t C, uint32_t ns, uint32_t n_query,
-        const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
-        const uint64_t *__restrict__ qchunk_off, uint64_t n_qchunks,
-        uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out,
-        lsmkv_key_t *__restrict__ keys_out, DevStatus *st)
+        uint32_t n_runs, const uint64_t *__restrict__ dir, uint32_t jcap, uint32_t C,
+        uint32_t ns, uint32_t n_query, const uint32_t *__restrict__ tokens,
+        const uint64_t *__restrict__ seq_off, const uint64_t *__restrict__ qchunk_off,
+        uint64_t n_qchunks, uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out,
+        lsmkv_key_t *__restrict__ keys_out, DevStatus *st, unsigned long long *next_query)
 {
-    const unsigned lane = lane_id();
-    const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    __shared__ uint64_t s_aggA[kProbeMaxWarps], s_aggB[kProbeMaxWarps];
+    __shared__ unsigned long long s_first_miss, s_q;
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
+    const uint64_t round_chunks = 32ull * W;
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    unsigned long long n_lookups = 0, n_hit = 0, n_empty = 0;
-    for (uint64_t q = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; q < n_query;
-         q += warps) {
+    unsigned long long n_lookups = 0;
+
+    for (;;) {
+        // queries are handed out one at a time: long and short ones balance across the CTAs
+        __syncthreads();
+        if (threadIdx.x == 0) s_q = atomicAdd(next_query, 1ull);
+        __syncthreads();
+        const uint64_t q = s_q;
+        if (q >= n_query) break;
         const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
         const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
         const uint64_t o0 = qchunk_off[q], o1 = qchunk_off[q + 1];
         if (s1 < s0 || o1 < o0 || o1 - o0 != nch || o1 > n_qchunks || nch > 0xFFFFFFFFull) {
-            if (lane == 0) { st_flag(st, LSMKV_ST_BAD_COUNT, q); hit_out[q] = 0; }
-            continue;
+            if (threadIdx.x == 0) { st_flag(st, LSMKV_ST_BAD_COUNT, q); hit_out[q] = 0; }
+            continue;                                        // uniform over the CTA
         }
+        const uint32_t *seq = tokens + s0;
         uint4 *recs = reinterpret_cast<uint4 *>(recs_out + o0);
-        uint64_t hit = nch, cA = 0, cB = 0;
+        uint64_t hit = nch, cA = 0, cB = 0;                  // cA/cB: prefix before this round
         bool done = false;
-        for (uint64_t base = 0; base < nch; base += 32) {
-            const uint64_t j = base + lane;
+        for (uint64_t base = 0; base < nch; base += round_chunks) {
+            const uint64_t j = base + 32ull * warp + lane;
             const bool valid = j < nch;
-            if (done && !keys_out) {                 // past the first miss: only zero-fill
+            if (done && !keys_out) {                         // past the first miss: zero-fill
                 if (valid) recs[j] = zero;
                 continue;
             }
-            const ChunkKey k = warp_chunk_keys(kc, tokens + s0, C, ns, base, nch, cA, cB);
+            if (threadIdx.x == 0) s_first_miss = ~0ull;
+            uint64_t hA, hB;
+            uint32_t first, last;
+            warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
+            if (lane == 31) { s_aggA[warp] = hA; s_aggB[warp] = hB; }
+            __syncthreads();
+            // prefix before this warp's block: chain the digests of the blocks before it
+            uint64_t pA = cA, pB = cB;
+            for (unsigned v = 0; v < W; ++v) {
+                if (v == warp) { hA = addmod61(mulmod61(pA, kc.pwA[lane]), hA);
+                                 hB = addmod61(mulmod61(pB, kc.pwB[lane]), hB); }
+                pA = addmod61(mulmod61(pA, kc.pwA[31]), s_aggA[v]);
+                pB = addmod61(mulmod61(pB, kc.pwB[31]), s_aggB[v]);
+            }
+            cA = pA; cB = pB;                                // valid when the round was full
+            ChunkKey k;
+            k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)j;
+            k.w1 = hA; k.w2 = hB;
+            k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
             if (done) {
                 if (valid) recs[j] = zero;
+                __syncthreads();                             // s_agg* are rewritten next round
                 continue;
             }
             uint4 val = zero;
-            const bool found = valid && lookup_runs(rt, n_runs, k, val);
-            const unsigned miss = __ballot_sync(0xFFFFFFFFu, valid && !found);
-            const unsigned first_miss = miss ? (unsigned)__ffs(miss) - 1u : 32u;
-            if (valid) recs[j] = lane < first_miss ? val : zero;
+            const bool found = valid && lookup_runs(rt, n_runs, dir, jcap, k, val);
             n_lookups += valid ? 1ull : 0ull;
-            if (miss) { hit = base + first_miss; done = true; }
+            const unsigned miss = __ballot_sync(0xFFFFFFFFu, valid && !found);
+            if (miss && lane == 0)
+                atomicMin(&s_first_miss, base + 32ull * warp + (unsigned)__ffs(miss) - 1ull);
+            __syncthreads();
+            const uint64_t fm = s_first_miss;
+            if (valid) recs[j] = j < fm ? val : zero;
+            if (fm != ~0ull) { hit = fm; done = true; }
+            __syncthreads();                                 // before s_first_miss is reset
         }
-        if (lane == 0) {
+        if (threadIdx.x == 0) {
             hit_out[q] = (uint32_t)hit;
-            n_hit += hit;
-            n_empty += hit == 0 ? 1ull : 0ull;
+            atomicAdd(&st->chunks_hit, (unsigned long long)hit);
+            if (hit == 0) atomicAdd(&st->empty_probes, 1ull);
         }
     }
-    // counters: lanes hold partial lookup counts, lane 0 holds hits / empties
 #pragma unroll
     for (unsigned d = 16; d; d >>= 1) n_lookups += __shfl_down_sync(0xFFFFFFFFu, n_lookups, d);
-    if (lane == 0) {
-        if (n_lookups) atomicAdd(&st->lookups, n_lookups);
-        if (n_hit) atomicAdd(&st->chunks_hit, n_hit);
-        if (n_empty) atomicAdd(&st->empty_probes, n_empty);
-    }
+    if (lane == 0 && n_lookups) atomicAdd(&st->lookups, n_lookups);
 }
 
 }  // namespace lsmkv
