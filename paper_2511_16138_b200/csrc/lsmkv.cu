@@ -244,8 +244,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->chunk_bytes = 2ull * g->n_layers * pb;
     fill_key_consts(ctx->kc, g->chunk_tokens);
     ctx->copy_mode = 0;
-    ctx->copy_stage_bytes = 32768;
-    ctx->copy_stages = 6;
+    ctx->copy_stage_bytes = 16384;
+    ctx->copy_stages = 12;
     ctx->copy_ctas_per_sm = 1;
     ctx->copy_l2_hint = 0;
     ctx->probe_warps_per_cta = 4;
