@@ -175,6 +175,30 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
                        const lsmkv_pool_t *pool);
 
 /*
+ * Flush: one sorted run out of a write batch (Sec. 2.2 "Updates": out-of-place writes are
+ * buffered and flushed as a sorted run). keys/vals [dev] hold n entries in arrival order,
+ * duplicates allowed; of equal keys the LAST arrival survives. Output [dev]: run_keys_out and
+ * run_vals_out need room for n entries; entries [0, *n_out) are the run (ascending, unique),
+ * entries [*n_out, n) are padding -- all-ones keys, which compare above every real key, with
+ * zero records -- so the buffers may be used as a run of length n without reading *n_out back.
+ * n_out [dev] receives the run length. Outputs must not overlap the inputs. n < 2^32 - 1.
+ * Uses (and may grow) the context's sort scratch: 88 bytes per entry.
+ */
+int lsmkv_flush_batch(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys,
+                      const lsmkv_val_t *vals, uint64_t n, lsmkv_key_t *run_keys_out,
+                      lsmkv_val_t *run_vals_out, uint64_t *n_out);
+
+/*
+ * Compaction: several runs ([host] array, newest first, as for lsmkv_probe_batch) merged into
+ * one: the union of their keys, each key with the record of the newest run that holds it
+ * (Sec. 2.2: compaction merges runs and removes obsolete entries). keys_out / vals_out [dev]
+ * need room for the sum of the run lengths and are padded like a flush; n_out [dev] receives
+ * the merged length. Sum of lengths < 2^32 - 1. Outputs must not overlap the input runs.
+ */
+int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint32_t n_runs,
+                     lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
+
+/*
  * Allocation-free decode (an addition of this library; the paper has no counterpart).
  *
  * Same result as lsmkv_decode_batch(), for callers that are not allowed to allocate device
@@ -227,6 +251,8 @@ int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out);
 #define LSMKV_K_PROBE 2
 #define LSMKV_K_PLAN 3
 #define LSMKV_K_UNPACK 4
+#define LSMKV_K_FLUSH 5
+#define LSMKV_K_MERGE 6
 #define LSMKV_K_CLASSES 8
 typedef struct {
     double ms[LSMKV_K_CLASSES];

@@ -13,6 +13,7 @@
 #include "lsmkv_copy.cuh"
 #include "lsmkv_keys.cuh"
 #include "lsmkv_probe.cuh"
+#include "lsmkv_sort.cuh"
 
 using namespace lsmkv;
 
@@ -27,6 +28,9 @@ struct lsmkv_ctx {
     // workspace: hit_off u64[ws_seq + 1] followed by plan u32[ws_chunks]
     void *d_ws;
     uint64_t ws_seq, ws_chunks;
+    // scratch of flush / compaction (key and index ping-pong buffers, records, block counts)
+    void *d_sort;
+    uint64_t sort_cap;
     // fence-pointer directory of the probe: u64[n_runs * (jcap + 1)]
     uint64_t *d_dir;
     uint64_t dir_cap;
@@ -160,6 +164,65 @@ int ensure_dir(lsmkv_ctx *ctx, uint64_t entries)
     return LSMKV_OK;
 }
 
+struct SortWs {
+    lsmkv_key_t *keys[2];
+    uint32_t *idx[2];
+    lsmkv_val_t *vals;
+    uint64_t *block_count;
+};
+
+size_t sort_ws_bytes(uint64_t n)
+{
+    return (size_t)n * (2 * 32 + 2 * 4 + 16) + ((size_t)n / kScanBlock + 4) * 8 + 256;
+}
+
+int ensure_sort(lsmkv_ctx *ctx, uint64_t n, SortWs *ws)
+{
+    if (n > ctx->sort_cap || !ctx->d_sort) {
+        void *p = nullptr;
+        cudaError_t e = cudaMalloc(&p, sort_ws_bytes(n));
+        if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
+        if (ctx->d_sort) cudaFree(ctx->d_sort);
+        ctx->d_sort = p;
+        ctx->sort_cap = n;
+    }
+    const uint64_t cap = ctx->sort_cap;
+    unsigned char *b = static_cast<unsigned char *>(ctx->d_sort);
+    ws->keys[0] = reinterpret_cast<lsmkv_key_t *>(b);
+    ws->keys[1] = reinterpret_cast<lsmkv_key_t *>(b + cap * 32);
+    ws->vals = reinterpret_cast<lsmkv_val_t *>(b + cap * 64);
+    ws->block_count = reinterpret_cast<uint64_t *>(b + cap * 80);
+    const size_t bc = ((size_t)cap / kScanBlock + 4) * 8;
+    ws->idx[0] = reinterpret_cast<uint32_t *>(b + cap * 80 + bc);
+    ws->idx[1] = ws->idx[0] + cap;
+    return LSMKV_OK;
+}
+
+// flag / scan / scatter: sorted keys + origin indices -> final run (+ padding) and its length
+int launch_dedupe(lsmkv_ctx *ctx, cudaStream_t s, const SortWs &ws, int buf, uint64_t n,
+                  const lsmkv_val_t *vals_in, int keep_last, lsmkv_key_t *keys_out,
+                  lsmkv_val_t *vals_out, uint64_t *n_out)
+{
+    const uint64_t blocks = (n + kScanBlock - 1) / kScanBlock;
+    k_dedupe_count<<<(unsigned)blocks, kScanBlock, 0, s>>>(ws.keys[buf], n, keep_last,
+                                                            ws.block_count);
+    k_scan_blocks<<<1, 1024, 0, s>>>(ws.block_count, blocks, n_out);
+    k_dedupe_scatter<<<(unsigned)blocks, kScanBlock, 0, s>>>(ws.keys[buf], ws.idx[buf], vals_in,
+                                                              n, keep_last, ws.block_count, n_out,
+                                                              keys_out, vals_out);
+    ctx->launches += 3;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
+unsigned merge_grid(const lsmkv_ctx *ctx, uint64_t n)
+{
+    uint64_t g = (n + 255) / 256;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 8;
+    if (g > cap) g = cap;
+    return g ? (unsigned)g : 1u;
+}
+
 constexpr uint64_t kDirMaxJ = 65536;   // chunk indices covered by the probe's directory
 
 uint64_t *ws_hit_off(lsmkv_ctx *ctx) { return static_cast<uint64_t *>(ctx->d_ws); }
@@ -287,6 +350,7 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     cudaDeviceSynchronize();
     if (ctx->d_ws) cudaFree(ctx->d_ws);
     if (ctx->d_dir) cudaFree(ctx->d_dir);
+    if (ctx->d_sort) cudaFree(ctx->d_sort);
     if (ctx->d_status) cudaFree(ctx->d_status);
     for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : ctx->free_events) cudaEventDestroy(e);
@@ -467,6 +531,102 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
     job.recs = recs;
     job.st = ctx->d_status;
     return launch_copy(ctx, s, job, ar, n_qchunks);
+}
+
+int lsmkv_flush_batch(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys,
+                      const lsmkv_val_t *vals, uint64_t n, lsmkv_key_t *run_keys_out,
+                      lsmkv_val_t *run_vals_out, uint64_t *n_out)
+{
+    if (!ctx || !n_out) return LSMKV_EINVAL;
+    if (n >= 0xFFFFFFFFull) return LSMKV_EINVAL;
+    if (n && (!keys || !vals || !run_keys_out || !run_vals_out || !aligned16(keys) ||
+              !aligned16(vals) || !aligned16(run_keys_out) || !aligned16(run_vals_out)))
+        return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n == 0) {
+        CU(ctx, cudaMemsetAsync(n_out, 0, sizeof(uint64_t), s));
+        return LSMKV_OK;
+    }
+    SortWs ws;
+    int rc = ensure_sort(ctx, n, &ws);
+    if (rc != LSMKV_OK) return rc;
+    LaunchTimer timer(ctx, s, LSMKV_K_FLUSH);
+    SegTable segs;
+    std::memset(&segs, 0, sizeof(segs));
+    const lsmkv_key_t *src = keys;
+    const uint32_t *src_idx = nullptr;
+    int buf = 0;
+    const unsigned grid = merge_grid(ctx, n);
+    for (uint64_t width = 1;; width *= 2) {
+        k_merge_level<<<grid, 256, 0, s>>>(src, src_idx, ws.keys[buf], ws.idx[buf], n, width, segs);
+        ++ctx->launches;
+        src = ws.keys[buf];
+        src_idx = ws.idx[buf];
+        if (width * 2 >= n) break;
+        buf ^= 1;
+    }
+    CU(ctx, cudaGetLastError());
+    return launch_dedupe(ctx, s, ws, buf, n, vals, /*keep_last=*/1, run_keys_out, run_vals_out,
+                         n_out);
+}
+
+int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint32_t n_runs,
+                     lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out)
+{
+    if (!ctx || !n_out || n_runs > LSMKV_MAX_RUNS || (n_runs && !runs)) return LSMKV_EINVAL;
+    uint64_t total = 0;
+    for (uint32_t r = 0; r < n_runs; ++r) {
+        if (runs[r].n && (!runs[r].keys || !runs[r].vals)) return LSMKV_EINVAL;
+        total += runs[r].n;
+    }
+    if (total >= 0xFFFFFFFFull) return LSMKV_EINVAL;
+    if (total && (!keys_out || !vals_out || !aligned16(keys_out) || !aligned16(vals_out)))
+        return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (total == 0) {
+        CU(ctx, cudaMemsetAsync(n_out, 0, sizeof(uint64_t), s));
+        return LSMKV_OK;
+    }
+    SortWs ws;
+    int rc = ensure_sort(ctx, total, &ws);
+    if (rc != LSMKV_OK) return rc;
+    LaunchTimer timer(ctx, s, LSMKV_K_MERGE);
+    // concatenate newest first; ties then resolve to the newer run
+    SegTable segs;
+    std::memset(&segs, 0, sizeof(segs));
+    uint64_t at = 0;
+    uint32_t n_seg = 0;
+    for (uint32_t r = 0; r < n_runs; ++r) {
+        if (runs[r].n == 0) continue;
+        CU(ctx, cudaMemcpyAsync(ws.keys[0] + at, runs[r].keys, runs[r].n * sizeof(lsmkv_key_t),
+                                cudaMemcpyDeviceToDevice, s));
+        CU(ctx, cudaMemcpyAsync(ws.vals + at, runs[r].vals, runs[r].n * sizeof(lsmkv_val_t),
+                                cudaMemcpyDeviceToDevice, s));
+        segs.start[n_seg++] = at;
+        at += runs[r].n;
+    }
+    segs.start[n_seg] = total;
+    segs.n_seg = n_seg;
+    int buf = 0;
+    const uint32_t *src_idx = nullptr;
+    const unsigned grid = merge_grid(ctx, total);
+    for (;;) {
+        k_merge_level<<<grid, 256, 0, s>>>(ws.keys[buf], src_idx, ws.keys[buf ^ 1], ws.idx[buf ^ 1],
+                                           total, 0, segs);
+        ++ctx->launches;
+        buf ^= 1;
+        src_idx = ws.idx[buf];
+        const uint32_t next = (segs.n_seg + 1) / 2;
+        for (uint32_t k = 0; k < next; ++k) segs.start[k] = segs.start[2 * k];
+        segs.start[next] = total;
+        segs.n_seg = next;
+        if (next <= 1) break;
+    }
+    CU(ctx, cudaGetLastError());
+    return launch_dedupe(ctx, s, ws, buf, total, ws.vals, /*keep_last=*/0, keys_out, vals_out,
+                         n_out);
 }
 
 int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out)

@@ -23,12 +23,12 @@ EXPORTS = (
     "lsmkv_probe_batch", "lsmkv_decode_batch", "lsmkv_last_status", "lsmkv_last_cuda_error",
     "lsmkv_launch_count", "lsmkv_set_tuning", "lsmkv_get_tuning", "lsmkv_strerror",
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
-    "lsmkv_decode_batch_static",
+    "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
 )
 ETOOBIG = -5
 STATIC_MAX_QUERIES, STATIC_MAX_CHUNKS = 4096, 262144
 K_KEYS, K_PACK, K_PROBE, K_PLAN, K_UNPACK, K_CLASSES = 0, 1, 2, 3, 4, 8
-K_NAMES = ("keys", "pack", "probe", "plan", "unpack")
+K_NAMES = ("keys", "pack", "probe", "plan", "unpack", "flush", "merge")
 
 
 class LsmkvError(RuntimeError):
@@ -121,6 +121,10 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch_static.argtypes = [C.POINTER(GeomStruct), C.c_int, vp, u32, vp, u64, vp,
                                             vp, C.POINTER(vp), C.POINTER(u64), u32, vp,
                                             C.POINTER(PoolStruct), vp]
+    L.lsmkv_flush_batch.restype = C.c_int
+    L.lsmkv_flush_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp, vp]
+    L.lsmkv_merge_runs.restype = C.c_int
+    L.lsmkv_merge_runs.argtypes = [vp, vp, C.POINTER(RunStruct), u32, vp, vp, vp]
     L.lsmkv_last_status.restype = C.c_int
     L.lsmkv_last_status.argtypes = [vp, vp, C.POINTER(StatusStruct)]
     L.lsmkv_last_cuda_error.restype = C.c_int
@@ -235,6 +239,23 @@ def lsmkv_decode_batch(ctx, stream, n_query, qchunk_off, n_qchunks, hit_chunks, 
     _check(ctx, rc, "lsmkv_decode_batch")
 
 
+def lsmkv_flush_batch(ctx, stream, keys, vals, n, run_keys_out, run_vals_out, n_out) -> None:
+    rc = lib().lsmkv_flush_batch(ctx, _stream(stream), _ptr(keys), _ptr(vals), n,
+                                 _ptr(run_keys_out), _ptr(run_vals_out), _ptr(n_out))
+    _check(ctx, rc, "lsmkv_flush_batch")
+
+
+def lsmkv_merge_runs(ctx, stream, runs, keys_out, vals_out, n_out) -> None:
+    """runs: sequence of (keys, vals, n), newest first."""
+    n_runs = len(runs)
+    arr = (RunStruct * max(1, n_runs))()
+    for i, (k, v, n) in enumerate(runs):
+        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    rc = lib().lsmkv_merge_runs(ctx, _stream(stream), arr, n_runs, _ptr(keys_out),
+                                _ptr(vals_out), _ptr(n_out))
+    _check(ctx, rc, "lsmkv_merge_runs")
+
+
 def lsmkv_decode_batch_static(geom: Geom, device, stream, n_query, qchunk_off, n_qchunks,
                               hit_chunks, recs, arenas, dst_page_table, pool,
                               status_out=None) -> None:
@@ -334,6 +355,12 @@ class Context:
                      dst_page_table, pool, stream=None):
         lsmkv_decode_batch(self.handle, stream, n_query, qchunk_off, n_qchunks, hit_chunks, recs,
                            arenas, dst_page_table, pool)
+
+    def flush_batch(self, keys, vals, n, run_keys_out, run_vals_out, n_out, stream=None):
+        lsmkv_flush_batch(self.handle, stream, keys, vals, n, run_keys_out, run_vals_out, n_out)
+
+    def merge_runs(self, runs, keys_out, vals_out, n_out, stream=None):
+        lsmkv_merge_runs(self.handle, stream, runs, keys_out, vals_out, n_out)
 
     def last_status(self, stream=None) -> dict:
         return lsmkv_last_status(self.handle, stream)
