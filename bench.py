@@ -1,6 +1,6 @@
 #!/usr/bin/env python
-"""Benchmark of the whole hot path: encode (chunk keys + records + pack) -> probe -> decode
-(unpack/scatter) over one batch of Llama-3-8B-shaped requests, on N GPUs of one node.
+"""Benchmark of the whole hot path: encode (chunk keys + records + pack) -> flush (keys become a
+sorted run) -> probe -> decode (unpack/scatter) over one batch of Llama-3-8B-shaped requests, on N GPUs of one node.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -216,7 +216,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2511_16138_b200 import hostindex, lsmkv, ranks
+    from paper_2511_16138_b200 import lsmkv, ranks
 
     rank, world, local_rank = ranks.rank_env()
     if world > 1:
@@ -309,28 +309,40 @@ def main():
         ctx.decode_batch(d["n_req"], d["coff"], d["n"], d["hit"], d["recs"],
                          [(arena, d["n"] * cb)], d["dst_pages"], dst_pool, stream=stream)
 
-    # ---- untimed preparation: the index (one sorted run per wave) from the encoder's own keys
+    # ---- untimed preparation: the index (one sorted run per wave), flushed on the device from
+    # the encoder's own keys; the padded flush output serves as the run, no count is read back
+    flush_ms = []
     for d in W:
         encode(d)
-        torch.cuda.synchronize()
-        keys = d["keys"].cpu().numpy().view(np.uint64).reshape(-1, 4)
-        vals = d["vals"].cpu().numpy().reshape(-1, 16)
-        rk, rv = hostindex.flush(keys, vals)
-        d["run_t"] = (up(rk), up(rv))
-        d["runs"] = [(d["run_t"][0], d["run_t"][1], len(rk))]
+        n = d["n"]
+        d["run_k"] = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+        d["run_v"] = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        d["run_n"] = torch.zeros(1, dtype=torch.int64, device=dev)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        ctx.flush_batch(d["keys"], d["vals"], n, d["run_k"], d["run_v"], d["run_n"], stream=stream)
+        f1.record(stream)
+        d["runs"] = [(d["run_k"], d["run_v"], n)]
         probe(d)
         decode(d)
         torch.cuda.synchronize()
-        # self-check of this wave (device side): every chunk is a hit; sampled pages restored
+        flush_ms.append(f0.elapsed_time(f1))
+        # self-check of this wave (device side): every chunk is a hit
         assert np.array_equal(d["hit"].cpu().numpy(), d["nch"].astype(np.int32)), "probe missed"
+        assert 0 < int(d["run_n"].item()) <= n
     st = ctx.last_status()
     assert st["flags"] == 0, st
 
+    def flush(d):
+        ctx.flush_batch(d["keys"], d["vals"], d["n"], d["run_k"], d["run_v"], d["run_n"],
+                        stream=stream)
+
     def step():
         for d in W:
-            encode(d)
+            encode(d)      # chunk keys + records + pack
+            flush(d)       # the batch's keys become the sorted run the probe searches
             probe(d)
-            decode(d)
+            decode(d)      # plan + unpack
 
     for _ in range(args.warmup):
         step()
@@ -368,7 +380,7 @@ def main():
     # ---- probe throughput on the probe-heavy workload (second half of the metric)
     probe_block = None
     if rank == 0 and not args.no_probe_block:
-        probe_block = probe_heavy_block(torch, lsmkv, hostindex, dev, local_rank, args.steps,
+        probe_block = probe_heavy_block(torch, lsmkv, dev, local_rank, args.steps,
                                         args.warmup)
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, single GPU runs only)
@@ -430,6 +442,7 @@ def main():
                 "kernel_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
                 "kernel_launches": {k: v[1] for k, v in prof.items()},
                 "lookups_per_step": status["lookups"] / args.steps,
+                "flush_ms_per_wave_in_prep": sum(flush_ms) / len(flush_ms),
             },
         }
         print(json.dumps(out))
@@ -437,11 +450,11 @@ def main():
         dist.destroy_process_group()
 
 
-def probe_heavy_block(torch, lsmkv, hostindex, dev, device_index, steps, warmup):
+def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
     """Probe throughput on the probe-heavy workload (configs[2]): 1M stored chunk keys in four
     sorted runs (900 / 9000 / 90000 / 900100 keys, 1% newer duplicates), 4096 queries of 2k-32k
-    tokens, 60% with a cached prefix. Keys come from the library's own encoder; the runs are
-    built on the host (untimed)."""
+    tokens, 60% with a cached prefix. Keys come from the library's own encoder and the runs from
+    its flush (both untimed here)."""
     g = lsmkv.Geom(8, 8, 128, page_tokens=16, chunk_tokens=16)
     w = synth.probe_heavy()
     nch = synth.chunk_counts(w.store.seq_off, 16)
@@ -463,14 +476,27 @@ def probe_heavy_block(torch, lsmkv, hostindex, dev, device_index, steps, warmup)
         keys = d_keys.cpu().numpy().view(np.uint64).reshape(-1, 4)
         vals = d_vals.cpu().numpy().reshape(-1, 16)
         runs, keep = [], []
-        for r in range(4):
+        for r in range(4):                      # deal the keys to the runs, flush each on the GPU
             sel = w.run_of_key == r
             dup = w.dup_idx[w.dup_run == r]
-            rk, rv = hostindex.flush(np.concatenate([keys[sel], keys[dup]]),
-                                     np.concatenate([vals[sel], vals[(dup + 7919) % n]]))
-            tk, tv = up(rk), up(rv)
-            keep.append((tk, tv))
-            runs.append((tk, tv, len(rk)))
+            bk = up(np.concatenate([keys[sel], keys[dup]]))
+            bv = up(np.concatenate([vals[sel], vals[(dup + 7919) % n]]))
+            m = int(sel.sum()) + len(dup)
+            tk = torch.empty(m * 32, dtype=torch.uint8, device=dev)
+            tv = torch.empty(m * 16, dtype=torch.uint8, device=dev)
+            tn = torch.zeros(1, dtype=torch.int64, device=dev)
+            ctx.flush_batch(bk, bv, m, tk, tv, tn)
+            keep.append((tk, tv, tn))
+            runs.append((tk, tv, m))
+        ctx.last_status()
+        ctx.profile_enable(True)
+        ctx.profile_read()
+        big = int((w.run_of_key == 3).sum())
+        for _ in range(3):
+            ctx.flush_batch(bk, bv, m, tk, tv, tn)
+        torch.cuda.synchronize()
+        flush_big_ms = ctx.profile_read()["flush"][0] / 3
+        ctx.profile_enable(False)
         qoff = synth.offsets(synth.chunk_counts(w.query.seq_off, 16))
         total = int(qoff[-1])
         d_tok, d_off, d_qoff = up(w.query.tokens), up(w.query.seq_off), up(qoff)
@@ -501,6 +527,7 @@ def probe_heavy_block(torch, lsmkv, hostindex, dev, device_index, steps, warmup)
                 "hit_chunks_per_s": st["chunks_hit"] / reps / ms * 1e3,
                 "query_tokens": int(len(w.query.tokens)), "stored_keys": n,
                 "algorithmic_GBps": algo_bytes / ms / 1e6,
+                "flush_ms_for_%d_keys" % big: flush_big_ms,
                 "bound": "L2 latency / instruction issue (not HBM)"}
     finally:
         ctx.close()
@@ -547,7 +574,6 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
         devs = {k: torch.empty(max(16, v.numel()), dtype=torch.uint8, device=dev) for k, v in pins.items()}
         prepared.append([d, b - a, c1 - c0, pins, devs, None])
     # untimed: the index of each sub-batch (its records point into this sub-batch's blobs)
-    from paper_2511_16138_b200 import hostindex
     keep = []
     for p in prepared:
         d, n_req, n, pins, devs, _ = p
@@ -555,13 +581,13 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
             devs[k][:pins[k].numel()].copy_(pins[k])
         ctx.encode_batch(n_req, devs["tokens"], devs["seq_off"], None, devs["coff"], n, None, None,
                          0, 0, d["keys"], d["vals"], None, 0, stream=stream)
+        tk = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+        tv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        tn = torch.zeros(1, dtype=torch.int64, device=dev)
+        ctx.flush_batch(d["keys"], d["vals"], n, tk, tv, tn, stream=stream)
         torch.cuda.synchronize()
-        rk, rv = hostindex.flush(d["keys"][:n * 32].cpu().numpy().view(np.uint64).reshape(-1, 4),
-                                 d["vals"][:n * 16].cpu().numpy().reshape(-1, 16))
-        tk = torch.from_numpy(rk.view(np.uint8).reshape(-1).copy()).to(dev)
-        tv = torch.from_numpy(rv.reshape(-1).copy()).to(dev)
-        keep.append((tk, tv))
-        p[5] = [(tk, tv, len(rk))]
+        keep.append((tk, tv, tn))
+        p[5] = [(tk, tv, n)]
     h2d = d2h = 0
     moved = 0
 

@@ -238,3 +238,31 @@ def oracle_decode_one(g, rec, blob_bytes):
     oracle.decode_batch(og, np.array([0, 1], np.uint64), np.array([1], np.uint32), r,
                         [np.ascontiguousarray(blob_bytes)], np.array([0], np.uint32), out)
     return out
+
+
+def gpu_flush_run(ctx, keys: np.ndarray, vals: np.ndarray):
+    """Flush on the device; returns the trimmed run as host arrays (keys [m,4], vals [m])."""
+    n = len(keys)
+    if n == 0:
+        return np.zeros((0, 4), np.uint64), np.zeros(0, VAL_DTYPE)
+    ok = torch.empty(n * 32, dtype=torch.uint8, device=DEV)
+    ov = torch.empty(n * 16, dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    ctx.flush_batch(dev(keys), dev(np.ascontiguousarray(vals)), n, ok, ov, cnt)
+    torch.cuda.synchronize()
+    m = int(cnt.item())
+    return (host(ok, np.uint64, n * 32).reshape(-1, 4)[:m].copy(),
+            host(ov, VAL_DTYPE, n * 16)[:m].copy())
+
+
+def gpu_merge_runs(ctx, runs):
+    total = sum(len(k) for k, _ in runs)
+    druns, keep = dev_runs(runs)
+    ok = torch.empty(max(1, total) * 32, dtype=torch.uint8, device=DEV)
+    ov = torch.empty(max(1, total) * 16, dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    ctx.merge_runs(druns, ok, ov, cnt)
+    torch.cuda.synchronize()
+    m = int(cnt.item())
+    return (host(ok, np.uint64, total * 32).reshape(-1, 4)[:m].copy(),
+            host(ov, VAL_DTYPE, total * 16)[:m].copy())

@@ -69,7 +69,7 @@ def encode_probe_decode_wave(ctx, g, batch, nch, src, dst, arena, rng, n_sample=
     o_keys, o_vals, _ = oracle.encode_batch(og, batch.tokens, batch.seq_off, None, coff, None,
                                             None, 0, 0, with_blob=False)
     assert np.array_equal(keys, o_keys) and np.array_equal(vals, o_vals)
-    run = hostindex.flush(keys, vals)
+    run = H.gpu_flush_run(ctx, keys, vals)
     o_run = oracle.flush(o_keys, o_vals)
     assert np.array_equal(run[0], o_run[0]) and np.array_equal(run[1], o_run[1])
     d_hit = torch.zeros(batch.n, dtype=torch.int32, device=H.DEV)
@@ -142,7 +142,7 @@ def test_config5_long_context_encode_probe_decode():
     rng = synth.rng_for(5, 5)
     with lsmkv.Context(g, 0) as ctx:
         keys, vals = encode_probe_decode_wave(ctx, g, w.store, nch, src, dst, arena, rng, width=4)
-        run = hostindex.flush(keys, vals)
+        run = H.gpu_flush_run(ctx, keys, vals)
         qn = synth.chunk_counts(w.query.seq_off, 16)
         qoff = synth.offsets(qn)
         hit, recs, qkeys, (d_qoff, d_hit, d_recs) = H.gpu_probe(ctx, w.query, qoff, [run])
@@ -188,8 +188,11 @@ def test_config3_probe_heavy_full():
             d = w.dup_idx[w.dup_run == r]
             dv = vals[d].copy()
             dv["offset"] = ((d + 7919) % n_blobs) * cb            # newer copy, different record
-            runs.append(hostindex.flush(np.concatenate([keys[sel], keys[d]]),
+            runs.append(H.gpu_flush_run(ctx, np.concatenate([keys[sel], keys[d]]),
                                         np.concatenate([vals[sel], dv])))
+            o_run = oracle.flush(np.concatenate([keys[sel], keys[d]]),
+                                 np.concatenate([vals[sel], dv]))
+            assert np.array_equal(runs[r][0], o_run[0]) and np.array_equal(runs[r][1], o_run[1])
         assert len(runs[3][0]) == 900_100
         qn = synth.chunk_counts(w.query.seq_off, 16)
         qoff = synth.offsets(qn)
@@ -334,10 +337,12 @@ def test_config4_gqa_multi_turn():
                 used += n
                 total_encoded += n
                 stored = nch.copy()
-                runs.insert(0, hostindex.flush(keys, vals))
+                runs.insert(0, H.gpu_flush_run(ctx, keys, vals))
                 o_runs.insert(0, oracle.flush(o_keys, o_vals))
+                assert np.array_equal(runs[0][0], o_runs[0][0])
+                assert np.array_equal(runs[0][1], o_runs[0][1])
                 if len(runs) > 4:                  # compaction of the two oldest runs
-                    runs[-2:] = [hostindex.merge_runs(runs[-2:])]
+                    runs[-2:] = [H.gpu_merge_runs(ctx, runs[-2:])]
                     o_runs[-2:] = [oracle.merge_runs(o_runs[-2:])]
                     assert np.array_equal(runs[-1][0], o_runs[-1][0])
                     assert np.array_equal(runs[-1][1], o_runs[-1][1])
