@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--requests", type=int, default=256, help="requests in the batch (256 = the named workload)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU baseline budget (0 = skip)")
+    ap.add_argument("--only-probe-block", action="store_true",
+                    help="run just the probe-heavy measurement (a small case for profiling)")
     ap.add_argument("--no-probe-block", action="store_true",
                     help="skip the probe-heavy measurement")
     ap.add_argument("--tuning", default="", help="name=value,... launch-shape knobs")
@@ -231,6 +233,12 @@ def main():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
+
+    if args.only_probe_block:
+        if rank == 0:
+            print(json.dumps({"probe": probe_heavy_block(torch, lsmkv, dev, local_rank,
+                                                         args.steps, args.warmup)}))
+        return
 
     g = lsmkv.Geom(**GEOM)
     cb, pb, L2 = g.chunk_bytes, g.page_bytes, 2 * g.n_layers
