@@ -15,6 +15,10 @@
  *   - Problems only the GPU can see (a page id beyond the pool, a record that points outside
  *     its arena, a misaligned buffer, a wait that ran out) never fault: the offending item is
  *     skipped and recorded in a device status block read back by lsmkv_last_status().
+ *   - A context is not thread-safe and orders nothing by itself: calls that share internal
+ *     scratch (two probes, two decodes, two flushes/merges, two host-buffer calls of the same
+ *     kind) must be ordered by the caller -- same stream, or events. A put on one stream and a
+ *     probe/decode on another are independent. Use one context per stream for more.
  *   - No call allocates device memory except lsmkv_create(), lsmkv_reserve() and a batch call
  *     whose batch is larger than any before it (the internal workspace grows; call
  *     lsmkv_reserve() up front to rule that out).
@@ -199,6 +203,45 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
 
 /*
+ * Host-buffer variants (the form the paper's service interface has: token sequences and
+ * tensors handed over by the serving process, App. B). Same results as the device-buffer
+ * calls; every pointer except `pool` and `runs[].keys/vals` is a HOST pointer (use pinned
+ * memory for full transfer speed; pageable memory works). The calls stage through device
+ * scratch owned by the context (grown on demand, bounded by the "host_stage_bytes" knob plus
+ * the descriptors; default 1 GiB of blobs per slice), enqueue all copies and kernels on
+ * `stream` and return; host outputs are valid, and host inputs may be reused, once the stream
+ * has reached the end of the call's work. Offsets (chunk_off / qchunk_off) are computed by
+ * the library from the sequence lengths.
+ *
+ * lsmkv_put_batch_host: put_batch. keys_out / vals_out / blob_out [host] receive what
+ *   lsmkv_encode_batch produces; *n_chunks_out (optional) is set before returning. blob_out
+ *   may be NULL together with page_table and pool (index-only).
+ * lsmkv_probe_batch_host: probe. hit_chunks_out [host n_query], recs_out [host, sum of
+ *   floor(len/C)], optional keys_out; *n_qchunks_out (optional) is set before returning.
+ * lsmkv_decode_batch_host: get_batch, tensor half. qchunk_off, hit_chunks, recs and
+ *   dst_page_table are host arrays (typically what lsmkv_probe_batch_host returned, after a
+ *   stream synchronisation); `arenas` are HOST base pointers of the tensor-log buffers indexed
+ *   by file_id. The blobs of the hit chunks are copied to the device slice by slice (blobs
+ *   adjacent in an arena travel as one copy) and scattered into the pool. Records are checked
+ *   on the host first: LSMKV_EINVAL and nothing enqueued if one points outside its arena.
+ */
+int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint32_t *tokens,
+                         const uint64_t *seq_off, const uint32_t *start_chunk,
+                         const uint32_t *page_table, const lsmkv_pool_t *pool, uint32_t file_id,
+                         uint64_t base_offset, lsmkv_key_t *keys_out, lsmkv_val_t *vals_out,
+                         void *blob_out, uint64_t blob_capacity, uint64_t *n_chunks_out);
+int lsmkv_probe_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
+                           const uint32_t *tokens, const uint64_t *seq_off,
+                           const lsmkv_run_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,
+                           lsmkv_val_t *recs_out, lsmkv_key_t *keys_out,
+                           uint64_t *n_qchunks_out);
+int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
+                            const uint64_t *qchunk_off, const uint32_t *hit_chunks,
+                            const lsmkv_val_t *recs, const void *const *arenas,
+                            const uint64_t *arena_bytes, uint32_t n_arenas,
+                            const uint32_t *dst_page_table, const lsmkv_pool_t *pool);
+
+/*
  * Allocation-free decode (an addition of this library; the paper has no counterpart).
  *
  * Same result as lsmkv_decode_batch(), for callers that are not allowed to allocate device
@@ -275,6 +318,7 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "copy_stages"       bulk copies in flight per CTA, 1..32 (reduced to fit shared memory)
  *   "copy_ctas_per_sm"  1..8        "copy_l2_hint"  0/1 = evict-first L2 policy on the copies
  *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..16
+ *   "host_stage_bytes"  blob bytes staged per slice by the host-buffer calls, 1 MiB..64 GiB
  */
 int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value);
 int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name);

@@ -3,6 +3,7 @@
 // payload bytes on the host.
 #include <cstdio>
 #include <cstdlib>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -38,7 +39,14 @@ struct lsmkv_ctx {
     uint64_t launches;
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
-    int64_t probe_warps_per_cta, simt_ctas_per_sm;
+    int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes;
+    // host-buffer calls: device staging and host scratch
+    void *d_io[3];
+    size_t io_cap[3];
+    std::vector<uint64_t> h_off_a;
+    struct HostScratch { void *p; size_t cap; cudaEvent_t done; bool used; };
+    HostScratch hs[2];
+    int hs_next;
     // optional per-kernel timing with CUDA events on the launching stream
     bool profiling;
     struct Timed { cudaEvent_t a, b; int cls; };
@@ -313,6 +321,7 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->copy_l2_hint = 0;
     ctx->probe_warps_per_cta = 4;
     ctx->simt_ctas_per_sm = 8;
+    ctx->host_stage_bytes = 1ll << 30;
 
     DeviceGuard guard(device);
     cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
@@ -351,6 +360,11 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     if (ctx->d_ws) cudaFree(ctx->d_ws);
     if (ctx->d_dir) cudaFree(ctx->d_dir);
     if (ctx->d_sort) cudaFree(ctx->d_sort);
+    for (void *p : ctx->d_io) if (p) cudaFree(p);
+    for (auto &h : ctx->hs) {
+        if (h.p) cudaFreeHost(h.p);
+        if (h.done) cudaEventDestroy(h.done);
+    }
     if (ctx->d_status) cudaFree(ctx->d_status);
     for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : ctx->free_events) cudaEventDestroy(e);
@@ -688,6 +702,7 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"copy_l2_hint", &ctx->copy_l2_hint, 0, 1},
         {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 16},
         {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
+        {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
     };
     for (auto &t : tab)
         if (std::strcmp(t.n, name) == 0) { *lo = t.lo; *hi = t.hi; return t.p; }
@@ -884,3 +899,5 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
     if (cudaGetLastError() != cudaSuccess) return LSMKV_ECUDA;
     return LSMKV_OK;
 }
+
+#include "lsmkv_hostio.cuh"

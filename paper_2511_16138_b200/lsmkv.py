@@ -24,6 +24,7 @@ EXPORTS = (
     "lsmkv_launch_count", "lsmkv_set_tuning", "lsmkv_get_tuning", "lsmkv_strerror",
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
+    "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
 )
 ETOOBIG = -5
 STATIC_MAX_QUERIES, STATIC_MAX_CHUNKS = 4096, 262144
@@ -121,6 +122,15 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch_static.argtypes = [C.POINTER(GeomStruct), C.c_int, vp, u32, vp, u64, vp,
                                             vp, C.POINTER(vp), C.POINTER(u64), u32, vp,
                                             C.POINTER(PoolStruct), vp]
+    L.lsmkv_put_batch_host.restype = C.c_int
+    L.lsmkv_put_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, vp, C.POINTER(PoolStruct), u32,
+                                       u64, vp, vp, vp, u64, C.POINTER(u64)]
+    L.lsmkv_probe_batch_host.restype = C.c_int
+    L.lsmkv_probe_batch_host.argtypes = [vp, vp, u32, vp, vp, C.POINTER(RunStruct), u32, vp, vp,
+                                         vp, C.POINTER(u64)]
+    L.lsmkv_decode_batch_host.restype = C.c_int
+    L.lsmkv_decode_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, C.POINTER(vp),
+                                          C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
     L.lsmkv_flush_batch.restype = C.c_int
     L.lsmkv_flush_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp, vp]
     L.lsmkv_merge_runs.restype = C.c_int
@@ -239,6 +249,61 @@ def lsmkv_decode_batch(ctx, stream, n_query, qchunk_off, n_qchunks, hit_chunks, 
     _check(ctx, rc, "lsmkv_decode_batch")
 
 
+def _hptr(x):
+    """host array (numpy, pinned torch tensor) / int / None -> address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    return x.data_ptr()
+
+
+def lsmkv_put_batch_host(ctx, stream, n_req, tokens, seq_off, start_chunk, page_table, pool,
+                         file_id, base_offset, keys_out, vals_out, blob_out, blob_capacity) -> int:
+    """Host buffers in and out (numpy arrays or pinned tensors). Returns the chunk count."""
+    p = _pool(pool)
+    n = C.c_uint64(0)
+    rc = lib().lsmkv_put_batch_host(ctx, _stream(stream), n_req, _hptr(tokens), _hptr(seq_off),
+                                    _hptr(start_chunk), _hptr(page_table),
+                                    C.byref(p) if p is not None else None, file_id, base_offset,
+                                    _hptr(keys_out), _hptr(vals_out), _hptr(blob_out),
+                                    blob_capacity, C.byref(n))
+    _check(ctx, rc, "lsmkv_put_batch_host")
+    return int(n.value)
+
+
+def lsmkv_probe_batch_host(ctx, stream, n_query, tokens, seq_off, runs, hit_chunks_out,
+                           recs_out, keys_out=None) -> int:
+    """runs: device runs (keys, vals, n), newest first; everything else host. Returns the
+    number of query chunks."""
+    n_runs = len(runs)
+    arr = (RunStruct * max(1, n_runs))()
+    for i, (k, v, n) in enumerate(runs):
+        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    total = C.c_uint64(0)
+    rc = lib().lsmkv_probe_batch_host(ctx, _stream(stream), n_query, _hptr(tokens),
+                                      _hptr(seq_off), arr, n_runs, _hptr(hit_chunks_out),
+                                      _hptr(recs_out), _hptr(keys_out), C.byref(total))
+    _check(ctx, rc, "lsmkv_probe_batch_host")
+    return int(total.value)
+
+
+def lsmkv_decode_batch_host(ctx, stream, n_query, qchunk_off, hit_chunks, recs, arenas,
+                            dst_page_table, pool) -> None:
+    """arenas: sequence of (host base, n_bytes) indexed by file_id; all arrays host."""
+    n = len(arenas)
+    bases = (C.c_void_p * max(1, n))(*[_hptr(a) for a, _ in arenas])
+    sizes = (C.c_uint64 * max(1, n))(*[b for _, b in arenas])
+    p = _pool(pool)
+    rc = lib().lsmkv_decode_batch_host(ctx, _stream(stream), n_query, _hptr(qchunk_off),
+                                       _hptr(hit_chunks), _hptr(recs), bases, sizes, n,
+                                       _hptr(dst_page_table),
+                                       C.byref(p) if p is not None else None)
+    _check(ctx, rc, "lsmkv_decode_batch_host")
+
+
 def lsmkv_flush_batch(ctx, stream, keys, vals, n, run_keys_out, run_vals_out, n_out) -> None:
     rc = lib().lsmkv_flush_batch(ctx, _stream(stream), _ptr(keys), _ptr(vals), n,
                                  _ptr(run_keys_out), _ptr(run_vals_out), _ptr(n_out))
@@ -355,6 +420,22 @@ class Context:
                      dst_page_table, pool, stream=None):
         lsmkv_decode_batch(self.handle, stream, n_query, qchunk_off, n_qchunks, hit_chunks, recs,
                            arenas, dst_page_table, pool)
+
+    def put_batch_host(self, n_req, tokens, seq_off, start_chunk, page_table, pool, file_id,
+                       base_offset, keys_out, vals_out, blob_out, blob_capacity, stream=None):
+        return lsmkv_put_batch_host(self.handle, stream, n_req, tokens, seq_off, start_chunk,
+                                    page_table, pool, file_id, base_offset, keys_out, vals_out,
+                                    blob_out, blob_capacity)
+
+    def probe_batch_host(self, n_query, tokens, seq_off, runs, hit_chunks_out, recs_out,
+                         keys_out=None, stream=None):
+        return lsmkv_probe_batch_host(self.handle, stream, n_query, tokens, seq_off, runs,
+                                      hit_chunks_out, recs_out, keys_out)
+
+    def decode_batch_host(self, n_query, qchunk_off, hit_chunks, recs, arenas, dst_page_table,
+                          pool, stream=None):
+        lsmkv_decode_batch_host(self.handle, stream, n_query, qchunk_off, hit_chunks, recs,
+                                arenas, dst_page_table, pool)
 
     def flush_batch(self, keys, vals, n, run_keys_out, run_vals_out, n_out, stream=None):
         lsmkv_flush_batch(self.handle, stream, keys, vals, n, run_keys_out, run_vals_out, n_out)
