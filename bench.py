@@ -542,10 +542,12 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
 
 
 def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream, barrier, world):
-    """Same path with HOST buffers: per sub-batch the request descriptors go host->device, the
-    packed blobs, keys and records come back to (pinned) host memory as a tensor-log writer
-    would want them, then the blobs go host->device again and are scattered into the pool; hit
-    lengths come back to the host. The KV pool itself lives on the GPU by nature."""
+    """Same path through the host-buffer entry points of the C ABI: per sub-batch the token
+    sequences and page tables are HOST arrays, the packed blobs, keys and records come back to
+    pinned host memory (where a tensor-log writer would take them), the probe returns hit
+    lengths and records to the host, and the decode copies the hit blobs from the host arena
+    back to the device and scatters them. The KV pool itself lives on the GPU by nature. Two
+    slots on two streams: the put of sub-batch i+1 overlaps the get of sub-batch i."""
     cb = g.chunk_bytes
     sub_cap = 2048                                   # chunks per sub-batch (4 GiB of blobs)
     subs = []
@@ -557,92 +559,94 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
             acc += int(nchw[r])
         subs.append((d, a, len(nchw)))
     max_n = max(int(d["nch"][a:b].sum()) for d, a, b in subs)
-    # two slots, so that the put side of sub-batch i (pack, device->host) overlaps the get side
-    # of sub-batch i-1 (host->device, scatter): PCIe is full duplex
+    max_req = max(b - a for d, a, b in subs)
     NS = 2
-    pin_blob = [torch.empty(max_n * cb, dtype=torch.uint8, pin_memory=True) for _ in range(NS)]
-    pin_keys = [torch.empty(max_n * 32, dtype=torch.uint8, pin_memory=True) for _ in range(NS)]
-    pin_vals = [torch.empty(max_n * 16, dtype=torch.uint8, pin_memory=True) for _ in range(NS)]
-    pin_hit = [torch.empty(4096, dtype=torch.int32, pin_memory=True) for _ in range(NS)]
-    stage = arena if arena.numel() >= 2 * NS * max_n * cb else \
-        torch.empty(2 * NS * max_n * cb, dtype=torch.uint8, device=dev)
-    put_arena = [stage[i * max_n * cb:(i + 1) * max_n * cb] for i in range(NS)]
-    get_arena = [stage[(NS + i) * max_n * cb:(NS + i + 1) * max_n * cb] for i in range(NS)]
+
+    def pin(nbytes):
+        return torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+
+    pin_blob = [pin(max_n * cb) for _ in range(NS)]
+    pin_keys = [pin(max_n * 32) for _ in range(NS)]
+    pin_vals = [pin(max_n * 16) for _ in range(NS)]
+    pin_hit = [pin(max_req * 4) for _ in range(NS)]
+    pin_recs = [pin(max_n * 16) for _ in range(NS)]
     s_put, s_get = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
+    def pinned(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
+
     prepared = []
     for d, a, b in subs:
         h = d["host"]
         t0, t1 = int(h["seq_off"][a]), int(h["seq_off"][b])
         c0, c1 = int(h["coff"][a]), int(h["coff"][b])
-        arrs = dict(tokens=h["tokens"][t0:t1], seq_off=(h["seq_off"][a:b + 1] - h["seq_off"][a]),
-                    coff=(h["coff"][a:b + 1] - h["coff"][a]), src=h["src_pages"][c0:c1],
-                    dst=h["dst_pages"][c0:c1])
-        pins = {k: torch.from_numpy(np.ascontiguousarray(v).view(np.uint8).copy()).pin_memory()
-                for k, v in arrs.items()}
-        devs = {k: torch.empty(max(16, v.numel()), dtype=torch.uint8, device=dev) for k, v in pins.items()}
-        prepared.append([d, b - a, c1 - c0, pins, devs, None])
+        seq_rel = (h["seq_off"][a:b + 1] - h["seq_off"][a]).astype(np.uint64)
+        qoff = (h["coff"][a:b + 1] - h["coff"][a]).astype(np.uint64)
+        p = dict(d=d, n_req=b - a, n=c1 - c0, tokens=pinned(h["tokens"][t0:t1]),
+                 seq_off=pinned(seq_rel), src=pinned(h["src_pages"][c0:c1]),
+                 dst=pinned(h["dst_pages"][c0:c1]), qoff=pinned(qoff), nch=d["nch"][a:b])
+        prepared.append(p)
     # untimed: the index of each sub-batch (its records point into this sub-batch's blobs)
-    keep = []
     for p in prepared:
-        d, n_req, n, pins, devs, _ = p
-        for k in pins:
-            devs[k][:pins[k].numel()].copy_(pins[k])
-        ctx.encode_batch(n_req, devs["tokens"], devs["seq_off"], None, devs["coff"], n, None, None,
-                         0, 0, d["keys"], d["vals"], None, 0, stream=stream)
+        n = p["n"]
+        ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, None, None, 0, 0,
+                           pin_keys[0], pin_vals[0], None, 0, stream=stream)
+        dk = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+        dv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        dk.copy_(pin_keys[0][:n * 32], non_blocking=True)
+        dv.copy_(pin_vals[0][:n * 16], non_blocking=True)
         tk = torch.empty(n * 32, dtype=torch.uint8, device=dev)
         tv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
         tn = torch.zeros(1, dtype=torch.int64, device=dev)
-        ctx.flush_batch(d["keys"], d["vals"], n, tk, tv, tn, stream=stream)
+        ctx.flush_batch(dk, dv, n, tk, tv, tn, stream=stream)
         torch.cuda.synchronize()
-        keep.append((tk, tv, tn))
-        p[5] = [(tk, tv, n)]
-    h2d = d2h = 0
-    moved = 0
-
+        p["run_t"] = (tk, tv, tn)
+        p["runs"] = [(tk, tv, n)]
+    h2d = d2h = moved = 0
     put_done = [torch.cuda.Event() for _ in range(NS)]
     slot_free = [torch.cuda.Event() for _ in range(NS)]
-    step_done = torch.cuda.Event()
 
-    def one_step():
+    def put(i):
+        nonlocal h2d, d2h
+        p, k_ = prepared[i], i % NS
+        s_put.wait_event(slot_free[k_])
+        ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, p["src"], src_pool, 0, 0,
+                           pin_keys[k_], pin_vals[k_], pin_blob[k_], max_n * cb, stream=s_put)
+        put_done[k_].record(s_put)
+        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["src"].numel()
+        d2h += p["n"] * (cb + 48)
+
+    def get(i):
         nonlocal h2d, d2h, moved
-        s_put.wait_event(step_done)          # descriptors of the previous step are still in use
-        for i, (d, n_req, n, pins, devs, runs) in enumerate(prepared):
-            k_ = i % NS
-            # ---- put side: descriptors in, pack, blobs + keys + records out to the host
-            with torch.cuda.stream(s_put):
-                s_put.wait_event(slot_free[k_])
-                for name in pins:
-                    devs[name][:pins[name].numel()].copy_(pins[name], non_blocking=True)
-                    h2d += pins[name].numel()
-                ctx.encode_batch(n_req, devs["tokens"], devs["seq_off"], None, devs["coff"], n,
-                                 devs["src"], src_pool, 0, 0, d["keys"], d["vals"], put_arena[k_],
-                                 n * cb, stream=s_put)
-                pin_blob[k_][:n * cb].copy_(put_arena[k_][:n * cb], non_blocking=True)
-                pin_keys[k_][:n * 32].copy_(d["keys"][:n * 32], non_blocking=True)
-                pin_vals[k_][:n * 16].copy_(d["vals"][:n * 16], non_blocking=True)
-                d2h += n * (cb + 48)
-                put_done[k_].record(s_put)
-            # ---- get side: probe, blobs back in from the host, scatter
-            with torch.cuda.stream(s_get):
-                s_get.wait_event(put_done[k_])
-                ctx.probe_batch(n_req, devs["tokens"], devs["seq_off"], devs["coff"], n, runs,
-                                d["hit"], d["recs"], None, stream=s_get)
-                pin_hit[k_][:n_req].copy_(d["hit"][:n_req], non_blocking=True)
-                d2h += n_req * 4
-                get_arena[k_][:n * cb].copy_(pin_blob[k_][:n * cb], non_blocking=True)
-                h2d += n * cb
-                ctx.decode_batch(n_req, devs["coff"], n, d["hit"], d["recs"],
-                                 [(get_arena[k_], n * cb)], devs["dst"], dst_pool, stream=s_get)
-                slot_free[k_].record(s_get)
-            moved += 2 * n * cb
-        step_done.record(s_get)
+        p, k_ = prepared[i], i % NS
+        n, n_req = p["n"], p["n_req"]
+        s_get.wait_event(put_done[k_])
+        ctx.probe_batch_host(n_req, p["tokens"], p["seq_off"], p["runs"], pin_hit[k_],
+                             pin_recs[k_], None, stream=s_get)
+        s_get.synchronize()                 # the host reads hit lengths and records
+        ctx.decode_batch_host(n_req, p["qoff"], pin_hit[k_], pin_recs[k_],
+                              [(pin_blob[k_], n * cb)], p["dst"], dst_pool, stream=s_get)
+        slot_free[k_].record(s_get)
+        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + n * (cb + 20) + 20
+        d2h += n_req * 4 + n * 16
+        moved += 2 * n * cb
+
+    def one_step(check=False):
+        put(0)
+        for i in range(len(prepared)):
+            if i + 1 < len(prepared):
+                put(i + 1)
+            get(i)
+            if check:
+                hits = pin_hit[i % NS][:prepared[i]["n_req"] * 4].numpy().view(np.uint32)
+                assert np.array_equal(hits, prepared[i]["nch"].astype(np.uint32)), "e2e probe missed"
 
     s_put.wait_stream(stream)
     s_get.wait_stream(stream)
-    one_step()                                      # warm-up (also faults in the pinned pages)
+    one_step(check=True)                    # warm-up (also faults in the pinned pages)
     barrier()
     st = ctx.last_status()
-    assert st["flags"] == 0 and st["chunks_decoded"] == sum(p[2] for p in prepared), st
+    assert st["flags"] == 0 and st["chunks_decoded"] == sum(p["n"] for p in prepared), st
     h2d = d2h = moved = 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -662,9 +666,11 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
     return {"value": ranks.whole_job_rate(moved, ms) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
             "steps": steps, "ms_per_step": ms / steps,
-            "note": "blobs, keys and records copied to pinned host memory and blobs copied back "
-                    "before the scatter; two slots on two streams so device->host and "
-                    "host->device transfers overlap; PCIe-bound"}
+            "api": "lsmkv_put_batch_host / lsmkv_probe_batch_host / lsmkv_decode_batch_host",
+            "note": "host buffers in and out through the C ABI: blobs, keys and records land in "
+                    "pinned host memory, hit blobs are copied back from it before the scatter; "
+                    "put and get sides run on two streams so both PCIe directions are busy; "
+                    "PCIe-bound"}
 
 
 if __name__ == "__main__":

@@ -45,8 +45,8 @@ struct lsmkv_ctx {
     size_t io_cap[3];
     std::vector<uint64_t> h_off_a;
     struct HostScratch { void *p; size_t cap; cudaEvent_t done; bool used; };
-    HostScratch hs[2];
-    int hs_next;
+    HostScratch hs[3][2];
+    int hs_next[3];
     // optional per-kernel timing with CUDA events on the launching stream
     bool profiling;
     struct Timed { cudaEvent_t a, b; int cls; };
@@ -361,10 +361,11 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     if (ctx->d_dir) cudaFree(ctx->d_dir);
     if (ctx->d_sort) cudaFree(ctx->d_sort);
     for (void *p : ctx->d_io) if (p) cudaFree(p);
-    for (auto &h : ctx->hs) {
-        if (h.p) cudaFreeHost(h.p);
-        if (h.done) cudaEventDestroy(h.done);
-    }
+    for (auto &kind : ctx->hs)
+        for (auto &h : kind) {
+            if (h.p) cudaFreeHost(h.p);
+            if (h.done) cudaEventDestroy(h.done);
+        }
     if (ctx->d_status) cudaFree(ctx->d_status);
     for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (auto e : ctx->free_events) cudaEventDestroy(e);

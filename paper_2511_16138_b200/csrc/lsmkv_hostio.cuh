@@ -36,19 +36,21 @@ int ensure_io(lsmkv_ctx *ctx, int kind, size_t bytes)
 
 size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 
-// Pinned host scratch for the small descriptor arrays a call uploads. Two slots alternate
-// between calls; a slot is reused only after the stream work of the call that used it last has
-// finished (its event), so the asynchronous uploads never read rewritten memory.
+// Pinned host scratch for the small descriptor arrays a call uploads. Every kind of call
+// (0 = put, 1 = probe, 2 = decode) alternates between two slots of its own; a slot is reused
+// only after the stream work of the call that used it last has finished (its event), so the
+// asynchronous uploads never read rewritten memory and a put never waits for a get.
 struct ScratchLease {
     lsmkv_ctx *ctx;
     lsmkv_ctx::HostScratch *slot;
     cudaStream_t s;
     unsigned char *p;
     size_t at;
-    ScratchLease(lsmkv_ctx *c, cudaStream_t st, size_t bytes) : ctx(c), slot(nullptr), s(st), p(nullptr), at(0)
+    ScratchLease(lsmkv_ctx *c, int kind, cudaStream_t st, size_t bytes)
+        : ctx(c), slot(nullptr), s(st), p(nullptr), at(0)
     {
-        lsmkv_ctx::HostScratch &h = c->hs[c->hs_next];
-        c->hs_next ^= 1;
+        lsmkv_ctx::HostScratch &h = c->hs[kind][c->hs_next[kind]];
+        c->hs_next[kind] ^= 1;
         if (h.used && h.done) cudaEventSynchronize(h.done);
         if (!h.done && cudaEventCreateWithFlags(&h.done, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
@@ -118,7 +120,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint64_t stage_chunks_max = std::max<uint64_t>(1, (uint64_t)ctx->host_stage_bytes / cb);
-    ScratchLease lease(ctx, s, (4 * (size_t)n_req + 8) * 8 + 64 * (size_t)n_req + 4096);
+    ScratchLease lease(ctx, 0, s, (4 * (size_t)n_req + 8) * 8 + 64 * (size_t)n_req + 4096);
     if (!lease.ok()) return LSMKV_ENOMEM;
     for (uint32_t a = 0; a < n_req;) {
         // slice [a, b): as many requests as fit the blob stage (always at least one)
@@ -205,7 +207,7 @@ extern "C" int lsmkv_probe_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_q
     uint32_t *d_hit = io.take<uint32_t>(n_query);
     lsmkv_val_t *d_recs = io.take<lsmkv_val_t>(total ? total : 1);
     lsmkv_key_t *d_keys = keys_out ? io.take<lsmkv_key_t>(total ? total : 1) : nullptr;
-    ScratchLease lease(ctx, s, (2 * (size_t)n_query + 4) * 8 + 256);
+    ScratchLease lease(ctx, 1, s, (2 * (size_t)n_query + 4) * 8 + 256);
     if (!lease.ok()) return LSMKV_ENOMEM;
     uint64_t *rel = lease.take<uint64_t>((size_t)n_query + 1);
     uint64_t *qo = lease.take<uint64_t>((size_t)n_query + 1);
@@ -267,7 +269,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
     const void *stage_arena[1] = {d_blob};
 
     const uint64_t n_slices = (total_hits + m_max - 1) / m_max;
-    ScratchLease lease(ctx, s, total_hits * 20 + n_slices * 96 + 4096);
+    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices * 96 + 4096);
     if (!lease.ok()) return LSMKV_ENOMEM;
     uint32_t q = 0;
     uint64_t j = 0, left = total_hits;
