@@ -109,6 +109,12 @@ def lib() -> C.CDLL:
                                    C.c_void_p]
         _lib.orc_merge_runs.restype = C.c_int64
         _lib.orc_merge_runs.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        _lib.orc_bloom_blocks.restype = C.c_uint64
+        _lib.orc_bloom_blocks.argtypes = [C.c_uint64]
+        _lib.orc_bloom_build.restype = None
+        _lib.orc_bloom_build.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_bloom_may_contain.restype = C.c_int
+        _lib.orc_bloom_may_contain.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         _lib.orc_probe_batch.restype = C.c_int
         _lib.orc_probe_batch.argtypes = [
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -241,6 +247,23 @@ def merge_runs(runs):
     if m < 0:
         raise OracleError(int(m))
     return ko[:m].copy(), vo[:m].copy()
+
+
+def bloom_blocks(n: int) -> int:
+    return int(lib().orc_bloom_blocks(n))
+
+
+def bloom_build(keys) -> np.ndarray:
+    """Bloom filter bytes (32 per block) of a set of keys."""
+    keys = _arr(keys, np.uint64).reshape(-1, 4)
+    out = np.zeros(32 * bloom_blocks(len(keys)), dtype=np.uint8)
+    lib().orc_bloom_build(_p(keys), len(keys), _p(out))
+    return out
+
+
+def bloom_may_contain(bloom: np.ndarray, key) -> bool:
+    key = _arr(key, np.uint64)
+    return bool(lib().orc_bloom_may_contain(_p(bloom), bloom.size // 32, _p(key)))
 
 
 def probe_batch(g: Geom, tokens, seq_off, qchunk_off, runs, want_keys: bool = False):

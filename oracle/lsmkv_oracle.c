@@ -266,6 +266,49 @@ int64_t orc_merge_runs(const orc_run *runs, uint32_t n_runs, orc_key *keys_out,
     return m;
 }
 
+/* ---- Bloom filter of a run (Sec. 2.2 "Point Lookups", App. B "Probe": filters let a lookup skip
+ * runs that cannot hold the key). Result-neutral: a filter may say "maybe" for an absent key but
+ * never "no" for a present one.
+ *
+ * Format (this build's): blocked filter, blocks of 256 bits (32 bytes), 10 bits per key:
+ *   n_blocks = max(1, ceil(10 * n / 256));   block(key) = floor(w1 * n_blocks / 2^61)
+ *   six bits per key inside its block, at positions (w2 >> 8i) & 255 for i = 0..5;
+ *   position p is bit (p & 7) of byte (p >> 3) of the block.
+ */
+uint64_t orc_bloom_blocks(uint64_t n)
+{
+    const uint64_t b = (10 * n + 255) / 256;
+    return b ? b : 1;
+}
+
+static uint64_t bloom_block_of(const orc_key *k, uint64_t n_blocks)
+{
+    return (uint64_t)(((unsigned __int128)k->w[1] * n_blocks) >> 61);
+}
+
+void orc_bloom_build(const orc_key *keys, uint64_t n, uint8_t *bloom /* 32 * orc_bloom_blocks(n) */)
+{
+    const uint64_t nb = orc_bloom_blocks(n);
+    memset(bloom, 0, nb * 32);
+    for (uint64_t i = 0; i < n; ++i) {
+        uint8_t *blk = bloom + 32 * bloom_block_of(&keys[i], nb);
+        for (int t = 0; t < 6; ++t) {
+            const unsigned p = (unsigned)((keys[i].w[2] >> (8 * t)) & 255u);
+            blk[p >> 3] |= (uint8_t)(1u << (p & 7u));
+        }
+    }
+}
+
+int orc_bloom_may_contain(const uint8_t *bloom, uint64_t n_blocks, const orc_key *key)
+{
+    const uint8_t *blk = bloom + 32 * bloom_block_of(key, n_blocks);
+    for (int t = 0; t < 6; ++t) {
+        const unsigned p = (unsigned)((key->w[2] >> (8 * t)) & 255u);
+        if (!(blk[p >> 3] & (1u << (p & 7u)))) return 0;
+    }
+    return 1;
+}
+
 /* ---- probe: longest cached prefix, first-miss rule ---------------------------------- */
 
 /*
