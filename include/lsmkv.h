@@ -77,11 +77,15 @@ typedef struct {
     uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens must equal page_tokens; flags = 0 */
 } lsmkv_geom_t;
 
-/* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i]. */
+/* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i].
+ * bloom (optional, NULL = none): the run's Bloom filter as built by lsmkv_bloom_build, with
+ * bloom_blocks 32-byte blocks; the probe then skips the run for keys the filter rules out. */
 typedef struct {
     const lsmkv_key_t *keys; /* [dev] */
     const lsmkv_val_t *vals; /* [dev] */
     uint64_t n;
+    const void *bloom;       /* [dev] or NULL */
+    uint64_t bloom_blocks;
 } lsmkv_run_t;
 
 /* The paged KV pool. */
@@ -201,6 +205,20 @@ int lsmkv_flush_batch(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys,
  */
 int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint32_t n_runs,
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
+
+/*
+ * Bloom filter of a run (Sec. 2.2 "Point Lookups", App. B "Probe": filters rule out runs that
+ * cannot hold a key). Result-neutral: probes return the same answers with or without it.
+ * Format: blocks of 256 bits; lsmkv_bloom_blocks(n) = max(1, ceil(10 n / 256)) blocks for n keys;
+ * a key goes to block floor(w1 * n_blocks / 2^61) and sets the six bits at positions
+ * (w2 >> 8i) & 255, i = 0..5 (position p = bit p&7 of byte p>>3 of the block). Entries whose
+ * w1 is not a digest (the all-ones padding of a flushed run) are ignored.
+ * lsmkv_bloom_build: keys [dev, n entries] -> bloom_out [dev, 32 * lsmkv_bloom_blocks(n) bytes,
+ * 16-byte aligned], cleared and filled on `stream`.
+ */
+uint64_t lsmkv_bloom_blocks(uint64_t n);
+int lsmkv_bloom_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uint64_t n,
+                      void *bloom_out);
 
 /*
  * Host-buffer variants (the form the paper's service interface has: token sequences and

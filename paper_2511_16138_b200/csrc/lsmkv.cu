@@ -450,9 +450,13 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
         if (runs[r].n && (!runs[r].keys || !runs[r].vals || !aligned16(runs[r].keys) ||
                           !aligned16(runs[r].vals)))
             return LSMKV_EINVAL;
+        if (runs[r].bloom && (runs[r].bloom_blocks == 0 || !aligned16(runs[r].bloom)))
+            return LSMKV_EINVAL;
         rt.keys[r] = runs[r].keys;
         rt.vals[r] = runs[r].vals;
         rt.n[r] = runs[r].n;
+        rt.bloom[r] = runs[r].n ? static_cast<const uint32_t *>(runs[r].bloom) : nullptr;
+        rt.bloom_blocks[r] = runs[r].bloom_blocks;
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -642,6 +646,30 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
     CU(ctx, cudaGetLastError());
     return launch_dedupe(ctx, s, ws, buf, total, ws.vals, /*keep_last=*/0, keys_out, vals_out,
                          n_out);
+}
+
+uint64_t lsmkv_bloom_blocks(uint64_t n)
+{
+    const uint64_t b = (10 * n + 255) / 256;
+    return b ? b : 1;
+}
+
+int lsmkv_bloom_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uint64_t n,
+                      void *bloom_out)
+{
+    if (!ctx || !bloom_out || !aligned16(bloom_out) || (n && (!keys || !aligned16(keys))))
+        return LSMKV_EINVAL;
+    if (n > (UINT64_MAX - 255) / 10) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t nb = lsmkv_bloom_blocks(n);
+    CU(ctx, cudaMemsetAsync(bloom_out, 0, nb * 32, s));
+    if (n) {
+        k_bloom_build<<<merge_grid(ctx, n), 256, 0, s>>>(keys, n, static_cast<uint32_t *>(bloom_out), nb);
+        ++ctx->launches;
+        CU(ctx, cudaGetLastError());
+    }
+    return LSMKV_OK;
 }
 
 int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out)

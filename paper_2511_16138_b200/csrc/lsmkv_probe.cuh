@@ -22,7 +22,43 @@ struct RunTable {
     const lsmkv_key_t *keys[LSMKV_MAX_RUNS];
     const lsmkv_val_t *vals[LSMKV_MAX_RUNS];
     uint64_t n[LSMKV_MAX_RUNS];
+    const uint32_t *bloom[LSMKV_MAX_RUNS];     // optional Bloom filter, 8 words per block
+    uint64_t bloom_blocks[LSMKV_MAX_RUNS];
 };
+
+constexpr uint64_t kDigestLimit = 1ull << 61;  // digests are < 2^61 - 1; padding keys are not
+
+// Bloom filter of a run: block floor(w1 * n_blocks / 2^61), six bits at (w2 >> 8i) & 255.
+__global__ void __launch_bounds__(256)
+k_bloom_build(const lsmkv_key_t *__restrict__ keys, uint64_t n, uint32_t *__restrict__ bloom,
+              uint64_t n_blocks)
+{
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(
+            reinterpret_cast<const unsigned long long *>(keys + i) + 1);   // w1, w2
+        if (a.x >= kDigestLimit) continue;                                  // padding entry
+        uint32_t *blk = bloom + 8ull * __umul64hi(a.x << 3, n_blocks);
+#pragma unroll
+        for (int t = 0; t < 6; ++t) {
+            const uint32_t p = (uint32_t)(a.y >> (8 * t)) & 255u;
+            atomicOr(blk + (p >> 5), 1u << (p & 31u));
+        }
+    }
+}
+
+__device__ __forceinline__ bool bloom_may_contain(const uint32_t *bloom, uint64_t n_blocks,
+                                                  const ChunkKey &k)
+{
+    const uint32_t *blk = bloom + 8ull * __umul64hi(k.w1 << 3, n_blocks);
+    bool ok = true;
+#pragma unroll
+    for (int t = 0; t < 6; ++t) {
+        const uint32_t p = (uint32_t)(k.w2 >> (8 * t)) & 255u;
+        ok = ok && ((__ldg(blk + (p >> 5)) >> (p & 31u)) & 1u);
+    }
+    return ok;
+}
 
 __device__ __forceinline__ uint64_t key_w(const lsmkv_key_t *e, int i)
 {
@@ -138,6 +174,7 @@ __device__ __forceinline__ bool lookup_runs(const RunTable &rt, uint32_t n_runs,
     const uint64_t j = k.w0 & 0xFFFFFFFFull;
     const uint64_t stride = (uint64_t)jcap + 1;
     for (uint32_t r = 0; r < n_runs; ++r) {
+        if (rt.bloom[r] && !bloom_may_contain(rt.bloom[r], rt.bloom_blocks[r], k)) continue;
         const lsmkv_key_t *keys = rt.keys[r];
         uint64_t lo, hi;
         if (j < jcap) {

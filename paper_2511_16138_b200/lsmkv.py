@@ -25,6 +25,7 @@ EXPORTS = (
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
+    "lsmkv_bloom_blocks", "lsmkv_bloom_build",
 )
 ETOOBIG = -5
 STATIC_MAX_QUERIES, STATIC_MAX_CHUNKS = 4096, 262144
@@ -48,7 +49,18 @@ class GeomStruct(C.Structure):
 
 
 class RunStruct(C.Structure):
-    _fields_ = [("keys", C.c_void_p), ("vals", C.c_void_p), ("n", C.c_uint64)]
+    _fields_ = [("keys", C.c_void_p), ("vals", C.c_void_p), ("n", C.c_uint64),
+                ("bloom", C.c_void_p), ("bloom_blocks", C.c_uint64)]
+
+
+def _run_array(runs):
+    """runs: sequence of (keys, vals, n) or (keys, vals, n, bloom, bloom_blocks)."""
+    arr = (RunStruct * max(1, len(runs)))()
+    for i, r in enumerate(runs):
+        arr[i].keys, arr[i].vals, arr[i].n = _ptr(r[0]), _ptr(r[1]), r[2]
+        if len(r) > 3 and r[3] is not None:
+            arr[i].bloom, arr[i].bloom_blocks = _ptr(r[3]), r[4]
+    return arr
 
 
 class PoolStruct(C.Structure):
@@ -131,6 +143,10 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch_host.restype = C.c_int
     L.lsmkv_decode_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, C.POINTER(vp),
                                           C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
+    L.lsmkv_bloom_blocks.restype = u64
+    L.lsmkv_bloom_blocks.argtypes = [u64]
+    L.lsmkv_bloom_build.restype = C.c_int
+    L.lsmkv_bloom_build.argtypes = [vp, vp, vp, u64, vp]
     L.lsmkv_flush_batch.restype = C.c_int
     L.lsmkv_flush_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp, vp]
     L.lsmkv_merge_runs.restype = C.c_int
@@ -227,9 +243,7 @@ def lsmkv_probe_batch(ctx, stream, n_query, tokens, seq_off, qchunk_off, n_qchun
                       hit_chunks_out, recs_out, keys_out=None) -> None:
     """runs: sequence of (keys, vals, n), newest first."""
     n_runs = len(runs)
-    arr = (RunStruct * max(1, n_runs))()
-    for i, (k, v, n) in enumerate(runs):
-        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    arr = _run_array(runs)
     rc = lib().lsmkv_probe_batch(ctx, _stream(stream), n_query, _ptr(tokens), _ptr(seq_off),
                                  _ptr(qchunk_off), n_qchunks, arr, n_runs,
                                  _ptr(hit_chunks_out), _ptr(recs_out), _ptr(keys_out))
@@ -279,9 +293,7 @@ def lsmkv_probe_batch_host(ctx, stream, n_query, tokens, seq_off, runs, hit_chun
     """runs: device runs (keys, vals, n), newest first; everything else host. Returns the
     number of query chunks."""
     n_runs = len(runs)
-    arr = (RunStruct * max(1, n_runs))()
-    for i, (k, v, n) in enumerate(runs):
-        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    arr = _run_array(runs)
     total = C.c_uint64(0)
     rc = lib().lsmkv_probe_batch_host(ctx, _stream(stream), n_query, _hptr(tokens),
                                       _hptr(seq_off), arr, n_runs, _hptr(hit_chunks_out),
@@ -304,6 +316,15 @@ def lsmkv_decode_batch_host(ctx, stream, n_query, qchunk_off, hit_chunks, recs, 
     _check(ctx, rc, "lsmkv_decode_batch_host")
 
 
+def lsmkv_bloom_blocks(n: int) -> int:
+    return int(lib().lsmkv_bloom_blocks(n))
+
+
+def lsmkv_bloom_build(ctx, stream, keys, n, bloom_out) -> None:
+    _check(ctx, lib().lsmkv_bloom_build(ctx, _stream(stream), _ptr(keys), n, _ptr(bloom_out)),
+           "lsmkv_bloom_build")
+
+
 def lsmkv_flush_batch(ctx, stream, keys, vals, n, run_keys_out, run_vals_out, n_out) -> None:
     rc = lib().lsmkv_flush_batch(ctx, _stream(stream), _ptr(keys), _ptr(vals), n,
                                  _ptr(run_keys_out), _ptr(run_vals_out), _ptr(n_out))
@@ -313,9 +334,7 @@ def lsmkv_flush_batch(ctx, stream, keys, vals, n, run_keys_out, run_vals_out, n_
 def lsmkv_merge_runs(ctx, stream, runs, keys_out, vals_out, n_out) -> None:
     """runs: sequence of (keys, vals, n), newest first."""
     n_runs = len(runs)
-    arr = (RunStruct * max(1, n_runs))()
-    for i, (k, v, n) in enumerate(runs):
-        arr[i].keys, arr[i].vals, arr[i].n = _ptr(k), _ptr(v), n
+    arr = _run_array(runs)
     rc = lib().lsmkv_merge_runs(ctx, _stream(stream), arr, n_runs, _ptr(keys_out),
                                 _ptr(vals_out), _ptr(n_out))
     _check(ctx, rc, "lsmkv_merge_runs")
@@ -436,6 +455,9 @@ class Context:
                           pool, stream=None):
         lsmkv_decode_batch_host(self.handle, stream, n_query, qchunk_off, hit_chunks, recs,
                                 arenas, dst_page_table, pool)
+
+    def bloom_build(self, keys, n, bloom_out, stream=None):
+        lsmkv_bloom_build(self.handle, stream, keys, n, bloom_out)
 
     def flush_batch(self, keys, vals, n, run_keys_out, run_vals_out, n_out, stream=None):
         lsmkv_flush_batch(self.handle, stream, keys, vals, n, run_keys_out, run_vals_out, n_out)
