@@ -510,20 +510,31 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
         d_tok, d_off, d_qoff = up(w.query.tokens), up(w.query.seq_off), up(qoff)
         d_hit = torch.zeros(w.query.n, dtype=torch.int32, device=dev)
         d_recs = torch.empty(total * 16, dtype=torch.uint8, device=dev)
-        for _ in range(max(3, warmup)):
-            ctx.probe_batch(w.query.n, d_tok, d_off, d_qoff, total, runs, d_hit, d_recs, None)
-        torch.cuda.synchronize()
-        assert np.array_equal(d_hit.cpu().numpy(), w.expected_hit.astype(np.int32))
-        ctx.last_status()
-        reps = max(5, steps)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
-            ctx.probe_batch(w.query.n, d_tok, d_off, d_qoff, total, runs, d_hit, d_recs, None)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / reps
-        st = ctx.last_status()
+        # the same runs with their Bloom filters attached
+        runs_bloom = []
+        for (tk, tv, m_) in runs:
+            nb = lsmkv.lsmkv_bloom_blocks(m_)
+            bl = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+            ctx.bloom_build(tk, m_, bl)
+            runs_bloom.append((tk, tv, m_, bl, nb))
+
+        def timed(rr):
+            for _ in range(max(3, warmup)):
+                ctx.probe_batch(w.query.n, d_tok, d_off, d_qoff, total, rr, d_hit, d_recs, None)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_hit.cpu().numpy(), w.expected_hit.astype(np.int32))
+            ctx.last_status()
+            reps = max(5, steps)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                ctx.probe_batch(w.query.n, d_tok, d_off, d_qoff, total, rr, d_hit, d_recs, None)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps, ctx.last_status(), reps
+
+        ms_plain, _, _ = timed(runs)
+        ms, st, reps = timed(runs_bloom)
         hit_tokens = int(w.expected_hit.sum()) * 16
         # least traffic any probe must do: tokens up to the first miss, one record per query
         # chunk, one hit length per query
@@ -531,6 +542,8 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
         return {"workload": "configs[2]: 1M stored chunk keys in 4 sorted runs, 4096 queries of "
                             "2k-32k tokens, 60% cached",
                 "ms_per_probe": ms, "query_chunks": total, "keys_per_s": total / ms * 1e3,
+                "ms_per_probe_without_bloom_filters": ms_plain,
+                "keys_per_s_without_bloom_filters": total / ms_plain * 1e3,
                 "lookups_per_s": st["lookups"] / reps / ms * 1e3,
                 "hit_chunks_per_s": st["chunks_hit"] / reps / ms * 1e3,
                 "query_tokens": int(len(w.query.tokens)), "stored_keys": n,
