@@ -115,6 +115,25 @@ def lib() -> C.CDLL:
         _lib.orc_bloom_build.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         _lib.orc_bloom_may_contain.restype = C.c_int
         _lib.orc_bloom_may_contain.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_xp12_slab_bound.restype = C.c_uint64
+        _lib.orc_xp12_slab_bound.argtypes = [C.c_uint64]
+        _lib.orc_xp12_dir_bytes.restype = C.c_uint64
+        _lib.orc_xp12_dir_bytes.argtypes = [C.c_void_p]
+        _lib.orc_xp12_chunk_bound.restype = C.c_uint64
+        _lib.orc_xp12_chunk_bound.argtypes = [C.c_void_p]
+        _lib.orc_xp12_slab_encode.restype = C.c_uint64
+        _lib.orc_xp12_slab_encode.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_xp12_slab_decode.restype = C.c_uint64
+        _lib.orc_xp12_slab_decode.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
+        _lib.orc_encode_batch_xp12.restype = C.c_int
+        _lib.orc_encode_batch_xp12.argtypes = [
+            C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint64,
+            C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_decode_batch_xp12.restype = C.c_int
+        _lib.orc_decode_batch_xp12.argtypes = [
+            C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+            C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         _lib.orc_probe_batch.restype = C.c_int
         _lib.orc_probe_batch.argtypes = [
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -301,5 +320,74 @@ def decode_batch(g: Geom, qchunk_off, hit, recs, arenas, dst_page_table, pool) -
     rc = lib().orc_decode_batch(C.byref(gc), len(hit), _p(qchunk_off), _p(hit), _p(recs), aptr,
                                 _p(abytes), len(arenas), _p(dst_page_table), ptrs,
                                 pool.shape[1])
+    if rc != OK:
+        raise OracleError(rc)
+
+
+# ---- compressing codec "xp12" ----------------------------------------------------------------
+
+def xp12_slab_encode(elems) -> np.ndarray:
+    """Compressed bytes of one slab of 16-bit elements."""
+    e = _arr(elems, np.uint16)
+    out = np.zeros(int(lib().orc_xp12_slab_bound(e.size)), dtype=np.uint8)
+    n = lib().orc_xp12_slab_encode(_p(e), e.size, _p(out))
+    return out[:n].copy()
+
+
+def xp12_slab_decode(blob, n_elems: int):
+    """Decoded 16-bit elements of one slab, or None if the bytes are malformed."""
+    b = _arr(blob, np.uint8)
+    out = np.zeros(n_elems, dtype=np.uint16)
+    used = lib().orc_xp12_slab_decode(_p(b), b.size, n_elems, _p(out))
+    return out if used else None
+
+
+def xp12_chunk_bound(g: Geom) -> int:
+    gc = g.c()
+    return int(lib().orc_xp12_chunk_bound(C.byref(gc)))
+
+
+def xp12_dir_bytes(g: Geom) -> int:
+    gc = g.c()
+    return int(lib().orc_xp12_dir_bytes(C.byref(gc)))
+
+
+def encode_batch_xp12(g: Geom, tokens, seq_off, start_chunk, chunk_off, page_table, pool,
+                      file_id: int, base_offset: int):
+    """Returns (keys, vals, blob bytes actually used)."""
+    tokens = _arr(tokens, np.uint32)
+    seq_off = _arr(seq_off, np.uint64)
+    chunk_off = _arr(chunk_off, np.uint64)
+    start_chunk = None if start_chunk is None else _arr(start_chunk, np.uint32)
+    page_table = _arr(page_table, np.uint32)
+    n_req = len(seq_off) - 1
+    n_chunks = int(chunk_off[-1]) if n_req else 0
+    keys = np.zeros((n_chunks, 4), dtype=np.uint64)
+    vals = np.zeros(n_chunks, dtype=VAL_DTYPE)
+    cap = n_chunks * xp12_chunk_bound(g)
+    blob = np.zeros(max(16, cap), dtype=np.uint8)
+    used = C.c_uint64(0)
+    gc = g.c()
+    rc = lib().orc_encode_batch_xp12(C.byref(gc), n_req, _p(tokens), _p(seq_off),
+                                     _p(start_chunk), _p(chunk_off), n_chunks, _p(page_table),
+                                     _pool_ptrs(pool), pool.shape[1], file_id, base_offset,
+                                     _p(keys), _p(vals), _p(blob), cap, C.byref(used))
+    if rc != OK:
+        raise OracleError(rc)
+    return keys, vals, blob[:used.value].copy()
+
+
+def decode_batch_xp12(g: Geom, qchunk_off, hit, recs, arenas, dst_page_table, pool) -> None:
+    qchunk_off = _arr(qchunk_off, np.uint64)
+    hit = _arr(hit, np.uint32)
+    recs = np.ascontiguousarray(recs, dtype=VAL_DTYPE)
+    dst_page_table = _arr(dst_page_table, np.uint32)
+    arenas = [np.ascontiguousarray(a, dtype=np.uint8) for a in arenas]
+    aptr = (C.c_void_p * max(1, len(arenas)))(*[a.ctypes.data for a in arenas])
+    abytes = np.array([a.size for a in arenas], dtype=np.uint64)
+    gc = g.c()
+    rc = lib().orc_decode_batch_xp12(C.byref(gc), len(hit), _p(qchunk_off), _p(hit), _p(recs),
+                                     aptr, _p(abytes), len(arenas), _p(dst_page_table),
+                                     _pool_ptrs(pool), pool.shape[1])
     if rc != OK:
         raise OracleError(rc)

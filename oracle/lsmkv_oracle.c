@@ -386,3 +386,183 @@ int orc_decode_batch(const orc_geom *g, uint32_t n_query, const uint64_t *qchunk
     }
     return ORC_OK;
 }
+
+/* ---- compressing batch codec "xp12" (Sec. 3.4 "Batch Codec Operations": the combined tensors
+ * of a batch are compressed before storage and decompressed together on load). The paper names
+ * no algorithm; this build's is lossless, so restored pages stay bit-exact: bf16 values are
+ * split into a sign+mantissa byte and an exponent, and the exponents of a page slab, which
+ * cluster in a narrow window below the slab's largest, are stored in 4 bits each.
+ *
+ * One slab of N 16-bit elements v = (s << 15) | (e << 7) | m  (N a multiple of 8):
+ *   e_max = largest e in the slab; base = max(0, e_max - 14); code = e - base if
+ *   base <= e <= base + 14, else 15 ("exception").  n_exc = number of exceptions.
+ *   mode 0 (packed), used when n_exc < N / 2:
+ *     [0..16)        header: u32 magic 0x32315058, u32 n_exc, u8 base, u8 mode, u16 0, u32 size
+ *     [16..16+N)     byte i = (s_i << 7) | m_i
+ *     [.. +N/2)      nibble codes, element i in byte i/2, even i in the low nibble
+ *     [.. +n_exc)    the raw e of every exception, in element order
+ *     zero padding to a multiple of 16; size = that total
+ *   mode 1 (raw), otherwise: the same header with n_exc = 0, base = 0, then the 2N raw bytes.
+ * One chunk: a directory of 2L+1 u32 (byte offset of every slab inside the chunk blob, last =
+ * the blob's size; zero-padded to a multiple of 16), then the slabs in blob order (K0 V0 K1 ...).
+ * Record of a chunk: {file_id, reserved = blob size, offset}; blobs are placed back to back.
+ */
+#define ORC_XP_MAGIC 0x32315058u
+
+static uint64_t round16(uint64_t x) { return (x + 15) & ~(uint64_t)15; }
+
+uint64_t orc_xp12_slab_bound(uint64_t n_elems) { return 16 + 2 * n_elems; }
+
+uint64_t orc_xp12_dir_bytes(const orc_geom *g) { return round16(4ull * (2ull * g->n_layers + 1)); }
+
+/* Returns the encoded size; out needs orc_xp12_slab_bound(n) bytes. */
+uint64_t orc_xp12_slab_encode(const uint16_t *in, uint64_t n, uint8_t *out)
+{
+    unsigned e_max = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const unsigned e = (in[i] >> 7) & 0xFF;
+        if (e > e_max) e_max = e;
+    }
+    const unsigned base = e_max > 14 ? e_max - 14 : 0;
+    uint64_t n_exc = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const unsigned e = (in[i] >> 7) & 0xFF;
+        if (e < base) ++n_exc;                 /* e > base + 14 cannot happen: base + 14 >= e_max */
+    }
+    uint32_t hdr[4] = {ORC_XP_MAGIC, 0, 0, 0};
+    uint64_t size;
+    if (n_exc < n / 2) {
+        size = round16(16 + n + n / 2 + n_exc);
+        memset(out, 0, size);
+        uint8_t *sm = out + 16, *codes = sm + n, *exc = codes + n / 2;
+        uint64_t k = 0;
+        for (uint64_t i = 0; i < n; ++i) {
+            const unsigned v = in[i], e = (v >> 7) & 0xFF;
+            sm[i] = (uint8_t)(((v >> 15) << 7) | (v & 0x7F));
+            unsigned code = 15;
+            if (e >= base) code = e - base; else exc[k++] = (uint8_t)e;
+            codes[i / 2] |= (uint8_t)(code << (4 * (i & 1)));
+        }
+        hdr[1] = (uint32_t)n_exc;
+        hdr[2] = base;                         /* base in byte 8, mode 0 in byte 9 */
+    } else {
+        size = 16 + 2 * n;
+        memcpy(out + 16, in, 2 * n);
+        hdr[2] = 1u << 8;                      /* mode 1 */
+    }
+    hdr[3] = (uint32_t)size;
+    memcpy(out, hdr, 16);
+    return size;
+}
+
+/* Returns the number of bytes consumed, or 0 if the slab is malformed. */
+uint64_t orc_xp12_slab_decode(const uint8_t *in, uint64_t avail, uint64_t n, uint16_t *out)
+{
+    uint32_t hdr[4];
+    if (avail < 16) return 0;
+    memcpy(hdr, in, 16);
+    const unsigned base = hdr[2] & 0xFF, mode = (hdr[2] >> 8) & 0xFF;
+    const uint64_t n_exc = hdr[1], size = hdr[3];
+    if (hdr[0] != ORC_XP_MAGIC || size > avail) return 0;
+    if (mode == 1) {
+        if (size != 16 + 2 * n) return 0;
+        memcpy(out, in + 16, 2 * n);
+        return size;
+    }
+    if (mode != 0 || size != round16(16 + n + n / 2 + n_exc)) return 0;
+    const uint8_t *sm = in + 16, *codes = sm + n, *exc = codes + n / 2;
+    uint64_t k = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const unsigned code = (codes[i / 2] >> (4 * (i & 1))) & 15;
+        unsigned e;
+        if (code == 15) { if (k >= n_exc) return 0; e = exc[k++]; } else e = base + code;
+        out[i] = (uint16_t)(((sm[i] >> 7) << 15) | (e << 7) | (sm[i] & 0x7F));
+    }
+    return k == n_exc ? size : 0;
+}
+
+/*
+ * put_batch with the compressing codec: as orc_encode_batch, but every chunk's blob is the
+ * directory + compressed slabs, blobs are placed back to back from blob_out (which needs
+ * n_chunks * orc_xp12_chunk_bound bytes), and records carry the blob size in `reserved`.
+ * *blob_bytes_out = total bytes written.
+ */
+uint64_t orc_xp12_chunk_bound(const orc_geom *g)
+{
+    return orc_xp12_dir_bytes(g) + 2ull * g->n_layers * orc_xp12_slab_bound(orc_page_bytes(g) / 2);
+}
+
+int orc_encode_batch_xp12(const orc_geom *g, uint32_t n_req, const uint32_t *tokens,
+                          const uint64_t *seq_off, const uint32_t *start_chunk,
+                          const uint64_t *chunk_off, uint64_t n_chunks,
+                          const uint32_t *page_table, const uint8_t *const *kv_ptrs,
+                          uint64_t num_pages, uint32_t file_id, uint64_t base_offset,
+                          orc_key *keys_out, orc_val *vals_out, uint8_t *blob_out,
+                          uint64_t blob_capacity, uint64_t *blob_bytes_out)
+{
+    if (!geom_ok(g) || g->elem_bytes != 2 || orc_page_bytes(g) % 16) return ORC_EINVAL;
+    /* keys exactly as in the identity codec */
+    int rc = orc_encode_batch(g, n_req, tokens, seq_off, start_chunk, chunk_off, n_chunks, NULL,
+                              NULL, 0, file_id, base_offset, keys_out, vals_out, NULL, 0);
+    if (rc != ORC_OK) return rc;
+    const uint64_t L = g->n_layers, pb = orc_page_bytes(g), ne = pb / 2;
+    const uint64_t dirb = orc_xp12_dir_bytes(g);
+    uint64_t at = 0;
+    for (uint64_t i = 0; i < n_chunks; ++i) {
+        if (blob_capacity - at < orc_xp12_chunk_bound(g)) return ORC_ECAPACITY;
+        const uint64_t page = page_table[i];
+        if (page >= num_pages) return ORC_EBADPAGE;
+        uint8_t *blob = blob_out + at;
+        uint32_t *dir = (uint32_t *)blob;
+        memset(blob, 0, dirb);
+        uint64_t pos = dirb;
+        for (uint64_t b = 0; b < 2 * L; ++b) {          /* blob order: K0 V0 K1 V1 ... */
+            const uint64_t buf = (b & 1) * L + (b >> 1);
+            dir[b] = (uint32_t)pos;
+            pos += orc_xp12_slab_encode((const uint16_t *)(kv_ptrs[buf] + page * pb), ne,
+                                        blob + pos);
+        }
+        dir[2 * L] = (uint32_t)pos;
+        vals_out[i].file_id = file_id;
+        vals_out[i].reserved = (uint32_t)pos;
+        vals_out[i].offset = base_offset + at;
+        at += pos;
+    }
+    if (blob_bytes_out) *blob_bytes_out = at;
+    return ORC_OK;
+}
+
+int orc_decode_batch_xp12(const orc_geom *g, uint32_t n_query, const uint64_t *qchunk_off,
+                          const uint32_t *hit, const orc_val *recs, const uint8_t *const *arenas,
+                          const uint64_t *arena_bytes, uint32_t n_arenas,
+                          const uint32_t *dst_page_table, uint8_t *const *kv_ptrs,
+                          uint64_t num_pages)
+{
+    if (!geom_ok(g) || g->elem_bytes != 2) return ORC_EINVAL;
+    const uint64_t L = g->n_layers, pb = orc_page_bytes(g), ne = pb / 2;
+    const uint64_t dirb = orc_xp12_dir_bytes(g);
+    for (uint32_t q = 0; q < n_query; ++q) {
+        if (hit[q] > qchunk_off[q + 1] - qchunk_off[q]) return ORC_EINVAL;
+        for (uint64_t j = 0; j < hit[q]; ++j) {
+            const uint64_t idx = qchunk_off[q] + j;
+            const orc_val rec = recs[idx];
+            if (rec.file_id >= n_arenas || rec.reserved < dirb) return ORC_EBADREC;
+            if (rec.offset > arena_bytes[rec.file_id] ||
+                arena_bytes[rec.file_id] - rec.offset < rec.reserved) return ORC_EBADREC;
+            const uint64_t page = dst_page_table[idx];
+            if (page >= num_pages) return ORC_EBADPAGE;
+            const uint8_t *blob = arenas[rec.file_id] + rec.offset;
+            const uint32_t *dir = (const uint32_t *)blob;
+            if (dir[2 * L] != rec.reserved) return ORC_EBADREC;
+            for (uint64_t b = 0; b < 2 * L; ++b) {
+                const uint64_t buf = (b & 1) * L + (b >> 1);
+                if (dir[b] < dirb || dir[b] > dir[b + 1] || dir[b + 1] > rec.reserved)
+                    return ORC_EBADREC;
+                if (!orc_xp12_slab_decode(blob + dir[b], dir[b + 1] - dir[b], ne,
+                                          (uint16_t *)(kv_ptrs[buf] + page * pb)))
+                    return ORC_EBADREC;
+            }
+        }
+    }
+    return ORC_OK;
+}
