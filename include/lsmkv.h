@@ -66,6 +66,11 @@ extern "C" {
 #define LSMKV_ST_BAD_COUNT 0x4u    /* chunk_off / qchunk_off / hit disagree with the sequence lengths */
 #define LSMKV_ST_MISALIGNED 0x8u   /* a pool buffer is not 16-byte aligned (skipped) */
 #define LSMKV_ST_WAIT_EXPIRED 0x10u /* a bounded wait inside a kernel gave up */
+#define LSMKV_ST_OVERFLOW 0x20u    /* compressing codec: a blob did not fit blob_capacity (chunk skipped, empty record) */
+
+/* lsmkv_geom_t.flags */
+#define LSMKV_CODEC_IDENTITY 0u    /* blobs are bit copies of the page slabs */
+#define LSMKV_CODEC_XP12 1u        /* lossless exponent packing of 16-bit float slabs (see below) */
 
 typedef struct lsmkv_ctx lsmkv_ctx;
 
@@ -74,7 +79,7 @@ typedef struct { uint32_t file_id, reserved; uint64_t offset; } lsmkv_val_t; /* 
 
 typedef struct {
     uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
-    uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens must equal page_tokens; flags = 0 */
+    uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens must equal page_tokens; flags = LSMKV_CODEC_* */
 } lsmkv_geom_t;
 
 /* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i].
@@ -205,6 +210,29 @@ int lsmkv_flush_batch(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys,
  */
 int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint32_t n_runs,
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
+
+/*
+ * Compressing codec LSMKV_CODEC_XP12 (Sec. 3.4 "Batch Codec Operations": combined tensors are
+ * compressed before storage and decompressed together on load; the paper names no algorithm,
+ * this one is lossless so restored pages stay bit-exact). Selected per context through
+ * lsmkv_geom_t.flags; needs elem_bytes == 2. It changes only blobs and records:
+ *   slab of N 16-bit elements v = s<<15 | e<<7 | m:  base = max(0, e_max - 14);
+ *     16-byte header {u32 0x32315058, u32 n_exc, u8 base, u8 mode, u16 0, u32 size}
+ *     mode 0: N bytes (s<<7 | m), N/2 bytes of 4-bit codes (e - base, 15 = below the window;
+ *             element i in byte i/2, even i in the low nibble), n_exc raw exponent bytes of the
+ *             code-15 elements in element order, zero padding to a multiple of 16
+ *     mode 1 (n_exc >= N/2): the 2N raw bytes
+ *   chunk blob: directory of 2L+1 u32 (byte offset of every slab, then the blob size; padded
+ *     to 16 bytes) followed by the slabs in blob order (K0 V0 K1 V1 ...)
+ *   records: {file_id, reserved = blob size, offset}; blobs are placed back to back, so
+ *     offset = base_offset + sum of the sizes of the chunks before it. Data-dependent: size
+ *     blob_out with lsmkv_encode_bound(); the bytes used are the last record's offset + size
+ *     - base_offset. A chunk that does not fit blob_capacity sets LSMKV_ST_OVERFLOW and gets
+ *     an all-zero-size record.
+ * lsmkv_decode_batch validates every directory entry and slab header (LSMKV_ST_BAD_RECORD).
+ * lsmkv_decode_batch_static supports the identity codec only.
+ */
+uint64_t lsmkv_encode_bound(const lsmkv_ctx *ctx, uint64_t n_chunks); /* worst-case blob bytes */
 
 /*
  * Bloom filter of a run (Sec. 2.2 "Point Lookups", App. B "Probe": filters rule out runs that

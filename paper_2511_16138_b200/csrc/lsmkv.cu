@@ -15,6 +15,7 @@
 #include "lsmkv_keys.cuh"
 #include "lsmkv_probe.cuh"
 #include "lsmkv_sort.cuh"
+#include "lsmkv_xp12.cuh"
 
 using namespace lsmkv;
 
@@ -32,6 +33,11 @@ struct lsmkv_ctx {
     // scratch of flush / compaction (key and index ping-pong buffers, records, block counts)
     void *d_sort;
     uint64_t sort_cap;
+    // compressing codec: 0 = identity, 1 = xp12; scratch of its encoder
+    uint32_t codec;
+    uint32_t xp_dir_bytes;
+    void *d_xp;
+    uint64_t xp_cap;     // chunks
     // fence-pointer directory of the probe: u64[n_runs * (jcap + 1)]
     uint64_t *d_dir;
     uint64_t dir_cap;
@@ -191,6 +197,7 @@ int ensure_sort(lsmkv_ctx *ctx, uint64_t n, SortWs *ws)
         cudaError_t e = cudaMalloc(&p, sort_ws_bytes(n));
         if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
         if (ctx->d_sort) cudaFree(ctx->d_sort);
+    if (ctx->d_xp) cudaFree(ctx->d_xp);
         ctx->d_sort = p;
         ctx->sort_cap = n;
     }
@@ -284,6 +291,54 @@ int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &
     return LSMKV_OK;
 }
 
+// put_batch with the compressing codec: measure slabs, lay blobs out, write them.
+int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_t *page_table,
+                const lsmkv_pool_t *pool, uint32_t file_id, uint64_t base_offset,
+                lsmkv_val_t *vals_out, void *blob_out, uint64_t blob_capacity)
+{
+    const uint64_t slabs = 2ull * ctx->geom.n_layers;
+    if (n_chunks > ctx->xp_cap || !ctx->d_xp) {
+        void *p = nullptr;
+        cudaError_t e = cudaMalloc(&p, (size_t)n_chunks * slabs * 12 + ((size_t)n_chunks + 2) * 8 + 256);
+        if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
+        if (ctx->d_xp) cudaFree(ctx->d_xp);
+        ctx->d_xp = p;
+        ctx->xp_cap = n_chunks;
+    }
+    XpJob job;
+    std::memset(&job, 0, sizeof(job));
+    job.n_layers = ctx->geom.n_layers;
+    job.page_bytes = (uint32_t)ctx->page_bytes;
+    job.n_elems = (uint32_t)(ctx->page_bytes / 2);
+    job.dir_bytes = ctx->xp_dir_bytes;
+    job.num_pages = pool->num_pages;
+    job.kv_ptrs = pool->kv_ptrs;
+    job.page_table = page_table;
+    job.n_chunks = n_chunks;
+    job.chunk_off = static_cast<uint64_t *>(ctx->d_xp);
+    job.slab_size = reinterpret_cast<uint32_t *>(job.chunk_off + ctx->xp_cap + 2);
+    job.slab_info = job.slab_size + ctx->xp_cap * slabs;
+    job.slab_nexc = job.slab_info + ctx->xp_cap * slabs;
+    job.blob = static_cast<unsigned char *>(blob_out);
+    job.blob_capacity = blob_capacity;
+    job.file_id = file_id;
+    job.base_offset = base_offset;
+    job.vals_out = vals_out;
+    job.st = ctx->d_status;
+    LaunchTimer timer(ctx, s, LSMKV_K_PACK);
+    uint64_t grid = n_chunks * slabs;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 8;
+    if (grid > cap) grid = cap;
+    k_xp_measure<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    k_xp_chunk_sizes<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
+    k_scan_blocks<<<1, 1024, 0, s>>>(job.chunk_off, n_chunks, job.chunk_off + n_chunks);
+    k_xp_layout<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
+    k_xp_pack<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    ctx->launches += 5;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
 unsigned warp_grid(const lsmkv_ctx *ctx, uint64_t n_warps_wanted, unsigned threads,
                    unsigned ctas_per_sm)
 {
@@ -303,10 +358,13 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     if (!out || !g) return LSMKV_EINVAL;
     *out = nullptr;
     if (!g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes || !g->page_tokens ||
-        g->chunk_tokens != g->page_tokens || g->flags != 0)
+        g->chunk_tokens != g->page_tokens || g->flags > LSMKV_CODEC_XP12)
         return LSMKV_EINVAL;
     const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
     if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
+    if (g->flags == LSMKV_CODEC_XP12 &&
+        (g->elem_bytes != 2 || 2ull * g->n_layers * (pb + 16) + 8ull * g->n_layers + 16 > 0xFFFFFFF0ull))
+        return LSMKV_EINVAL;
     lsmkv_ctx *ctx = new (std::nothrow) lsmkv_ctx();   // value-initialised: all fields zero
     if (!ctx) return LSMKV_ENOMEM;
     ctx->geom = *g;
@@ -314,6 +372,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->page_bytes = pb;
     ctx->chunk_bytes = 2ull * g->n_layers * pb;
     fill_key_consts(ctx->kc, g->chunk_tokens);
+    ctx->codec = g->flags;
+    ctx->xp_dir_bytes = (uint32_t)((4ull * (2ull * g->n_layers + 1) + 15) & ~15ull);
     ctx->copy_mode = 0;
     ctx->copy_stage_bytes = 16384;
     ctx->copy_stages = 12;
@@ -360,6 +420,7 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
     if (ctx->d_ws) cudaFree(ctx->d_ws);
     if (ctx->d_dir) cudaFree(ctx->d_dir);
     if (ctx->d_sort) cudaFree(ctx->d_sort);
+    if (ctx->d_xp) cudaFree(ctx->d_xp);
     for (void *p : ctx->d_io) if (p) cudaFree(p);
     for (auto &kind : ctx->hs)
         for (auto &h : kind) {
@@ -397,8 +458,12 @@ int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint3
     const bool with_blob = blob_out != nullptr;
     if (with_blob) {
         if (!page_table || !pool || !pool->kv_ptrs || !aligned16(blob_out)) return LSMKV_EINVAL;
-        if (n_chunks > UINT64_MAX / ctx->chunk_bytes) return LSMKV_EINVAL;
-        if (blob_capacity < n_chunks * ctx->chunk_bytes) return LSMKV_ECAPACITY;
+        if (n_chunks > UINT64_MAX / (ctx->chunk_bytes + 65536)) return LSMKV_EINVAL;
+        if (ctx->codec == LSMKV_CODEC_IDENTITY && blob_capacity < n_chunks * ctx->chunk_bytes)
+            return LSMKV_ECAPACITY;
+        if (ctx->codec == LSMKV_CODEC_XP12 &&
+            (blob_capacity < n_chunks * ctx->xp_dir_bytes || (base_offset & 15u)))
+            return LSMKV_ECAPACITY;
     } else if (page_table || pool) {
         return LSMKV_EINVAL;
     }
@@ -416,6 +481,9 @@ int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint3
     ++ctx->launches;
     CU(ctx, cudaGetLastError());
     if (!with_blob) return LSMKV_OK;
+    if (ctx->codec == LSMKV_CODEC_XP12)
+        return encode_xp12(ctx, s, n_chunks, page_table, pool, file_id, base_offset, vals_out,
+                           blob_out, blob_capacity);
 
     CopyJob job;
     std::memset(&job, 0, sizeof(job));
@@ -531,12 +599,35 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
         ++ctx->launches;
         CU(ctx, cudaGetLastError());
         k_plan_fill<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
-            n_query, qchunk_off, hit_off, recs, ar, n_arenas, ctx->chunk_bytes, plan,
-            ctx->d_status);
+            n_query, qchunk_off, hit_off, recs, ar, n_arenas, ctx->chunk_bytes,
+            ctx->codec == LSMKV_CODEC_XP12 ? ctx->xp_dir_bytes + 16u : 0u, plan, ctx->d_status);
         ++ctx->launches;
         CU(ctx, cudaGetLastError());
     }
 
+    if (ctx->codec == LSMKV_CODEC_XP12) {
+        XpUnpackJob uj;
+        std::memset(&uj, 0, sizeof(uj));
+        uj.n_layers = ctx->geom.n_layers;
+        uj.page_bytes = (uint32_t)ctx->page_bytes;
+        uj.n_elems = (uint32_t)(ctx->page_bytes / 2);
+        uj.dir_bytes = ctx->xp_dir_bytes;
+        uj.num_pages = pool->num_pages;
+        uj.kv_ptrs = pool->kv_ptrs;
+        uj.page_table = dst_page_table;
+        uj.n_items_dev = hit_off + n_query;
+        uj.plan = plan;
+        uj.recs = recs;
+        uj.st = ctx->d_status;
+        LaunchTimer timer(ctx, s, LSMKV_K_UNPACK);
+        uint64_t grid = n_qchunks * 2ull * ctx->geom.n_layers;
+        const uint64_t cap = (uint64_t)ctx->sm_count * 8;
+        if (grid > cap) grid = cap;
+        k_xp_unpack<<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        ++ctx->launches;
+        CU(ctx, cudaGetLastError());
+        return LSMKV_OK;
+    }
     CopyJob job;
     std::memset(&job, 0, sizeof(job));
     job.unpack = 1;
@@ -646,6 +737,14 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
     CU(ctx, cudaGetLastError());
     return launch_dedupe(ctx, s, ws, buf, total, ws.vals, /*keep_last=*/0, keys_out, vals_out,
                          n_out);
+}
+
+uint64_t lsmkv_encode_bound(const lsmkv_ctx *ctx, uint64_t n_chunks)
+{
+    if (!ctx) return 0;
+    if (ctx->codec == LSMKV_CODEC_XP12)
+        return n_chunks * (ctx->xp_dir_bytes + 2ull * ctx->geom.n_layers * (16 + ctx->page_bytes));
+    return n_chunks * ctx->chunk_bytes;
 }
 
 uint64_t lsmkv_bloom_blocks(uint64_t n)
@@ -891,7 +990,7 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
         const uint64_t fill_cap = (uint64_t)sd->sm_count * 8;
         if (fill_grid > fill_cap) fill_grid = fill_cap;
         k_plan_fill<<<(unsigned)fill_grid, 256, 0, s>>>(n_query, qchunk_off, hit_off, recs, ar,
-                                                        n_arenas, cb, plan, st);
+                                                        n_arenas, cb, 0u, plan, st);
         CopyJob job;
         std::memset(&job, 0, sizeof(job));
         job.unpack = 1;

@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(256)
 k_plan_fill(uint32_t n_query, const uint64_t *__restrict__ qchunk_off,
             const uint64_t *__restrict__ hit_off, const lsmkv_val_t *__restrict__ recs,
             const __grid_constant__ ArenaTable ar, uint32_t n_arenas, uint64_t chunk_bytes,
-            uint32_t *__restrict__ plan, DevStatus *st)
+            uint32_t min_coded_bytes, uint32_t *__restrict__ plan, DevStatus *st)
 {
     const unsigned lane = lane_id();
     const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -261,8 +261,12 @@ k_plan_fill(uint32_t n_query, const uint64_t *__restrict__ qchunk_off,
             const uint64_t idx = o0 + j;
             const uint4 r = __ldg(reinterpret_cast<const uint4 *>(recs + idx));
             const uint64_t off = (uint64_t)r.z | ((uint64_t)r.w << 32);
+            // identity codec: blobs are chunk_bytes long; compressing codec (min_coded_bytes
+            // != 0): the record carries its blob's size
+            const uint64_t need = min_coded_bytes ? r.y : chunk_bytes;
             bool ok = r.x < n_arenas && (off & 15u) == 0;
-            if (ok) ok = off <= ar.bytes[r.x] && ar.bytes[r.x] - off >= chunk_bytes;
+            if (min_coded_bytes) ok = ok && r.y >= min_coded_bytes && (r.y & 15u) == 0;
+            if (ok) ok = off <= ar.bytes[r.x] && ar.bytes[r.x] - off >= need;
             if (!ok) st_flag(st, LSMKV_ST_BAD_RECORD, idx);
             plan[t0 + j] = ok ? (uint32_t)idx : kSkip;
         }

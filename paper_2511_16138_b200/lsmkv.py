@@ -25,8 +25,10 @@ EXPORTS = (
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
-    "lsmkv_bloom_blocks", "lsmkv_bloom_build",
+    "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound",
 )
+ST_OVERFLOW = 32
+CODEC_IDENTITY, CODEC_XP12 = 0, 1
 ETOOBIG = -5
 STATIC_MAX_QUERIES, STATIC_MAX_CHUNKS = 4096, 262144
 K_KEYS, K_PACK, K_PROBE, K_PLAN, K_UNPACK, K_CLASSES = 0, 1, 2, 3, 4, 8
@@ -143,6 +145,8 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch_host.restype = C.c_int
     L.lsmkv_decode_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, C.POINTER(vp),
                                           C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
+    L.lsmkv_encode_bound.restype = u64
+    L.lsmkv_encode_bound.argtypes = [vp, u64]
     L.lsmkv_bloom_blocks.restype = u64
     L.lsmkv_bloom_blocks.argtypes = [u64]
     L.lsmkv_bloom_build.restype = C.c_int
@@ -316,6 +320,10 @@ def lsmkv_decode_batch_host(ctx, stream, n_query, qchunk_off, hit_chunks, recs, 
     _check(ctx, rc, "lsmkv_decode_batch_host")
 
 
+def lsmkv_encode_bound(ctx, n_chunks: int) -> int:
+    return int(lib().lsmkv_encode_bound(ctx, n_chunks))
+
+
 def lsmkv_bloom_blocks(n: int) -> int:
     return int(lib().lsmkv_bloom_blocks(n))
 
@@ -455,6 +463,9 @@ class Context:
                           pool, stream=None):
         lsmkv_decode_batch_host(self.handle, stream, n_query, qchunk_off, hit_chunks, recs,
                                 arenas, dst_page_table, pool)
+
+    def encode_bound(self, n_chunks: int) -> int:
+        return lsmkv_encode_bound(self.handle, n_chunks)
 
     def bloom_build(self, keys, n, bloom_out, stream=None):
         lsmkv_bloom_build(self.handle, stream, keys, n, bloom_out)

@@ -266,3 +266,51 @@ def gpu_merge_runs(ctx, runs):
     m = int(cnt.item())
     return (host(ok, np.uint64, total * 32).reshape(-1, 4)[:m].copy(),
             host(ov, VAL_DTYPE, total * 16)[:m].copy())
+
+
+def roundtrip_xp12(g: lsmkv.Geom, store, query, seed=0):
+    """Whole path with the compressing codec: encode, flush on the device, probe, decode into a
+    zeroed pool; every output against the oracle's."""
+    og = ogeom(g)
+    rng = np.random.default_rng(seed)
+    C = g.chunk_tokens
+    nch = synth.chunk_counts(store.seq_off, C)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    qoff = synth.offsets(synth.chunk_counts(query.seq_off, C))
+    nq = int(qoff[-1])
+    num_pages = max(n, nq) + 3
+    pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
+    src_pages = synth.random_pages(rng, num_pages, n)
+    dst_pages = synth.random_pages(rng, num_pages, nq)
+    o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, store.tokens, store.seq_off, None, coff,
+                                                      src_pages, pool_np, 0, 0)
+    o_run = oracle.flush(o_keys, o_vals)
+    o_hit, o_recs, _, _ = oracle.probe_batch(og, query.tokens, query.seq_off, qoff, [o_run])
+    o_dst = np.zeros_like(pool_np)
+    oracle.decode_batch_xp12(og, qoff, o_hit, o_recs, [o_blob], dst_pages, o_dst)
+    with lsmkv.Context(g, 0) as ctx:
+        pool = DevPool(g, num_pages, pool_np)
+        bound = ctx.encode_bound(n)
+        d_keys = torch.zeros(n * 32, dtype=torch.uint8, device=DEV)
+        d_vals = torch.zeros(n * 16, dtype=torch.uint8, device=DEV)
+        d_blob = torch.zeros(bound, dtype=torch.uint8, device=DEV)
+        ctx.encode_batch(store.n, dev(store.tokens), dev(store.seq_off), None, dev(coff), n,
+                         dev(src_pages), pool.table, 0, 0, d_keys, d_vals, d_blob, bound)
+        torch.cuda.synchronize()
+        keys = host(d_keys, np.uint64, n * 32).reshape(-1, 4)
+        vals = host(d_vals, VAL_DTYPE, n * 16)
+        assert np.array_equal(keys, o_keys) and np.array_equal(vals, o_vals)
+        used = int(vals["offset"][-1]) + int(vals["reserved"][-1])
+        assert np.array_equal(d_blob[:used].cpu().numpy(), o_blob)
+        run = gpu_flush_run(ctx, keys, vals)
+        assert np.array_equal(run[0], o_run[0]) and np.array_equal(run[1], o_run[1])
+        hit, recs, _, (d_qoff, d_hit, d_recs) = gpu_probe(ctx, query, qoff, [run], want_keys=False)
+        assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
+        dst = DevPool(g, num_pages)
+        ctx.decode_batch(query.n, d_qoff, nq, d_hit, d_recs, [(d_blob, used)], dev(dst_pages),
+                         dst.table)
+        torch.cuda.synchronize()
+        assert np.array_equal(dst.numpy(), o_dst)
+        assert_status_clean(ctx)
+    return dict(hit=o_hit, ratio=used / (n * g.chunk_bytes))
