@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU baseline budget (0 = skip)")
     ap.add_argument("--only-probe-block", action="store_true",
                     help="run just the probe-heavy measurement (a small case for profiling)")
+    ap.add_argument("--no-xp12-block", action="store_true",
+                    help="skip the compressing-codec measurement")
     ap.add_argument("--no-probe-block", action="store_true",
                     help="skip the probe-heavy measurement")
     ap.add_argument("--tuning", default="", help="name=value,... launch-shape knobs")
@@ -385,6 +387,12 @@ def main():
         e2e = run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream,
                       barrier, world)
 
+    # ---- the compressing codec on the first wave (reported beside the identity codec)
+    xp_block = None
+    if rank == 0 and not args.no_xp12_block:
+        xp_block = xp12_block(torch, lsmkv, dev, local_rank, W[0], src_bufs, src_pool, dst_bufs,
+                              dst_pool, arena, stream)
+
     # ---- probe throughput on the probe-heavy workload (second half of the metric)
     probe_block = None
     if rank == 0 and not args.no_probe_block:
@@ -441,6 +449,7 @@ def main():
                          "avg_launch_ms": copy_ms / max(1, copy_launches)},
             "cpu_baseline": cpu,
             "probe": probe_block,
+            "codec_xp12": xp_block,
             "phases": {
                 "pack_GBps_payload": payload * args.steps / (prof["pack"][0] * 1e-3) / 1e9,
                 "unpack_GBps_payload": payload * args.steps / (prof["unpack"][0] * 1e-3) / 1e9,
@@ -550,6 +559,55 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
                 "algorithmic_GBps": algo_bytes / ms / 1e6,
                 "flush_ms_for_%d_keys" % big: flush_big_ms,
                 "bound": "L2 latency / instruction issue (not HBM)"}
+    finally:
+        ctx.close()
+
+
+def xp12_block(torch, lsmkv, dev, device_index, d, src_bufs, src_pool, dst_bufs, dst_pool, arena,
+               stream, reps=3):
+    """The compressing codec (lossless exponent packing) on the first wave of the workload:
+    compression ratio and pack / unpack rates in raw payload bytes per second."""
+    g = lsmkv.Geom(**dict(GEOM, flags=lsmkv.CODEC_XP12))
+    cb = g.chunk_bytes
+    ctx = lsmkv.Context(g, device_index)
+    try:
+        n, n_req = d["n"], d["n_req"]
+        cap = min(arena.numel(), ctx.encode_bound(n))
+        vals = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        hit = torch.from_numpy(d["nch"].astype(np.int32)).to(dev)
+
+        def enc():
+            ctx.encode_batch(n_req, d["tokens"], d["seq_off"], None, d["coff"], n, d["src_pages"],
+                             src_pool, 0, 0, d["keys"], vals, arena, cap, stream=stream)
+
+        def dec():
+            ctx.decode_batch(n_req, d["coff"], n, hit, vals, [(arena, cap)], d["dst_pages"],
+                             dst_pool, stream=stream)
+
+        enc(); dec()
+        torch.cuda.synchronize()
+        st = ctx.last_status()
+        assert st["flags"] == 0, st
+        v = vals.cpu().numpy().view(np.uint64).reshape(-1, 2)
+        used = int(v[-1, 1]) + int(v[-1, 0] >> np.uint64(32))
+        sp = torch.from_numpy(d["host"]["src_pages"][:512].astype(np.int64)).to(dev)
+        dp = torch.from_numpy(d["host"]["dst_pages"][:512].astype(np.int64)).to(dev)
+        for sb, db in zip(src_bufs, dst_bufs):
+            assert torch.equal(sb[sp], db[dp]), "xp12 round trip differs"
+        ctx.profile_enable(True)
+        ctx.profile_read()
+        for _ in range(reps):
+            enc(); dec()
+        torch.cuda.synchronize()
+        prof = ctx.profile_read()
+        pack_ms, unpack_ms = prof["pack"][0] / reps, prof["unpack"][0] / reps
+        return {"codec": "xp12 (lossless bf16 exponent packing)", "chunks": n,
+                "raw_GiB": n * cb / 2**30, "ratio": used / (n * cb),
+                "pack_GBps_raw_payload": n * cb / pack_ms / 1e6,
+                "unpack_GBps_raw_payload": n * cb / unpack_ms / 1e6,
+                "pack_ms": pack_ms, "unpack_ms": unpack_ms,
+                "pack_hbm_GBps_algorithmic": (2 * n * cb + used) / pack_ms / 1e6,
+                "unpack_hbm_GBps_algorithmic": (n * cb + used) / unpack_ms / 1e6}
     finally:
         ctx.close()
 

@@ -365,6 +365,8 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "copy_ctas_per_sm"  1..8        "copy_l2_hint"  0/1 = evict-first L2 policy on the copies
  *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..16
  *   "host_stage_bytes"  blob bytes staged per slice by the host-buffer calls, 1 MiB..64 GiB
+ *   "xp_generic"        1 = compressing codec always uses its generic kernels (0 = fast kernels
+ *                       for slabs of 8192 / 16384 / 32768 elements)
  */
 int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value);
 int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name);

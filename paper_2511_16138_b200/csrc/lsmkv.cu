@@ -45,7 +45,7 @@ struct lsmkv_ctx {
     uint64_t launches;
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
-    int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes;
+    int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
     size_t io_cap[3];
@@ -329,11 +329,20 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
     uint64_t grid = n_chunks * slabs;
     const uint64_t cap = (uint64_t)ctx->sm_count * 8;
     if (grid > cap) grid = cap;
-    k_xp_measure<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    // common slab sizes take the fast kernels (2048 * {4, 8, 16} elements), the rest the generic
+    const uint32_t sweeps = job.n_elems % 2048u == 0 && !ctx->xp_generic ? job.n_elems / 2048u : 0;
+    const size_t list_bytes = job.n_elems;
+    if (sweeps == 4) k_xp_measure_fast<4><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    else if (sweeps == 8) k_xp_measure_fast<8><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    else if (sweeps == 16) k_xp_measure_fast<16><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    else k_xp_measure<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
     k_xp_chunk_sizes<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
     k_scan_blocks<<<1, 1024, 0, s>>>(job.chunk_off, n_chunks, job.chunk_off + n_chunks);
     k_xp_layout<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
-    k_xp_pack<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    if (sweeps == 4) k_xp_pack_fast<4><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
+    else if (sweeps == 8) k_xp_pack_fast<8><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
+    else if (sweeps == 16) k_xp_pack_fast<16><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
+    else k_xp_pack<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
     ctx->launches += 5;
     CU(ctx, cudaGetLastError());
     return LSMKV_OK;
@@ -623,7 +632,11 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
         uint64_t grid = n_qchunks * 2ull * ctx->geom.n_layers;
         const uint64_t cap = (uint64_t)ctx->sm_count * 8;
         if (grid > cap) grid = cap;
-        k_xp_unpack<<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        const uint32_t sweeps = uj.n_elems % 2048u == 0 && !ctx->xp_generic ? uj.n_elems / 2048u : 0;
+        if (sweeps == 4) k_xp_unpack_fast<4><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        else if (sweeps == 8) k_xp_unpack_fast<8><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        else if (sweeps == 16) k_xp_unpack_fast<16><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        else k_xp_unpack<<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
         ++ctx->launches;
         CU(ctx, cudaGetLastError());
         return LSMKV_OK;
@@ -831,6 +844,7 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 16},
         {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
         {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
+        {"xp_generic", &ctx->xp_generic, 0, 1},
     };
     for (auto &t : tab)
         if (std::strcmp(t.n, name) == 0) { *lo = t.lo; *hi = t.hi; return t.p; }

@@ -34,14 +34,19 @@ def mixed_pool(rng, g, num_pages):
                 v[b, p][m] = 0x0001                                          # many exceptions
             elif kind == 4:
                 v[b, p][: n // 2] = 0                                        # exactly half below
-            elif kind == 5:
-                v[b, p] = rng.choice(np.array([0x7F80, 0xFF80, 0x7FC1, 0x8000, 0x3F80], np.uint16), n)
+            elif kind == 5:                                                  # inf / nan: e_max = 255
+                v[b, p] = rng.choice(np.array([0x7F80, 0xFF80, 0x7FC1, 0x8000, 0x3F80, 0x0001,
+                                               0x8001, 0x7F00, 0xFF7F], np.uint16), n)
     return pool
 
 
-@pytest.mark.parametrize("g", [geom(3, 2, 16, 4), geom(2, 8, 128, 16), geom(2, 1, 24, 3),
-                               geom(1, 4, 128, 64)])
-def test_encode_and_decode_equal_the_oracle(g):
+@pytest.mark.parametrize("g,generic", [(geom(3, 2, 16, 4), 0), (geom(2, 8, 128, 16), 0),
+                                       (geom(2, 8, 128, 16), 1), (geom(2, 1, 24, 3), 0),
+                                       (geom(1, 4, 128, 64), 0), (geom(1, 4, 128, 64), 1),
+                                       (geom(2, 8, 64, 16), 0)])
+def test_encode_and_decode_equal_the_oracle(g, generic):
+    """Slabs of 128, 16384, 72, 32768 and 8192 elements: fast kernels where they apply (and the
+    generic ones forced on the same shapes)."""
     og = H.ogeom(g)
     rng = np.random.default_rng(g.page_bytes)
     C = g.chunk_tokens
@@ -56,6 +61,7 @@ def test_encode_and_decode_equal_the_oracle(g):
     o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, b.tokens, b.seq_off, None, coff, pages,
                                                       pool_np, 5, 1024)
     with lsmkv.Context(g, 0) as ctx:
+        ctx.set_tuning("xp_generic", generic)
         bound = ctx.encode_bound(n)
         assert bound == n * oracle.xp12_chunk_bound(og)
         pool = H.DevPool(g, num_pages, pool_np)
