@@ -540,10 +540,13 @@ k_xp_pack_fast(const __grid_constant__ XpJob job)
         const uint32_t base2 = base | (base << 16);
         const uint32_t k_first = warp * SWEEPS * 32 + lane;       // this lane's first uint4
         uint32_t warp_count = 0;
-#pragma unroll 4
+        uint4 qs[SWEEPS];                                         // all loads in flight at once
+#pragma unroll
+        for (int s = 0; s < SWEEPS; ++s) qs[s] = __ldcs(s4 + k_first + s * 32);
+#pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
             const uint32_t k = k_first + s * 32;
-            const uint4 q = __ldcs(s4 + k);
+            const uint4 q = qs[s];
             uint32_t x0, x1, x2, x3;
             const uint32_t c32 = xpfast::code_byte(q.x, base2, x0) |
                                  (xpfast::code_byte(q.y, base2, x1) << 8) |
@@ -634,14 +637,19 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
         const unsigned char *sm = in, *codes = in + N, *exc = codes + N / 2;
         const uint32_t k_first = warp * SWEEPS * 32 + lane;
         const uint32_t base2 = base | (base << 16);
+        uint2 sms[SWEEPS];                                       // all loads in flight at once
+        uint32_t cds[SWEEPS];
+#pragma unroll
+        for (int s = 0; s < SWEEPS; ++s) {
+            sms[s] = __ldcs(reinterpret_cast<const uint2 *>(sm + 8ull * (k_first + s * 32)));
+            cds[s] = __ldcs(reinterpret_cast<const uint32_t *>(codes + 4ull * (k_first + s * 32)));
+        }
         // exceptions before this warp's segment (only when the slab has any)
         uint32_t at_warp = 0;
         if (n_exc) {                                             // uniform over the CTA
             uint32_t mine = 0, mask;
 #pragma unroll
-            for (int s = 0; s < SWEEPS; ++s)
-                mine += xpfast::count_f_nibbles(
-                    __ldg(reinterpret_cast<const uint32_t *>(codes + 4ull * (k_first + s * 32))), mask);
+            for (int s = 0; s < SWEEPS; ++s) mine += xpfast::count_f_nibbles(cds[s], mask);
 #pragma unroll
             for (int d = 16; d; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
             if (lane == 0) warp_total[warp] = mine;
@@ -659,11 +667,11 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
                 continue;
             }
         }
-#pragma unroll 4
+#pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
             const uint32_t k = k_first + s * 32;
-            const uint2 smv = __ldcs(reinterpret_cast<const uint2 *>(sm + 8ull * k));
-            const uint32_t c32 = __ldcs(reinterpret_cast<const uint32_t *>(codes + 4ull * k));
+            const uint2 smv = sms[s];
+            const uint32_t c32 = cds[s];
             uint32_t w[4];
             // word t: elements 2t, 2t+1
             const uint32_t s2[4] = {__byte_perm(smv.x, 0, 0x4140), __byte_perm(smv.x, 0, 0x4342),
