@@ -261,7 +261,11 @@ int lsmkv_bloom_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uin
  *
  * lsmkv_put_batch_host: put_batch. keys_out / vals_out / blob_out [host] receive what
  *   lsmkv_encode_batch produces; *n_chunks_out (optional) is set before returning. blob_out
- *   may be NULL together with page_table and pool (index-only).
+ *   may be NULL together with page_table and pool (index-only). *blob_bytes_out (optional) =
+ *   bytes placed in blob_out. With the compressing codec blob sizes depend on the data: the
+ *   call then synchronises `stream` once per slice, copies back exactly the bytes produced
+ *   (blobs stay back to back across slices) and returns LSMKV_ECAPACITY if blob_out is too
+ *   small; with the identity codec it never synchronises.
  * lsmkv_probe_batch_host: probe. hit_chunks_out [host n_query], recs_out [host, sum of
  *   floor(len/C)], optional keys_out; *n_qchunks_out (optional) is set before returning.
  * lsmkv_decode_batch_host: get_batch, tensor half. qchunk_off, hit_chunks, recs and
@@ -275,7 +279,8 @@ int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uin
                          const uint64_t *seq_off, const uint32_t *start_chunk,
                          const uint32_t *page_table, const lsmkv_pool_t *pool, uint32_t file_id,
                          uint64_t base_offset, lsmkv_key_t *keys_out, lsmkv_val_t *vals_out,
-                         void *blob_out, uint64_t blob_capacity, uint64_t *n_chunks_out);
+                         void *blob_out, uint64_t blob_capacity, uint64_t *n_chunks_out,
+                         uint64_t *blob_bytes_out);
 int lsmkv_probe_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
                            const uint32_t *tokens, const uint64_t *seq_off,
                            const lsmkv_run_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,

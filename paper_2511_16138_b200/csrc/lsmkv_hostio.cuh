@@ -94,10 +94,12 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
                                     const lsmkv_pool_t *pool, uint32_t file_id,
                                     uint64_t base_offset, lsmkv_key_t *keys_out,
                                     lsmkv_val_t *vals_out, void *blob_out,
-                                    uint64_t blob_capacity, uint64_t *n_chunks_out)
+                                    uint64_t blob_capacity, uint64_t *n_chunks_out,
+                                    uint64_t *blob_bytes_out)
 {
     if (!ctx) return LSMKV_EINVAL;
     if (n_chunks_out) *n_chunks_out = 0;
+    if (blob_bytes_out) *blob_bytes_out = 0;
     if (n_req == 0) return LSMKV_OK;
     if (!tokens || !seq_off || !keys_out || !vals_out) return LSMKV_EINVAL;
     const bool with_blob = blob_out != nullptr;
@@ -115,11 +117,16 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     const uint64_t n_chunks = coff[n_req];
     if (n_chunks_out) *n_chunks_out = n_chunks;
     if (n_chunks == 0) return LSMKV_OK;
-    if (with_blob && blob_capacity / cb < n_chunks) return LSMKV_ECAPACITY;
+    const bool coded = with_blob && ctx->codec != LSMKV_CODEC_IDENTITY;
+    if (with_blob && !coded && blob_capacity / cb < n_chunks) return LSMKV_ECAPACITY;
+    // bytes one chunk can take in the stage (worst case of the codec)
+    const uint64_t slot = coded ? lsmkv_encode_bound(ctx, 1) : cb;
+    if (with_blob && !coded && blob_bytes_out) *blob_bytes_out = n_chunks * cb;
 
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const uint64_t stage_chunks_max = std::max<uint64_t>(1, (uint64_t)ctx->host_stage_bytes / cb);
+    const uint64_t stage_chunks_max = std::max<uint64_t>(1, (uint64_t)ctx->host_stage_bytes / slot);
+    uint64_t host_used = 0;                          // compressing codec: bytes placed so far
     ScratchLease lease(ctx, 0, s, (4 * (size_t)n_req + 8) * 8 + 64 * (size_t)n_req + 4096);
     if (!lease.ok()) return LSMKV_ENOMEM;
     for (uint32_t a = 0; a < n_req;) {
@@ -132,7 +139,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
         if (m == 0) { a = b; continue; }
         size_t need = pad256(nt * 4) + 2 * pad256(((size_t)nr + 1) * 8) + pad256((size_t)nr * 4) +
                       pad256(m * 4) + pad256(m * 32) + pad256(m * 16) +
-                      (with_blob ? pad256(m * cb) : 0) + 4096;
+                      (with_blob ? pad256(m * slot) : 0) + 4096;
         int rc = ensure_io(ctx, 0, need);
         if (rc != LSMKV_OK) return rc;
         IoLayout io(ctx->d_io[0]);
@@ -143,7 +150,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
         uint32_t *d_pages = io.take<uint32_t>(m);
         lsmkv_key_t *d_keys = io.take<lsmkv_key_t>(m);
         lsmkv_val_t *d_vals = io.take<lsmkv_val_t>(m);
-        unsigned char *d_blob = with_blob ? io.take<unsigned char>(m * cb) : nullptr;
+        unsigned char *d_blob = with_blob ? io.take<unsigned char>(m * slot) : nullptr;
         // offsets relative to the slice, in pinned scratch that lives until the call's work ends
         uint64_t *rel = lease.take<uint64_t>(2 * ((size_t)nr + 1));
         for (uint32_t k = 0; k <= nr; ++k) {
@@ -160,14 +167,27 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
             CU(ctx, cudaMemcpyAsync(d_pages, page_table + coff[a], m * 4, cudaMemcpyHostToDevice, s));
         rc = lsmkv_encode_batch(ctx, stream, nr, d_tok, d_seq, start_chunk ? d_start : nullptr,
                                 d_coff, m, with_blob ? d_pages : nullptr, with_blob ? pool : nullptr,
-                                file_id, base_offset + coff[a] * cb, d_keys, d_vals, d_blob,
-                                with_blob ? m * cb : 0);
+                                file_id, base_offset + (coded ? host_used : coff[a] * cb), d_keys,
+                                d_vals, d_blob, with_blob ? m * slot : 0);
         if (rc != LSMKV_OK) return rc;
         CU(ctx, cudaMemcpyAsync(keys_out + coff[a], d_keys, m * 32, cudaMemcpyDeviceToHost, s));
         CU(ctx, cudaMemcpyAsync(vals_out + coff[a], d_vals, m * 16, cudaMemcpyDeviceToHost, s));
-        if (with_blob)
+        if (coded) {
+            // blob sizes depend on the data: wait for this slice's records, then copy exactly
+            // the bytes it produced behind the previous slice's
+            CU(ctx, cudaStreamSynchronize(s));
+            const lsmkv_val_t &last = vals_out[coff[b] - 1];
+            if (last.reserved == 0) return LSMKV_ECAPACITY;   // stage overflow (flagged on device)
+            const uint64_t used = last.offset + last.reserved - (base_offset + host_used);
+            if (blob_capacity - host_used < used) return LSMKV_ECAPACITY;
+            CU(ctx, cudaMemcpyAsync(static_cast<unsigned char *>(blob_out) + host_used, d_blob, used,
+                                    cudaMemcpyDeviceToHost, s));
+            host_used += used;
+            if (blob_bytes_out) *blob_bytes_out = host_used;
+        } else if (with_blob) {
             CU(ctx, cudaMemcpyAsync(static_cast<unsigned char *>(blob_out) + coff[a] * cb, d_blob,
                                     m * cb, cudaMemcpyDeviceToHost, s));
+        }
         a = b;
     }
     return LSMKV_OK;
@@ -239,76 +259,94 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
         !arenas || !arena_bytes || n_arenas == 0)
         return LSMKV_EINVAL;
     const uint64_t cb = ctx->chunk_bytes;
+    const bool coded = ctx->codec != LSMKV_CODEC_IDENTITY;
     // the hit chunks in order, validated on the host (nothing is enqueued if one is bad)
-    uint64_t total_hits = 0;
+    uint64_t total_hits = 0, max_len = coded ? 0 : cb, min_len = coded ? ~0ull : cb, sum_len = 0;
     for (uint32_t q = 0; q < n_query; ++q) {
         if (qchunk_off[q + 1] < qchunk_off[q] || hit_chunks[q] > qchunk_off[q + 1] - qchunk_off[q])
             return LSMKV_EINVAL;
         for (uint64_t j = 0; j < hit_chunks[q]; ++j) {
             const lsmkv_val_t &r = recs[qchunk_off[q] + j];
+            const uint64_t len = coded ? r.reserved : cb;
             if (r.file_id >= n_arenas || !arenas[r.file_id] || r.offset > arena_bytes[r.file_id] ||
-                arena_bytes[r.file_id] - r.offset < cb)
+                arena_bytes[r.file_id] - r.offset < len || (coded && (len < 32 || (len & 15))))
                 return LSMKV_EINVAL;
+            max_len = std::max(max_len, len);
+            min_len = std::min(min_len, len);
+            sum_len += len;
         }
         total_hits += hit_chunks[q];
     }
     if (total_hits == 0) return LSMKV_OK;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const uint64_t stage_chunks = std::max<uint64_t>(1, (uint64_t)ctx->host_stage_bytes / cb);
+    // a slice holds at most m_max chunks and stage_bytes bytes of blobs (at least one blob)
+    const uint64_t stage_bytes_max = std::max<uint64_t>((uint64_t)ctx->host_stage_bytes, max_len);
+    const uint64_t stage_chunks = std::max<uint64_t>(1, stage_bytes_max / min_len);
     const uint64_t m_max = std::min<uint64_t>(stage_chunks, total_hits);
-    size_t need = pad256(m_max * cb) + pad256(m_max * 16) + pad256(m_max * 4) + 3 * 256 + 4096;
+    const uint64_t blob_stage = coded ? stage_bytes_max : m_max * cb;
+    size_t need = pad256(blob_stage) + pad256(m_max * 16) + pad256(m_max * 4) + 3 * 256 + 4096;
     int rc = ensure_io(ctx, 2, need);
     if (rc != LSMKV_OK) return rc;
     IoLayout io(ctx->d_io[2]);
-    unsigned char *d_blob = io.take<unsigned char>(m_max * cb);
+    unsigned char *d_blob = io.take<unsigned char>(blob_stage);
     lsmkv_val_t *d_recs = io.take<lsmkv_val_t>(m_max);
     uint32_t *d_pages = io.take<uint32_t>(m_max);
     uint64_t *d_qoff = io.take<uint64_t>(2);
     uint32_t *d_hit = io.take<uint32_t>(1);
     const void *stage_arena[1] = {d_blob};
 
-    const uint64_t n_slices = (total_hits + m_max - 1) / m_max;
-    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices * 96 + 4096);
+    // descriptors of all hit chunks (each slice uploads its part), plus 32 bytes per slice
+    // every slice stages at least one chunk, and at least half the stage unless blobs are huge
+    uint64_t n_slices_max = total_hits;
+    if (max_len <= blob_stage / 2)
+        n_slices_max = std::min<uint64_t>(total_hits, 2 * (sum_len / blob_stage) + total_hits / m_max + 2);
+    n_slices_max = std::min<uint64_t>(n_slices_max, 1u << 20);
+    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices_max * 48 + 4096);
     if (!lease.ok()) return LSMKV_ENOMEM;
+    lsmkv_val_t *srecs_all = lease.take<lsmkv_val_t>(total_hits);
+    uint32_t *spages_all = lease.take<uint32_t>(total_hits);
     uint32_t q = 0;
-    uint64_t j = 0, left = total_hits;
+    uint64_t j = 0, left = total_hits, done = 0, slices = 0;
     while (q < n_query && left) {
-        // one slice: up to m_max hit chunks, their blobs gathered into the stage in hit order;
-        // blobs that sit back to back in a host arena travel as one copy
+        // one slice: up to m_max hit chunks and blob_stage bytes, blobs gathered into the stage
+        // in hit order; blobs that sit back to back in a host arena travel as one copy
         const uint64_t cap = std::min<uint64_t>(m_max, left);
-        lsmkv_val_t *srecs = lease.take<lsmkv_val_t>(cap);
-        uint32_t *spages = lease.take<uint32_t>(cap);
-        uint64_t m = 0;
-        uint64_t run_first = 0;              // first slot of the pending contiguous copy
+        lsmkv_val_t *srecs = srecs_all + done;
+        uint32_t *spages = spages_all + done;
+        uint64_t m = 0, at = 0;              // chunks and bytes staged in this slice
+        uint64_t run_dst = 0;                // stage offset of the pending contiguous copy
         const unsigned char *run_src = nullptr;
-        uint64_t run_len = 0;
+        uint64_t run_bytes = 0;
         while (q < n_query && m < cap) {
             if (j >= hit_chunks[q]) { ++q; j = 0; continue; }
             const uint64_t idx = qchunk_off[q] + j;
             const lsmkv_val_t &r = recs[idx];
+            const uint64_t len = coded ? r.reserved : cb;
+            if (at + len > blob_stage) break;                    // slice is full (m >= 1 here)
             const unsigned char *src = static_cast<const unsigned char *>(arenas[r.file_id]) + r.offset;
-            const uint64_t slot = m;
-            if (run_len && src == run_src + run_len * cb) {
-                ++run_len;
+            if (run_bytes && src == run_src + run_bytes) {
+                run_bytes += len;
             } else {
-                if (run_len)
-                    CU(ctx, cudaMemcpyAsync(d_blob + run_first * cb, run_src, run_len * cb,
+                if (run_bytes)
+                    CU(ctx, cudaMemcpyAsync(d_blob + run_dst, run_src, run_bytes,
                                             cudaMemcpyHostToDevice, s));
-                run_first = slot;
+                run_dst = at;
                 run_src = src;
-                run_len = 1;
+                run_bytes = len;
             }
-            srecs[m] = lsmkv_val_t{0, 0, slot * cb};
+            srecs[m] = lsmkv_val_t{0, coded ? r.reserved : 0u, at};
             spages[m] = dst_page_table[idx];
+            at += len;
             ++m;
             ++j;
         }
-        if (run_len)
-            CU(ctx, cudaMemcpyAsync(d_blob + run_first * cb, run_src, run_len * cb,
-                                    cudaMemcpyHostToDevice, s));
+        if (run_bytes)
+            CU(ctx, cudaMemcpyAsync(d_blob + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
         if (m == 0) break;
         left -= m;
+        done += m;
+        if (++slices > n_slices_max) return LSMKV_EINVAL;     // cannot happen: see the bound above
         uint64_t *qoff2 = lease.take<uint64_t>(2);
         uint32_t *hit1 = lease.take<uint32_t>(1);
         qoff2[0] = 0;
@@ -318,7 +356,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
         CU(ctx, cudaMemcpyAsync(d_pages, spages, m * 4, cudaMemcpyHostToDevice, s));
         CU(ctx, cudaMemcpyAsync(d_qoff, qoff2, 16, cudaMemcpyHostToDevice, s));
         CU(ctx, cudaMemcpyAsync(d_hit, hit1, 4, cudaMemcpyHostToDevice, s));
-        const uint64_t stage_bytes = m * cb;
+        const uint64_t stage_bytes = at;
         rc = lsmkv_decode_batch(ctx, stream, 1, d_qoff, m, d_hit, d_recs, stage_arena, &stage_bytes,
                                 1, d_pages, pool);
         if (rc != LSMKV_OK) return rc;

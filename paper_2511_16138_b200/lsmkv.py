@@ -138,7 +138,7 @@ def lib() -> C.CDLL:
                                             C.POINTER(PoolStruct), vp]
     L.lsmkv_put_batch_host.restype = C.c_int
     L.lsmkv_put_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, vp, C.POINTER(PoolStruct), u32,
-                                       u64, vp, vp, vp, u64, C.POINTER(u64)]
+                                       u64, vp, vp, vp, u64, C.POINTER(u64), C.POINTER(u64)]
     L.lsmkv_probe_batch_host.restype = C.c_int
     L.lsmkv_probe_batch_host.argtypes = [vp, vp, u32, vp, vp, C.POINTER(RunStruct), u32, vp, vp,
                                          vp, C.POINTER(u64)]
@@ -279,17 +279,20 @@ def _hptr(x):
 
 
 def lsmkv_put_batch_host(ctx, stream, n_req, tokens, seq_off, start_chunk, page_table, pool,
-                         file_id, base_offset, keys_out, vals_out, blob_out, blob_capacity) -> int:
-    """Host buffers in and out (numpy arrays or pinned tensors). Returns the chunk count."""
+                         file_id, base_offset, keys_out, vals_out, blob_out, blob_capacity,
+                         want_bytes: bool = False):
+    """Host buffers in and out (numpy arrays or pinned tensors). Returns the chunk count, or
+    (chunk count, blob bytes placed) with ``want_bytes``."""
     p = _pool(pool)
     n = C.c_uint64(0)
+    nb = C.c_uint64(0)
     rc = lib().lsmkv_put_batch_host(ctx, _stream(stream), n_req, _hptr(tokens), _hptr(seq_off),
                                     _hptr(start_chunk), _hptr(page_table),
                                     C.byref(p) if p is not None else None, file_id, base_offset,
                                     _hptr(keys_out), _hptr(vals_out), _hptr(blob_out),
-                                    blob_capacity, C.byref(n))
+                                    blob_capacity, C.byref(n), C.byref(nb))
     _check(ctx, rc, "lsmkv_put_batch_host")
-    return int(n.value)
+    return (int(n.value), int(nb.value)) if want_bytes else int(n.value)
 
 
 def lsmkv_probe_batch_host(ctx, stream, n_query, tokens, seq_off, runs, hit_chunks_out,
@@ -449,10 +452,11 @@ class Context:
                            arenas, dst_page_table, pool)
 
     def put_batch_host(self, n_req, tokens, seq_off, start_chunk, page_table, pool, file_id,
-                       base_offset, keys_out, vals_out, blob_out, blob_capacity, stream=None):
+                       base_offset, keys_out, vals_out, blob_out, blob_capacity, stream=None,
+                       want_bytes=False):
         return lsmkv_put_batch_host(self.handle, stream, n_req, tokens, seq_off, start_chunk,
                                     page_table, pool, file_id, base_offset, keys_out, vals_out,
-                                    blob_out, blob_capacity)
+                                    blob_out, blob_capacity, want_bytes)
 
     def probe_batch_host(self, n_query, tokens, seq_off, runs, hit_chunks_out, recs_out,
                          keys_out=None, stream=None):

@@ -126,3 +126,62 @@ def test_host_calls_reject_bad_arguments_before_enqueuing():
         torch.cuda.synchronize()
         assert n == 2 and list(vals["offset"]) == [64, 64 + cb] and list(vals["file_id"]) == [3, 3]
         assert ctx.put_batch_host(0, toks, off, None, None, None, 0, 0, keys, vals, None, 0) == 0
+
+
+@pytest.mark.parametrize("stage", [1 << 20, 1 << 30])
+def test_host_buffers_with_the_compressing_codec(stage):
+    """put / probe / decode through host memory with variable-size blobs: byte-identical to the
+    oracle's blobs laid back to back, across slices."""
+    g = lsmkv.Geom(n_layers=2, n_kv_heads=8, head_dim=64, page_tokens=16, chunk_tokens=16,
+                   flags=lsmkv.CODEC_XP12)                      # 16 KiB slabs, 64 KiB chunks
+    og = H.ogeom(g)
+    rng = np.random.default_rng(21)
+    w = synth.llama_requests(n_req=12, min_len=100, max_len=700, config_id=73)
+    b = w.batch
+    nch = synth.chunk_counts(b.seq_off, 16)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    num_pages = n + 9
+    pool_np = synth.random_pool_bytes(rng, 4, num_pages, g.page_bytes)
+    pool_np.view(np.uint16)[:, ::7, ::5] = 0x0001               # sprinkle exceptions
+    pages = synth.random_pages(rng, num_pages, n)
+    o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, b.tokens, b.seq_off, None, coff, pages,
+                                                      pool_np, 2, 256)
+    with lsmkv.Context(g, 0) as ctx:
+        ctx.set_tuning("host_stage_bytes", stage)
+        pool = H.DevPool(g, num_pages, pool_np)
+        keys = np.zeros((n, 4), np.uint64)
+        vals = np.zeros(n, VAL_DTYPE)
+        blob = np.zeros(ctx.encode_bound(n), np.uint8)
+        got_n, used = ctx.put_batch_host(b.n, b.tokens, b.seq_off, None, pages, pool.table, 2, 256,
+                                         keys, vals, blob, blob.size, want_bytes=True)
+        torch.cuda.synchronize()
+        assert got_n == n and used == o_blob.size
+        assert np.array_equal(keys, o_keys) and np.array_equal(vals, o_vals)
+        assert np.array_equal(blob[:used], o_blob)
+        # too small a host buffer is reported
+        with pytest.raises(lsmkv.LsmkvError) as e:
+            ctx.put_batch_host(b.n, b.tokens, b.seq_off, None, pages, pool.table, 2, 256, keys,
+                               vals, blob, used - 16)
+        assert e.value.code == lsmkv.ECAPACITY
+        torch.cuda.synchronize()
+        ctx.last_status()
+        run = oracle.flush(o_keys, o_vals)
+        druns, keep = H.dev_runs([run])
+        hit = np.zeros(b.n, np.uint32)
+        recs = np.zeros(n, VAL_DTYPE)
+        ctx.probe_batch_host(b.n, b.tokens, b.seq_off, druns, hit, recs)
+        torch.cuda.synchronize()
+        assert np.array_equal(hit, nch.astype(np.uint32))
+        arena = np.concatenate([np.zeros(256, np.uint8), o_blob])
+        arenas = [np.zeros(16, np.uint8), np.zeros(16, np.uint8), arena]   # file_id 2
+        dst_pages = synth.random_pages(rng, num_pages, n)
+        o_dst = np.zeros_like(pool_np)
+        oracle.decode_batch_xp12(og, coff, hit, recs, arenas, dst_pages, o_dst)
+        dst = H.DevPool(g, num_pages)
+        ctx.decode_batch_host(b.n, coff, hit, recs, [(a, a.size) for a in arenas], dst_pages,
+                              dst.table)
+        torch.cuda.synchronize()
+        assert np.array_equal(dst.numpy(), o_dst)
+        st = ctx.last_status()
+        assert st["flags"] == 0 and st["chunks_decoded"] == n
