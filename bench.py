@@ -381,17 +381,26 @@ def main():
     moved_all = ranks.sum_over_ranks(2 * payload, dev)   # bytes packed + unpacked, all ranks
     value = ranks.whole_job_rate(moved_all, ms_step) / 1e9
 
-    # ---- end to end: host buffers in, host buffers out, through the same C-ABI calls
-    e2e = None
-    if args.e2e_steps > 0:
-        e2e = run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream,
-                      barrier, world)
-
     # ---- the compressing codec on the first wave (reported beside the identity codec)
     xp_block = None
     if rank == 0 and not args.no_xp12_block:
         xp_block = xp12_block(torch, lsmkv, dev, local_rank, W[0], src_bufs, src_pool, dst_bufs,
                               dst_pool, arena, stream)
+
+    # ---- end to end: host buffers in, host buffers out, through the same C-ABI calls
+    e2e = e2e_xp = None
+    if args.e2e_steps > 0:
+        del arena                                    # the host-buffer calls stage on their own
+        torch.cuda.empty_cache()
+        e2e = run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barrier,
+                      world, "identity")
+        if not args.no_xp12_block:
+            ctx_xp = lsmkv.Context(lsmkv.Geom(**dict(GEOM, flags=lsmkv.CODEC_XP12)), local_rank)
+            try:
+                e2e_xp = run_e2e(args, torch, lsmkv, ctx_xp, g, W, src_pool, dst_pool, dev, stream,
+                                 barrier, world, "xp12")
+            finally:
+                ctx_xp.close()
 
     # ---- probe throughput on the probe-heavy workload (second half of the metric)
     probe_block = None
@@ -435,7 +444,7 @@ def main():
                        "tuning": {k: ctx.get_tuning(k) for k in
                                   ("copy_mode", "copy_stage_bytes", "copy_stages",
                                    "copy_ctas_per_sm", "copy_l2_hint")}},
-            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "e2e": e2e, "e2e_codec_xp12": e2e_xp, "gpu_launches": int(launches), "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "k_copy_slabs (pack + unpack launches)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_source": peak_src,
@@ -612,15 +621,17 @@ def xp12_block(torch, lsmkv, dev, device_index, d, src_bufs, src_pool, dst_bufs,
         ctx.close()
 
 
-def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, stream, barrier, world):
+def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barrier, world,
+            label):
     """Same path through the host-buffer entry points of the C ABI: per sub-batch the token
     sequences and page tables are HOST arrays, the packed blobs, keys and records come back to
     pinned host memory (where a tensor-log writer would take them), the probe returns hit
     lengths and records to the host, and the decode copies the hit blobs from the host arena
     back to the device and scatters them. The KV pool itself lives on the GPU by nature. Two
-    slots on two streams: the put of sub-batch i+1 overlaps the get of sub-batch i."""
+    slots on two streams: the get of sub-batch i is enqueued, then the put of sub-batch i+1,
+    so both PCIe directions are busy. `ctx` decides the codec (identity or compressing)."""
     cb = g.chunk_bytes
-    sub_cap = 2048                                   # chunks per sub-batch (4 GiB of blobs)
+    sub_cap = 2048                                   # chunks per sub-batch (4 GiB of raw blobs)
     subs = []
     for d in W:
         nchw, a, acc = d["nch"], 0, 0
@@ -632,11 +643,12 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
     max_n = max(int(d["nch"][a:b].sum()) for d, a, b in subs)
     max_req = max(b - a for d, a, b in subs)
     NS = 2
+    blob_cap = ctx.encode_bound(max_n)
 
     def pin(nbytes):
         return torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
 
-    pin_blob = [pin(max_n * cb) for _ in range(NS)]
+    pin_blob = [pin(blob_cap) for _ in range(NS)]
     pin_keys = [pin(max_n * 32) for _ in range(NS)]
     pin_vals = [pin(max_n * 16) for _ in range(NS)]
     pin_hit = [pin(max_req * 4) for _ in range(NS)]
@@ -657,15 +669,19 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
                  seq_off=pinned(seq_rel), src=pinned(h["src_pages"][c0:c1]),
                  dst=pinned(h["dst_pages"][c0:c1]), qoff=pinned(qoff), nch=d["nch"][a:b])
         prepared.append(p)
-    # untimed: the index of each sub-batch (its records point into this sub-batch's blobs)
+    # untimed: a real put of each sub-batch gives its records; flushed on the device they are
+    # the sub-batch's index (a put is deterministic, so the timed puts reproduce them)
     for p in prepared:
         n = p["n"]
-        ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, None, None, 0, 0,
-                           pin_keys[0], pin_vals[0], None, 0, stream=stream)
-        dk = torch.empty(n * 32, dtype=torch.uint8, device=dev)
-        dv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
-        dk.copy_(pin_keys[0][:n * 32], non_blocking=True)
-        dv.copy_(pin_vals[0][:n * 16], non_blocking=True)
+        _, used = ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, p["src"],
+                                     src_pool, 0, 0, pin_keys[0], pin_vals[0], pin_blob[0],
+                                     blob_cap, stream=stream, want_bytes=True)
+        torch.cuda.synchronize()
+        if used == 0:                                # identity codec: size is known up front
+            used = n * cb
+        p["blob_bytes"] = used
+        dk = pin_keys[0][:n * 32].to(dev)
+        dv = pin_vals[0][:n * 16].to(dev)
         tk = torch.empty(n * 32, dtype=torch.uint8, device=dev)
         tv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
         tn = torch.zeros(1, dtype=torch.int64, device=dev)
@@ -682,10 +698,10 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
         p, k_ = prepared[i], i % NS
         s_put.wait_event(slot_free[k_])
         ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, p["src"], src_pool, 0, 0,
-                           pin_keys[k_], pin_vals[k_], pin_blob[k_], max_n * cb, stream=s_put)
+                           pin_keys[k_], pin_vals[k_], pin_blob[k_], blob_cap, stream=s_put)
         put_done[k_].record(s_put)
         h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["src"].numel()
-        d2h += p["n"] * (cb + 48)
+        d2h += p["blob_bytes"] + p["n"] * 48
 
     def get(i):
         nonlocal h2d, d2h, moved
@@ -696,24 +712,26 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
                              pin_recs[k_], None, stream=s_get)
         s_get.synchronize()                 # the host reads hit lengths and records
         ctx.decode_batch_host(n_req, p["qoff"], pin_hit[k_], pin_recs[k_],
-                              [(pin_blob[k_], n * cb)], p["dst"], dst_pool, stream=s_get)
+                              [(pin_blob[k_], p["blob_bytes"])], p["dst"], dst_pool, stream=s_get)
         slot_free[k_].record(s_get)
-        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + n * (cb + 20) + 20
+        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["blob_bytes"] + n * 20 + 20
         d2h += n_req * 4 + n * 16
         moved += 2 * n * cb
 
     def one_step(check=False):
         put(0)
         for i in range(len(prepared)):
+            get(i)                          # enqueued first: its transfers run while ...
             if i + 1 < len(prepared):
-                put(i + 1)
-            get(i)
+                put(i + 1)                  # ... the next put goes the other way
             if check:
+                s_get.synchronize()
                 hits = pin_hit[i % NS][:prepared[i]["n_req"] * 4].numpy().view(np.uint32)
                 assert np.array_equal(hits, prepared[i]["nch"].astype(np.uint32)), "e2e probe missed"
 
     s_put.wait_stream(stream)
     s_get.wait_stream(stream)
+    ctx.last_status()
     one_step(check=True)                    # warm-up (also faults in the pinned pages)
     barrier()
     st = ctx.last_status()
@@ -736,12 +754,12 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, arena, dev, strea
     ctx.last_status()
     return {"value": ranks.whole_job_rate(moved, ms) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
-            "steps": steps, "ms_per_step": ms / steps,
+            "steps": steps, "ms_per_step": ms / steps, "codec": label,
             "api": "lsmkv_put_batch_host / lsmkv_probe_batch_host / lsmkv_decode_batch_host",
             "note": "host buffers in and out through the C ABI: blobs, keys and records land in "
                     "pinned host memory, hit blobs are copied back from it before the scatter; "
                     "put and get sides run on two streams so both PCIe directions are busy; "
-                    "PCIe-bound"}
+                    "value counts raw (uncompressed) payload bytes; PCIe-bound"}
 
 
 if __name__ == "__main__":

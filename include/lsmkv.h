@@ -358,6 +358,9 @@ int lsmkv_profile_read(lsmkv_ctx *ctx, lsmkv_profile_t *out /* [host] */);
 /* The cudaError_t behind the last LSMKV_ECUDA of this context (0 if none). */
 int lsmkv_last_cuda_error(const lsmkv_ctx *ctx);
 
+/* Source line (in the library's own files) of the CUDA call behind that error, 0 if unknown. */
+int lsmkv_last_cuda_line(const lsmkv_ctx *ctx);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
 

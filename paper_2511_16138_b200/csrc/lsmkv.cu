@@ -42,6 +42,7 @@ struct lsmkv_ctx {
     uint64_t *d_dir;
     uint64_t dir_cap;
     int last_cuda;
+    int last_cuda_line;   // source line of the failing CUDA call (diagnostics)
     uint64_t launches;
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
@@ -73,9 +74,9 @@ struct DeviceGuard {
     ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
-int cuda_fail(lsmkv_ctx *ctx, cudaError_t e)
+int cuda_fail(lsmkv_ctx *ctx, cudaError_t e, int line = 0)
 {
-    if (ctx) ctx->last_cuda = (int)e;
+    if (ctx) { ctx->last_cuda = (int)e; ctx->last_cuda_line = line; }
     cudaGetLastError();   // clear the sticky-less error state
     return LSMKV_ECUDA;
 }
@@ -83,7 +84,7 @@ int cuda_fail(lsmkv_ctx *ctx, cudaError_t e)
 #define CU(ctx, call)                                            \
     do {                                                         \
         cudaError_t e__ = (call);                                \
-        if (e__ != cudaSuccess) return cuda_fail((ctx), e__);    \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__, __LINE__); \
     } while (0)
 
 // (a * b) mod (2^61 - 1) on the host, for the power tables only
@@ -161,6 +162,7 @@ int ensure_workspace(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
     if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
     if (ctx->d_ws) cudaFree(ctx->d_ws);   // waits for work that may still use the old one
     ctx->d_ws = p;
+    cudaGetLastError();   // drop any stale last-error left by the allocation calls
     ctx->ws_seq = ns;
     ctx->ws_chunks = nc;
     return LSMKV_OK;
@@ -174,6 +176,7 @@ int ensure_dir(lsmkv_ctx *ctx, uint64_t entries)
     if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
     if (ctx->d_dir) cudaFree(ctx->d_dir);   // waits for work that may still use the old one
     ctx->d_dir = static_cast<uint64_t *>(p);
+    cudaGetLastError();   // drop any stale last-error left by the allocation calls
     ctx->dir_cap = entries;
     return LSMKV_OK;
 }
@@ -199,6 +202,7 @@ int ensure_sort(lsmkv_ctx *ctx, uint64_t n, SortWs *ws)
         if (ctx->d_sort) cudaFree(ctx->d_sort);
     if (ctx->d_xp) cudaFree(ctx->d_xp);
         ctx->d_sort = p;
+    cudaGetLastError();   // drop any stale last-error left by the allocation calls
         ctx->sort_cap = n;
     }
     const uint64_t cap = ctx->sort_cap;
@@ -304,6 +308,9 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
         if (ctx->d_xp) cudaFree(ctx->d_xp);
         ctx->d_xp = p;
         ctx->xp_cap = n_chunks;
+        // A successful allocation can still leave a stale entry in the runtime's last-error
+        // slot (seen on this driver); drop it so the launch checks below report only launches.
+        cudaGetLastError();
     }
     XpJob job;
     std::memset(&job, 0, sizeof(job));
@@ -830,6 +837,8 @@ int lsmkv_profile_read(lsmkv_ctx *ctx, lsmkv_profile_t *out)
 }
 
 int lsmkv_last_cuda_error(const lsmkv_ctx *ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int lsmkv_last_cuda_line(const lsmkv_ctx *ctx) { return ctx ? ctx->last_cuda_line : 0; }
 
 uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx) { return ctx ? ctx->launches : 0; }
 

@@ -30,6 +30,7 @@ int ensure_io(lsmkv_ctx *ctx, int kind, size_t bytes)
     if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
     if (ctx->d_io[kind]) cudaFree(ctx->d_io[kind]);   // waits for work that may still use it
     ctx->d_io[kind] = p;
+    cudaGetLastError();   // drop any stale last-error left by the allocation calls
     ctx->io_cap[kind] = bytes;
     return LSMKV_OK;
 }

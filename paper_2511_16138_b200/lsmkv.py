@@ -25,7 +25,7 @@ EXPORTS = (
     "lsmkv_format_version", "lsmkv_profile_enable", "lsmkv_profile_read",
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
-    "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound",
+    "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
 )
 ST_OVERFLOW = 32
 CODEC_IDENTITY, CODEC_XP12 = 0, 1
@@ -36,10 +36,10 @@ K_NAMES = ("keys", "pack", "probe", "plan", "unpack", "flush", "merge")
 
 
 class LsmkvError(RuntimeError):
-    def __init__(self, code: int, where: str, cuda: int = 0):
+    def __init__(self, code: int, where: str, cuda: int = 0, line: int = 0):
         msg = f"{where}: {strerror(code)} ({code})"
         if cuda:
-            msg += f", cudaError {cuda}"
+            msg += f", cudaError {cuda}" + (f" at library line {line}" if line else "")
         super().__init__(msg)
         self.code = code
         self.cuda = cuda
@@ -159,6 +159,8 @@ def lib() -> C.CDLL:
     L.lsmkv_last_status.argtypes = [vp, vp, C.POINTER(StatusStruct)]
     L.lsmkv_last_cuda_error.restype = C.c_int
     L.lsmkv_last_cuda_error.argtypes = [vp]
+    L.lsmkv_last_cuda_line.restype = C.c_int
+    L.lsmkv_last_cuda_line.argtypes = [vp]
     L.lsmkv_launch_count.restype = u64
     L.lsmkv_launch_count.argtypes = [vp]
     L.lsmkv_set_tuning.restype = C.c_int
@@ -204,7 +206,8 @@ def _stream(stream):
 
 def _check(ctx, rc: int, where: str):
     if rc != OK:
-        raise LsmkvError(rc, where, lib().lsmkv_last_cuda_error(ctx) if ctx else 0)
+        raise LsmkvError(rc, where, lib().lsmkv_last_cuda_error(ctx) if ctx else 0,
+                         lib().lsmkv_last_cuda_line(ctx) if ctx else 0)
 
 
 # ---- the C entry points, one to one ------------------------------------------------------
