@@ -703,29 +703,42 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
         h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["src"].numel()
         d2h += p["blob_bytes"] + p["n"] * 48
 
-    def get(i):
-        nonlocal h2d, d2h, moved
+    def probe(i):
+        nonlocal h2d, d2h
         p, k_ = prepared[i], i % NS
-        n, n_req = p["n"], p["n_req"]
         s_get.wait_event(put_done[k_])
-        ctx.probe_batch_host(n_req, p["tokens"], p["seq_off"], p["runs"], pin_hit[k_],
+        ctx.probe_batch_host(p["n_req"], p["tokens"], p["seq_off"], p["runs"], pin_hit[k_],
                              pin_recs[k_], None, stream=s_get)
         s_get.synchronize()                 # the host reads hit lengths and records
-        ctx.decode_batch_host(n_req, p["qoff"], pin_hit[k_], pin_recs[k_],
+        h2d += p["tokens"].numel() + p["seq_off"].numel()
+        d2h += p["n_req"] * 4 + p["n"] * 16
+
+    def decode(i):
+        nonlocal h2d, moved
+        p, k_ = prepared[i], i % NS
+        ctx.decode_batch_host(p["n_req"], p["qoff"], pin_hit[k_], pin_recs[k_],
                               [(pin_blob[k_], p["blob_bytes"])], p["dst"], dst_pool, stream=s_get)
         slot_free[k_].record(s_get)
-        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["blob_bytes"] + n * 20 + 20
-        d2h += n_req * 4 + n * 16
-        moved += 2 * n * cb
+        h2d += p["blob_bytes"] + p["n"] * 20 + 20
+        moved += 2 * p["n"] * cb
+
+    # Transfers of one direction are served in the order they were issued, across streams. With
+    # the identity codec a put never blocks the host, so the next put is issued first (its
+    # small uploads then sit in front of the get's large one); with the compressing codec a
+    # put synchronises per slice, so the get is issued first and runs under it.
+    put_first = label == "identity"
 
     def one_step(check=False):
         put(0)
         for i in range(len(prepared)):
-            get(i)                          # enqueued first: its transfers run while ...
-            if i + 1 < len(prepared):
-                put(i + 1)                  # ... the next put goes the other way
+            probe(i)
+            nxt = i + 1 < len(prepared)
+            if put_first and nxt:
+                put(i + 1)
+            decode(i)
+            if not put_first and nxt:
+                put(i + 1)
             if check:
-                s_get.synchronize()
                 hits = pin_hit[i % NS][:prepared[i]["n_req"] * 4].numpy().view(np.uint32)
                 assert np.array_equal(hits, prepared[i]["nch"].astype(np.uint32)), "e2e probe missed"
 

@@ -51,6 +51,7 @@ struct lsmkv_ctx {
     void *d_io[3];
     size_t io_cap[3];
     std::vector<uint64_t> h_off_a;
+    std::vector<uint32_t> h_cuts;
     struct HostScratch { void *p; size_t cap; cudaEvent_t done; bool used; };
     HostScratch hs[3][2];
     int hs_next[3];

@@ -37,6 +37,25 @@ int ensure_io(lsmkv_ctx *ctx, int kind, size_t bytes)
 
 size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 
+// Large transfers go out in pieces: copies of one direction are served in issue order even
+// when they sit on different streams, so one multi-GiB copy would hold up every small copy
+// another stream issues in the same direction (and with it that stream's kernels). With
+// bounded pieces a put on one stream and a get on another keep both PCIe directions busy.
+constexpr size_t kCopyPiece = 32u << 20;
+
+cudaError_t copy_pieces(void *dst, const void *src, size_t bytes, cudaMemcpyKind kind,
+                        cudaStream_t s)
+{
+    unsigned char *d = static_cast<unsigned char *>(dst);
+    const unsigned char *p = static_cast<const unsigned char *>(src);
+    for (size_t at = 0; at < bytes; at += kCopyPiece) {
+        const size_t n = std::min(kCopyPiece, bytes - at);
+        const cudaError_t e = cudaMemcpyAsync(d + at, p + at, n, kind, s);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 // Pinned host scratch for the small descriptor arrays a call uploads. Every kind of call
 // (0 = put, 1 = probe, 2 = decode) alternates between two slots of its own; a slot is reused
 // only after the stream work of the call that used it last has finished (its event), so the
@@ -127,47 +146,69 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint64_t stage_chunks_max = std::max<uint64_t>(1, (uint64_t)ctx->host_stage_bytes / slot);
-    uint64_t host_used = 0;                          // compressing codec: bytes placed so far
-    ScratchLease lease(ctx, 0, s, (4 * (size_t)n_req + 8) * 8 + 64 * (size_t)n_req + 4096);
-    if (!lease.ok()) return LSMKV_ENOMEM;
+    // slices [a, b): as many requests as fit the blob stage (always at least one)
+    std::vector<uint32_t> &cuts = ctx->h_cuts;
+    cuts.clear();
+    uint64_t m_max = 0;
     for (uint32_t a = 0; a < n_req;) {
-        // slice [a, b): as many requests as fit the blob stage (always at least one)
         uint32_t b = a + 1;
         while (b < n_req && coff[b + 1] - coff[a] <= stage_chunks_max) ++b;
-        const uint32_t nr = b - a;
-        const uint64_t m = coff[b] - coff[a];
-        const uint64_t t0 = seq_off[a], nt = seq_off[b] - t0;
-        if (m == 0) { a = b; continue; }
-        size_t need = pad256(nt * 4) + 2 * pad256(((size_t)nr + 1) * 8) + pad256((size_t)nr * 4) +
-                      pad256(m * 4) + pad256(m * 32) + pad256(m * 16) +
-                      (with_blob ? pad256(m * slot) : 0) + 4096;
-        int rc = ensure_io(ctx, 0, need);
-        if (rc != LSMKV_OK) return rc;
-        IoLayout io(ctx->d_io[0]);
-        uint32_t *d_tok = io.take<uint32_t>(nt);
-        uint64_t *d_seq = io.take<uint64_t>((size_t)nr + 1);
-        uint64_t *d_coff = io.take<uint64_t>((size_t)nr + 1);
-        uint32_t *d_start = io.take<uint32_t>(nr);
-        uint32_t *d_pages = io.take<uint32_t>(m);
-        lsmkv_key_t *d_keys = io.take<lsmkv_key_t>(m);
-        lsmkv_val_t *d_vals = io.take<lsmkv_val_t>(m);
-        unsigned char *d_blob = with_blob ? io.take<unsigned char>(m * slot) : nullptr;
-        // offsets relative to the slice, in pinned scratch that lives until the call's work ends
-        uint64_t *rel = lease.take<uint64_t>(2 * ((size_t)nr + 1));
-        for (uint32_t k = 0; k <= nr; ++k) {
-            rel[k] = seq_off[a + k] - t0;
-            rel[(size_t)nr + 1 + k] = coff[a + k] - coff[a];
+        cuts.push_back(a);
+        m_max = std::max(m_max, coff[b] - coff[a]);
+        a = b;
+    }
+    cuts.push_back(n_req);
+    const size_t n_slices = cuts.size() - 1;
+    const uint64_t t_first = seq_off[0], nt = seq_off[n_req] - t_first;
+
+    // device scratch: every descriptor of the call (uploaded once, up front), one blob stage
+    const size_t n_rel = (size_t)n_req + n_slices;        // sum over slices of (requests + 1)
+    size_t need = pad256(nt * 4) + 2 * pad256(n_rel * 8) + pad256((size_t)n_req * 4) +
+                  pad256(n_chunks * 4) + pad256(m_max * 32) + pad256(m_max * 16) +
+                  (with_blob ? pad256(m_max * slot) : 0) + 4096;
+    int rc = ensure_io(ctx, 0, need);
+    if (rc != LSMKV_OK) return rc;
+    IoLayout io(ctx->d_io[0]);
+    uint32_t *d_tok = io.take<uint32_t>(nt ? nt : 1);
+    uint64_t *d_seq = io.take<uint64_t>(n_rel);
+    uint64_t *d_coff = io.take<uint64_t>(n_rel);
+    uint32_t *d_start = io.take<uint32_t>(n_req);
+    uint32_t *d_pages = io.take<uint32_t>(n_chunks);
+    lsmkv_key_t *d_keys = io.take<lsmkv_key_t>(m_max);
+    lsmkv_val_t *d_vals = io.take<lsmkv_val_t>(m_max);
+    unsigned char *d_blob = with_blob ? io.take<unsigned char>(m_max * slot) : nullptr;
+
+    ScratchLease lease(ctx, 0, s, 2 * n_rel * 8 + 256);
+    if (!lease.ok()) return LSMKV_ENOMEM;
+    uint64_t *h_seq = lease.take<uint64_t>(n_rel), *h_coff = lease.take<uint64_t>(n_rel);
+    size_t at = 0;
+    for (size_t k = 0; k < n_slices; ++k) {              // offsets relative to each slice
+        const uint32_t a = cuts[k], b = cuts[k + 1];
+        for (uint32_t r = a; r <= b; ++r) {
+            h_seq[at + (r - a)] = seq_off[r] - seq_off[a];
+            h_coff[at + (r - a)] = coff[r] - coff[a];
         }
-        CU(ctx, cudaMemcpyAsync(d_tok, tokens + t0, nt * 4, cudaMemcpyHostToDevice, s));
-        CU(ctx, cudaMemcpyAsync(d_seq, rel, ((size_t)nr + 1) * 8, cudaMemcpyHostToDevice, s));
-        CU(ctx, cudaMemcpyAsync(d_coff, rel + nr + 1, ((size_t)nr + 1) * 8,
-                                cudaMemcpyHostToDevice, s));
-        if (start_chunk)
-            CU(ctx, cudaMemcpyAsync(d_start, start_chunk + a, (size_t)nr * 4, cudaMemcpyHostToDevice, s));
-        if (with_blob)
-            CU(ctx, cudaMemcpyAsync(d_pages, page_table + coff[a], m * 4, cudaMemcpyHostToDevice, s));
-        rc = lsmkv_encode_batch(ctx, stream, nr, d_tok, d_seq, start_chunk ? d_start : nullptr,
-                                d_coff, m, with_blob ? d_pages : nullptr, with_blob ? pool : nullptr,
+        at += (size_t)(b - a) + 1;
+    }
+    if (nt) CU(ctx, copy_pieces(d_tok, tokens + t_first, nt * 4, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(d_seq, h_seq, n_rel * 8, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(d_coff, h_coff, n_rel * 8, cudaMemcpyHostToDevice, s));
+    if (start_chunk)
+        CU(ctx, cudaMemcpyAsync(d_start, start_chunk, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
+    if (with_blob)
+        CU(ctx, copy_pieces(d_pages, page_table, n_chunks * 4, cudaMemcpyHostToDevice, s));
+
+    uint64_t host_used = 0;                          // compressing codec: bytes placed so far
+    at = 0;
+    for (size_t k = 0; k < n_slices; ++k) {
+        const uint32_t a = cuts[k], b = cuts[k + 1], nr = b - a;
+        const uint64_t m = coff[b] - coff[a];
+        const size_t rel_at = at;
+        at += (size_t)nr + 1;
+        if (m == 0) continue;
+        rc = lsmkv_encode_batch(ctx, stream, nr, d_tok + (seq_off[a] - t_first), d_seq + rel_at,
+                                start_chunk ? d_start + a : nullptr, d_coff + rel_at, m,
+                                with_blob ? d_pages + coff[a] : nullptr, with_blob ? pool : nullptr,
                                 file_id, base_offset + (coded ? host_used : coff[a] * cb), d_keys,
                                 d_vals, d_blob, with_blob ? m * slot : 0);
         if (rc != LSMKV_OK) return rc;
@@ -181,15 +222,14 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
             if (last.reserved == 0) return LSMKV_ECAPACITY;   // stage overflow (flagged on device)
             const uint64_t used = last.offset + last.reserved - (base_offset + host_used);
             if (blob_capacity - host_used < used) return LSMKV_ECAPACITY;
-            CU(ctx, cudaMemcpyAsync(static_cast<unsigned char *>(blob_out) + host_used, d_blob, used,
-                                    cudaMemcpyDeviceToHost, s));
+            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + host_used, d_blob, used,
+                                cudaMemcpyDeviceToHost, s));
             host_used += used;
             if (blob_bytes_out) *blob_bytes_out = host_used;
         } else if (with_blob) {
-            CU(ctx, cudaMemcpyAsync(static_cast<unsigned char *>(blob_out) + coff[a] * cb, d_blob,
-                                    m * cb, cudaMemcpyDeviceToHost, s));
+            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + coff[a] * cb, d_blob, m * cb,
+                                cudaMemcpyDeviceToHost, s));
         }
-        a = b;
     }
     return LSMKV_OK;
 }
@@ -279,87 +319,99 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
         total_hits += hit_chunks[q];
     }
     if (total_hits == 0) return LSMKV_OK;
+    if (total_hits >= 0xFFFFFFFFull) return LSMKV_EINVAL;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // a slice holds at most m_max chunks and stage_bytes bytes of blobs (at least one blob)
-    const uint64_t stage_bytes_max = std::max<uint64_t>((uint64_t)ctx->host_stage_bytes, max_len);
-    const uint64_t stage_chunks = std::max<uint64_t>(1, stage_bytes_max / min_len);
-    const uint64_t m_max = std::min<uint64_t>(stage_chunks, total_hits);
-    const uint64_t blob_stage = coded ? stage_bytes_max : m_max * cb;
-    size_t need = pad256(blob_stage) + pad256(m_max * 16) + pad256(m_max * 4) + 3 * 256 + 4096;
+    // a slice holds at most blob_stage bytes of blobs (always at least one blob)
+    const uint64_t blob_stage = std::max<uint64_t>((uint64_t)ctx->host_stage_bytes, max_len);
+
+    // pass 1 (host): where each slice starts, then the stage-relative records and destination
+    // pages of every hit chunk, in hit order
+    std::vector<uint64_t> &first = ctx->h_off_a;                     // first hit of every slice
+    first.clear();
+    uint64_t k = 0, at = 0, m_max = 0;
+    for (uint32_t q = 0; q < n_query; ++q) {
+        for (uint64_t j = 0; j < hit_chunks[q]; ++j, ++k) {
+            const uint64_t len = coded ? recs[qchunk_off[q] + j].reserved : cb;
+            if (first.empty() || at + len > blob_stage) { first.push_back(k); at = 0; }
+            at += len;
+        }
+    }
+    first.push_back(total_hits);
+    const size_t n_slices = first.size() - 1;
+    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices * 24 + 4096);
+    if (!lease.ok()) return LSMKV_ENOMEM;
+    lsmkv_val_t *h_recs = lease.take<lsmkv_val_t>(total_hits);
+    uint32_t *h_pages = lease.take<uint32_t>(total_hits);
+    uint64_t *h_qoff = lease.take<uint64_t>(2 * n_slices);           // {0, m} per slice
+    uint32_t *h_hit = lease.take<uint32_t>(n_slices);                // m per slice
+    k = 0;
+    size_t sl_at = 0;
+    for (uint32_t q = 0; q < n_query; ++q) {
+        for (uint64_t j = 0; j < hit_chunks[q]; ++j, ++k) {
+            const uint64_t idx = qchunk_off[q] + j;
+            if (sl_at + 1 < first.size() && k == first[sl_at + 1]) ++sl_at;
+            if (k == first[sl_at]) at = 0;
+            h_recs[k] = lsmkv_val_t{0, coded ? recs[idx].reserved : 0u, at};
+            h_pages[k] = dst_page_table[idx];
+            at += coded ? recs[idx].reserved : cb;
+        }
+    }
+    for (size_t sl = 0; sl < n_slices; ++sl) {
+        m_max = std::max(m_max, first[sl + 1] - first[sl]);
+        h_qoff[2 * sl] = 0;
+        h_qoff[2 * sl + 1] = first[sl + 1] - first[sl];
+        h_hit[sl] = (uint32_t)(first[sl + 1] - first[sl]);
+    }
+    (void)m_max;
+
+    size_t need = pad256(blob_stage) + pad256(total_hits * 16) + pad256(total_hits * 4) +
+                  pad256(n_slices * 16) + pad256(n_slices * 4) + 4096;
     int rc = ensure_io(ctx, 2, need);
     if (rc != LSMKV_OK) return rc;
     IoLayout io(ctx->d_io[2]);
     unsigned char *d_blob = io.take<unsigned char>(blob_stage);
-    lsmkv_val_t *d_recs = io.take<lsmkv_val_t>(m_max);
-    uint32_t *d_pages = io.take<uint32_t>(m_max);
-    uint64_t *d_qoff = io.take<uint64_t>(2);
-    uint32_t *d_hit = io.take<uint32_t>(1);
+    lsmkv_val_t *d_recs = io.take<lsmkv_val_t>(total_hits);
+    uint32_t *d_pages = io.take<uint32_t>(total_hits);
+    uint64_t *d_qoff = io.take<uint64_t>(2 * n_slices);
+    uint32_t *d_hit = io.take<uint32_t>(n_slices);
     const void *stage_arena[1] = {d_blob};
+    // every descriptor goes up first, so that nothing small queues behind the blob copies
+    CU(ctx, copy_pieces(d_recs, h_recs, total_hits * 16, cudaMemcpyHostToDevice, s));
+    CU(ctx, copy_pieces(d_pages, h_pages, total_hits * 4, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(d_qoff, h_qoff, n_slices * 16, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(d_hit, h_hit, n_slices * 4, cudaMemcpyHostToDevice, s));
 
-    // descriptors of all hit chunks (each slice uploads its part), plus 32 bytes per slice
-    // every slice stages at least one chunk, and at least half the stage unless blobs are huge
-    uint64_t n_slices_max = total_hits;
-    if (max_len <= blob_stage / 2)
-        n_slices_max = std::min<uint64_t>(total_hits, 2 * (sum_len / blob_stage) + total_hits / m_max + 2);
-    n_slices_max = std::min<uint64_t>(n_slices_max, 1u << 20);
-    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices_max * 48 + 4096);
-    if (!lease.ok()) return LSMKV_ENOMEM;
-    lsmkv_val_t *srecs_all = lease.take<lsmkv_val_t>(total_hits);
-    uint32_t *spages_all = lease.take<uint32_t>(total_hits);
+    // pass 2: per slice, the blobs go to the stage in hit order (blobs that sit back to back in
+    // a host arena travel as one run of copies) and are scattered into the pool
+    k = 0;
     uint32_t q = 0;
-    uint64_t j = 0, left = total_hits, done = 0, slices = 0;
-    while (q < n_query && left) {
-        // one slice: up to m_max hit chunks and blob_stage bytes, blobs gathered into the stage
-        // in hit order; blobs that sit back to back in a host arena travel as one copy
-        const uint64_t cap = std::min<uint64_t>(m_max, left);
-        lsmkv_val_t *srecs = srecs_all + done;
-        uint32_t *spages = spages_all + done;
-        uint64_t m = 0, at = 0;              // chunks and bytes staged in this slice
-        uint64_t run_dst = 0;                // stage offset of the pending contiguous copy
+    uint64_t j = 0;
+    for (size_t sl = 0; sl < n_slices; ++sl) {
+        const uint64_t m = first[sl + 1] - first[sl];
+        uint64_t run_dst = 0, run_bytes = 0, stage_used = 0;
         const unsigned char *run_src = nullptr;
-        uint64_t run_bytes = 0;
-        while (q < n_query && m < cap) {
-            if (j >= hit_chunks[q]) { ++q; j = 0; continue; }
-            const uint64_t idx = qchunk_off[q] + j;
-            const lsmkv_val_t &r = recs[idx];
+        for (uint64_t c = 0; c < m; ++c, ++k) {
+            while (j >= hit_chunks[q]) { ++q; j = 0; }
+            const lsmkv_val_t &r = recs[qchunk_off[q] + j];
+            ++j;
             const uint64_t len = coded ? r.reserved : cb;
-            if (at + len > blob_stage) break;                    // slice is full (m >= 1 here)
             const unsigned char *src = static_cast<const unsigned char *>(arenas[r.file_id]) + r.offset;
             if (run_bytes && src == run_src + run_bytes) {
                 run_bytes += len;
             } else {
                 if (run_bytes)
-                    CU(ctx, cudaMemcpyAsync(d_blob + run_dst, run_src, run_bytes,
-                                            cudaMemcpyHostToDevice, s));
-                run_dst = at;
+                    CU(ctx, copy_pieces(d_blob + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
+                run_dst = h_recs[k].offset;
                 run_src = src;
                 run_bytes = len;
             }
-            srecs[m] = lsmkv_val_t{0, coded ? r.reserved : 0u, at};
-            spages[m] = dst_page_table[idx];
-            at += len;
-            ++m;
-            ++j;
+            stage_used = h_recs[k].offset + len;
         }
         if (run_bytes)
-            CU(ctx, cudaMemcpyAsync(d_blob + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
-        if (m == 0) break;
-        left -= m;
-        done += m;
-        if (++slices > n_slices_max) return LSMKV_EINVAL;     // cannot happen: see the bound above
-        uint64_t *qoff2 = lease.take<uint64_t>(2);
-        uint32_t *hit1 = lease.take<uint32_t>(1);
-        qoff2[0] = 0;
-        qoff2[1] = m;
-        *hit1 = (uint32_t)m;
-        CU(ctx, cudaMemcpyAsync(d_recs, srecs, m * 16, cudaMemcpyHostToDevice, s));
-        CU(ctx, cudaMemcpyAsync(d_pages, spages, m * 4, cudaMemcpyHostToDevice, s));
-        CU(ctx, cudaMemcpyAsync(d_qoff, qoff2, 16, cudaMemcpyHostToDevice, s));
-        CU(ctx, cudaMemcpyAsync(d_hit, hit1, 4, cudaMemcpyHostToDevice, s));
-        const uint64_t stage_bytes = at;
-        rc = lsmkv_decode_batch(ctx, stream, 1, d_qoff, m, d_hit, d_recs, stage_arena, &stage_bytes,
-                                1, d_pages, pool);
+            CU(ctx, copy_pieces(d_blob + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
+        rc = lsmkv_decode_batch(ctx, stream, 1, d_qoff + 2 * sl, m, d_hit + sl, d_recs + first[sl],
+                                stage_arena, &stage_used, 1, d_pages + first[sl], pool);
         if (rc != LSMKV_OK) return rc;
     }
     return LSMKV_OK;
