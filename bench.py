@@ -223,8 +223,9 @@ def main():
     from paper_2511_16138_b200 import lsmkv, ranks
 
     rank, world, local_rank = ranks.rank_env()
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:    # launched by torch.distributed.run
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -232,7 +233,7 @@ def main():
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
+        if dist.is_initialized():
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -472,7 +473,7 @@ def main():
             },
         }
         print(json.dumps(out))
-    if world > 1:
+    if dist.is_initialized():
         dist.destroy_process_group()
 
 
