@@ -136,3 +136,23 @@ def test_bad_inputs_are_flagged_and_skipped_without_faulting():
         assert e.value.code == lsmkv.ECAPACITY
         with pytest.raises(lsmkv.LsmkvError):
             ctx.set_tuning("no_such_knob", 1)
+
+
+def test_extreme_token_ids_and_namespace():
+    """Token ids up to 2^32-1 (t + 1 needs 33 bits), the largest namespace, and sequences built
+    from the token triples whose digest is exactly zero."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "digest_zero_sequences.json")) as f:
+        zero = json.load(f)["zero_digest"]
+    g = lsmkv.Geom(2, 1, 32, page_tokens=3, chunk_tokens=3, ns=0xFFFFFFFF)   # 192-byte pages
+    rng = np.random.default_rng(12)
+    seqs = [np.full(3 * 40, 0xFFFFFFFF, dtype=np.uint32),
+            rng.integers(2**32 - 5, 2**32, 3 * 33 + 1, dtype=np.uint64).astype(np.uint32),
+            np.array(zero[0] * 7, dtype=np.uint32),          # lane A digest returns to 0 every chunk
+            np.array(zero[1] * 5 + [1, 2], dtype=np.uint32),
+            np.zeros(3 * 35, dtype=np.uint32)]
+    store = synth.make_batch(seqs)
+    query = synth.make_batch([s.copy() for s in seqs] + [np.array(zero[0] * 9, dtype=np.uint32)])
+    out = H.roundtrip(g, store, query, n_runs=2, seed=13)
+    assert list(out["hit"]) == [40, 33, 7, 5, 35, 7]
