@@ -489,8 +489,13 @@ int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint3
 
     {
         LaunchTimer timer(ctx, s, LSMKV_K_KEYS);
-        const unsigned grid = warp_grid(ctx, n_req, 128, 16);
-        k_encode_keys<<<grid, 128, 0, s>>>(ctx->kc, ctx->geom.chunk_tokens, ctx->geom.ns, n_req,
+        // few long requests: wide CTAs; many requests: narrower ones, more of them resident
+        const unsigned warps = n_req < (unsigned)ctx->sm_count ? 8u : 4u;
+        uint64_t grid = n_req;
+        const uint64_t cap = (uint64_t)ctx->sm_count * (2048u / (warps * 32u));
+        if (grid > cap) grid = cap;
+        k_encode_keys<<<(unsigned)grid, warps * 32u, 0, s>>>(ctx->kc, ctx->geom.chunk_tokens,
+                                           ctx->geom.ns, n_req,
                                            tokens, seq_off, start_chunk, chunk_off, n_chunks,
                                            file_id, base_offset, ctx->chunk_bytes, keys_out,
                                            vals_out, ctx->d_status);

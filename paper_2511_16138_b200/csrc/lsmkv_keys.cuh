@@ -144,6 +144,43 @@ __device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const u
     return k;
 }
 
+constexpr int kKeyMaxWarps = 16;
+
+// One CTA of W warps, 32*W consecutive chunks starting at `base`: warp w hashes the 32-chunk
+// block base + 32*w, the block digests are exchanged through shared memory and chained, so every
+// thread ends up with the key of chunk base + 32*warp + lane. cA/cB carry the digest of the
+// prefix before `base` from round to round (same value in every thread). Contains one
+// __syncthreads(); the caller must put another one between two calls (s_agg* are rewritten).
+__device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
+                                                   uint32_t C, uint32_t ns, uint64_t base,
+                                                   uint64_t nch, uint64_t &cA, uint64_t &cB,
+                                                   uint64_t *s_aggA, uint64_t *s_aggB)
+{
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
+    uint64_t hA, hB;
+    uint32_t first, last;
+    warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
+    if (lane == 31) { s_aggA[warp] = hA; s_aggB[warp] = hB; }
+    __syncthreads();
+    uint64_t pA = cA, pB = cB;                 // prefix before block v, advanced block by block
+    for (unsigned v = 0; v < W; ++v) {
+        if (v == warp) {
+            hA = addmod61(mulmod61(pA, kc.pwA[lane]), hA);
+            hB = addmod61(mulmod61(pB, kc.pwB[lane]), hB);
+        }
+        pA = addmod61(mulmod61(pA, kc.pwA[31]), s_aggA[v]);
+        pB = addmod61(mulmod61(pB, kc.pwB[31]), s_aggB[v]);
+    }
+    cA = pA;                                   // meaningful when the round was full
+    cB = pB;
+    ChunkKey k;
+    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)(base + 32ull * warp + lane);
+    k.w1 = hA;
+    k.w2 = hB;
+    k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
+    return k;
+}
+
 __device__ __forceinline__ void store_key(lsmkv_key_t *dst, const ChunkKey &k)
 {
     ulonglong2 *p = reinterpret_cast<ulonglong2 *>(dst);
@@ -151,8 +188,9 @@ __device__ __forceinline__ void store_key(lsmkv_key_t *dst, const ChunkKey &k)
     p[1] = make_ulonglong2(k.w2, k.w3);
 }
 
-// put_batch keys + records: one warp per request.
-__global__ void __launch_bounds__(128)
+// put_batch keys + records: one CTA per request at a time (requests handed out round-robin),
+// 32 * W chunks per round.
+__global__ void __launch_bounds__(512)
 k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uint32_t n_req,
               const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
               const uint32_t *__restrict__ start_chunk, const uint64_t *__restrict__ chunk_off,
@@ -160,24 +198,24 @@ k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uin
               lsmkv_key_t *__restrict__ keys_out, lsmkv_val_t *__restrict__ vals_out,
               DevStatus *st)
 {
-    const unsigned lane = lane_id();
-    const uint64_t warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-    for (uint64_t r = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n_req;
-         r += warps) {
+    __shared__ uint64_t s_aggA[kKeyMaxWarps], s_aggB[kKeyMaxWarps];
+    const uint64_t round_chunks = 32ull * (blockDim.x >> 5);
+    for (uint64_t r = blockIdx.x; r < n_req; r += gridDim.x) {
         const uint64_t s0 = seq_off[r], s1 = seq_off[r + 1];
         const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
         const uint64_t start = start_chunk ? start_chunk[r] : 0;
         const uint64_t cnt = nch > start ? nch - start : 0;
         const uint64_t o0 = chunk_off[r], o1 = chunk_off[r + 1];
         if (s1 < s0 || o1 < o0 || o1 - o0 != cnt || o1 > n_chunks || nch > 0xFFFFFFFFull) {
-            if (lane == 0) st_flag(st, LSMKV_ST_BAD_COUNT, r);
-            continue;
+            if (threadIdx.x == 0) st_flag(st, LSMKV_ST_BAD_COUNT, r);
+            continue;                                        // uniform over the CTA
         }
         if (cnt == 0) continue;
         uint64_t cA = 0, cB = 0;
-        for (uint64_t base = 0; base < nch; base += 32) {
-            const ChunkKey k = warp_chunk_keys(kc, tokens + s0, C, ns, base, nch, cA, cB);
-            const uint64_t j = base + lane;
+        for (uint64_t base = 0; base < nch; base += round_chunks) {
+            const ChunkKey k = cta_chunk_keys(kc, tokens + s0, C, ns, base, nch, cA, cB, s_aggA,
+                                              s_aggB);
+            const uint64_t j = base + threadIdx.x;           // = base + 32 * warp + lane
             if (j >= start && j < nch) {
                 const uint64_t i = o0 + (j - start);
                 store_key(keys_out + i, k);
@@ -189,8 +227,9 @@ k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uin
                 v.w = (uint32_t)(off >> 32);
                 *reinterpret_cast<uint4 *>(vals_out + i) = v;
             }
+            __syncthreads();
         }
-        if (lane == 0) atomicAdd(&st->chunks_encoded, (unsigned long long)cnt);
+        if (threadIdx.x == 0) atomicAdd(&st->chunks_encoded, (unsigned long long)cnt);
     }
 }
 

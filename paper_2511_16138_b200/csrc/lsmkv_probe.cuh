@@ -193,8 +193,6 @@ __device__ __forceinline__ bool lookup_runs(const RunTable &rt, uint32_t n_runs,
     return false;
 }
 
-constexpr int kProbeMaxWarps = 16;
-
 __global__ void __launch_bounds__(512)
 k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable rt,
         uint32_t n_runs, const uint64_t *__restrict__ dir, uint32_t jcap, uint32_t C,
@@ -203,7 +201,7 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         uint64_t n_qchunks, uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out,
         lsmkv_key_t *__restrict__ keys_out, DevStatus *st, unsigned long long *next_query)
 {
-    __shared__ uint64_t s_aggA[kProbeMaxWarps], s_aggB[kProbeMaxWarps];
+    __shared__ uint64_t s_aggA[kKeyMaxWarps], s_aggB[kKeyMaxWarps];
     __shared__ unsigned long long s_first_miss, s_q;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
     const uint64_t round_chunks = 32ull * W;
@@ -236,24 +234,7 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                 continue;
             }
             if (threadIdx.x == 0) s_first_miss = ~0ull;
-            uint64_t hA, hB;
-            uint32_t first, last;
-            warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
-            if (lane == 31) { s_aggA[warp] = hA; s_aggB[warp] = hB; }
-            __syncthreads();
-            // prefix before this warp's block: chain the digests of the blocks before it
-            uint64_t pA = cA, pB = cB;
-            for (unsigned v = 0; v < W; ++v) {
-                if (v == warp) { hA = addmod61(mulmod61(pA, kc.pwA[lane]), hA);
-                                 hB = addmod61(mulmod61(pB, kc.pwB[lane]), hB); }
-                pA = addmod61(mulmod61(pA, kc.pwA[31]), s_aggA[v]);
-                pB = addmod61(mulmod61(pB, kc.pwB[31]), s_aggB[v]);
-            }
-            cA = pA; cB = pB;                                // valid when the round was full
-            ChunkKey k;
-            k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)j;
-            k.w1 = hA; k.w2 = hB;
-            k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
+            const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, cA, cB, s_aggA, s_aggB);
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
             if (done) {
                 if (valid) recs[j] = zero;
