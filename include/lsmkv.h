@@ -10,7 +10,8 @@
  *     except that device work enqueued by the call reads/writes the [dev] buffers until the
  *     stream reaches the point following the call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Every
- *     batch call only enqueues work and returns; none of them synchronises.
+ *     batch call only enqueues work and returns; none of them synchronises (one documented
+ *     exception: lsmkv_put_batch_host with the compressing codec).
  *   - Return value: 0 = enqueued, negative = LSMKV_E* and nothing was enqueued.
  *   - Problems only the GPU can see (a page id beyond the pool, a record that points outside
  *     its arena, a misaligned buffer, a wait that ran out) never fault: the offending item is
@@ -19,9 +20,10 @@
  *     scratch (two probes, two decodes, two flushes/merges, two host-buffer calls of the same
  *     kind) must be ordered by the caller -- same stream, or events. A put on one stream and a
  *     probe/decode on another are independent. Use one context per stream for more.
- *   - No call allocates device memory except lsmkv_create(), lsmkv_reserve() and a batch call
- *     whose batch is larger than any before it (the internal workspace grows; call
- *     lsmkv_reserve() up front to rule that out).
+ *   - No call allocates device memory except lsmkv_create(), lsmkv_reserve() and a call whose
+ *     batch is larger than any before it (the internal scratch of that kind of call grows;
+ *     lsmkv_reserve() pre-sizes the scratch of probe and decode, a first full-size call that
+ *     of flush, merge, the compressing codec and the host-buffer calls).
  *
  * Formats (version 1). The paper states properties (key order follows token-prefix order;
  * index values are a file identifier plus a byte offset; a batch's tensors are stored
@@ -32,7 +34,8 @@
  *             w3 = (first token of chunk j << 32) | last token of chunk j
  *   digest  h <- 0; per token t: h <- (h*BASE + t + 1) mod (2^61 - 1), canonical in [0, 2^61-1)
  *             BASE_A = 0x0B4E0EF37BC32127, BASE_B = 0x16A09E667F3BCC90
- *   record  {u32 file_id, u32 reserved = 0, u64 offset}; the blob length is chunk_bytes
+ *   record  {u32 file_id, u32 reserved, u64 offset}; identity codec: reserved = 0 and the blob
+ *             length is chunk_bytes; compressing codec: reserved = the blob's length
  *   pool    2L buffers: K of layers 0..L-1, then V of layers 0..L-1, each
  *             [num_pages][page_tokens][n_kv_heads][head_dim] elements (a page slab of
  *             page_bytes = page_tokens*n_kv_heads*head_dim*elem_bytes is contiguous)
