@@ -134,6 +134,8 @@ def lib() -> C.CDLL:
         _lib.orc_decode_batch_xp12.argtypes = [
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
+        _lib.orc_relocate_records.restype = C.c_uint64
+        _lib.orc_relocate_records.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32]
         _lib.orc_probe_batch.restype = C.c_int
         _lib.orc_probe_batch.argtypes = [
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -391,3 +393,14 @@ def decode_batch_xp12(g: Geom, qchunk_off, hit, recs, arenas, dst_page_table, po
                                      _pool_ptrs(pool), pool.shape[1])
     if rc != OK:
         raise OracleError(rc)
+
+
+RELOC_DTYPE = np.dtype([("old_file", "<u4"), ("new_file", "<u4"), ("delta", "<u8")])
+
+
+def relocate_records(vals, table):
+    """Copy of ``vals`` with the relocation table applied, and the number of records changed."""
+    v = np.ascontiguousarray(vals, dtype=VAL_DTYPE).copy()
+    t = np.ascontiguousarray(table, dtype=RELOC_DTYPE)
+    changed = lib().orc_relocate_records(_p(v), len(v), _p(t), len(t))
+    return v, int(changed)

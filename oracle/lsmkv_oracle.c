@@ -566,3 +566,27 @@ int orc_decode_batch_xp12(const orc_geom *g, uint32_t n_query, const uint64_t *q
     }
     return ORC_OK;
 }
+
+/* ---- tensor-file merging (Sec. 3.4 "Automatic Tensor File Merging"): when adjacent tensor files
+ * are merged into one, the file identifier and offset stored in the index are updated. A
+ * relocation entry says: records of file `old_file` now live in `new_file`, `delta` bytes
+ * further in. Records of files not in the table stay as they are. Returns the number of
+ * records changed.
+ */
+typedef struct { uint32_t old_file, new_file; uint64_t delta; } orc_reloc;
+
+uint64_t orc_relocate_records(orc_val *vals, uint64_t n, const orc_reloc *table, uint32_t n_table)
+{
+    uint64_t changed = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        for (uint32_t t = 0; t < n_table; ++t) {
+            if (vals[i].file_id == table[t].old_file) {      /* first matching entry applies */
+                vals[i].file_id = table[t].new_file;
+                vals[i].offset += table[t].delta;
+                ++changed;
+                break;
+            }
+        }
+    }
+    return changed;
+}

@@ -132,3 +132,27 @@ def test_merge_runs_equals_dict_union_newest_wins():
         assert (a is None) == (b is None)
         if a is not None:
             assert a[0] == b[0]
+
+
+def test_relocate_records_equals_a_numpy_rewrite():
+    """Merging tensor files moves records: file ids are renamed and offsets shifted; records of
+    other files are untouched."""
+    rng = np.random.default_rng(8)
+    v = np.zeros(500, dtype=VAL_DTYPE)
+    v["file_id"] = rng.integers(0, 6, 500)
+    v["reserved"] = rng.integers(0, 99, 500)
+    v["offset"] = rng.integers(0, 1 << 40, 500)
+    table = np.array([(1, 0, 1 << 33), (2, 0, 5 << 33), (4, 3, 4096)], dtype=oracle.RELOC_DTYPE)
+    got, changed = oracle.relocate_records(v, table)
+    want = v.copy()
+    for old, new, delta in table.tolist():
+        m = v["file_id"] == old
+        want["file_id"][m] = new
+        want["offset"][m] = v["offset"][m] + np.uint64(delta)
+    assert np.array_equal(got, want) and changed == int(np.isin(v["file_id"], [1, 2, 4]).sum())
+    assert np.array_equal(got["reserved"], v["reserved"])
+    # chained names are not followed: 0 -> 7 does not re-move what 1 -> 0 just moved
+    got2, _ = oracle.relocate_records(v, np.array([(1, 0, 8), (0, 7, 16)], dtype=oracle.RELOC_DTYPE))
+    assert set(got2["file_id"][v["file_id"] == 1]) == {0}
+    assert np.array_equal(got2["offset"][v["file_id"] == 0], v["offset"][v["file_id"] == 0] + np.uint64(16))
+    assert oracle.relocate_records(v, np.zeros(0, oracle.RELOC_DTYPE))[1] == 0
