@@ -215,6 +215,18 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
 
 /*
+ * Record relocation (Sec. 3.4 "Automatic Tensor File Merging": when tensor files are merged,
+ * the file_id + offset values in the index are updated). Every record of vals [dev, n entries,
+ * rewritten in place -- typically the vals array of a run] whose file_id equals table[t].old_file
+ * gets file_id = table[t].new_file and offset += table[t].delta; the first matching entry
+ * applies, other records are untouched. table [host], n_table <= 64. changed_out [dev,
+ * optional] receives the number of records rewritten.
+ */
+typedef struct { uint32_t old_file, new_file; uint64_t delta; } lsmkv_reloc_t;
+int lsmkv_relocate_records(lsmkv_ctx *ctx, void *stream, lsmkv_val_t *vals, uint64_t n,
+                           const lsmkv_reloc_t *table, uint32_t n_table, uint64_t *changed_out);
+
+/*
  * Compressing codec LSMKV_CODEC_XP12 (Sec. 3.4 "Batch Codec Operations": combined tensors are
  * compressed before storage and decompressed together on load; the paper names no algorithm,
  * this one is lossless so restored pages stay bit-exact). Selected per context through

@@ -765,6 +765,31 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
                          n_out);
 }
 
+int lsmkv_relocate_records(lsmkv_ctx *ctx, void *stream, lsmkv_val_t *vals, uint64_t n,
+                           const lsmkv_reloc_t *table, uint32_t n_table, uint64_t *changed_out)
+{
+    if (!ctx || (n && (!vals || !aligned16(vals))) || n_table > (uint32_t)kMaxReloc ||
+        (n_table && !table))
+        return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (changed_out) CU(ctx, cudaMemsetAsync(changed_out, 0, sizeof(uint64_t), s));
+    if (n == 0 || n_table == 0) return LSMKV_OK;
+    RelocTable tab;
+    std::memset(&tab, 0, sizeof(tab));
+    tab.n = n_table;
+    for (uint32_t t = 0; t < n_table; ++t) {
+        tab.old_file[t] = table[t].old_file;
+        tab.new_file[t] = table[t].new_file;
+        tab.delta[t] = table[t].delta;
+    }
+    k_relocate_records<<<merge_grid(ctx, n), 256, 0, s>>>(
+        vals, n, tab, reinterpret_cast<unsigned long long *>(changed_out));
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
 uint64_t lsmkv_encode_bound(const lsmkv_ctx *ctx, uint64_t n_chunks)
 {
     if (!ctx) return 0;

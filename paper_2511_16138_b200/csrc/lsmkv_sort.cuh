@@ -180,4 +180,37 @@ k_dedupe_scatter(const lsmkv_key_t *__restrict__ keys, const uint32_t *__restric
     }
 }
 
+// Tensor-file merging: records of a merged file get their new file id and shifted offset.
+constexpr int kMaxReloc = 64;
+struct RelocTable {
+    uint32_t old_file[kMaxReloc], new_file[kMaxReloc];
+    uint64_t delta[kMaxReloc];
+    uint32_t n;
+};
+
+__global__ void __launch_bounds__(256)
+k_relocate_records(lsmkv_val_t *__restrict__ vals, uint64_t n, const __grid_constant__ RelocTable tab,
+                   unsigned long long *__restrict__ changed_out)
+{
+    unsigned long long mine = 0;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        uint4 r = reinterpret_cast<uint4 *>(vals)[i];
+        for (uint32_t t = 0; t < tab.n; ++t) {
+            if (r.x == tab.old_file[t]) {                    // first matching entry applies
+                const uint64_t off = ((uint64_t)r.z | ((uint64_t)r.w << 32)) + tab.delta[t];
+                r.x = tab.new_file[t];
+                r.z = (uint32_t)off;
+                r.w = (uint32_t)(off >> 32);
+                reinterpret_cast<uint4 *>(vals)[i] = r;
+                ++mine;
+                break;
+            }
+        }
+    }
+#pragma unroll
+    for (unsigned d = 16; d; d >>= 1) mine += __shfl_down_sync(0xFFFFFFFFu, mine, d);
+    if (lane_id() == 0 && mine && changed_out) atomicAdd(changed_out, mine);
+}
+
 }  // namespace lsmkv

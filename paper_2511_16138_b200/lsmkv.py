@@ -26,6 +26,7 @@ EXPORTS = (
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
     "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
+    "lsmkv_relocate_records",
 )
 ST_OVERFLOW = 32
 CODEC_IDENTITY, CODEC_XP12 = 0, 1
@@ -74,6 +75,10 @@ class StatusStruct(C.Structure):
                 ("chunks_encoded", C.c_uint64), ("lookups", C.c_uint64),
                 ("chunks_hit", C.c_uint64), ("empty_probes", C.c_uint64),
                 ("chunks_decoded", C.c_uint64)]
+
+
+class RelocStruct(C.Structure):
+    _fields_ = [("old_file", C.c_uint32), ("new_file", C.c_uint32), ("delta", C.c_uint64)]
 
 
 class ProfileStruct(C.Structure):
@@ -145,6 +150,8 @@ def lib() -> C.CDLL:
     L.lsmkv_decode_batch_host.restype = C.c_int
     L.lsmkv_decode_batch_host.argtypes = [vp, vp, u32, vp, vp, vp, C.POINTER(vp),
                                           C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
+    L.lsmkv_relocate_records.restype = C.c_int
+    L.lsmkv_relocate_records.argtypes = [vp, vp, vp, u64, C.POINTER(RelocStruct), u32, vp]
     L.lsmkv_encode_bound.restype = u64
     L.lsmkv_encode_bound.argtypes = [vp, u64]
     L.lsmkv_bloom_blocks.restype = u64
@@ -326,6 +333,14 @@ def lsmkv_decode_batch_host(ctx, stream, n_query, qchunk_off, hit_chunks, recs, 
     _check(ctx, rc, "lsmkv_decode_batch_host")
 
 
+def lsmkv_relocate_records(ctx, stream, vals, n, table, changed_out=None) -> None:
+    """table: sequence of (old_file, new_file, delta)."""
+    arr = (RelocStruct * max(1, len(table)))(*[RelocStruct(*t) for t in table])
+    rc = lib().lsmkv_relocate_records(ctx, _stream(stream), _ptr(vals), n, arr, len(table),
+                                      _ptr(changed_out))
+    _check(ctx, rc, "lsmkv_relocate_records")
+
+
 def lsmkv_encode_bound(ctx, n_chunks: int) -> int:
     return int(lib().lsmkv_encode_bound(ctx, n_chunks))
 
@@ -470,6 +485,9 @@ class Context:
                           pool, stream=None):
         lsmkv_decode_batch_host(self.handle, stream, n_query, qchunk_off, hit_chunks, recs,
                                 arenas, dst_page_table, pool)
+
+    def relocate_records(self, vals, n, table, changed_out=None, stream=None):
+        lsmkv_relocate_records(self.handle, stream, vals, n, table, changed_out)
 
     def encode_bound(self, n_chunks: int) -> int:
         return lsmkv_encode_bound(self.handle, n_chunks)

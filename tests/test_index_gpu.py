@@ -129,3 +129,25 @@ def test_flush_argument_checks():
             ctx.flush_batch(None, z, 1, z, z, z)
         with pytest.raises(lsmkv.LsmkvError):
             ctx.merge_runs([(z, z, 1)] * 65, z, z, z)
+
+
+def test_relocate_records_equals_oracle():
+    rng = np.random.default_rng(31)
+    n = 70001
+    v = np.zeros(n, dtype=VAL_DTYPE)
+    v["file_id"] = rng.integers(0, 7, n)
+    v["reserved"] = rng.integers(0, 2**32, n, dtype=np.uint64).astype(np.uint32)
+    v["offset"] = rng.integers(0, 1 << 44, n, dtype=np.uint64)
+    table = [(1, 0, 1 << 35), (2, 0, 3 << 35), (5, 4, 4096), (0, 9, 16)]
+    want, changed = oracle.relocate_records(v, np.array(table, dtype=oracle.RELOC_DTYPE))
+    with lsmkv.Context(G, 0) as ctx:
+        dv = H.dev(v)
+        cnt = torch.full((1,), -1, dtype=torch.int64, device=H.DEV)
+        ctx.relocate_records(dv, n, table, cnt)
+        torch.cuda.synchronize()
+        assert np.array_equal(H.host(dv, VAL_DTYPE, n * 16), want) and int(cnt.item()) == changed
+        ctx.relocate_records(dv, n, [], cnt)                   # empty table: nothing changes
+        torch.cuda.synchronize()
+        assert np.array_equal(H.host(dv, VAL_DTYPE, n * 16), want) and int(cnt.item()) == 0
+        with pytest.raises(lsmkv.LsmkvError):
+            ctx.relocate_records(dv, n, [(0, 1, 0)] * 65, cnt)
