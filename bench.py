@@ -220,7 +220,9 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2511_16138_b200 import lsmkv, ranks
+    from paper_2511_16138_b200 import build, lsmkv, ranks
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        build.build()          # no-op when liblsmkv.so is newer than its sources
 
     rank, world, local_rank = ranks.rank_env()
     if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:    # launched by torch.distributed.run

@@ -8,6 +8,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Compile the CUDA library (nvcc, in-tree) when it is missing or older than its sources,
+    so that a fresh checkout tests the code it contains."""
+    from paper_2511_16138_b200 import build
+    build.build()
+    yield
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
