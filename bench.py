@@ -223,6 +223,10 @@ def main():
     from paper_2511_16138_b200 import build, lsmkv, ranks
     if int(os.environ.get("LOCAL_RANK", "0")) == 0:
         build.build()          # no-op when liblsmkv.so is newer than its sources
+    else:                      # the other ranks of the node wait for local rank 0's build
+        t_wait = time.time()
+        while build._stale() and time.time() - t_wait < 300:
+            time.sleep(0.5)
 
     rank, world, local_rank = ranks.rank_env()
     if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:    # launched by torch.distributed.run
