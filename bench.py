@@ -638,7 +638,7 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
     slots on two streams: the get of sub-batch i is enqueued, then the put of sub-batch i+1,
     so both PCIe directions are busy. `ctx` decides the codec (identity or compressing)."""
     cb = g.chunk_bytes
-    sub_cap = 2048                                   # chunks per sub-batch (4 GiB of raw blobs)
+    sub_cap = 2048 if world == 1 else 1024           # chunks per sub-batch (4 or 2 GiB of raw blobs)
     subs = []
     for d in W:
         nchw, a, acc = d["nch"], 0, 0
