@@ -156,3 +156,15 @@ def test_extreme_token_ids_and_namespace():
     query = synth.make_batch([s.copy() for s in seqs] + [np.array(zero[0] * 9, dtype=np.uint32)])
     out = H.roundtrip(g, store, query, n_runs=2, seed=13)
     assert list(out["hit"]) == [40, 33, 7, 5, 35, 7]
+
+
+@pytest.mark.parametrize("tuning", [{"probe_warps_per_cta": 1}, {"probe_warps_per_cta": 2},
+                                    {"probe_warps_per_cta": 16}, {"copy_ctas_per_sm": 4, "copy_stages": 3},
+                                    {"copy_mode": 1, "simt_ctas_per_sm": 1}])
+def test_launch_shapes_do_not_change_results(tuning):
+    """Every tuning knob is a launch shape only: long sequences (many rounds per query whatever
+    the CTA width), several runs, start chunks -- same bytes as the oracle."""
+    g = lsmkv.Geom(2, 2, 32, page_tokens=16, chunk_tokens=16)
+    w = synth.long_context(n_req=5, seq_len=16 * 530 + 7, shared=16 * 200, n_mutate=16 * 40 + 3)
+    start = np.array([0, 3, 200, 529, 600], dtype=np.uint32)
+    H.roundtrip(g, w.store, w.query, start_chunk=start, n_runs=3, tuning=tuning, seed=17)
