@@ -690,16 +690,16 @@ int lsmkv_flush_batch(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys,
     LaunchTimer timer(ctx, s, LSMKV_K_FLUSH);
     SegTable segs;
     std::memset(&segs, 0, sizeof(segs));
-    const lsmkv_key_t *src = keys;
-    const uint32_t *src_idx = nullptr;
+    // tiles of kSortTile entries are sorted in shared memory, then merged level by level
     int buf = 0;
+    k_tile_sort<<<(unsigned)((n + kSortTile - 1) / kSortTile), kSortTile / 2, 0, s>>>(
+        keys, ws.keys[0], ws.idx[0], n);
+    ++ctx->launches;
     const unsigned grid = merge_grid(ctx, n);
-    for (uint64_t width = 1;; width *= 2) {
-        k_merge_level<<<grid, 256, 0, s>>>(src, src_idx, ws.keys[buf], ws.idx[buf], n, width, segs);
+    for (uint64_t width = kSortTile; width < n; width *= 2) {
+        k_merge_level<<<grid, 256, 0, s>>>(ws.keys[buf], ws.idx[buf], ws.keys[buf ^ 1],
+                                           ws.idx[buf ^ 1], n, width, segs);
         ++ctx->launches;
-        src = ws.keys[buf];
-        src_idx = ws.idx[buf];
-        if (width * 2 >= n) break;
         buf ^= 1;
     }
     CU(ctx, cudaGetLastError());

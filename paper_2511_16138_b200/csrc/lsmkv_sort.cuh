@@ -3,8 +3,9 @@
 //
 // Both are built on one primitive, a stable pairwise merge by ranks: every element finds, with
 // one binary search in the sibling segment, how many sibling elements precede it, and that
-// count plus its own offset is its output position. A flush is a bottom-up merge sort with that
-// primitive (segments of 1, 2, 4, ... elements); a compaction concatenates the runs newest
+// count plus its own offset is its output position. A flush sorts tiles of 512 entries in shared
+// memory and then merges bottom-up with that primitive (segments of 512, 1024, ... elements); a
+// compaction concatenates the runs newest
 // first and merges neighbouring segments level by level. Ties keep left-before-right, so equal
 // keys stay in arrival order (flush: the last one survives) or in age order (compaction: the
 // first, i.e. newest, survives). A flag/scan/scatter pass then drops the losers, gathers the
@@ -89,6 +90,51 @@ k_merge_level(const lsmkv_key_t *__restrict__ src, const uint32_t *__restrict__ 
         }
         store_key4(dst + base + rank, x);
         dst_idx[base + rank] = src_idx ? src_idx[i] : (uint32_t)i;
+    }
+}
+
+// First step of a flush: every CTA sorts one tile of kSortTile entries in shared memory with a
+// bitonic network on (key, arrival index) -- the index makes the order total, so the result is
+// the stable order -- and the merge levels start from segments of kSortTile instead of 1.
+constexpr int kSortTile = 512;
+
+__device__ __forceinline__ bool entry_less(const Key4 &a, uint32_t ia, const Key4 &b, uint32_t ib)
+{
+    if (a.w0 != b.w0) return a.w0 < b.w0;
+    if (a.w1 != b.w1) return a.w1 < b.w1;
+    if (a.w2 != b.w2) return a.w2 < b.w2;
+    if (a.w3 != b.w3) return a.w3 < b.w3;
+    return ia < ib;
+}
+
+__global__ void __launch_bounds__(kSortTile / 2)
+k_tile_sort(const lsmkv_key_t *__restrict__ src, lsmkv_key_t *__restrict__ dst,
+            uint32_t *__restrict__ dst_idx, uint64_t n)
+{
+    __shared__ Key4 sk[kSortTile];
+    __shared__ uint32_t si[kSortTile];
+    const uint64_t tile0 = (uint64_t)blockIdx.x * kSortTile;
+    for (unsigned t = threadIdx.x; t < kSortTile; t += blockDim.x) {
+        const uint64_t i = tile0 + t;
+        if (i < n) { sk[t] = load_key(src + i); si[t] = (uint32_t)i; }
+        else { sk[t] = Key4{~0ull, ~0ull, ~0ull, ~0ull}; si[t] = 0xFFFFFFFFu; }   // sorts last
+    }
+    __syncthreads();
+    for (unsigned k = 2; k <= kSortTile; k <<= 1) {
+        for (unsigned j = k >> 1; j > 0; j >>= 1) {
+            const unsigned t = threadIdx.x;
+            const unsigned i = 2 * t - (t & (j - 1)), l = i + j;
+            const bool up = (i & k) == 0;
+            const Key4 a = sk[i], b = sk[l];
+            const uint32_t ia = si[i], ib = si[l];
+            const bool swap = up ? entry_less(b, ib, a, ia) : entry_less(a, ia, b, ib);
+            if (swap) { sk[i] = b; sk[l] = a; si[i] = ib; si[l] = ia; }
+            __syncthreads();
+        }
+    }
+    for (unsigned t = threadIdx.x; t < kSortTile; t += blockDim.x) {
+        const uint64_t i = tile0 + t;
+        if (i < n) { store_key4(dst + i, sk[t]); dst_idx[i] = si[t]; }
     }
 }
 

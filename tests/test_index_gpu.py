@@ -48,7 +48,7 @@ def check_padding(k, v, m):
     assert np.all(k[m:] == np.uint64(2**64 - 1)) and not v[m:].view(np.uint8).any()
 
 
-@pytest.mark.parametrize("n", [0, 1, 2, 3, 255, 256, 1000, 1025, 4097, 70000])
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 255, 256, 511, 512, 513, 1000, 1024, 1025, 4097, 70000])
 def test_flush_equals_oracle(n):
     rng = np.random.default_rng(n + 1)
     keys, vals = rand_batch(rng, n)
