@@ -460,7 +460,7 @@ def main():
                          # (traffic / algorithmic bytes = 0.9866), scaled by chunk count
                          "traffic": NCU_TRAFFIC_RATIO * algo_bytes_per_launch,
                          "traffic_source": "ncu dram__bytes_read+write on a 774-chunk launch, "
-                                           "scaled by chunks (profiles/k_copy_slabs_bulk__llama8b.md)",
+                                           "scaled by chunks (ncu summary committed with the repository)",
                          "algorithmic_bytes_per_launch": algo_bytes_per_launch,
                          "avg_launch_ms": copy_ms / max(1, copy_launches)},
             "cpu_baseline": cpu,
