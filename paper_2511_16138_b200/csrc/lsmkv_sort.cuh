@@ -111,13 +111,16 @@ __global__ void __launch_bounds__(kSortTile / 2)
 k_tile_sort(const lsmkv_key_t *__restrict__ src, lsmkv_key_t *__restrict__ dst,
             uint32_t *__restrict__ dst_idx, uint64_t n)
 {
-    __shared__ Key4 sk[kSortTile];
+    // one array per key word: neighbouring threads touch neighbouring words (no bank conflicts)
+    __shared__ uint64_t s0[kSortTile], s1[kSortTile], s2[kSortTile], s3[kSortTile];
     __shared__ uint32_t si[kSortTile];
     const uint64_t tile0 = (uint64_t)blockIdx.x * kSortTile;
     for (unsigned t = threadIdx.x; t < kSortTile; t += blockDim.x) {
         const uint64_t i = tile0 + t;
-        if (i < n) { sk[t] = load_key(src + i); si[t] = (uint32_t)i; }
-        else { sk[t] = Key4{~0ull, ~0ull, ~0ull, ~0ull}; si[t] = 0xFFFFFFFFu; }   // sorts last
+        Key4 k{~0ull, ~0ull, ~0ull, ~0ull};                  // beyond the end: sorts last
+        uint32_t id = 0xFFFFFFFFu;
+        if (i < n) { k = load_key(src + i); id = (uint32_t)i; }
+        s0[t] = k.w0; s1[t] = k.w1; s2[t] = k.w2; s3[t] = k.w3; si[t] = id;
     }
     __syncthreads();
     for (unsigned k = 2; k <= kSortTile; k <<= 1) {
@@ -125,16 +128,22 @@ k_tile_sort(const lsmkv_key_t *__restrict__ src, lsmkv_key_t *__restrict__ dst,
             const unsigned t = threadIdx.x;
             const unsigned i = 2 * t - (t & (j - 1)), l = i + j;
             const bool up = (i & k) == 0;
-            const Key4 a = sk[i], b = sk[l];
+            const Key4 a{s0[i], s1[i], s2[i], s3[i]}, b{s0[l], s1[l], s2[l], s3[l]};
             const uint32_t ia = si[i], ib = si[l];
             const bool swap = up ? entry_less(b, ib, a, ia) : entry_less(a, ia, b, ib);
-            if (swap) { sk[i] = b; sk[l] = a; si[i] = ib; si[l] = ia; }
+            if (swap) {
+                s0[i] = b.w0; s1[i] = b.w1; s2[i] = b.w2; s3[i] = b.w3; si[i] = ib;
+                s0[l] = a.w0; s1[l] = a.w1; s2[l] = a.w2; s3[l] = a.w3; si[l] = ia;
+            }
             __syncthreads();
         }
     }
     for (unsigned t = threadIdx.x; t < kSortTile; t += blockDim.x) {
         const uint64_t i = tile0 + t;
-        if (i < n) { store_key4(dst + i, sk[t]); dst_idx[i] = si[t]; }
+        if (i < n) {
+            store_key4(dst + i, Key4{s0[t], s1[t], s2[t], s3[t]});
+            dst_idx[i] = si[t];
+        }
     }
 }
 
