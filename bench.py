@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU baseline budget (0 = skip)")
     ap.add_argument("--only-probe-block", action="store_true",
                     help="run just the probe-heavy measurement (a small case for profiling)")
+    ap.add_argument("--no-shapes-block", action="store_true",
+                    help="skip the pack/unpack rates on the other workloads' KV shapes")
     ap.add_argument("--no-xp12-block", action="store_true",
                     help="skip the compressing-codec measurement")
     ap.add_argument("--no-probe-block", action="store_true",
@@ -428,6 +430,7 @@ def main():
                "sample": f"first {s_req} requests = {s_n} chunks ({s_n * cb / 2**30:.2f} GiB per "
                          f"direction), {passes} passes in {el:.1f} s; host cpus={os.cpu_count()}"}
 
+    shapes_block = None
     if rank == 0:
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(peaks_path):
@@ -435,6 +438,14 @@ def main():
                 peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
         else:
             peak, peak_src = 6650.0, "fallback"
+        n_waves_used = len(W)
+        if not args.no_shapes_block:
+            # everything of the main workload can go now: the other shapes need the room
+            del src_bufs, dst_bufs, src_pool, dst_pool, W
+            if args.e2e_steps <= 0:
+                del arena
+            torch.cuda.empty_cache()
+            shapes_block = other_shapes_block(torch, lsmkv, dev, local_rank, peak)
         copy_ms = prof["pack"][0] + prof["unpack"][0]
         copy_launches = prof["pack"][1] + prof["unpack"][1]
         algo_bytes_per_launch = 2.0 * (2 * payload * args.steps) / max(1, copy_launches)
@@ -445,7 +456,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
             "config": {"workload": WORKLOAD, "requests": args.requests, "chunks": total_chunks,
-                       "payload_GiB_per_direction": payload / 2**30, "waves": len(W),
+                       "payload_GiB_per_direction": payload / 2**30, "waves": n_waves_used,
                        "l2": "inputs larger than L2 (each wave moves >30 GiB)",
                        "payload_dtype": "bf16 bit patterns (opaque)", "key_arithmetic": "u64",
                        "tuning": {k: ctx.get_tuning(k) for k in
@@ -466,6 +477,7 @@ def main():
             "cpu_baseline": cpu,
             "probe": probe_block,
             "codec_xp12": xp_block,
+            "other_shapes": shapes_block,
             "phases": {
                 "pack_GBps_payload": payload * args.steps / (prof["pack"][0] * 1e-3) / 1e9,
                 "unpack_GBps_payload": payload * args.steps / (prof["unpack"][0] * 1e-3) / 1e9,
@@ -481,6 +493,84 @@ def main():
         print(json.dumps(out))
     if dist.is_initialized():
         dist.destroy_process_group()
+
+
+def other_shapes_block(torch, lsmkv, dev, device_index, peak):
+    """Pack / unpack rates on the KV shapes of the other named workloads (identity codec, one
+    resident wave each, random page tables): the GQA shape with 64-token pages, the 80-layer
+    long-context shape, and the tiny 4-layer shape (launch-latency territory)."""
+    shapes = [
+        ("configs[3] GQA 28x4x128, page 64", dict(n_layers=28, n_kv_heads=4, head_dim=128,
+                                                  page_tokens=64, chunk_tokens=64), 6144),
+        ("configs[4] long-context 80x8x128, page 16", dict(n_layers=80, n_kv_heads=8,
+                                                          head_dim=128), 8192),
+        ("configs[0] tiny 4x8x128, page 16", dict(n_layers=4, n_kv_heads=8, head_dim=128), 1024),
+    ]
+    out = []
+    for name, gd, n in shapes:
+        g = lsmkv.Geom(**gd)
+        cb, pb = g.chunk_bytes, g.page_bytes
+        free, _ = torch.cuda.mem_get_info()
+        n = int(min(n, free * 0.8 / (3 * cb)))
+        ctx = lsmkv.Context(g, device_index)
+        src = dst = arena = None
+        try:
+            C = g.chunk_tokens
+            n_req = max(1, n // 256)
+            per = n // n_req
+            n = per * n_req
+            rng = synth.rng_for(9, g.n_layers)
+            tokens = rng.integers(0, 128000, n * C, dtype=np.uint32)
+            seq_off = (np.arange(n_req + 1, dtype=np.uint64) * np.uint64(per * C))
+            coff = (np.arange(n_req + 1, dtype=np.uint64) * np.uint64(per))
+
+            def up(a):
+                return torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).to(dev)
+
+            gen = torch.Generator(device=dev)
+            gen.manual_seed(9)
+            src = [torch.randn(n * pb // 2, dtype=torch.bfloat16, device=dev,
+                               generator=gen).view(torch.uint8).view(n, pb) for _ in range(2 * g.n_layers)]
+            dst = [torch.zeros((n, pb), dtype=torch.uint8, device=dev) for _ in range(2 * g.n_layers)]
+            sp, dp = lsmkv.pool_table(src), lsmkv.pool_table(dst)
+            arena = torch.empty(n * cb, dtype=torch.uint8, device=dev)
+            d_tok, d_off, d_coff = up(tokens), up(seq_off), up(coff)
+            src_pages, dst_pages = synth.random_pages(rng, n, n), synth.random_pages(rng, n, n)
+            d_sp, d_dp = up(src_pages), up(dst_pages)
+            keys = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+            vals = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+            hit = torch.full((n_req,), per, dtype=torch.int32, device=dev)
+
+            def once():
+                ctx.encode_batch(n_req, d_tok, d_off, None, d_coff, n, d_sp, sp, 0, 0, keys, vals,
+                                 arena, n * cb)
+                ctx.decode_batch(n_req, d_coff, n, hit, vals, [(arena, n * cb)], d_dp, dp)
+
+            for _ in range(3):
+                once()
+            torch.cuda.synchronize()
+            idx_s = torch.from_numpy(src_pages[:256].astype(np.int64)).to(dev)
+            idx_d = torch.from_numpy(dst_pages[:256].astype(np.int64)).to(dev)
+            assert all(torch.equal(a[idx_s], b[idx_d]) for a, b in zip(src, dst)), name
+            assert ctx.last_status()["flags"] == 0
+            ctx.profile_enable(True)
+            ctx.profile_read()
+            reps = 5
+            for _ in range(reps):
+                once()
+            torch.cuda.synchronize()
+            prof = ctx.profile_read()
+            pm, um = prof["pack"][0] / reps, prof["unpack"][0] / reps
+            out.append({"shape": name, "chunks": n, "chunk_MiB": cb / 2**20,
+                        "payload_GiB": n * cb / 2**30,
+                        "pack_GBps_payload": n * cb / pm / 1e6, "unpack_GBps_payload": n * cb / um / 1e6,
+                        "pack_hbm_frac_of_peak": 2 * n * cb / pm / 1e6 / peak,
+                        "unpack_hbm_frac_of_peak": 2 * n * cb / um / 1e6 / peak})
+        finally:
+            ctx.close()
+            del src, dst, arena
+            torch.cuda.empty_cache()
+    return out
 
 
 def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
