@@ -136,6 +136,10 @@ def lib() -> C.CDLL:
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint64]
         _lib.orc_relocate_records.restype = C.c_uint64
         _lib.orc_relocate_records.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32]
+        _lib.orc_xprobe_batch.restype = C.c_int
+        _lib.orc_xprobe_batch.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p,
+                                          C.c_void_p]
         _lib.orc_probe_batch.restype = C.c_int
         _lib.orc_probe_batch.argtypes = [
             C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -404,3 +408,42 @@ def relocate_records(vals, table):
     t = np.ascontiguousarray(table, dtype=RELOC_DTYPE)
     changed = lib().orc_relocate_records(_p(v), len(v), _p(t), len(t))
     return v, int(changed)
+
+
+# ---- exact prefix index ----------------------------------------------------------------------
+
+class _XRun(C.Structure):
+    _fields_ = [("tokens", C.c_void_p), ("seq_off", C.c_void_p), ("n_seq", C.c_uint32),
+                ("vals", C.c_void_p), ("chunk_off", C.c_void_p)]
+
+
+def xprobe_batch(g: Geom, tokens, seq_off, qchunk_off, xruns):
+    """xruns: list (newest first) of (tokens u32, seq_off u64[n+1], vals VAL_DTYPE per chunk in
+    sequence-major order). Returns (hit u32[Q], recs VAL_DTYPE[total query chunks])."""
+    tokens = _arr(tokens, np.uint32)
+    seq_off = _arr(seq_off, np.uint64)
+    qchunk_off = _arr(qchunk_off, np.uint64)
+    nq = len(seq_off) - 1
+    total = int(qchunk_off[-1]) if nq else 0
+    arr = (_XRun * max(1, len(xruns)))()
+    keep = []
+    for i, (t, so, v) in enumerate(xruns):
+        t = _arr(t, np.uint32)
+        so = _arr(so, np.uint64)
+        v = np.ascontiguousarray(v, dtype=VAL_DTYPE)
+        nch = (np.diff(so.astype(np.int64)) // g.chunk_tokens).astype(np.uint64)
+        co = np.zeros(len(so), dtype=np.uint64)
+        np.cumsum(nch, out=co[1:])
+        assert len(v) == int(co[-1])
+        keep.append((t, so, v, co))
+        arr[i].tokens, arr[i].seq_off, arr[i].n_seq = t.ctypes.data, so.ctypes.data, len(so) - 1
+        arr[i].vals, arr[i].chunk_off = v.ctypes.data, co.ctypes.data
+    hit = np.zeros(nq, dtype=np.uint32)
+    recs = np.zeros(total, dtype=VAL_DTYPE)
+    gc = g.c()
+    rc = lib().orc_xprobe_batch(C.byref(gc), nq, _p(tokens), _p(seq_off), _p(qchunk_off), arr,
+                                len(xruns), _p(hit), _p(recs))
+    del keep
+    if rc != OK:
+        raise OracleError(rc)
+    return hit, recs

@@ -590,3 +590,86 @@ uint64_t orc_relocate_records(orc_val *vals, uint64_t n, const orc_reloc *table,
     }
     return changed;
 }
+
+/* ---- exact prefix index ("xrun"): the index keyed by the token prefixes themselves, so that key
+ * order IS prefix order and nothing depends on a digest (Sec. 3.1/3.2: keys keep the structure
+ * of token prefixes; lexicographic order coincides with prefix order).
+ *
+ * One xrun holds whole stored sequences (every chunk prefix 0..nch_s-1 of every sequence s), so
+ * the chunk prefixes of a query present in it form an interval [0, m): m = the largest number
+ * of whole chunks the query shares with any stored sequence = max_s floor(lcp(Q, s) / C).
+ * Several sequences may hold the same chunk prefix; its record is that of the OWNER: the
+ * smallest such sequence in token-lexicographic order (a sequence that is a prefix of another
+ * is smaller; identical sequences: the earlier arrival is smaller).
+ * Across runs (newest first): hit = max over runs of m_run; the record of chunk j comes from
+ * the newest run with m_run > j.
+ *
+ * Everything below is the definition by brute force: no sorting, no tree.
+ */
+typedef struct {
+    const uint32_t *tokens;     /* arena */
+    const uint64_t *seq_off;    /* [n_seq + 1] */
+    uint32_t n_seq;
+    const orc_val *vals;        /* records per chunk, sequence-major: chunk_off[s] + j */
+    const uint64_t *chunk_off;  /* [n_seq + 1] prefix sums of floor(len_s / C) */
+} orc_xrun;
+
+static uint64_t lcp_tokens(const uint32_t *a, uint64_t na, const uint32_t *b, uint64_t nb)
+{
+    const uint64_t n = na < nb ? na : nb;
+    uint64_t i = 0;
+    while (i < n && a[i] == b[i]) ++i;
+    return i;
+}
+
+/* token-lexicographic order; a proper prefix is smaller; equal strings compare by index */
+static int seq_less(const orc_xrun *x, uint32_t s, uint32_t t)
+{
+    const uint32_t *a = x->tokens + x->seq_off[s], *b = x->tokens + x->seq_off[t];
+    const uint64_t na = x->seq_off[s + 1] - x->seq_off[s], nb = x->seq_off[t + 1] - x->seq_off[t];
+    const uint64_t l = lcp_tokens(a, na, b, nb);
+    if (l < na && l < nb) return a[l] < b[l];
+    if (na != nb) return na < nb;
+    return s < t;
+}
+
+int orc_xprobe_batch(const orc_geom *g, uint32_t n_query, const uint32_t *tokens,
+                     const uint64_t *seq_off, const uint64_t *qchunk_off, const orc_xrun *runs,
+                     uint32_t n_runs, uint32_t *hit_out, orc_val *recs_out)
+{
+    if (!geom_ok(g)) return ORC_EINVAL;
+    const uint64_t C = g->chunk_tokens;
+    for (uint32_t q = 0; q < n_query; ++q) {
+        const uint32_t *Q = tokens + seq_off[q];
+        const uint64_t len = seq_off[q + 1] - seq_off[q], nch = len / C;
+        if (qchunk_off[q + 1] - qchunk_off[q] != nch) return ORC_EINVAL;
+        orc_val *recs = recs_out + qchunk_off[q];
+        memset(recs, 0, nch * sizeof(orc_val));
+        uint64_t hit = 0;
+        for (uint32_t r = 0; r < n_runs; ++r) {              /* newest first */
+            const orc_xrun *x = &runs[r];
+            uint64_t m = 0;
+            for (uint32_t s = 0; s < x->n_seq; ++s) {
+                const uint64_t l = lcp_tokens(Q, len, x->tokens + x->seq_off[s],
+                                              x->seq_off[s + 1] - x->seq_off[s]) / C;
+                if (l > m) m = l;
+            }
+            /* chunks [hit, m) are new through this run: older runs only add beyond what newer
+             * ones gave, newer runs keep what they already decided */
+            for (uint64_t j = hit; j < m; ++j) {
+                int have = 0;
+                uint32_t owner = 0;
+                for (uint32_t s = 0; s < x->n_seq; ++s) {
+                    const uint64_t l = lcp_tokens(Q, len, x->tokens + x->seq_off[s],
+                                                  x->seq_off[s + 1] - x->seq_off[s]);
+                    if (l < (j + 1) * C) continue;          /* s does not hold this prefix */
+                    if (!have || seq_less(x, s, owner)) { owner = s; have = 1; }
+                }
+                recs[j] = x->vals[x->chunk_off[owner] + j];
+            }
+            if (m > hit) hit = m;
+        }
+        hit_out[q] = (uint32_t)hit;
+    }
+    return ORC_OK;
+}
