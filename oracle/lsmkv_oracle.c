@@ -595,12 +595,13 @@ uint64_t orc_relocate_records(orc_val *vals, uint64_t n, const orc_reloc *table,
  * order IS prefix order and nothing depends on a digest (Sec. 3.1/3.2: keys keep the structure
  * of token prefixes; lexicographic order coincides with prefix order).
  *
- * One xrun holds whole stored sequences (every chunk prefix 0..nch_s-1 of every sequence s), so
- * the chunk prefixes of a query present in it form an interval [0, m): m = the largest number
- * of whole chunks the query shares with any stored sequence = max_s floor(lcp(Q, s) / C).
- * Several sequences may hold the same chunk prefix; its record is that of the OWNER: the
- * smallest such sequence in token-lexicographic order (a sequence that is a prefix of another
- * is smaller; identical sequences: the earlier arrival is smaller).
+ * One xrun holds whole stored sequences, each with one record per whole chunk (the records of
+ * chunks it shares with an earlier sequence are copies of that sequence's records). The chunk
+ * prefixes of a query Q present in it form an interval [0, m), m = floor(L / C), L = the
+ * longest token prefix Q shares with any stored sequence. All of Q's records from that run
+ * come from ONE stored sequence, the NEIGHBOUR of Q: among the sequences that reach L, the
+ * largest one not above Q in token-lexicographic order (a sequence that is a prefix of another
+ * is smaller; identical sequences order by arrival), and if none is, the smallest one above Q.
  * Across runs (newest first): hit = max over runs of m_run; the record of chunk j comes from
  * the newest run with m_run > j.
  *
@@ -622,15 +623,12 @@ static uint64_t lcp_tokens(const uint32_t *a, uint64_t na, const uint32_t *b, ui
     return i;
 }
 
-/* token-lexicographic order; a proper prefix is smaller; equal strings compare by index */
-static int seq_less(const orc_xrun *x, uint32_t s, uint32_t t)
+/* token-lexicographic three-way comparison; a proper prefix is smaller */
+static int tok_cmp(const uint32_t *a, uint64_t na, const uint32_t *b, uint64_t nb)
 {
-    const uint32_t *a = x->tokens + x->seq_off[s], *b = x->tokens + x->seq_off[t];
-    const uint64_t na = x->seq_off[s + 1] - x->seq_off[s], nb = x->seq_off[t + 1] - x->seq_off[t];
     const uint64_t l = lcp_tokens(a, na, b, nb);
-    if (l < na && l < nb) return a[l] < b[l];
-    if (na != nb) return na < nb;
-    return s < t;
+    if (l < na && l < nb) return a[l] < b[l] ? -1 : 1;
+    return na < nb ? -1 : na > nb ? 1 : 0;
 }
 
 int orc_xprobe_batch(const orc_geom *g, uint32_t n_query, const uint32_t *tokens,
@@ -648,26 +646,35 @@ int orc_xprobe_batch(const orc_geom *g, uint32_t n_query, const uint32_t *tokens
         uint64_t hit = 0;
         for (uint32_t r = 0; r < n_runs; ++r) {              /* newest first */
             const orc_xrun *x = &runs[r];
-            uint64_t m = 0;
+            uint64_t L = 0;
             for (uint32_t s = 0; s < x->n_seq; ++s) {
                 const uint64_t l = lcp_tokens(Q, len, x->tokens + x->seq_off[s],
-                                              x->seq_off[s + 1] - x->seq_off[s]) / C;
-                if (l > m) m = l;
+                                              x->seq_off[s + 1] - x->seq_off[s]);
+                if (l > L) L = l;
             }
-            /* chunks [hit, m) are new through this run: older runs only add beyond what newer
-             * ones gave, newer runs keep what they already decided */
-            for (uint64_t j = hit; j < m; ++j) {
-                int have = 0;
-                uint32_t owner = 0;
-                for (uint32_t s = 0; s < x->n_seq; ++s) {
-                    const uint64_t l = lcp_tokens(Q, len, x->tokens + x->seq_off[s],
-                                                  x->seq_off[s + 1] - x->seq_off[s]);
-                    if (l < (j + 1) * C) continue;          /* s does not hold this prefix */
-                    if (!have || seq_less(x, s, owner)) { owner = s; have = 1; }
+            const uint64_t m = L / C;
+            if (m <= hit) continue;      /* newer runs already decided everything this one has */
+            int have_lo = 0, have_hi = 0;
+            uint32_t lo = 0, hi = 0;     /* largest reaching-L sequence <= Q; smallest one > Q */
+            for (uint32_t s = 0; s < x->n_seq; ++s) {
+                const uint32_t *S = x->tokens + x->seq_off[s];
+                const uint64_t ns = x->seq_off[s + 1] - x->seq_off[s];
+                if (lcp_tokens(Q, len, S, ns) != L) continue;
+                if (tok_cmp(S, ns, Q, len) <= 0) {
+                    if (!have_lo || tok_cmp(S, ns, x->tokens + x->seq_off[lo],
+                                            x->seq_off[lo + 1] - x->seq_off[lo]) >= 0) {
+                        lo = s;          /* >= : among identical sequences the later arrival */
+                        have_lo = 1;
+                    }
+                } else if (!have_hi || tok_cmp(S, ns, x->tokens + x->seq_off[hi],
+                                               x->seq_off[hi + 1] - x->seq_off[hi]) < 0) {
+                    hi = s;              /* <  : among identical sequences the earlier arrival */
+                    have_hi = 1;
                 }
-                recs[j] = x->vals[x->chunk_off[owner] + j];
             }
-            if (m > hit) hit = m;
+            const uint32_t owner = have_lo ? lo : hi;
+            for (uint64_t j = hit; j < m; ++j) recs[j] = x->vals[x->chunk_off[owner] + j];
+            hit = m;
         }
         hit_out[q] = (uint32_t)hit;
     }

@@ -21,8 +21,9 @@ def make_xrun(g, batch, file_id):
 
 
 def py_expected(C, query, stores):
-    """The definition with Python tuples: per run, longest shared whole chunks; owner = smallest
-    sequence (tuple order: a prefix is smaller; ties by index) among those holding the prefix."""
+    """The definition with Python tuples (tuple order: a prefix is smaller). Per run: L = longest
+    shared token prefix; the records come from the neighbour of Q among the sequences reaching L:
+    the largest (sequence, arrival) not above Q, else the smallest above."""
     hits, recs = [], []
     for q in range(query.n):
         Q = tuple(int(t) for t in query.seq(q))
@@ -32,17 +33,24 @@ def py_expected(C, query, stores):
         for (batch, vals) in stores:                         # newest first
             seqs = [tuple(int(t) for t in batch.seq(s)) for s in range(batch.n)]
             coff = np.concatenate([[0], np.cumsum([len(s) // C for s in seqs])])
+
             def shared(s):
                 n = 0
                 while n < min(len(Q), len(s)) and Q[n] == s[n]:
                     n += 1
                 return n
-            m = max([shared(s) // C for s in seqs] + [0])
+            L = max([shared(s) for s in seqs] + [0])
+            m = L // C
+            if m <= hit:
+                continue
+            reach = [i for i, s in enumerate(seqs) if shared(s) == L]
+            below = [i for i in reach if seqs[i] <= Q]
+            above = [i for i in reach if seqs[i] > Q]
+            owner = (max(below, key=lambda i: (seqs[i], i)) if below
+                     else min(above, key=lambda i: (seqs[i], i)))
             for j in range(hit, m):
-                holders = [i for i, s in enumerate(seqs) if shared(s) >= (j + 1) * C]
-                owner = min(holders, key=lambda i: (seqs[i], i))
                 rec[j] = (int(vals["file_id"][coff[owner] + j]), int(vals["offset"][coff[owner] + j]))
-            hit = max(hit, m)
+            hit = m
         hits.append(hit)
         recs.append(rec)
     return hits, recs
