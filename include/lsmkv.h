@@ -215,6 +215,50 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
 
 /*
+ * Exact prefix index (Sec. 3.1/3.2: keys that keep the structure of token prefixes, so that key
+ * order is prefix order). An "xrun" indexes WHOLE stored sequences by their tokens themselves:
+ * no digest takes part, so two different prefixes can never be confused. The caller keeps, on
+ * the device and alive while the xrun is in use: the token arena and offsets of the stored
+ * sequences, and one record per whole chunk of every sequence, sequence-major (the records of
+ * chunks a sequence shares with an earlier one are copies of that one's records -- what a probe
+ * returned for them before the put). lsmkv_xrun_build writes the two index arrays:
+ *   order_out     [dev] u32[n_seq]: sequence numbers in token-lexicographic order (a sequence
+ *                 that is a prefix of another comes first; identical sequences by number)
+ *   chunk_off_out [dev] u64[n_seq + 1]: prefix sums of floor(len_s / C), the row of sequence s
+ *                 in the record array
+ * n_seq < 2^32 - 1. Uses (and may grow) the context's sort scratch. A sequence with
+ * seq_off[s + 1] < seq_off[s] sets LSMKV_ST_BAD_COUNT and counts as empty.
+ */
+typedef struct {
+    const uint32_t *tokens;      /* [dev] arena of the stored sequences */
+    const uint64_t *seq_off;     /* [dev] u64[n_seq + 1] */
+    const lsmkv_val_t *vals;     /* [dev] records, 16-byte aligned: vals[chunk_off[s] + j] */
+    const uint32_t *order;       /* [dev] from lsmkv_xrun_build */
+    const uint64_t *chunk_off;   /* [dev] from lsmkv_xrun_build */
+    uint32_t n_seq;
+    uint32_t reserved;           /* 0 */
+} lsmkv_xrun_t;
+
+int lsmkv_xrun_build(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
+                     const uint64_t *seq_off, uint32_t n_seq, uint32_t *order_out,
+                     uint64_t *chunk_off_out);
+
+/*
+ * Probe of xruns ([host] array, newest first, n_runs <= LSMKV_MAX_RUNS; queries laid out as for
+ * lsmkv_probe_batch). Per run, the whole chunks of the longest token prefix the query shares
+ * with any stored sequence are present; hit_chunks_out[q] is the largest such count over the
+ * runs, and chunk j takes its record from the newest run that reaches beyond j. Within a run
+ * the records come from the query's neighbour in token order among the sequences sharing that
+ * longest prefix: the largest one not above the query, else the smallest one above it.
+ * recs_out [dev, n_qchunks entries, 16-byte aligned]: records of the hit chunks, zeros after.
+ * Errors as lsmkv_probe_batch (LSMKV_ST_BAD_COUNT for a query whose counts disagree).
+ */
+int lsmkv_xprobe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint32_t *tokens,
+                       const uint64_t *seq_off, const uint64_t *qchunk_off, uint64_t n_qchunks,
+                       const lsmkv_xrun_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,
+                       lsmkv_val_t *recs_out);
+
+/*
  * Record relocation (Sec. 3.4 "Automatic Tensor File Merging": when tensor files are merged,
  * the file_id + offset values in the index are updated). Every record of vals [dev, n entries,
  * rewritten in place -- typically the vals array of a run] whose file_id equals table[t].old_file

@@ -447,3 +447,18 @@ def xprobe_batch(g: Geom, tokens, seq_off, qchunk_off, xruns):
     if rc != OK:
         raise OracleError(rc)
     return hit, recs
+
+
+def xrun_order(tokens, seq_off) -> np.ndarray:
+    """Sequence numbers in token-lexicographic order (prefix first, identical ones by number)."""
+    tokens = _arr(tokens, np.uint32)
+    seq_off = _arr(seq_off, np.uint64)
+    n = len(seq_off) - 1
+    out = np.zeros(n, dtype=np.uint32)
+    L = lib()
+    L.orc_xrun_order.restype = C.c_int
+    L.orc_xrun_order.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
+    rc = L.orc_xrun_order(_p(tokens), _p(seq_off), n, _p(out))
+    if rc != OK:
+        raise OracleError(rc)
+    return out

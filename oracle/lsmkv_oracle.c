@@ -680,3 +680,26 @@ int orc_xprobe_batch(const orc_geom *g, uint32_t n_query, const uint32_t *tokens
     }
     return ORC_OK;
 }
+
+/* The sorted order an xrun is searched in: sequence numbers by token-lexicographic order, a
+ * proper prefix first, identical sequences by number. Library sort with the comparison above. */
+static const orc_xrun *g_sort_run;
+static int order_cmp(const void *pa, const void *pb)
+{
+    const uint32_t a = *(const uint32_t *)pa, b = *(const uint32_t *)pb;
+    const orc_xrun *x = g_sort_run;
+    const int c = tok_cmp(x->tokens + x->seq_off[a], x->seq_off[a + 1] - x->seq_off[a],
+                          x->tokens + x->seq_off[b], x->seq_off[b + 1] - x->seq_off[b]);
+    return c ? c : (a < b ? -1 : a > b ? 1 : 0);
+}
+
+int orc_xrun_order(const uint32_t *tokens, const uint64_t *seq_off, uint32_t n_seq,
+                   uint32_t *order_out)
+{
+    orc_xrun x = { tokens, seq_off, n_seq, NULL, NULL };
+    for (uint32_t s = 0; s < n_seq; ++s) order_out[s] = s;
+    g_sort_run = &x;
+    qsort(order_out, n_seq, sizeof(uint32_t), order_cmp);
+    g_sort_run = NULL;
+    return ORC_OK;
+}

@@ -16,6 +16,7 @@
 #include "lsmkv_probe.cuh"
 #include "lsmkv_sort.cuh"
 #include "lsmkv_xp12.cuh"
+#include "lsmkv_xrun.cuh"
 
 using namespace lsmkv;
 
@@ -763,6 +764,75 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
     CU(ctx, cudaGetLastError());
     return launch_dedupe(ctx, s, ws, buf, total, ws.vals, /*keep_last=*/0, keys_out, vals_out,
                          n_out);
+}
+
+int lsmkv_xrun_build(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
+                     const uint64_t *seq_off, uint32_t n_seq, uint32_t *order_out,
+                     uint64_t *chunk_off_out)
+{
+    if (!ctx || !chunk_off_out || n_seq == 0xFFFFFFFFu) return LSMKV_EINVAL;
+    if (n_seq && (!seq_off || !order_out)) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n_seq == 0) {
+        CU(ctx, cudaMemsetAsync(chunk_off_out, 0, sizeof(uint64_t), s));
+        return LSMKV_OK;
+    }
+    SortWs ws;
+    int rc = ensure_sort(ctx, n_seq, &ws);
+    if (rc != LSMKV_OK) return rc;
+    LaunchTimer timer(ctx, s, LSMKV_K_FLUSH);
+    k_xrun_init<<<merge_grid(ctx, n_seq), 256, 0, s>>>(seq_off, n_seq, ctx->geom.chunk_tokens,
+                                                       ws.idx[0], chunk_off_out, ctx->d_status);
+    k_scan_blocks<<<1, 1024, 0, s>>>(chunk_off_out, n_seq, chunk_off_out + n_seq);
+    ctx->launches += 2;
+    int buf = 0;
+    // one warp per element; the grid covers the elements once or caps at 8 CTAs per SM
+    const unsigned grid = warp_grid(ctx, n_seq, 256, 8);
+    for (uint64_t width = 1; width < n_seq; width *= 2) {
+        k_xrun_merge_level<<<grid, 256, 0, s>>>(tokens, seq_off, ws.idx[buf], ws.idx[buf ^ 1],
+                                                n_seq, width);
+        ++ctx->launches;
+        buf ^= 1;
+    }
+    CU(ctx, cudaGetLastError());
+    CU(ctx, cudaMemcpyAsync(order_out, ws.idx[buf], (size_t)n_seq * sizeof(uint32_t),
+                            cudaMemcpyDeviceToDevice, s));
+    return LSMKV_OK;
+}
+
+int lsmkv_xprobe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint32_t *tokens,
+                       const uint64_t *seq_off, const uint64_t *qchunk_off, uint64_t n_qchunks,
+                       const lsmkv_xrun_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,
+                       lsmkv_val_t *recs_out)
+{
+    if (!ctx) return LSMKV_EINVAL;
+    if (n_query == 0) return LSMKV_OK;
+    if (!seq_off || !qchunk_off || !hit_chunks_out) return LSMKV_EINVAL;
+    if (n_qchunks && (!tokens || !recs_out || !aligned16(recs_out))) return LSMKV_EINVAL;
+    if (n_runs > LSMKV_MAX_RUNS || (n_runs && !runs)) return LSMKV_EINVAL;
+    XRunTable rt;
+    std::memset(&rt, 0, sizeof(rt));
+    for (uint32_t r = 0; r < n_runs; ++r) {
+        if (runs[r].n_seq && (!runs[r].seq_off || !runs[r].order || !runs[r].chunk_off ||
+                              !runs[r].vals || !aligned16(runs[r].vals)))
+            return LSMKV_EINVAL;
+        rt.tokens[r] = runs[r].tokens;
+        rt.seq_off[r] = runs[r].seq_off;
+        rt.vals[r] = runs[r].vals;
+        rt.order[r] = runs[r].order;
+        rt.chunk_off[r] = runs[r].chunk_off;
+        rt.n_seq[r] = runs[r].n_seq;
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
+    k_xprobe<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
+        rt, n_runs, ctx->geom.chunk_tokens, n_query, tokens, seq_off, qchunk_off, n_qchunks,
+        hit_chunks_out, recs_out, ctx->d_status);
+    ++ctx->launches;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
 }
 
 int lsmkv_relocate_records(lsmkv_ctx *ctx, void *stream, lsmkv_val_t *vals, uint64_t n,

@@ -1,0 +1,166 @@
+// Exact prefix index ("xrun"): stored sequences ordered by their tokens, so key order is prefix
+// order and a lookup compares tokens, never digests (Sec. 3.1/3.2: keys that keep the prefix
+// structure). Build = a rank-merge sort of sequence ids with a warp-cooperative token comparison;
+// probe = one binary search per (query, run) that skips the tokens both bounds already share.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "lsmkv.h"
+#include "lsmkv_common.cuh"
+
+namespace lsmkv {
+
+struct SeqView {
+    const uint32_t *tok;
+    uint64_t len;
+};
+
+__device__ __forceinline__ SeqView seq_view(const uint32_t *__restrict__ tokens,
+                                            const uint64_t *__restrict__ seq_off, uint64_t s)
+{
+    const uint64_t a = __ldg(seq_off + s), b = __ldg(seq_off + s + 1);
+    return SeqView{tokens + a, b >= a ? b - a : 0};
+}
+
+// Warp-cooperative: length of the common token prefix of a and b, starting the comparison at
+// `from` (the caller knows the first `from` tokens agree). Every lane returns the same value.
+__device__ __forceinline__ uint64_t warp_lcp(const SeqView &a, const SeqView &b, uint64_t from)
+{
+    const uint64_t n = a.len < b.len ? a.len : b.len;
+    const unsigned lane = lane_id();
+    for (uint64_t i = from; i < n; i += 32) {
+        const uint64_t k = i + lane;
+        const bool differ = k < n && __ldg(a.tok + k) != __ldg(b.tok + k);
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, differ);
+        if (m) return i + (unsigned)__ffs(m) - 1u;
+    }
+    return n;
+}
+
+// a < b in token order given their common prefix length l; a proper prefix is smaller; equal
+// strings order by the tie-break ids.
+__device__ __forceinline__ bool seq_less_at(const SeqView &a, const SeqView &b, uint64_t l,
+                                            uint32_t ia, uint32_t ib)
+{
+    if (l < a.len && l < b.len) return __ldg(a.tok + l) < __ldg(b.tok + l);
+    if (a.len != b.len) return a.len < b.len;
+    return ia < ib;
+}
+
+__global__ void __launch_bounds__(256)
+k_xrun_init(const uint64_t *__restrict__ seq_off, uint32_t n_seq, uint32_t C,
+            uint32_t *__restrict__ order, uint64_t *__restrict__ chunk_cnt, DevStatus *st)
+{
+    for (uint64_t s = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n_seq;
+         s += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t a = seq_off[s], b = seq_off[s + 1];
+        if (b < a) st_flag(st, LSMKV_ST_BAD_COUNT, s);
+        order[s] = (uint32_t)s;
+        chunk_cnt[s] = b >= a ? (b - a) / C : 0;
+    }
+}
+
+// One merge level over sequence ids, one warp per element: its rank among the sibling segment
+// comes from a binary search with the token comparison. The order is total (ties by id), so the
+// two halves never hold equal elements.
+__global__ void __launch_bounds__(256)
+k_xrun_merge_level(const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
+                   const uint32_t *__restrict__ src, uint32_t *__restrict__ dst, uint64_t n,
+                   uint64_t width)
+{
+    const uint64_t warp0 = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    for (uint64_t i = warp0; i < n; i += n_warps) {
+        const uint64_t base = i / (2 * width) * (2 * width);
+        const uint64_t mid = min(n, base + width), end = min(n, base + 2 * width);
+        const uint32_t x = __ldg(src + i);
+        const SeqView vx = seq_view(tokens, seq_off, x);
+        uint64_t lo, hi;
+        if (i < mid) { lo = mid; hi = end; } else { lo = base; hi = mid; }
+        const uint64_t first = lo;
+        while (lo < hi) {                                    // sibling elements below x
+            const uint64_t m = lo + ((hi - lo) >> 1);
+            const uint32_t y = __ldg(src + m);
+            const SeqView vy = seq_view(tokens, seq_off, y);
+            const uint64_t l = warp_lcp(vy, vx, 0);
+            if (seq_less_at(vy, vx, l, y, x)) lo = m + 1; else hi = m;
+        }
+        const uint64_t own = i < mid ? i - base : i - mid;
+        if (lane_id() == 0) dst[base + own + (lo - first)] = x;
+    }
+}
+
+constexpr int kMaxXRuns = LSMKV_MAX_RUNS;
+
+struct XRunTable {
+    const uint32_t *tokens[kMaxXRuns];
+    const uint64_t *seq_off[kMaxXRuns];
+    const lsmkv_val_t *vals[kMaxXRuns];
+    const uint32_t *order[kMaxXRuns];
+    const uint64_t *chunk_off[kMaxXRuns];
+    uint32_t n_seq[kMaxXRuns];
+};
+
+// One warp per query. Per run, newest first: the position of the query among the sorted stored
+// sequences; the longer of the prefixes shared with the two neighbours is the longest prefix
+// shared with anything in the run, and that neighbour (the lower one on a tie) lends its records.
+__global__ void __launch_bounds__(256)
+k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint32_t n_query,
+         const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
+         const uint64_t *__restrict__ qchunk_off, uint64_t n_qchunks,
+         uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out, DevStatus *st)
+{
+    const unsigned lane = lane_id();
+    const uint64_t warp0 = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (uint64_t q = warp0; q < n_query; q += n_warps) {
+        const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
+        const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
+        const uint64_t o0 = qchunk_off[q], o1 = qchunk_off[q + 1];
+        if (s1 < s0 || o1 < o0 || o1 - o0 != nch || o1 > n_qchunks || nch > 0xFFFFFFFFull) {
+            if (lane == 0) { st_flag(st, LSMKV_ST_BAD_COUNT, q); hit_out[q] = 0; }
+            continue;
+        }
+        const SeqView Q{tokens + s0, s1 - s0};
+        uint4 *recs = reinterpret_cast<uint4 *>(recs_out + o0);
+        uint64_t hit = 0;
+        for (uint32_t r = 0; r < n_runs; ++r) {
+            const uint32_t n = rt.n_seq[r];
+            if (n == 0 || hit >= nch) continue;
+            // invariant: order[lo - 1] <= Q < order[hi]; l_lo / l_hi = tokens Q shares with them
+            uint64_t lo = 0, hi = n, l_lo = 0, l_hi = 0;
+            uint32_t s_lo = 0, s_hi = 0;
+            bool have_lo = false, have_hi = false;
+            while (lo < hi) {
+                const uint64_t m = lo + ((hi - lo) >> 1);
+                const uint32_t y = __ldg(rt.order[r] + m);
+                const SeqView vy = seq_view(rt.tokens[r], rt.seq_off[r], y);
+                // everything between the bounds shares at least min(l_lo, l_hi) tokens with Q
+                const uint64_t from = have_lo && have_hi ? (l_lo < l_hi ? l_lo : l_hi) : 0;
+                const uint64_t l = warp_lcp(vy, Q, from);
+                const bool above = l < vy.len && (l >= Q.len || __ldg(vy.tok + l) > __ldg(Q.tok + l));
+                if (above) { hi = m; l_hi = l; s_hi = y; have_hi = true; }
+                else { lo = m + 1; l_lo = l; s_lo = y; have_lo = true; }
+            }
+            const bool use_lo = have_lo && (!have_hi || l_lo >= l_hi);
+            const uint64_t L = use_lo ? l_lo : l_hi;
+            const uint64_t m_chunks = L / C;
+            if (m_chunks <= hit) continue;
+            const uint32_t owner = use_lo ? s_lo : s_hi;
+            const uint4 *src = reinterpret_cast<const uint4 *>(rt.vals[r]) +
+                               __ldg(rt.chunk_off[r] + owner);
+            for (uint64_t j = hit + lane; j < m_chunks; j += 32) recs[j] = __ldg(src + j);
+            hit = m_chunks;
+        }
+        for (uint64_t j = hit + lane; j < nch; j += 32) recs[j] = zero;
+        if (lane == 0) {
+            hit_out[q] = (uint32_t)hit;
+            atomicAdd(&st->chunks_hit, (unsigned long long)hit);
+            if (hit == 0) atomicAdd(&st->empty_probes, 1ull);
+        }
+    }
+}
+
+}  // namespace lsmkv

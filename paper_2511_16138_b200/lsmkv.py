@@ -26,7 +26,7 @@ EXPORTS = (
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
     "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
-    "lsmkv_relocate_records",
+    "lsmkv_relocate_records", "lsmkv_xrun_build", "lsmkv_xprobe_batch",
 )
 ST_OVERFLOW = 32
 CODEC_IDENTITY, CODEC_XP12 = 0, 1
@@ -44,6 +44,12 @@ class LsmkvError(RuntimeError):
         super().__init__(msg)
         self.code = code
         self.cuda = cuda
+
+
+class XRunStruct(C.Structure):
+    _fields_ = [("tokens", C.c_void_p), ("seq_off", C.c_void_p), ("vals", C.c_void_p),
+                ("order", C.c_void_p), ("chunk_off", C.c_void_p), ("n_seq", C.c_uint32),
+                ("reserved", C.c_uint32)]
 
 
 class GeomStruct(C.Structure):
@@ -152,6 +158,11 @@ def lib() -> C.CDLL:
                                           C.POINTER(u64), u32, vp, C.POINTER(PoolStruct)]
     L.lsmkv_relocate_records.restype = C.c_int
     L.lsmkv_relocate_records.argtypes = [vp, vp, vp, u64, C.POINTER(RelocStruct), u32, vp]
+    L.lsmkv_xrun_build.restype = C.c_int
+    L.lsmkv_xrun_build.argtypes = [vp, vp, vp, vp, u32, vp, vp]
+    L.lsmkv_xprobe_batch.restype = C.c_int
+    L.lsmkv_xprobe_batch.argtypes = [vp, vp, u32, vp, vp, vp, u64, C.POINTER(XRunStruct), u32,
+                                     vp, vp]
     L.lsmkv_encode_bound.restype = u64
     L.lsmkv_encode_bound.argtypes = [vp, u64]
     L.lsmkv_bloom_blocks.restype = u64
@@ -341,6 +352,24 @@ def lsmkv_relocate_records(ctx, stream, vals, n, table, changed_out=None) -> Non
     _check(ctx, rc, "lsmkv_relocate_records")
 
 
+def lsmkv_xrun_build(ctx, stream, tokens, seq_off, n_seq, order_out, chunk_off_out) -> None:
+    rc = lib().lsmkv_xrun_build(ctx, _stream(stream), _ptr(tokens), _ptr(seq_off), n_seq,
+                                _ptr(order_out), _ptr(chunk_off_out))
+    _check(ctx, rc, "lsmkv_xrun_build")
+
+
+def lsmkv_xprobe_batch(ctx, stream, n_query, tokens, seq_off, qchunk_off, n_qchunks, xruns,
+                       hit_chunks_out, recs_out) -> None:
+    """xruns: sequence of (tokens, seq_off, vals, order, chunk_off, n_seq), newest first."""
+    arr = (XRunStruct * max(1, len(xruns)))()
+    for i, (t, so, v, o, co, n) in enumerate(xruns):
+        arr[i] = XRunStruct(_ptr(t), _ptr(so), _ptr(v), _ptr(o), _ptr(co), n, 0)
+    rc = lib().lsmkv_xprobe_batch(ctx, _stream(stream), n_query, _ptr(tokens), _ptr(seq_off),
+                                  _ptr(qchunk_off), n_qchunks, arr, len(xruns),
+                                  _ptr(hit_chunks_out), _ptr(recs_out))
+    _check(ctx, rc, "lsmkv_xprobe_batch")
+
+
 def lsmkv_encode_bound(ctx, n_chunks: int) -> int:
     return int(lib().lsmkv_encode_bound(ctx, n_chunks))
 
@@ -485,6 +514,14 @@ class Context:
                           pool, stream=None):
         lsmkv_decode_batch_host(self.handle, stream, n_query, qchunk_off, hit_chunks, recs,
                                 arenas, dst_page_table, pool)
+
+    def xrun_build(self, tokens, seq_off, n_seq, order_out, chunk_off_out, stream=None):
+        lsmkv_xrun_build(self.handle, stream, tokens, seq_off, n_seq, order_out, chunk_off_out)
+
+    def xprobe_batch(self, n_query, tokens, seq_off, qchunk_off, n_qchunks, xruns,
+                     hit_chunks_out, recs_out, stream=None):
+        lsmkv_xprobe_batch(self.handle, stream, n_query, tokens, seq_off, qchunk_off, n_qchunks,
+                           xruns, hit_chunks_out, recs_out)
 
     def relocate_records(self, vals, n, table, changed_out=None, stream=None):
         lsmkv_relocate_records(self.handle, stream, vals, n, table, changed_out)

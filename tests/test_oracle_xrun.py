@@ -118,3 +118,13 @@ def test_planted_hits_and_newest_run_wins():
     assert [int(r["file_id"]) for r in recs[a:a + 3]] == [9, 9, 7]
     hit2, _ = oracle.xprobe_batch(g, w.query.tokens, w.query.seq_off, qoff, [])
     assert not hit2.any()
+
+
+def test_order_is_pythons_tuple_order():
+    rng = np.random.default_rng(5)
+    seqs = [rng.integers(0, 3, rng.integers(0, 9), dtype=np.uint32) for _ in range(300)]
+    seqs += [np.array([2**32 - 1, 0], np.uint32), np.array([2**31, 5], np.uint32),
+             np.array([], np.uint32), np.array([], np.uint32)]
+    b = synth.make_batch(seqs)
+    want = sorted(range(b.n), key=lambda i: (tuple(int(t) for t in b.seq(i)), i))
+    assert list(oracle.xrun_order(b.tokens, b.seq_off)) == want
