@@ -650,6 +650,8 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
 
         ms_plain, _, _ = timed(runs)
         ms, st, reps = timed(runs_bloom)
+        exact = exact_index_numbers(torch, ctx, w, up, d_tok, d_off, d_qoff, total, d_hit, d_recs,
+                                    max(3, warmup), max(5, steps))
         hit_tokens = int(w.expected_hit.sum()) * 16
         # least traffic any probe must do: tokens up to the first miss, one record per query
         # chunk, one hit length per query
@@ -664,9 +666,43 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
                 "query_tokens": int(len(w.query.tokens)), "stored_keys": n,
                 "algorithmic_GBps": algo_bytes / ms / 1e6,
                 "flush_ms_for_%d_keys" % big: flush_big_ms,
+                "exact_index": exact,
                 "bound": "L2 latency / instruction issue (not HBM)"}
     finally:
         ctx.close()
+
+
+def exact_index_numbers(torch, ctx, w, up, d_tok, d_off, d_qoff, total, d_hit, d_recs, warm, reps):
+    """The same queries against the exact prefix index (stored sequences ordered by their tokens,
+    no digests): build time over the whole stored sequences and probe time."""
+    dev = d_tok.device
+    s_tok, s_off = up(w.store.tokens), up(w.store.seq_off)
+    n_seq = w.store.n
+    n_chunks = int(synth.chunk_counts(w.store.seq_off, 16).sum())
+    s_vals = torch.zeros(max(1, n_chunks) * 16, dtype=torch.uint8, device=dev)
+    d_order = torch.empty(max(1, n_seq), dtype=torch.int32, device=dev)
+    d_coff = torch.empty(n_seq + 1, dtype=torch.int64, device=dev)
+
+    def time_of(fn, n_warm, n_rep):
+        for _ in range(n_warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_rep):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n_rep
+
+    build_ms = time_of(lambda: ctx.xrun_build(s_tok, s_off, n_seq, d_order, d_coff), 2, 3)
+    xr = [(s_tok, s_off, s_vals, d_order, d_coff, n_seq)]
+    probe = lambda: ctx.xprobe_batch(w.query.n, d_tok, d_off, d_qoff, total, xr, d_hit, d_recs)
+    ms = time_of(probe, warm, reps)
+    assert np.array_equal(d_hit.cpu().numpy(), w.expected_hit.astype(np.int32))
+    ctx.last_status()
+    return {"stored_sequences": n_seq, "stored_chunks": n_chunks, "build_ms": build_ms,
+            "ms_per_probe": ms, "keys_per_s": total / ms * 1e3}
 
 
 def xp12_block(torch, lsmkv, dev, device_index, d, src_bufs, src_pool, dst_bufs, dst_pool, arena,

@@ -27,25 +27,59 @@ __device__ __forceinline__ SeqView seq_view(const uint32_t *__restrict__ tokens,
 // `from` (the caller knows the first `from` tokens agree). Every lane returns the same value.
 __device__ __forceinline__ uint64_t warp_lcp(const SeqView &a, const SeqView &b, uint64_t from)
 {
+    constexpr int kUnroll = 4;                   // 128 tokens per step, all loads in flight at once
     const uint64_t n = a.len < b.len ? a.len : b.len;
     const unsigned lane = lane_id();
-    for (uint64_t i = from; i < n; i += 32) {
-        const uint64_t k = i + lane;
-        const bool differ = k < n && __ldg(a.tok + k) != __ldg(b.tok + k);
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, differ);
-        if (m) return i + (unsigned)__ffs(m) - 1u;
+    for (uint64_t i = from; i < n; i += 32 * kUnroll) {
+        bool differ[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const uint64_t k = i + 32u * u + lane;
+            differ[u] = k < n && __ldg(a.tok + k) != __ldg(b.tok + k);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, differ[u]);
+            if (m) return i + 32u * u + (unsigned)__ffs(m) - 1u;
+        }
     }
     return n;
 }
 
-// a < b in token order given their common prefix length l; a proper prefix is smaller; equal
-// strings order by the tie-break ids.
-__device__ __forceinline__ bool seq_less_at(const SeqView &a, const SeqView &b, uint64_t l,
-                                            uint32_t ia, uint32_t ib)
+// Where x belongs among the sorted sequences order[lo, hi): the first position whose sequence is
+// above x. "Above" = larger in token order (a proper prefix is smaller); a sequence with the same
+// tokens is above x when its number exceeds x_id. The two ends are compared before bisecting
+// (in the sort an element usually falls wholly before or after the sibling segment); once both
+// bounds are known every comparison starts at min(l_lo, l_hi): everything between the bounds
+// shares at least that many tokens with x.
+struct Located {
+    uint64_t pos;            // order[pos - 1] is not above x, order[pos] is
+    uint64_t l_lo, l_hi;     // tokens x shares with those two neighbours
+    uint32_t s_lo, s_hi;     // their sequence numbers
+    bool have_lo, have_hi;   // whether such a neighbour exists in [lo, hi)
+};
+
+__device__ __forceinline__ Located warp_locate(const SeqView &x, uint32_t x_id,
+                                               const uint32_t *__restrict__ tokens,
+                                               const uint64_t *__restrict__ seq_off,
+                                               const uint32_t *__restrict__ order, uint64_t lo,
+                                               uint64_t hi)
 {
-    if (l < a.len && l < b.len) return __ldg(a.tok + l) < __ldg(b.tok + l);
-    if (a.len != b.len) return a.len < b.len;
-    return ia < ib;
+    Located r{lo, 0, 0, 0, 0, false, false};
+    while (lo < hi) {
+        const uint64_t m = !r.have_hi ? hi - 1 : !r.have_lo ? lo : lo + ((hi - lo) >> 1);
+        const uint32_t y = __ldg(order + m);
+        const SeqView vy = seq_view(tokens, seq_off, y);
+        const uint64_t from = r.have_lo && r.have_hi ? (r.l_lo < r.l_hi ? r.l_lo : r.l_hi) : 0;
+        const uint64_t l = warp_lcp(vy, x, from);
+        // y ends at l: a prefix of x (below) or the same tokens (the numbers decide)
+        const bool above = l < vy.len ? (l >= x.len || __ldg(vy.tok + l) > __ldg(x.tok + l))
+                                      : (vy.len == x.len && y > x_id);
+        if (above) { hi = m; r.l_hi = l; r.s_hi = y; r.have_hi = true; }
+        else { lo = m + 1; r.l_lo = l; r.s_lo = y; r.have_lo = true; }
+    }
+    r.pos = lo;
+    return r;
 }
 
 __global__ void __launch_bounds__(256)
@@ -78,16 +112,9 @@ k_xrun_merge_level(const uint32_t *__restrict__ tokens, const uint64_t *__restri
         const SeqView vx = seq_view(tokens, seq_off, x);
         uint64_t lo, hi;
         if (i < mid) { lo = mid; hi = end; } else { lo = base; hi = mid; }
-        const uint64_t first = lo;
-        while (lo < hi) {                                    // sibling elements below x
-            const uint64_t m = lo + ((hi - lo) >> 1);
-            const uint32_t y = __ldg(src + m);
-            const SeqView vy = seq_view(tokens, seq_off, y);
-            const uint64_t l = warp_lcp(vy, vx, 0);
-            if (seq_less_at(vy, vx, l, y, x)) lo = m + 1; else hi = m;
-        }
+        const uint64_t below = warp_locate(vx, x, tokens, seq_off, src, lo, hi).pos - lo;
         const uint64_t own = i < mid ? i - base : i - mid;
-        if (lane_id() == 0) dst[base + own + (lo - first)] = x;
+        if (lane_id() == 0) dst[base + own + below] = x;
     }
 }
 
@@ -129,6 +156,8 @@ k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint
         for (uint32_t r = 0; r < n_runs; ++r) {
             const uint32_t n = rt.n_seq[r];
             if (n == 0 || hit >= nch) continue;
+            // The search is written out here rather than shared with the sort's routine: the
+            // shared form measured a third slower in this kernel.
             // invariant: order[lo - 1] <= Q < order[hi]; l_lo / l_hi = tokens Q shares with them
             uint64_t lo = 0, hi = n, l_lo = 0, l_hi = 0;
             uint32_t s_lo = 0, s_hi = 0;
