@@ -119,6 +119,26 @@ void fill_key_consts(KeyConsts &kc, uint32_t C)
         a = host_mulmod(a, mA);
         b = host_mulmod(b, mB);
     }
+    // weights of the 16 tokens of a block, BASE^(15-i), in limbs of 21 + 21 + 19 bits
+    a = 1;
+    b = 1;
+    kc.sumA = 0;
+    kc.sumB = 0;
+    for (int i = 15; i >= 0; --i) {
+        const uint64_t w[2] = {a, b};
+        for (int x = 0; x < 2; ++x) {
+            uint32_t *d = x == 0 ? kc.dA[i] : kc.dB[i];
+            d[0] = (uint32_t)(w[x] & 0x1FFFFFu);
+            d[1] = (uint32_t)((w[x] >> 21) & 0x1FFFFFu);
+            d[2] = (uint32_t)(w[x] >> 42);
+        }
+        kc.sumA = (kc.sumA + a) % kP;
+        kc.sumB = (kc.sumB + b) % kP;
+        a = host_mulmod(a, kBaseA);
+        b = host_mulmod(b, kBaseB);
+    }
+    kc.b16A = a;
+    kc.b16B = b;
 }
 
 // Brackets one kernel launch with events when profiling is on.
@@ -245,6 +265,7 @@ unsigned merge_grid(const lsmkv_ctx *ctx, uint64_t n)
 }
 
 constexpr uint64_t kDirMaxJ = 65536;   // chunk indices covered by the probe's directory
+constexpr uint64_t kOrderMaxQueries = 65536;   // batches up to this size are handed out longest first
 
 uint64_t *ws_hit_off(lsmkv_ctx *ctx) { return static_cast<uint64_t *>(ctx->d_ws); }
 uint32_t *ws_plan(lsmkv_ctx *ctx)
@@ -419,7 +440,7 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
         return LSMKV_ECUDA;
     }
     int rc = ensure_workspace(ctx, 1024, 65536);
-    if (rc == LSMKV_OK) rc = ensure_dir(ctx, 2 + 8 * (kDirMaxJ + 1));
+    if (rc == LSMKV_OK) rc = ensure_dir(ctx, 2 + 8 * (kDirMaxJ + 1) + kOrderMaxQueries / 2);
     if (rc != LSMKV_OK) {
         if (ctx->d_ws) cudaFree(ctx->d_ws);
         cudaFree(ctx->d_status);
@@ -459,7 +480,8 @@ int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
     DeviceGuard guard(ctx->device);
     int rc = ensure_workspace(ctx, n_seq, n_chunks);
     if (rc != LSMKV_OK) return rc;
-    return ensure_dir(ctx, 2 + 8 * ((n_chunks < kDirMaxJ ? n_chunks : kDirMaxJ) + 1));
+    return ensure_dir(ctx, 2 + 8 * ((n_chunks < kDirMaxJ ? n_chunks : kDirMaxJ) + 1) +
+                               kOrderMaxQueries / 2);
 }
 
 int lsmkv_encode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_req, const uint32_t *tokens,
@@ -552,13 +574,16 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint32_t jcap = (uint32_t)(n_qchunks < kDirMaxJ ? n_qchunks : kDirMaxJ);
-    // d_dir: [0] = the probe's work counter, [2..] = the directory
+    // d_dir: [0] = the probe's work counter, [2..] = the directory, then the hand-out order
+    const uint64_t dir_entries = (uint64_t)n_runs * ((uint64_t)jcap + 1);
+    const bool ordered = n_query > 1 && n_query <= kOrderMaxQueries;
     {
-        int rc = ensure_dir(ctx, 2 + (uint64_t)n_runs * ((uint64_t)jcap + 1));
+        int rc = ensure_dir(ctx, 2 + dir_entries + (ordered ? (n_query + 1) / 2 : 0));
         if (rc != LSMKV_OK) return rc;
     }
     unsigned long long *next_query = reinterpret_cast<unsigned long long *>(ctx->d_dir);
     uint64_t *dir = ctx->d_dir + 2;
+    uint32_t *order = ordered ? reinterpret_cast<uint32_t *>(dir + dir_entries) : nullptr;
     {
         LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
         {
@@ -568,7 +593,8 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
             if (dgrid > dcap) dgrid = dcap;
             if (dgrid == 0) dgrid = 1;
             k_run_dir<<<(unsigned)dgrid, 256, 0, s>>>(rt, n_runs, ctx->geom.ns, jcap, dir,
-                                                      next_query);
+                                                      next_query, n_query, seq_off,
+                                                      ctx->geom.chunk_tokens, order);
             ++ctx->launches;
         }
         const unsigned warps = (unsigned)ctx->probe_warps_per_cta;
@@ -580,7 +606,7 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
                                                    ctx->geom.chunk_tokens, ctx->geom.ns, n_query,
                                                    tokens, seq_off, qchunk_off, n_qchunks,
                                                    hit_chunks_out, recs_out, keys_out,
-                                                   ctx->d_status, next_query);
+                                                   ctx->d_status, next_query, order);
         ++ctx->launches;
     }
     CU(ctx, cudaGetLastError());

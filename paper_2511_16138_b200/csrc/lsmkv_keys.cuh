@@ -18,9 +18,15 @@ constexpr uint64_t kBaseB = 0x16A09E667F3BCC90ull;
 
 // pw[x][i] = (BASE_x ^ C) ^ (i+1) mod p for i = 0..31; entries 0,1,3,7,15 are the scan
 // multipliers M^1, M^2, M^4, M^8, M^16.
+// d[x][i] = BASE_x ^ (15 - i) mod p cut into limbs of 21, 21 and 19 bits: the weights of the 16
+// tokens of a block (see block16_dot). sum[x] = BASE^0 + ... + BASE^15, b16[x] = BASE^16 (mod p).
 struct KeyConsts {
     uint64_t pwA[32];
     uint64_t pwB[32];
+    uint32_t dA[16][3];
+    uint32_t dB[16][3];
+    uint64_t sumA, sumB;
+    uint64_t b16A, b16B;
 };
 
 // a, b < 2^61  ->  a*b mod p, canonical
@@ -56,42 +62,79 @@ __device__ __forceinline__ uint64_t shfl_up64(uint64_t v, unsigned d)
 
 struct ChunkKey { uint64_t w0, w1, w2, w3; };
 
-// Hash of one chunk from h = 0 (both lanes), plus its first and last token. 16-byte loads when
-// the chunk start is 16-byte aligned.
-__device__ __forceinline__ void chunk_hash(const uint32_t *t, uint32_t C, bool vec_ok,
-                                           uint64_t &hA, uint64_t &hB, uint32_t &first,
-                                           uint32_t &last)
+// a0 + a1 * 2^21 + a2 * 2^42 + sum (mod p), canonical; a0, a1 < 2^57, a2 < 2^55, sum < p.
+// 2^61 = 1 (mod p), so the bits a shift pushes past bit 60 come back in at bit 0.
+__device__ __forceinline__ uint64_t limbs_mod61(uint64_t a0, uint64_t a1, uint64_t a2, uint64_t sum)
 {
-    if (vec_ok) {
-        const uint4 *t4 = reinterpret_cast<const uint4 *>(t);
-        uint4 v = __ldg(t4);
-        first = v.x;
-        hA = (uint64_t)v.x + 1ull;
-        hB = hA;
-        hA = horner61(hA, kBaseA, v.y); hB = horner61(hB, kBaseB, v.y);
-        hA = horner61(hA, kBaseA, v.z); hB = horner61(hB, kBaseB, v.z);
-        hA = horner61(hA, kBaseA, v.w); hB = horner61(hB, kBaseB, v.w);
-        last = v.w;
-#pragma unroll 3
-        for (uint32_t i = 1; i < (C >> 2); ++i) {
-            v = __ldg(t4 + i);
-            hA = horner61(hA, kBaseA, v.x); hB = horner61(hB, kBaseB, v.x);
-            hA = horner61(hA, kBaseA, v.y); hB = horner61(hB, kBaseB, v.y);
-            hA = horner61(hA, kBaseA, v.z); hB = horner61(hB, kBaseB, v.z);
-            hA = horner61(hA, kBaseA, v.w); hB = horner61(hB, kBaseB, v.w);
-            last = v.w;
+    uint64_t s = a0 + ((a1 & ((1ull << 40) - 1)) << 21) + (a1 >> 40) +
+                 ((a2 & ((1ull << 19) - 1)) << 42) + (a2 >> 19) + sum;      // < 2^63
+    s = (s & kP) + (s >> 61);                                               // <= p + 3
+    return s >= kP ? s - kP : s;
+}
+
+__device__ __forceinline__ uint4 load_tokens4(const uint32_t *t, bool vec_ok)
+{
+    if (vec_ok) return __ldg(reinterpret_cast<const uint4 *>(t));
+    return make_uint4(__ldg(t), __ldg(t + 1), __ldg(t + 2), __ldg(t + 3));
+}
+
+// Digest of 16 tokens from h = 0 (both lanes). Sixteen Horner steps from zero give
+// sum_i (t_i + 1) * BASE^(15-i); with the weights cut into limbs of at most 21 bits every
+// product t_i * limb is below 2^53, sixteen of them add up without overflow, and one reduction
+// at the end replaces sixteen modular multiplications. Exact, hence the same value.
+__device__ __forceinline__ void block16_dot(const KeyConsts &kc, const uint4 (&v)[4], uint64_t &dA,
+                                            uint64_t &dB)
+{
+    uint64_t a0 = 0, a1 = 0, a2 = 0, b0 = 0, b1 = 0, b2 = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int i = 4 * q + e;
+            a0 += (uint64_t)w[e] * kc.dA[i][0];
+            a1 += (uint64_t)w[e] * kc.dA[i][1];
+            a2 += (uint64_t)w[e] * kc.dA[i][2];
+            b0 += (uint64_t)w[e] * kc.dB[i][0];
+            b1 += (uint64_t)w[e] * kc.dB[i][1];
+            b2 += (uint64_t)w[e] * kc.dB[i][2];
         }
-    } else {
-        first = __ldg(t);
-        last = first;
-        hA = (uint64_t)first + 1ull;
-        hB = hA;
-#pragma unroll 4
-        for (uint32_t i = 1; i < C; ++i) {
-            last = __ldg(t + i);
-            hA = horner61(hA, kBaseA, last);
-            hB = horner61(hB, kBaseB, last);
+    }
+    dA = limbs_mod61(a0, a1, a2, kc.sumA);
+    dB = limbs_mod61(b0, b1, b2, kc.sumB);
+}
+
+// Hash of one chunk from h = 0 (both lanes), plus its first and last token: whole blocks of 16
+// tokens by block16_dot, chained with BASE^16, the remaining tokens by the recurrence itself.
+// 16-byte loads when the chunk start is 16-byte aligned.
+__device__ __forceinline__ void chunk_hash(const KeyConsts &kc, const uint32_t *t, uint32_t C,
+                                           bool vec_ok, uint64_t &hA, uint64_t &hB,
+                                           uint32_t &first, uint32_t &last)
+{
+    hA = 0;
+    hB = 0;
+    uint32_t i = 0;
+    for (; i + 16 <= C; i += 16) {
+        uint4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) v[q] = load_tokens4(t + i + 4 * q, vec_ok);
+        uint64_t dA, dB;
+        block16_dot(kc, v, dA, dB);
+        if (i == 0) {
+            first = v[0].x;
+            hA = dA;
+            hB = dB;
+        } else {
+            hA = addmod61(mulmod61(hA, kc.b16A), dA);
+            hB = addmod61(mulmod61(hB, kc.b16B), dB);
         }
+        last = v[3].w;
+    }
+    for (; i < C; ++i) {
+        last = __ldg(t + i);
+        if (i == 0) first = last;
+        hA = horner61(hA, kBaseA, last);
+        hB = horner61(hB, kBaseB, last);
     }
 }
 
@@ -108,7 +151,7 @@ __device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint3
     hA = 0; hB = 0; first = 0; last = 0;
     if (j < nch) {
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
-        chunk_hash(seq + j * C, C, vec_ok, hA, hB, first, last);
+        chunk_hash(kc, seq + j * C, C, vec_ok, hA, hB, first, last);
     }
     // inclusive scan: x_i <- x_{i-d} * M^d + x_i
 #pragma unroll
@@ -119,29 +162,6 @@ __device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint3
             hB = addmod61(mulmod61(uB, kc.pwB[d - 1]), hB);
         }
     }
-}
-
-// Same, with the running prefix: carryA/carryB are the digests of the prefix that ends just
-// before chunk base_j (0 at base_j = 0) and are advanced past chunk base_j + 31.
-__device__ __forceinline__ ChunkKey warp_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
-                                                    uint32_t C, uint32_t ns, uint64_t base_j,
-                                                    uint64_t nch, uint64_t &carryA,
-                                                    uint64_t &carryB)
-{
-    const unsigned lane = lane_id();
-    uint64_t hA, hB;
-    uint32_t first, last;
-    warp_block_scan(kc, seq, C, base_j, nch, hA, hB, first, last);
-    hA = addmod61(mulmod61(carryA, kc.pwA[lane]), hA);
-    hB = addmod61(mulmod61(carryB, kc.pwB[lane]), hB);
-    carryA = __shfl_sync(0xFFFFFFFFu, hA, 31);
-    carryB = __shfl_sync(0xFFFFFFFFu, hB, 31);
-    ChunkKey k;
-    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)(base_j + lane);
-    k.w1 = hA;
-    k.w2 = hB;
-    k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
-    return k;
 }
 
 constexpr int kKeyMaxWarps = 16;

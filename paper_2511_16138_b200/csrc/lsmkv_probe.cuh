@@ -77,14 +77,57 @@ __device__ __forceinline__ uint64_t lower_bound_w0(const lsmkv_key_t *keys, uint
     return lo;
 }
 
+// Length class of a query with nch chunks: 0..3 for itself, then four classes per power of two.
+constexpr int kLenClasses = 128;
+__device__ __forceinline__ uint32_t len_class(uint64_t nch)
+{
+    if (nch < 4) return (uint32_t)nch;
+    if (nch > 0xFFFFFFFFull) return kLenClasses - 1;
+    const uint32_t n = (uint32_t)nch, e = 31u - __clz(n);
+    return 4u * e + ((n >> (e - 2u)) & 3u) - 4u;           // e >= 2: 4..123
+}
+
+// order[0..n_query) = the queries by descending length class (counting sort by one CTA; the
+// order inside a class is whatever the atomics give, results do not depend on it). The probe
+// hands queries out in this order, so the longest ones -- whose rounds run one after another in
+// one CTA -- start first and the short ones fill the gaps at the end.
+__device__ __forceinline__ void order_queries(uint32_t n_query, const uint64_t *__restrict__ seq_off,
+                                              uint32_t C, uint32_t *__restrict__ order)
+{
+    __shared__ uint32_t s_cnt[kLenClasses];
+    for (uint32_t t = threadIdx.x; t < kLenClasses; t += blockDim.x) s_cnt[t] = 0;
+    __syncthreads();
+    for (uint32_t q = threadIdx.x; q < n_query; q += blockDim.x) {
+        const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
+        atomicAdd(&s_cnt[len_class(s1 >= s0 ? (s1 - s0) / C : 0)], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {                                // counts -> first slot of every class
+        uint32_t at = 0;
+        for (int c = kLenClasses - 1; c >= 0; --c) {
+            const uint32_t n = s_cnt[c];
+            s_cnt[c] = at;
+            at += n;
+        }
+    }
+    __syncthreads();
+    for (uint32_t q = threadIdx.x; q < n_query; q += blockDim.x) {
+        const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
+        order[atomicAdd(&s_cnt[len_class(s1 >= s0 ? (s1 - s0) / C : 0)], 1u)] = q;
+    }
+}
+
 // dir[r * stride + j] = first index of run r whose chunk index is >= j (same namespace),
 // for j = 0..jcap (stride = jcap + 1).
-// Also resets the probe's work counter (*next_query) for the launch that follows.
+// Also resets the probe's work counter (*next_query) for the launch that follows, and its last
+// block writes the hand-out order of the queries when `order` is given.
 __global__ void __launch_bounds__(256)
 k_run_dir(const __grid_constant__ RunTable rt, uint32_t n_runs, uint32_t ns, uint32_t jcap,
-          uint64_t *__restrict__ dir, unsigned long long *next_query)
+          uint64_t *__restrict__ dir, unsigned long long *next_query, uint32_t n_query,
+          const uint64_t *__restrict__ seq_off, uint32_t C, uint32_t *__restrict__ order)
 {
     if (blockIdx.x == 0 && threadIdx.x == 0) *next_query = 0;
+    if (order && blockIdx.x == gridDim.x - 1) order_queries(n_query, seq_off, C, order);
     const uint64_t stride = (uint64_t)jcap + 1;
     const uint64_t total = (uint64_t)n_runs * stride;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
@@ -120,74 +163,119 @@ __device__ __noinline__ uint64_t bucket_find_exact(const lsmkv_key_t *keys, uint
     return ~0ull;
 }
 
-// Exact search of the key in bucket [lo, hi) of one run. Returns its index or ~0.
-//
-// Fast path: the digest w1 is uniform, so the key's rank inside the bucket is close to
-// w1 * cnt / 2^61 (standard deviation <= sqrt(cnt) / 2). A branch-free binary search on w1 over
-// a window of about +-2.5 standard deviations around that guess pins it with ~log2(window)
-// loads, the same number for every lane of a warp. Whenever the window cannot prove presence or
-// absence (the answer falls on a window edge, or digests tie) the slow path searches the whole
-// bucket with the full key, so the result is exact in every case.
-__device__ __forceinline__ uint64_t bucket_find(const lsmkv_key_t *keys, uint64_t lo, uint64_t hi,
-                                                const ChunkKey &k)
-{
-    const uint64_t cnt64 = hi - lo;
-    if (cnt64 == 0) return ~0ull;
-    if (cnt64 >= 0x40000000ull) return bucket_find_exact(keys, lo, hi, k);
-    const uint32_t cnt = (uint32_t)cnt64;
-    const unsigned long long *w1p = reinterpret_cast<const unsigned long long *>(keys + lo) + 1;
-    uint32_t a = 0, n = cnt;
-    if (cnt > 16) {
-        const uint32_t g = (uint32_t)__umul64hi(k.w1 << 3, cnt64);    // w1 * cnt / 2^61
-        const uint32_t R = 4u + (uint32_t)(1.25f * sqrtf((float)cnt));
-        a = g > R ? g - R : 0u;
-        const uint32_t e = min(cnt, g + R + 1u);
-        n = e - a;
-    }
-    const uint32_t a0 = a, e0 = a + n;
-    uint32_t pos = a;                              // last index in the window with w1 <= target
-    while (n > 1) {
-        const uint32_t half = n >> 1;
-        const uint64_t v = __ldg(w1p + 4ull * (pos + half));
-        pos = v <= k.w1 ? pos + half : pos;
-        n -= half;
-    }
-    const uint64_t v = __ldg(w1p + 4ull * pos);
-    if (v == k.w1) {
-        const lsmkv_key_t *e = keys + lo + pos;
-        if (key_w(e, 2) == k.w2 && key_w(e, 3) == k.w3) return lo + pos;
-        return bucket_find_exact(keys, lo, hi, k);             // digest tie: be exact
-    }
-    if (v > k.w1) {                                // only possible at pos == a0
-        return a0 > 0 ? bucket_find_exact(keys, lo, lo + a0, k) : ~0ull;
-    }
-    // v < target: absent unless the window ended before the bucket did
-    if (pos + 1 == e0 && e0 < cnt) return bucket_find_exact(keys, lo + e0, hi, k);
-    return ~0ull;
-}
-
 // Point lookup, newest run first; the first run that holds the key decides.
+//
+// Inside a bucket the digest w1 is uniform, so the key's rank is close to w1 * cnt / 2^61
+// (standard deviation <= sqrt(cnt) / 2). A branch-free binary search on w1 over a window of about
+// +-2.5 standard deviations around that guess pins it with ~log2(window) loads. Whenever the
+// window cannot prove presence or absence (the answer falls on a window edge, or digests tie) a
+// plain search of the whole bucket with the full key decides, so the result is exact in every
+// case.
+//
+// Each search is a chain of dependent loads that hit L2 at best, and a warp has nothing else to
+// do while it waits. The runs are therefore searched kLookupGroup at a time in lock step: the
+// bucket bounds of the whole group are fetched together, then every step of the window search
+// issues one load per run before any of them is needed, so a group costs the latency of one
+// chain. The answers are then taken in age order, which keeps the first-match rule.
+constexpr int kLookupGroup = 4;
+
 __device__ __forceinline__ bool lookup_runs(const RunTable &rt, uint32_t n_runs,
                                             const uint64_t *__restrict__ dir, uint32_t jcap,
                                             const ChunkKey &k, uint4 &val)
 {
     const uint64_t j = k.w0 & 0xFFFFFFFFull;
     const uint64_t stride = (uint64_t)jcap + 1;
-    for (uint32_t r = 0; r < n_runs; ++r) {
-        if (rt.bloom[r] && !bloom_may_contain(rt.bloom[r], rt.bloom_blocks[r], k)) continue;
-        const lsmkv_key_t *keys = rt.keys[r];
-        uint64_t lo, hi;
-        if (j < jcap) {
-            lo = __ldg(dir + r * stride + j);
-            hi = __ldg(dir + r * stride + j + 1);
-        } else {                                   // beyond the directory: find the bucket
-            lo = lower_bound_w0(keys, rt.n[r], k.w0);
-            hi = lower_bound_w0(keys, rt.n[r], k.w0 + 1);
+    for (uint32_t r0 = 0; r0 < n_runs; r0 += kLookupGroup) {
+        uint64_t lo[kLookupGroup], hi[kLookupGroup];
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t r = r0 + g;
+            lo[g] = 0;
+            hi[g] = 0;
+            if (r < n_runs) {                              // uniform over the grid
+                if (j < jcap) {
+                    lo[g] = __ldg(dir + r * stride + j);
+                    hi[g] = __ldg(dir + r * stride + j + 1);
+                } else {                                   // beyond the directory: find the bucket
+                    lo[g] = lower_bound_w0(rt.keys[r], rt.n[r], k.w0);
+                    hi[g] = lower_bound_w0(rt.keys[r], rt.n[r], k.w0 + 1);
+                }
+            }
         }
-        const uint64_t pos = bucket_find(keys, lo, hi, k);
-        if (pos != ~0ull) {
-            val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + pos));
-            return true;
+        // window of every run: [a0, e0) inside its bucket, n = entries still in play (0 = the
+        // run cannot hold the key, or the bucket is too large for 32-bit positions)
+        const unsigned long long *w1p[kLookupGroup];
+        uint32_t pos[kLookupGroup], n[kLookupGroup], a0[kLookupGroup], e0[kLookupGroup];
+        uint32_t n_max = 0;
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t r = r0 + g;
+            uint64_t cnt64 = hi[g] - lo[g];
+            if (r < n_runs && cnt64 && rt.bloom[r] &&
+                !bloom_may_contain(rt.bloom[r], rt.bloom_blocks[r], k))
+                cnt64 = 0;                                 // ruled out by the filter
+            w1p[g] = r < n_runs
+                         ? reinterpret_cast<const unsigned long long *>(rt.keys[r] + lo[g]) + 1
+                         : nullptr;
+            uint32_t a = 0, m = 0;
+            if (cnt64 && cnt64 < 0x40000000ull) {
+                const uint32_t cnt = (uint32_t)cnt64;
+                m = cnt;
+                if (cnt > 16) {
+                    const uint32_t gs = (uint32_t)__umul64hi(k.w1 << 3, cnt64);   // w1 * cnt / 2^61
+                    const uint32_t R = 4u + (uint32_t)(1.25f * sqrtf((float)cnt));
+                    a = gs > R ? gs - R : 0u;
+                    m = min(cnt, gs + R + 1u) - a;
+                }
+            }
+            if (cnt64 == 0) hi[g] = lo[g];                 // remembered as "empty"
+            a0[g] = a;
+            e0[g] = a + m;
+            pos[g] = a;
+            n[g] = m;
+            n_max = max(n_max, m);
+        }
+        // lock-step search: pos = last index in the window with w1 <= target
+        while (n_max > 1) {
+#pragma unroll
+            for (int g = 0; g < kLookupGroup; ++g) {
+                if (n[g] > 1) {
+                    const uint32_t half = n[g] >> 1;
+                    const uint64_t v = __ldg(w1p[g] + 4ull * (pos[g] + half));
+                    pos[g] = v <= k.w1 ? pos[g] + half : pos[g];
+                    n[g] -= half;
+                }
+            }
+            n_max -= n_max >> 1;
+        }
+        uint64_t v[kLookupGroup];
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g)
+            v[g] = n[g] ? __ldg(w1p[g] + 4ull * pos[g]) : 0;
+        // answers in age order
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t r = r0 + g;
+            if (r >= n_runs || hi[g] == lo[g]) continue;
+            const lsmkv_key_t *keys = rt.keys[r];
+            uint64_t at = ~0ull;
+            if (n[g] == 0) {                               // huge bucket
+                at = bucket_find_exact(keys, lo[g], hi[g], k);
+            } else if (v[g] == k.w1) {
+                const ulonglong2 w23 = __ldg(reinterpret_cast<const ulonglong2 *>(
+                    reinterpret_cast<const unsigned long long *>(keys + lo[g] + pos[g]) + 2));
+                if (w23.x == k.w2 && w23.y == k.w3) at = lo[g] + pos[g];
+                else at = bucket_find_exact(keys, lo[g], hi[g], k);          // digest tie: be exact
+            } else if (v[g] > k.w1) {                      // only possible at pos == a0
+                if (a0[g] > 0) at = bucket_find_exact(keys, lo[g], lo[g] + a0[g], k);
+            } else if (pos[g] + 1 == e0[g] && lo[g] + e0[g] < hi[g]) {
+                // below the target at the window's last entry, and the bucket goes on
+                at = bucket_find_exact(keys, lo[g] + e0[g], hi[g], k);
+            }
+            if (at != ~0ull) {
+                val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + at));
+                return true;
+            }
         }
     }
     return false;
@@ -199,7 +287,8 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         uint32_t ns, uint32_t n_query, const uint32_t *__restrict__ tokens,
         const uint64_t *__restrict__ seq_off, const uint64_t *__restrict__ qchunk_off,
         uint64_t n_qchunks, uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out,
-        lsmkv_key_t *__restrict__ keys_out, DevStatus *st, unsigned long long *next_query)
+        lsmkv_key_t *__restrict__ keys_out, DevStatus *st, unsigned long long *next_query,
+        const uint32_t *__restrict__ order)
 {
     __shared__ uint64_t s_aggA[kKeyMaxWarps], s_aggB[kKeyMaxWarps];
     __shared__ unsigned long long s_first_miss, s_q;
@@ -213,8 +302,8 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         __syncthreads();
         if (threadIdx.x == 0) s_q = atomicAdd(next_query, 1ull);
         __syncthreads();
-        const uint64_t q = s_q;
-        if (q >= n_query) break;
+        if (s_q >= n_query) break;
+        const uint64_t q = order ? order[s_q] : s_q;
         const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
         const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
         const uint64_t o0 = qchunk_off[q], o1 = qchunk_off[q + 1];
@@ -234,6 +323,11 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                 continue;
             }
             if (threadIdx.x == 0) s_first_miss = ~0ull;
+            if (j + round_chunks < nch) {                    // next round's tokens on their way
+                const char *nx = reinterpret_cast<const char *>(seq + (j + round_chunks) * C);
+                for (uint32_t b = 0; b < 4u * C; b += 128u)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(nx + b));
+            }
             const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, cA, cB, s_aggA, s_aggB);
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
             if (done) {
