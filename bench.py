@@ -337,11 +337,14 @@ def main():
         d["run_k"] = torch.empty(n * 32, dtype=torch.uint8, device=dev)
         d["run_v"] = torch.empty(n * 16, dtype=torch.uint8, device=dev)
         d["run_n"] = torch.zeros(1, dtype=torch.int64, device=dev)
+        d["hidx_buckets"] = lsmkv.lsmkv_hindex_buckets(n)
+        d["hidx"] = torch.empty(d["hidx_buckets"] * 32, dtype=torch.uint8, device=dev)
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
         ctx.flush_batch(d["keys"], d["vals"], n, d["run_k"], d["run_v"], d["run_n"], stream=stream)
+        ctx.hindex_build(d["run_k"], n, d["hidx"], stream=stream)
         f1.record(stream)
-        d["runs"] = [(d["run_k"], d["run_v"], n)]
+        d["runs"] = [(d["run_k"], d["run_v"], n, None, 0, d["hidx"], d["hidx_buckets"])]
         probe(d)
         decode(d)
         torch.cuda.synchronize()
@@ -355,11 +358,12 @@ def main():
     def flush(d):
         ctx.flush_batch(d["keys"], d["vals"], d["n"], d["run_k"], d["run_v"], d["run_n"],
                         stream=stream)
+        ctx.hindex_build(d["run_k"], d["n"], d["hidx"], stream=stream)
 
     def step():
         for d in W:
             encode(d)      # chunk keys + records + pack
-            flush(d)       # the batch's keys become the sorted run the probe searches
+            flush(d)       # the batch's keys become the sorted run (+ its hash index) the probe reads
             probe(d)
             decode(d)      # plan + unpack
 
@@ -632,6 +636,21 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
             bl = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
             ctx.bloom_build(tk, m_, bl)
             runs_bloom.append((tk, tv, m_, bl, nb))
+        # the same runs with their hash indexes attached (build time measured on the big run)
+        runs_hashed, hidx_ms = [], 0.0
+        for (tk, tv, m_) in runs:
+            nb = lsmkv.lsmkv_hindex_buckets(m_)
+            hx = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+            ctx.hindex_build(tk, m_, hx)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(3):
+                ctx.hindex_build(tk, m_, hx)
+            e1.record()
+            torch.cuda.synchronize()
+            hidx_ms = e0.elapsed_time(e1) / 3                  # the last (largest) run's
+            runs_hashed.append((tk, tv, m_, None, 0, hx, nb))
 
         def timed(rr):
             for _ in range(max(3, warmup)):
@@ -649,7 +668,8 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
             return e0.elapsed_time(e1) / reps, ctx.last_status(), reps
 
         ms_plain, _, _ = timed(runs)
-        ms, st, reps = timed(runs_bloom)
+        ms_bloom, _, _ = timed(runs_bloom)
+        ms, st, reps = timed(runs_hashed)
         exact = exact_index_numbers(torch, ctx, w, up, d_tok, d_off, d_qoff, total, d_hit, d_recs,
                                     max(3, warmup), max(5, steps))
         hit_tokens = int(w.expected_hit.sum()) * 16
@@ -659,8 +679,11 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
         return {"workload": "configs[2]: 1M stored chunk keys in 4 sorted runs, 4096 queries of "
                             "2k-32k tokens, 60% cached",
                 "ms_per_probe": ms, "query_chunks": total, "keys_per_s": total / ms * 1e3,
-                "ms_per_probe_without_bloom_filters": ms_plain,
-                "keys_per_s_without_bloom_filters": total / ms_plain * 1e3,
+                "lookup": "hash index per run (built when the run is written)",
+                "hash_index_build_ms_for_%d_keys" % big: hidx_ms,
+                "ms_per_probe_searching_sorted_runs": ms_plain,
+                "keys_per_s_searching_sorted_runs": total / ms_plain * 1e3,
+                "ms_per_probe_searching_with_bloom_filters": ms_bloom,
                 "lookups_per_s": st["lookups"] / reps / ms * 1e3,
                 "hit_chunks_per_s": st["chunks_hit"] / reps / ms * 1e3,
                 "query_tokens": int(len(w.query.tokens)), "stored_keys": n,

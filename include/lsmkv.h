@@ -87,13 +87,19 @@ typedef struct {
 
 /* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i].
  * bloom (optional, NULL = none): the run's Bloom filter as built by lsmkv_bloom_build, with
- * bloom_blocks 32-byte blocks; the probe then skips the run for keys the filter rules out. */
+ * bloom_blocks 32-byte blocks; the probe then skips the run for keys the filter rules out.
+ * hindex (optional, NULL = none): the run's hash index as built by lsmkv_hindex_build, with
+ * hindex_buckets 32-byte buckets. When every non-empty run of a probe brings one, point lookups
+ * go through the hash indexes instead of searching the sorted keys (and ignore the Bloom
+ * filters, which the tables make redundant); otherwise the probe ignores the hash indexes. */
 typedef struct {
     const lsmkv_key_t *keys; /* [dev] */
     const lsmkv_val_t *vals; /* [dev] */
     uint64_t n;
     const void *bloom;       /* [dev] or NULL */
     uint64_t bloom_blocks;
+    const void *hindex;      /* [dev] or NULL */
+    uint64_t hindex_buckets;
 } lsmkv_run_t;
 
 /* The paged KV pool. */
@@ -306,6 +312,26 @@ uint64_t lsmkv_encode_bound(const lsmkv_ctx *ctx, uint64_t n_chunks); /* worst-c
 uint64_t lsmkv_bloom_blocks(uint64_t n);
 int lsmkv_bloom_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uint64_t n,
                       void *bloom_out);
+
+/*
+ * Hash index of a run (Sec. 2.2 "Point Lookups": a run carries auxiliary structures -- fence
+ * pointers, filters -- built once when the run is written, so that a point lookup touches as
+ * little of the run as possible; this one plays both parts for runs that live in device memory).
+ * Result-neutral: probes return the same answers with or without it.
+ * Format: lsmkv_hindex_buckets(n) = max(1, ceil(n / 2)) buckets of eight u32 slots. A slot is 0
+ * (empty) or (w2 & 0xFF) << 24 | (i + 1) for the key at position i of the run. A key's home
+ * bucket is floor(w1 * n_buckets / 2^61); it occupies the first slot that was free at its
+ * insertion, scanning from slot 0 of the home bucket through the following buckets (wrapping
+ * around). Lookups scan in the same order and stop at the first empty slot. Which of several
+ * keys of one bucket got which slot depends on the order of insertion and is not specified.
+ * Entries whose w1 is not a digest (the all-ones padding of a flushed run) are left out.
+ * n <= 2^24 - 2 (LSMKV_EINVAL beyond; such a run is probed without a hash index).
+ * lsmkv_hindex_build: keys [dev, n entries] -> hindex_out [dev, 32 * lsmkv_hindex_buckets(n)
+ * bytes, 16-byte aligned], cleared and filled on `stream`.
+ */
+uint64_t lsmkv_hindex_buckets(uint64_t n);
+int lsmkv_hindex_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uint64_t n,
+                       void *hindex_out);
 
 /*
  * Host-buffer variants (the form the paper's service interface has: token sequences and

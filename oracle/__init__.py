@@ -115,6 +115,13 @@ def lib() -> C.CDLL:
         _lib.orc_bloom_build.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         _lib.orc_bloom_may_contain.restype = C.c_int
         _lib.orc_bloom_may_contain.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_hindex_buckets.restype = C.c_uint64
+        _lib.orc_hindex_buckets.argtypes = [C.c_uint64]
+        _lib.orc_hindex_build.restype = C.c_int
+        _lib.orc_hindex_build.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        _lib.orc_hindex_find.restype = C.c_uint64
+        _lib.orc_hindex_find.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64,
+                                         C.c_void_p]
         _lib.orc_xp12_slab_bound.restype = C.c_uint64
         _lib.orc_xp12_slab_bound.argtypes = [C.c_uint64]
         _lib.orc_xp12_dir_bytes.restype = C.c_uint64
@@ -289,6 +296,30 @@ def bloom_build(keys) -> np.ndarray:
 def bloom_may_contain(bloom: np.ndarray, key) -> bool:
     key = _arr(key, np.uint64)
     return bool(lib().orc_bloom_may_contain(_p(bloom), bloom.size // 32, _p(key)))
+
+
+def hindex_buckets(n: int) -> int:
+    return int(lib().orc_hindex_buckets(n))
+
+
+def hindex_build(keys) -> np.ndarray:
+    """Hash index (u32 slots, 8 per bucket) of a run's keys, inserted by ascending position."""
+    keys = _arr(keys, np.uint64).reshape(-1, 4)
+    out = np.zeros(8 * hindex_buckets(len(keys)), dtype=np.uint32)
+    rc = lib().orc_hindex_build(_p(keys), len(keys), _p(out))
+    if rc != OK:
+        raise OracleError(rc)
+    return out
+
+
+def hindex_find(table: np.ndarray, keys, key) -> int:
+    """Position of `key` in the run `keys` by the table's lookup rule, or -1. Works on any valid
+    table of the run, whatever the order its keys were inserted in."""
+    keys = _arr(keys, np.uint64).reshape(-1, 4)
+    key = _arr(key, np.uint64)
+    table = _arr(table, np.uint32)
+    at = int(lib().orc_hindex_find(_p(table), table.size // 8, _p(keys), len(keys), _p(key)))
+    return -1 if at == 2**64 - 1 else at
 
 
 def probe_batch(g: Geom, tokens, seq_off, qchunk_off, runs, want_keys: bool = False):

@@ -309,6 +309,66 @@ int orc_bloom_may_contain(const uint8_t *bloom, uint64_t n_blocks, const orc_key
     return 1;
 }
 
+/* ---- hash index of a run -------------------------------------------------------------- */
+
+/*
+ * Sec. 2.2 "Point Lookups": a run carries auxiliary structures, built when the run is written,
+ * that let a point lookup touch as little of the run as possible. For runs held in memory a
+ * hash table over the run's keys does that: it answers "where in the run is this key, if
+ * anywhere" without a search. Results of lookups never depend on it.
+ *
+ * Format (this build's): n_buckets = max(1, ceil(n / 2)) buckets of eight u32 slots.
+ *   slot = 0 (empty) or (w2 & 0xFF) << 24 | (i + 1) for the key at position i of the run;
+ *   home bucket of a key = floor(w1 * n_buckets / 2^61);
+ *   a key takes the first empty slot found scanning slot 0..7 of its home bucket, then of the
+ *   following buckets, wrapping around; a lookup scans the same way, compares the full key
+ *   wherever the 8-bit tag matches, and stops at the first empty slot.
+ * Keys whose w1 is not a digest (>= 2^61: the padding of a flushed run) are left out.
+ * Inserting in a different order gives a different, equally valid table; this builder inserts
+ * by ascending position. n <= 2^24 - 2.
+ */
+uint64_t orc_hindex_buckets(uint64_t n)
+{
+    const uint64_t b = n / 2 + (n & 1);
+    return b ? b : 1;
+}
+
+static uint64_t hindex_home(const orc_key *k, uint64_t n_buckets)
+{
+    return (uint64_t)(((unsigned __int128)k->w[1] * n_buckets) >> 61);
+}
+
+int orc_hindex_build(const orc_key *keys, uint64_t n, uint32_t *table /* 8 * orc_hindex_buckets(n) */)
+{
+    if (n > (1ull << 24) - 2) return ORC_EINVAL;
+    const uint64_t nb = orc_hindex_buckets(n), slots = 8 * nb;
+    memset(table, 0, slots * sizeof(uint32_t));
+    for (uint64_t i = 0; i < n; ++i) {
+        if (keys[i].w[1] >> 61) continue;
+        uint64_t s = 8 * hindex_home(&keys[i], nb);
+        while (table[s]) s = s + 1 == slots ? 0 : s + 1;      /* at most n of >= 4n slots are taken */
+        table[s] = (uint32_t)((keys[i].w[2] & 0xFFu) << 24) | (uint32_t)(i + 1);
+    }
+    return ORC_OK;
+}
+
+/* position of `key` in the run according to the table, or UINT64_MAX */
+uint64_t orc_hindex_find(const uint32_t *table, uint64_t n_buckets, const orc_key *keys,
+                         uint64_t n, const orc_key *key)
+{
+    const uint64_t slots = 8 * n_buckets;
+    const uint32_t tag = (uint32_t)(key->w[2] & 0xFFu);
+    uint64_t s = 8 * hindex_home(key, n_buckets);
+    for (uint64_t seen = 0; seen < slots; ++seen) {
+        const uint32_t w = table[s];
+        if (w == 0) return UINT64_MAX;
+        const uint64_t at = (uint64_t)(w & 0xFFFFFFu) - 1;
+        if ((w >> 24) == tag && at < n && memcmp(&keys[at], key, sizeof(orc_key)) == 0) return at;
+        s = s + 1 == slots ? 0 : s + 1;
+    }
+    return UINT64_MAX;
+}
+
 /* ---- probe: longest cached prefix, first-miss rule ---------------------------------- */
 
 /*

@@ -559,6 +559,7 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     if (n_runs > LSMKV_MAX_RUNS || (n_runs && !runs)) return LSMKV_EINVAL;
     RunTable rt;
     std::memset(&rt, 0, sizeof(rt));
+    bool hashed = true;   // every non-empty run brings its hash index: no directory, no searches
     for (uint32_t r = 0; r < n_runs; ++r) {
         if (runs[r].n && (!runs[r].keys || !runs[r].vals || !aligned16(runs[r].keys) ||
                           !aligned16(runs[r].vals)))
@@ -570,12 +571,20 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
         rt.n[r] = runs[r].n;
         rt.bloom[r] = runs[r].n ? static_cast<const uint32_t *>(runs[r].bloom) : nullptr;
         rt.bloom_blocks[r] = runs[r].bloom_blocks;
+        if (runs[r].hindex && (runs[r].hindex_buckets == 0 || !aligned16(runs[r].hindex) ||
+                               runs[r].n > kHidxMaxKeys))
+            return LSMKV_EINVAL;
+        rt.hidx[r] = static_cast<const uint32_t *>(runs[r].hindex);
+        rt.hidx_buckets[r] = runs[r].hindex_buckets;
+        if (runs[r].n && !runs[r].hindex) hashed = false;
     }
+    if (n_runs == 0) hashed = false;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint32_t jcap = (uint32_t)(n_qchunks < kDirMaxJ ? n_qchunks : kDirMaxJ);
     // d_dir: [0] = the probe's work counter, [2..] = the directory, then the hand-out order
-    const uint64_t dir_entries = (uint64_t)n_runs * ((uint64_t)jcap + 1);
+    const uint32_t dir_runs = hashed ? 0 : n_runs;
+    const uint64_t dir_entries = (uint64_t)dir_runs * ((uint64_t)jcap + 1);
     const bool ordered = n_query > 1 && n_query <= kOrderMaxQueries;
     {
         int rc = ensure_dir(ctx, 2 + dir_entries + (ordered ? (n_query + 1) / 2 : 0));
@@ -587,12 +596,11 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     {
         LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
         {
-            const uint64_t entries = (uint64_t)n_runs * ((uint64_t)jcap + 1);
-            uint64_t dgrid = (entries + 255) / 256;
+            uint64_t dgrid = (dir_entries + 255) / 256;
             const uint64_t dcap = (uint64_t)ctx->sm_count * 8;
             if (dgrid > dcap) dgrid = dcap;
             if (dgrid == 0) dgrid = 1;
-            k_run_dir<<<(unsigned)dgrid, 256, 0, s>>>(rt, n_runs, ctx->geom.ns, jcap, dir,
+            k_run_dir<<<(unsigned)dgrid, 256, 0, s>>>(rt, dir_runs, ctx->geom.ns, jcap, dir,
                                                       next_query, n_query, seq_off,
                                                       ctx->geom.chunk_tokens, order);
             ++ctx->launches;
@@ -602,11 +610,12 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
         uint64_t grid = n_query;
         const uint64_t cap = (uint64_t)ctx->sm_count * (2048u / threads);
         if (grid > cap) grid = cap;
-        k_probe<<<(unsigned)grid, threads, 0, s>>>(ctx->kc, rt, n_runs, dir, jcap,
-                                                   ctx->geom.chunk_tokens, ctx->geom.ns, n_query,
-                                                   tokens, seq_off, qchunk_off, n_qchunks,
-                                                   hit_chunks_out, recs_out, keys_out,
-                                                   ctx->d_status, next_query, order);
+        auto kern = hashed ? k_probe<true> : k_probe<false>;
+        kern<<<(unsigned)grid, threads, 0, s>>>(ctx->kc, rt, n_runs, dir, jcap,
+                                                ctx->geom.chunk_tokens, ctx->geom.ns, n_query,
+                                                tokens, seq_off, qchunk_off, n_qchunks,
+                                                hit_chunks_out, recs_out, keys_out,
+                                                ctx->d_status, next_query, order);
         ++ctx->launches;
     }
     CU(ctx, cudaGetLastError());
@@ -912,6 +921,31 @@ int lsmkv_bloom_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uin
     CU(ctx, cudaMemsetAsync(bloom_out, 0, nb * 32, s));
     if (n) {
         k_bloom_build<<<merge_grid(ctx, n), 256, 0, s>>>(keys, n, static_cast<uint32_t *>(bloom_out), nb);
+        ++ctx->launches;
+        CU(ctx, cudaGetLastError());
+    }
+    return LSMKV_OK;
+}
+
+uint64_t lsmkv_hindex_buckets(uint64_t n)
+{
+    const uint64_t b = n / 2 + (n & 1);
+    return b ? b : 1;
+}
+
+int lsmkv_hindex_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, uint64_t n,
+                       void *hindex_out)
+{
+    if (!ctx || !hindex_out || !aligned16(hindex_out) || (n && (!keys || !aligned16(keys))))
+        return LSMKV_EINVAL;
+    if (n > kHidxMaxKeys) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t nb = lsmkv_hindex_buckets(n);
+    LaunchTimer timer(ctx, s, LSMKV_K_FLUSH);   // part of writing a run
+    CU(ctx, cudaMemsetAsync(hindex_out, 0, nb * 32, s));
+    if (n) {
+        k_hidx_build<<<merge_grid(ctx, n), 256, 0, s>>>(keys, n, static_cast<uint32_t *>(hindex_out), nb);
         ++ctx->launches;
         CU(ctx, cudaGetLastError());
     }

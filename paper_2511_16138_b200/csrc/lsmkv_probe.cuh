@@ -24,6 +24,8 @@ struct RunTable {
     uint64_t n[LSMKV_MAX_RUNS];
     const uint32_t *bloom[LSMKV_MAX_RUNS];     // optional Bloom filter, 8 words per block
     uint64_t bloom_blocks[LSMKV_MAX_RUNS];
+    const uint32_t *hidx[LSMKV_MAX_RUNS];      // optional hash index, 8 slots per bucket
+    uint64_t hidx_buckets[LSMKV_MAX_RUNS];
 };
 
 constexpr uint64_t kDigestLimit = 1ull << 61;  // digests are < 2^61 - 1; padding keys are not
@@ -281,6 +283,152 @@ __device__ __forceinline__ bool lookup_runs(const RunTable &rt, uint32_t n_runs,
     return false;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Hash index of a run: a table of 32-byte buckets of eight 4-byte slots that maps a key to its
+// position in the sorted run. A slot is 0 (empty) or (w2 & 0xFF) << 24 | (position + 1). A key's
+// home bucket is floor(w1 * n_buckets / 2^61); it sits in the first slot that was free when it
+// was inserted, scanning the home bucket's slots 0..7 and then the following buckets (wrapping).
+// Slots never empty again, so a lookup that scans in the same order may stop at the first empty
+// slot: the key is not in the run. With n_buckets = ceil(n / 2) a bucket holds two keys on
+// average and all eight slots of a bucket are taken for about one key in a thousand, so nearly
+// every lookup is one 32-byte load, plus the key and record of the one slot whose tag matches.
+// The sorted run stays what it is (merges and range scans use it); the table only replaces the
+// binary search of a point lookup.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kHidxSlots = 8;
+constexpr uint64_t kHidxMaxKeys = (1ull << 24) - 2;        // position + 1 must fit 24 bits
+
+__device__ __forceinline__ uint64_t hidx_home(uint64_t w1, uint64_t n_buckets)
+{
+    return __umul64hi(w1 << 3, n_buckets);
+}
+
+__global__ void __launch_bounds__(256)
+k_hidx_build(const lsmkv_key_t *__restrict__ keys, uint64_t n, uint32_t *__restrict__ hidx,
+             uint64_t n_buckets)
+{
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+         i += (uint64_t)gridDim.x * blockDim.x) {
+        const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(
+            reinterpret_cast<const unsigned long long *>(keys + i) + 1);   // w1, w2
+        if (a.x >= kDigestLimit) continue;                                  // padding entry
+        const uint32_t entry = (((uint32_t)a.y & 0xFFu) << 24) | (uint32_t)(i + 1);
+        uint64_t b = hidx_home(a.x, n_buckets);
+        bool placed = false;
+        for (uint64_t it = 0; it < n_buckets && !placed; ++it) {            // slots >= 4 n: ends
+            for (uint32_t t = 0; t < kHidxSlots && !placed; ++t)
+                placed = atomicCAS(hidx + kHidxSlots * b + t, 0u, entry) == 0u;
+            b = b + 1 == n_buckets ? 0 : b + 1;
+        }
+    }
+}
+
+__device__ __forceinline__ bool key_equals(const lsmkv_key_t *e, const ChunkKey &k)
+{
+    const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(e);
+    const ulonglong2 a = __ldg(p), b = __ldg(p + 1);
+    return a.x == k.w0 && a.y == k.w1 && b.x == k.w2 && b.y == k.w3;
+}
+
+// The lookup rule, slot by slot (any table, any fill). Returns the position or ~0.
+__device__ __noinline__ uint64_t hidx_find(const uint32_t *hidx, uint64_t n_buckets,
+                                           const lsmkv_key_t *keys, uint64_t n, const ChunkKey &k)
+{
+    const uint32_t tag = (uint32_t)k.w2 & 0xFFu;
+    uint64_t b = hidx_home(k.w1, n_buckets);
+    for (uint64_t it = 0; it < n_buckets; ++it) {
+        for (uint32_t t = 0; t < kHidxSlots; ++t) {
+            const uint32_t w = __ldg(hidx + kHidxSlots * b + t);
+            if (w == 0) return ~0ull;
+            const uint64_t at = (uint64_t)(w & 0xFFFFFFu) - 1;
+            if ((w >> 24) == tag && at < n && key_equals(keys + at, k)) return at;
+        }
+        b = b + 1 == n_buckets ? 0 : b + 1;
+    }
+    return ~0ull;
+}
+
+// Point lookup through the hash indexes, newest run first. The home buckets of kLookupGroup
+// runs are fetched together, then the keys and records of their candidates, so a group costs
+// two dependent loads; the rare cases the home bucket cannot settle go slot by slot.
+__device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_runs,
+                                                 const ChunkKey &k, uint4 &val)
+{
+    const uint32_t tag = (uint32_t)k.w2 & 0xFFu;
+    for (uint32_t r0 = 0; r0 < n_runs; r0 += kLookupGroup) {
+        uint4 lo[kLookupGroup], hi[kLookupGroup];
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t r = r0 + g;
+            lo[g] = make_uint4(0, 0, 0, 0);
+            hi[g] = lo[g];
+            if (r < n_runs && rt.n[r]) {
+                const uint4 *bkt = reinterpret_cast<const uint4 *>(
+                    rt.hidx[r] + kHidxSlots * hidx_home(k.w1, rt.hidx_buckets[r]));
+                lo[g] = __ldg(bkt);
+                hi[g] = __ldg(bkt + 1);
+            }
+        }
+        // first slot that is empty or carries the key's tag: cand = position + 1 of a tag match,
+        // 0 if an empty slot came first; open = neither in this bucket
+        uint32_t cand[kLookupGroup];
+        bool open[kLookupGroup];
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t w[8] = {lo[g].x, lo[g].y, lo[g].z, lo[g].w,
+                                   hi[g].x, hi[g].y, hi[g].z, hi[g].w};
+            cand[g] = 0;
+            open[g] = true;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const bool stop = open[g] && (w[t] == 0 || (w[t] >> 24) == tag);
+                if (stop) {
+                    cand[g] = w[t] & 0xFFFFFFu;
+                    open[g] = false;
+                }
+            }
+            if (r0 + g < n_runs && cand[g] > rt.n[r0 + g]) {   // not a position of this run
+                cand[g] = 0;
+                open[g] = true;
+            }
+        }
+        ulonglong2 ka[kLookupGroup], kb[kLookupGroup];
+        uint4 rec[kLookupGroup];
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            if (cand[g]) {
+                const uint32_t r = r0 + g;
+                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (cand[g] - 1));
+                ka[g] = __ldg(p);
+                kb[g] = __ldg(p + 1);
+                rec[g] = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (cand[g] - 1)));
+            }
+        }
+        // answers in age order
+#pragma unroll
+        for (int g = 0; g < kLookupGroup; ++g) {
+            const uint32_t r = r0 + g;
+            if (r >= n_runs || rt.n[r] == 0) continue;
+            if (cand[g]) {
+                if (ka[g].x == k.w0 && ka[g].y == k.w1 && kb[g].x == k.w2 && kb[g].y == k.w3) {
+                    val = rec[g];
+                    return true;
+                }
+                open[g] = true;                            // another key with the same tag
+            }
+            if (open[g]) {
+                const uint64_t at = hidx_find(rt.hidx[r], rt.hidx_buckets[r], rt.keys[r], rt.n[r], k);
+                if (at != ~0ull) {
+                    val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + at));
+                    return true;
+                }
+            }
+        }
+    }
+    return false;
+}
+
+template <bool HASHED>
 __global__ void __launch_bounds__(512)
 k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable rt,
         uint32_t n_runs, const uint64_t *__restrict__ dir, uint32_t jcap, uint32_t C,
@@ -336,7 +484,8 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                 continue;
             }
             uint4 val = zero;
-            const bool found = valid && lookup_runs(rt, n_runs, dir, jcap, k, val);
+            const bool found = valid && (HASHED ? lookup_runs_hash(rt, n_runs, k, val)
+                                                : lookup_runs(rt, n_runs, dir, jcap, k, val));
             n_lookups += valid ? 1ull : 0ull;
             const unsigned miss = __ballot_sync(0xFFFFFFFFu, valid && !found);
             if (miss && lane == 0)

@@ -26,6 +26,7 @@ EXPORTS = (
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
     "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
+    "lsmkv_hindex_buckets", "lsmkv_hindex_build",
     "lsmkv_relocate_records", "lsmkv_xrun_build", "lsmkv_xprobe_batch",
 )
 ST_OVERFLOW = 32
@@ -59,16 +60,20 @@ class GeomStruct(C.Structure):
 
 class RunStruct(C.Structure):
     _fields_ = [("keys", C.c_void_p), ("vals", C.c_void_p), ("n", C.c_uint64),
-                ("bloom", C.c_void_p), ("bloom_blocks", C.c_uint64)]
+                ("bloom", C.c_void_p), ("bloom_blocks", C.c_uint64),
+                ("hindex", C.c_void_p), ("hindex_buckets", C.c_uint64)]
 
 
 def _run_array(runs):
-    """runs: sequence of (keys, vals, n) or (keys, vals, n, bloom, bloom_blocks)."""
+    """runs: sequence of (keys, vals, n), (keys, vals, n, bloom, bloom_blocks) or
+    (keys, vals, n, bloom, bloom_blocks, hindex, hindex_buckets); bloom / hindex may be None."""
     arr = (RunStruct * max(1, len(runs)))()
     for i, r in enumerate(runs):
         arr[i].keys, arr[i].vals, arr[i].n = _ptr(r[0]), _ptr(r[1]), r[2]
         if len(r) > 3 and r[3] is not None:
             arr[i].bloom, arr[i].bloom_blocks = _ptr(r[3]), r[4]
+        if len(r) > 5 and r[5] is not None:
+            arr[i].hindex, arr[i].hindex_buckets = _ptr(r[5]), r[6]
     return arr
 
 
@@ -169,6 +174,10 @@ def lib() -> C.CDLL:
     L.lsmkv_bloom_blocks.argtypes = [u64]
     L.lsmkv_bloom_build.restype = C.c_int
     L.lsmkv_bloom_build.argtypes = [vp, vp, vp, u64, vp]
+    L.lsmkv_hindex_buckets.restype = u64
+    L.lsmkv_hindex_buckets.argtypes = [u64]
+    L.lsmkv_hindex_build.restype = C.c_int
+    L.lsmkv_hindex_build.argtypes = [vp, vp, vp, u64, vp]
     L.lsmkv_flush_batch.restype = C.c_int
     L.lsmkv_flush_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp, vp]
     L.lsmkv_merge_runs.restype = C.c_int
@@ -378,6 +387,15 @@ def lsmkv_bloom_blocks(n: int) -> int:
     return int(lib().lsmkv_bloom_blocks(n))
 
 
+def lsmkv_hindex_buckets(n: int) -> int:
+    return int(lib().lsmkv_hindex_buckets(n))
+
+
+def lsmkv_hindex_build(ctx, stream, keys, n, hindex_out) -> None:
+    _check(ctx, lib().lsmkv_hindex_build(ctx, _stream(stream), _ptr(keys), n, _ptr(hindex_out)),
+           "lsmkv_hindex_build")
+
+
 def lsmkv_bloom_build(ctx, stream, keys, n, bloom_out) -> None:
     _check(ctx, lib().lsmkv_bloom_build(ctx, _stream(stream), _ptr(keys), n, _ptr(bloom_out)),
            "lsmkv_bloom_build")
@@ -531,6 +549,9 @@ class Context:
 
     def bloom_build(self, keys, n, bloom_out, stream=None):
         lsmkv_bloom_build(self.handle, stream, keys, n, bloom_out)
+
+    def hindex_build(self, keys, n, hindex_out, stream=None):
+        lsmkv_hindex_build(self.handle, stream, keys, n, hindex_out)
 
     def flush_batch(self, keys, vals, n, run_keys_out, run_vals_out, n_out, stream=None):
         lsmkv_flush_batch(self.handle, stream, keys, vals, n, run_keys_out, run_vals_out, n_out)

@@ -38,7 +38,7 @@ def test_library_builds_and_exports_every_declared_symbol():
 
 def test_binding_struct_layouts_match_the_header():
     assert ctypes.sizeof(lsmkv.GeomStruct) == 32
-    assert ctypes.sizeof(lsmkv.RunStruct) == 40
+    assert ctypes.sizeof(lsmkv.RunStruct) == 56
     assert ctypes.sizeof(lsmkv.PoolStruct) == 16
     assert ctypes.sizeof(lsmkv.StatusStruct) == 56
     assert VAL_DTYPE.itemsize == lsmkv.VAL_BYTES == 16 and lsmkv.KEY_BYTES == 32
