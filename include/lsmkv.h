@@ -456,7 +456,7 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "copy_stage_bytes"  bytes per bulk copy, multiple of 16, 16..131072 (clamped to page_bytes)
  *   "copy_stages"       bulk copies in flight per CTA, 1..32 (reduced to fit shared memory)
  *   "copy_ctas_per_sm"  1..8        "copy_l2_hint"  0/1 = evict-first L2 policy on the copies
- *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..16
+ *   "simt_ctas_per_sm"  1..32       "probe_warps_per_cta"  1..8
  *   "host_stage_bytes"  blob bytes staged per slice by the host-buffer calls, 1 MiB..64 GiB
  *   "xp_generic"        1 = compressing codec always uses its generic kernels (0 = fast kernels
  *                       for slabs of 8192 / 16384 / 32768 elements)

@@ -1011,7 +1011,7 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"copy_stages", &ctx->copy_stages, 1, 32},
         {"copy_ctas_per_sm", &ctx->copy_ctas_per_sm, 1, 8},
         {"copy_l2_hint", &ctx->copy_l2_hint, 0, 1},
-        {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 16},
+        {"probe_warps_per_cta", &ctx->probe_warps_per_cta, 1, 8},
         {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
         {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
         {"xp_generic", &ctx->xp_generic, 0, 1},

@@ -50,6 +50,24 @@ __device__ __forceinline__ uint64_t addmod61(uint64_t a, uint64_t b)  // a, b < 
     return s >= kP ? s - kP : s;
 }
 
+// The scans below keep their intermediate values only partly reduced -- any representative below
+// 2^62 -- and take the canonical one (fold61) once at the end; the value mod p is the same.
+// a, b < 2^62  ->  a*b mod p, below 2^61 + 8
+__device__ __forceinline__ uint64_t mulmod61_lazy(uint64_t a, uint64_t b)
+{
+    const uint64_t lo = a * b;
+    const uint64_t hi = __umul64hi(a, b);               // product < 2^124, hi < 2^60
+    const uint64_t s = (lo & kP) + ((lo >> 61) | (hi << 3));   // < 2^61 + 2^63
+    return (s & kP) + (s >> 61);
+}
+
+// a*m + b mod p for a, m, b < 2^62, below 2^61 + 8
+__device__ __forceinline__ uint64_t muladd61_lazy(uint64_t a, uint64_t m, uint64_t b)
+{
+    const uint64_t s = mulmod61_lazy(a, m) + b;         // < 2^63
+    return (s & kP) + (s >> 61);
+}
+
 __device__ __forceinline__ uint64_t horner61(uint64_t h, uint64_t base, uint32_t token)
 {
     return fold61(mulmod61(h, base) + (uint64_t)token + 1ull);   // < p + 2^32 < 2^62
@@ -140,7 +158,8 @@ __device__ __forceinline__ void chunk_hash(const KeyConsts &kc, const uint32_t *
 
 // One warp, 32 consecutive chunks j = base_j + lane of the sequence starting at `seq`: every
 // lane gets the digests of tokens [base_j*C, (j+1)*C), i.e. relative to the start of this
-// 32-chunk block (no carry yet). Lanes with j >= nch hold garbage. All 32 lanes must call.
+// 32-chunk block (no carry yet), partly reduced. Lanes with j >= nch hold garbage. All 32 lanes
+// must call.
 __device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint32_t *seq,
                                                 uint32_t C, uint64_t base_j, uint64_t nch,
                                                 uint64_t &hA, uint64_t &hB, uint32_t &first,
@@ -158,41 +177,59 @@ __device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint3
     for (unsigned d = 1; d < 32; d <<= 1) {
         const uint64_t uA = shfl_up64(hA, d), uB = shfl_up64(hB, d);
         if (lane >= d) {
-            hA = addmod61(mulmod61(uA, kc.pwA[d - 1]), hA);
-            hB = addmod61(mulmod61(uB, kc.pwB[d - 1]), hB);
+            hA = muladd61_lazy(uA, kc.pwA[d - 1], hA);
+            hB = muladd61_lazy(uB, kc.pwB[d - 1], hB);
         }
     }
 }
 
 constexpr int kKeyMaxWarps = 16;
 
-// One CTA of W warps, 32*W consecutive chunks starting at `base`: warp w hashes the 32-chunk
-// block base + 32*w, the block digests are exchanged through shared memory and chained, so every
-// thread ends up with the key of chunk base + 32*warp + lane. cA/cB carry the digest of the
-// prefix before `base` from round to round (same value in every thread). Contains one
-// __syncthreads(); the caller must put another one between two calls (s_agg* are rewritten).
+// Shared-memory exchange of a CTA that hashes one sequence round by round.
+struct KeyShared {
+    uint64_t aggA[kKeyMaxWarps], aggB[kKeyMaxWarps];   // digest of each warp's 32-chunk block
+    uint64_t carryA[2], carryB[2];                     // prefix before the round, by round parity
+};
+
+// Before the first round of a sequence (followed by a __syncthreads() before round 0).
+__device__ __forceinline__ void key_rounds_begin(KeyShared &sh)
+{
+    if (threadIdx.x == 0) { sh.carryA[0] = 0; sh.carryB[0] = 0; }
+}
+
+// One round of a CTA: its first `wact` warps hash 32*wact consecutive chunks starting at `base`
+// (warp w the 32-chunk block base + 32*w). The block digests are exchanged through shared
+// memory; warp w chains the w blocks before its own onto the prefix the previous round left, so
+// every thread of an active warp ends up with the key of chunk base + 32*warp + lane. The last
+// active warp leaves the prefix behind the round for round `rnd + 1`. Warps >= wact get an
+// unspecified key. Contains one __syncthreads(); the caller must put another one between two
+// calls (the exchange is rewritten).
 __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
                                                    uint32_t C, uint32_t ns, uint64_t base,
-                                                   uint64_t nch, uint64_t &cA, uint64_t &cB,
-                                                   uint64_t *s_aggA, uint64_t *s_aggB)
+                                                   uint64_t nch, unsigned rnd, unsigned wact,
+                                                   KeyShared &sh)
 {
-    const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
-    uint64_t hA, hB;
-    uint32_t first, last;
-    warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
-    if (lane == 31) { s_aggA[warp] = hA; s_aggB[warp] = hB; }
-    __syncthreads();
-    uint64_t pA = cA, pB = cB;                 // prefix before block v, advanced block by block
-    for (unsigned v = 0; v < W; ++v) {
-        if (v == warp) {
-            hA = addmod61(mulmod61(pA, kc.pwA[lane]), hA);
-            hB = addmod61(mulmod61(pB, kc.pwB[lane]), hB);
-        }
-        pA = addmod61(mulmod61(pA, kc.pwA[31]), s_aggA[v]);
-        pB = addmod61(mulmod61(pB, kc.pwB[31]), s_aggB[v]);
+    const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
+    uint64_t hA = 0, hB = 0;
+    uint32_t first = 0, last = 0;
+    if (warp < wact) {
+        warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
+        if (lane == 31) { sh.aggA[warp] = hA; sh.aggB[warp] = hB; }
     }
-    cA = pA;                                   // meaningful when the round was full
-    cB = pB;
+    __syncthreads();
+    if (warp < wact) {
+        uint64_t pA = sh.carryA[rnd & 1u], pB = sh.carryB[rnd & 1u];   // prefix before block 0
+        for (unsigned v = 0; v < warp; ++v) {                          // ... before block `warp`
+            pA = muladd61_lazy(pA, kc.pwA[31], sh.aggA[v]);
+            pB = muladd61_lazy(pB, kc.pwB[31], sh.aggB[v]);
+        }
+        hA = fold61(muladd61_lazy(pA, kc.pwA[lane], hA));
+        hB = fold61(muladd61_lazy(pB, kc.pwB[lane], hB));
+        if (warp == wact - 1 && lane == 31) {          // meaningful when the round was full
+            sh.carryA[(rnd + 1u) & 1u] = hA;
+            sh.carryB[(rnd + 1u) & 1u] = hB;
+        }
+    }
     ChunkKey k;
     k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)(base + 32ull * warp + lane);
     k.w1 = hA;
@@ -218,8 +255,9 @@ k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uin
               lsmkv_key_t *__restrict__ keys_out, lsmkv_val_t *__restrict__ vals_out,
               DevStatus *st)
 {
-    __shared__ uint64_t s_aggA[kKeyMaxWarps], s_aggB[kKeyMaxWarps];
-    const uint64_t round_chunks = 32ull * (blockDim.x >> 5);
+    __shared__ KeyShared sh;
+    const unsigned W = blockDim.x >> 5;
+    const uint64_t round_chunks = 32ull * W;
     for (uint64_t r = blockIdx.x; r < n_req; r += gridDim.x) {
         const uint64_t s0 = seq_off[r], s1 = seq_off[r + 1];
         const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
@@ -231,10 +269,11 @@ k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uin
             continue;                                        // uniform over the CTA
         }
         if (cnt == 0) continue;
-        uint64_t cA = 0, cB = 0;
-        for (uint64_t base = 0; base < nch; base += round_chunks) {
-            const ChunkKey k = cta_chunk_keys(kc, tokens + s0, C, ns, base, nch, cA, cB, s_aggA,
-                                              s_aggB);
+        key_rounds_begin(sh);
+        __syncthreads();
+        unsigned rnd = 0;
+        for (uint64_t base = 0; base < nch; base += round_chunks, ++rnd) {
+            const ChunkKey k = cta_chunk_keys(kc, tokens + s0, C, ns, base, nch, rnd, W, sh);
             const uint64_t j = base + threadIdx.x;           // = base + 32 * warp + lane
             if (j >= start && j < nch) {
                 const uint64_t i = o0 + (j - start);

@@ -349,8 +349,9 @@ __device__ __noinline__ uint64_t hidx_find(const uint32_t *hidx, uint64_t n_buck
 }
 
 // Point lookup through the hash indexes, newest run first. The home buckets of kLookupGroup
-// runs are fetched together, then the keys and records of their candidates, so a group costs
-// two dependent loads; the rare cases the home bucket cannot settle go slot by slot.
+// runs are fetched together, then the key and record of each candidate in age order, so a group
+// costs two dependent loads as a rule; the rare cases the home bucket cannot settle go slot by
+// slot.
 __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_runs,
                                                  const ChunkKey &k, uint4 &val)
 {
@@ -392,26 +393,18 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
                 open[g] = true;
             }
         }
-        ulonglong2 ka[kLookupGroup], kb[kLookupGroup];
-        uint4 rec[kLookupGroup];
-#pragma unroll
-        for (int g = 0; g < kLookupGroup; ++g) {
-            if (cand[g]) {
-                const uint32_t r = r0 + g;
-                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (cand[g] - 1));
-                ka[g] = __ldg(p);
-                kb[g] = __ldg(p + 1);
-                rec[g] = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (cand[g] - 1)));
-            }
-        }
-        // answers in age order
+        // answers in age order; a candidate's key and record are fetched together (as a rule
+        // one run of the group has a candidate, so this is one more dependent load)
 #pragma unroll
         for (int g = 0; g < kLookupGroup; ++g) {
             const uint32_t r = r0 + g;
             if (r >= n_runs || rt.n[r] == 0) continue;
             if (cand[g]) {
-                if (ka[g].x == k.w0 && ka[g].y == k.w1 && kb[g].x == k.w2 && kb[g].y == k.w3) {
-                    val = rec[g];
+                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (cand[g] - 1));
+                const ulonglong2 ka = __ldg(p), kb = __ldg(p + 1);
+                const uint4 rec = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (cand[g] - 1)));
+                if (ka.x == k.w0 && ka.y == k.w1 && kb.x == k.w2 && kb.y == k.w3) {
+                    val = rec;
                     return true;
                 }
                 open[g] = true;                            // another key with the same tag
@@ -429,7 +422,7 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
 }
 
 template <bool HASHED>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(256, 3)
 k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable rt,
         uint32_t n_runs, const uint64_t *__restrict__ dir, uint32_t jcap, uint32_t C,
         uint32_t ns, uint32_t n_query, const uint32_t *__restrict__ tokens,
@@ -438,10 +431,9 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         lsmkv_key_t *__restrict__ keys_out, DevStatus *st, unsigned long long *next_query,
         const uint32_t *__restrict__ order)
 {
-    __shared__ uint64_t s_aggA[kKeyMaxWarps], s_aggB[kKeyMaxWarps];
+    __shared__ KeyShared sh;
     __shared__ unsigned long long s_first_miss, s_q;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
-    const uint64_t round_chunks = 32ull * W;
     const uint4 zero = make_uint4(0, 0, 0, 0);
     unsigned long long n_lookups = 0;
 
@@ -449,6 +441,7 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         // queries are handed out one at a time: long and short ones balance across the CTAs
         __syncthreads();
         if (threadIdx.x == 0) s_q = atomicAdd(next_query, 1ull);
+        key_rounds_begin(sh);
         __syncthreads();
         if (s_q >= n_query) break;
         const uint64_t q = order ? order[s_q] : s_q;
@@ -461,26 +454,30 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         }
         const uint32_t *seq = tokens + s0;
         uint4 *recs = reinterpret_cast<uint4 *>(recs_out + o0);
-        uint64_t hit = nch, cA = 0, cB = 0;                  // cA/cB: prefix before this round
+        uint64_t hit = nch, base = 0;
         bool done = false;
-        for (uint64_t base = 0; base < nch; base += round_chunks) {
+        // Round 0 is one warp's 32 chunks -- four queries in ten never get past it -- the
+        // later rounds take 32 chunks per warp of the CTA.
+        for (unsigned rnd = 0; base < nch; ++rnd) {
+            const unsigned wact = (rnd == 0 && !keys_out) ? 1u : W;
+            const uint64_t span = 32ull * wact;
             const uint64_t j = base + 32ull * warp + lane;
-            const bool valid = j < nch;
-            if (done && !keys_out) {                         // past the first miss: zero-fill
-                if (valid) recs[j] = zero;
-                continue;
-            }
+            const bool valid = warp < wact && j < nch;
             if (threadIdx.x == 0) s_first_miss = ~0ull;
-            if (j + round_chunks < nch) {                    // next round's tokens on their way
-                const char *nx = reinterpret_cast<const char *>(seq + (j + round_chunks) * C);
-                for (uint32_t b = 0; b < 4u * C; b += 128u)
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(nx + b));
+            if (!done) {                                     // next round's tokens on their way
+                const uint64_t jn = base + span + 32ull * warp + lane;
+                if (jn < nch) {
+                    const char *nx = reinterpret_cast<const char *>(seq + jn * C);
+                    for (uint32_t b = 0; b < 4u * C; b += 128u)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(nx + b));
+                }
             }
-            const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, cA, cB, s_aggA, s_aggB);
+            const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, rnd, wact, sh);
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
-            if (done) {
+            if (done) {                                      // only the keys were wanted
                 if (valid) recs[j] = zero;
-                __syncthreads();                             // s_agg* are rewritten next round
+                __syncthreads();                             // the exchange is rewritten next round
+                base += span;
                 continue;
             }
             uint4 val = zero;
@@ -493,8 +490,16 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
             __syncthreads();
             const uint64_t fm = s_first_miss;
             if (valid) recs[j] = j < fm ? val : zero;
-            if (fm != ~0ull) { hit = fm; done = true; }
             __syncthreads();                                 // before s_first_miss is reset
+            base += span;
+            if (fm != ~0ull) {
+                hit = fm;
+                done = true;
+                if (!keys_out) {                             // nothing left but zeros
+                    for (uint64_t z = base + threadIdx.x; z < nch; z += blockDim.x) recs[z] = zero;
+                    break;
+                }
+            }
         }
         if (threadIdx.x == 0) {
             hit_out[q] = (uint32_t)hit;

@@ -159,7 +159,7 @@ def test_extreme_token_ids_and_namespace():
 
 
 @pytest.mark.parametrize("tuning", [{"probe_warps_per_cta": 1}, {"probe_warps_per_cta": 2},
-                                    {"probe_warps_per_cta": 16}, {"copy_ctas_per_sm": 4, "copy_stages": 3},
+                                    {"probe_warps_per_cta": 8}, {"copy_ctas_per_sm": 4, "copy_stages": 3},
                                     {"copy_mode": 1, "simt_ctas_per_sm": 1}])
 def test_launch_shapes_do_not_change_results(tuning):
     """Every tuning knob is a launch shape only: long sequences (many rounds per query whatever
