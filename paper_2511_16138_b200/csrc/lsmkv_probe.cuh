@@ -432,7 +432,9 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         const uint32_t *__restrict__ order)
 {
     __shared__ KeyShared sh;
-    __shared__ unsigned long long s_first_miss, s_q;
+    // first miss of a round, by round mod 3: round r takes its minimum in slot r % 3 while
+    // thread 0 resets slot (r + 1) % 3, whose last readers were two barriers ago
+    __shared__ unsigned long long s_first_miss[3], s_q;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5, W = blockDim.x >> 5;
     const uint4 zero = make_uint4(0, 0, 0, 0);
     unsigned long long n_lookups = 0;
@@ -440,7 +442,10 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
     for (;;) {
         // queries are handed out one at a time: long and short ones balance across the CTAs
         __syncthreads();
-        if (threadIdx.x == 0) s_q = atomicAdd(next_query, 1ull);
+        if (threadIdx.x == 0) {
+            s_q = atomicAdd(next_query, 1ull);
+            s_first_miss[0] = ~0ull;
+        }
         key_rounds_begin(sh);
         __syncthreads();
         if (s_q >= n_query) break;
@@ -463,7 +468,6 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
             const uint64_t span = 32ull * wact;
             const uint64_t j = base + 32ull * warp + lane;
             const bool valid = warp < wact && j < nch;
-            if (threadIdx.x == 0) s_first_miss = ~0ull;
             if (!done) {                                     // next round's tokens on their way
                 const uint64_t jn = base + span + 32ull * warp + lane;
                 if (jn < nch) {
@@ -473,6 +477,7 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                 }
             }
             const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, rnd, wact, sh);
+            if (threadIdx.x == 0) s_first_miss[(rnd + 1u) % 3u] = ~0ull;
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
             if (done) {                                      // only the keys were wanted
                 if (valid) recs[j] = zero;
@@ -486,11 +491,11 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
             n_lookups += valid ? 1ull : 0ull;
             const unsigned miss = __ballot_sync(0xFFFFFFFFu, valid && !found);
             if (miss && lane == 0)
-                atomicMin(&s_first_miss, base + 32ull * warp + (unsigned)__ffs(miss) - 1ull);
+                atomicMin(&s_first_miss[rnd % 3u],
+                          base + 32ull * warp + (unsigned)__ffs(miss) - 1ull);
             __syncthreads();
-            const uint64_t fm = s_first_miss;
+            const uint64_t fm = s_first_miss[rnd % 3u];
             if (valid) recs[j] = j < fm ? val : zero;
-            __syncthreads();                                 // before s_first_miss is reset
             base += span;
             if (fm != ~0ull) {
                 hit = fm;
