@@ -690,9 +690,41 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
                 "algorithmic_GBps": algo_bytes / ms / 1e6,
                 "flush_ms_for_%d_keys" % big: flush_big_ms,
                 "exact_index": exact,
-                "bound": "L2 latency / instruction issue (not HBM)"}
+                "roofline": probe_roofline(torch, device_index, ms),
+                "bound": "instruction issue and dependent L2 loads (not HBM)"}
     finally:
         ctx.close()
+
+
+# Warp instructions of one k_probe<true> launch on this workload: ncu smsp__inst_executed.sum of
+# the capture summarised under profiles/ (k_probe, probe-heavy workload). Set to None whenever the
+# kernel changes until the counter has been taken again.
+PROBE_WARP_INSTRUCTIONS = 69272798
+
+
+def probe_roofline(torch, device_index, ms):
+    """The probe is integer arithmetic plus dependent loads, so its ceiling is the rate at which
+    the SMs can issue instructions: SMs x 4 schedulers x 1 warp instruction per cycle x the
+    maximum SM clock."""
+    props = torch.cuda.get_device_properties(device_index)
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+        mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+    except Exception:
+        mhz = 1965.0
+    peak = props.multi_processor_count * 4 * mhz * 1e6 / 1e9          # G warp instructions / s
+    if PROBE_WARP_INSTRUCTIONS is None:
+        return {"bound": "alu", "kernel": "k_probe<true>", "achieved": None, "peak": peak,
+                "unit": "G warp instructions/s", "frac": None}
+    achieved = PROBE_WARP_INSTRUCTIONS / ms / 1e6
+    return {"bound": "alu", "kernel": "k_probe<true>", "achieved": achieved, "peak": peak,
+            "unit": "G warp instructions/s", "frac": achieved / peak,
+            "peak_source": "SMs x 4 warp schedulers x max SM clock (%d x 4 x %.0f MHz)"
+                           % (props.multi_processor_count, mhz),
+            "instructions_per_launch": PROBE_WARP_INSTRUCTIONS,
+            "instructions_source": "ncu smsp__inst_executed.sum of one launch on this workload"}
 
 
 def exact_index_numbers(torch, ctx, w, up, d_tok, d_off, d_qoff, total, d_hit, d_recs, warm, reps):
