@@ -76,19 +76,42 @@ def dev_runs(runs):
     return out, keep
 
 
+def with_hindex(ctx, druns):
+    """The same device runs with their hash indexes attached (the form the benchmark probes)."""
+    out, keep = [], []
+    for r in druns:
+        dk, dv, n = r[0], r[1], r[2]
+        nb = lsmkv.lsmkv_hindex_buckets(n)
+        t = torch.full((nb * 32,), 0xFF, dtype=torch.uint8, device=DEV)
+        ctx.hindex_build(dk, n, t)
+        keep.append(t)
+        out.append((dk, dv, n, None, 0, t, nb))
+    return out, keep
+
+
 def gpu_probe(ctx, batch, qoff, runs, want_keys=True):
+    """Probe twice -- searching the sorted runs, then through their hash indexes -- and insist
+    on identical outputs; returns those of the second."""
     nq, total = batch.n, int(qoff[-1])
     d_tok, d_off, d_qoff = dev(batch.tokens), dev(batch.seq_off), dev(qoff)
-    d_hit = torch.full((max(4, nq),), 0x7FFFFFFF, dtype=torch.int32, device=DEV)
-    d_recs = torch.full((max(1, total) * 16,), 0xAB, dtype=torch.uint8, device=DEV)
-    d_keys = torch.zeros(max(1, total) * 32, dtype=torch.uint8, device=DEV) if want_keys else None
     druns, keep = dev_runs(runs)
-    ctx.probe_batch(nq, d_tok, d_off, d_qoff, total, druns, d_hit, d_recs, d_keys)
-    torch.cuda.synchronize()
-    hit = d_hit.cpu().numpy().view(np.uint32)[:nq]
-    recs = host(d_recs, VAL_DTYPE, total * 16)
-    keys = host(d_keys, np.uint64, total * 32).reshape(-1, 4) if want_keys else None
-    return hit, recs, keys, (d_qoff, d_hit, d_recs)
+    hruns, hkeep = with_hindex(ctx, druns)
+    outs = []
+    for rr in (druns, hruns):
+        d_hit = torch.full((max(4, nq),), 0x7FFFFFFF, dtype=torch.int32, device=DEV)
+        d_recs = torch.full((max(1, total) * 16,), 0xAB, dtype=torch.uint8, device=DEV)
+        d_keys = (torch.zeros(max(1, total) * 32, dtype=torch.uint8, device=DEV)
+                  if want_keys else None)
+        ctx.probe_batch(nq, d_tok, d_off, d_qoff, total, rr, d_hit, d_recs, d_keys)
+        torch.cuda.synchronize()
+        hit = d_hit.cpu().numpy().view(np.uint32)[:nq]
+        recs = host(d_recs, VAL_DTYPE, total * 16)
+        keys = host(d_keys, np.uint64, total * 32).reshape(-1, 4) if want_keys else None
+        outs.append((hit, recs, keys, (d_qoff, d_hit, d_recs)))
+    a, b = outs
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert (a[2] is None and b[2] is None) or np.array_equal(a[2], b[2])
+    return b
 
 
 def assert_status_clean(ctx):
@@ -156,7 +179,7 @@ def roundtrip(g: lsmkv.Geom, store, query, start_chunk=None, n_runs=1, num_pages
         assert np.array_equal(dst.numpy(), o_dst), "restored pool differs"
         status = assert_status_clean(ctx)
         assert status["chunks_encoded"] == n
-        assert status["chunks_hit"] == int(o_hit.sum()) * 2       # two probes
+        assert status["chunks_hit"] == int(o_hit.sum()) * 4       # two calls, each probing both ways
         assert status["chunks_decoded"] == int(o_hit.sum())
     return dict(hit=o_hit, n=n, status=status)
 

@@ -75,10 +75,18 @@ def encode_probe_decode_wave(ctx, g, batch, nch, src, dst, arena, rng, n_sample=
     d_hit = torch.zeros(batch.n, dtype=torch.int32, device=H.DEV)
     d_recs = torch.empty(n * 16, dtype=torch.uint8, device=H.DEV)
     druns, keep = H.dev_runs([run])
+    hruns, hkeep = H.with_hindex(ctx, druns)            # the form the benchmark probes
     ctx.probe_batch(batch.n, d_tok, d_off, d_coff, n, druns, d_hit, d_recs, None)
+    torch.cuda.synchronize()
+    hit_searched = d_hit.cpu().numpy().view(np.uint32).copy()
+    recs_searched = down(d_recs, VAL_DTYPE, n * 16).copy()
+    d_hit.zero_()
+    d_recs.fill_(0xAB)
+    ctx.probe_batch(batch.n, d_tok, d_off, d_coff, n, hruns, d_hit, d_recs, None)
     torch.cuda.synchronize()
     hit = d_hit.cpu().numpy().view(np.uint32)
     recs = down(d_recs, VAL_DTYPE, n * 16)
+    assert np.array_equal(hit, hit_searched) and np.array_equal(recs, recs_searched)
     o_hit, o_recs, _, _ = oracle.probe_batch(og, batch.tokens, batch.seq_off, coff, [run])
     assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
     assert np.array_equal(hit, nch.astype(np.uint32))
@@ -203,8 +211,8 @@ def test_config3_probe_heavy_full():
         assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
         assert np.array_equal(hit, w.expected_hit.astype(np.uint32))
         st = ctx.last_status()
-        assert st["flags"] == 0 and st["chunks_hit"] == int(hit.sum())
-        assert st["empty_probes"] == int((hit == 0).sum())
+        assert st["flags"] == 0 and st["chunks_hit"] == 2 * int(hit.sum())   # probed both ways
+        assert st["empty_probes"] == 2 * int((hit == 0).sum())
 
         # decode the hits in waves of queries into a 64 GiB pool
         num_pages = 131072
