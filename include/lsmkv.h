@@ -250,6 +250,24 @@ int lsmkv_xrun_build(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
                      uint64_t *chunk_off_out);
 
 /*
+ * Compaction of two xruns (Sec. 2.2 "Updates": runs are merged as the index grows). The caller
+ * has laid run B's sequences behind run A's in ONE arena: tokens / seq_off describe n_a + n_b
+ * sequences, A's first (the record arrays are concatenated the same way, B's rows behind A's).
+ *   order_a [dev] u32[n_a]: A's sequences (numbers 0..n_a-1) in token order, from a build or merge
+ *   order_b [dev] u32[n_b]: B's sequences in token order, numbered 0..n_b-1 within B as
+ *           lsmkv_xrun_build returned them for B alone; the call adds n_a to every number
+ *   order_out [dev] u32[n_a + n_b] and chunk_off_out [dev] u64[n_a + n_b + 1]: the index arrays of
+ *           the merged run, equal to what lsmkv_xrun_build gives for the whole arena at the price
+ *           of one merge step instead of a sort. order_out must not overlap the inputs.
+ * A number outside its part sets LSMKV_ST_BAD_COUNT (that entry is replaced, the result is then
+ * not a valid order). n_a + n_b < 2^32 - 1. Uses (and may grow) the context's sort scratch.
+ */
+int lsmkv_xrun_merge(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
+                     const uint64_t *seq_off, const uint32_t *order_a, uint32_t n_a,
+                     const uint32_t *order_b, uint32_t n_b, uint32_t *order_out,
+                     uint64_t *chunk_off_out);
+
+/*
  * Probe of xruns ([host] array, newest first, n_runs <= LSMKV_MAX_RUNS; queries laid out as for
  * lsmkv_probe_batch). Per run, the whole chunks of the longest token prefix the query shares
  * with any stored sequence are present; hit_chunks_out[q] is the largest such count over the

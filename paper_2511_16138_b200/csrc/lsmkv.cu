@@ -836,6 +836,36 @@ int lsmkv_xrun_build(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
     return LSMKV_OK;
 }
 
+int lsmkv_xrun_merge(lsmkv_ctx *ctx, void *stream, const uint32_t *tokens,
+                     const uint64_t *seq_off, const uint32_t *order_a, uint32_t n_a,
+                     const uint32_t *order_b, uint32_t n_b, uint32_t *order_out,
+                     uint64_t *chunk_off_out)
+{
+    const uint64_t n = (uint64_t)n_a + n_b;
+    if (!ctx || !chunk_off_out || n >= 0xFFFFFFFFull) return LSMKV_EINVAL;
+    if (n && (!seq_off || !order_out)) return LSMKV_EINVAL;
+    if ((n_a && !order_a) || (n_b && !order_b)) return LSMKV_EINVAL;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n == 0) {
+        CU(ctx, cudaMemsetAsync(chunk_off_out, 0, sizeof(uint64_t), s));
+        return LSMKV_OK;
+    }
+    SortWs ws;
+    int rc = ensure_sort(ctx, n, &ws);
+    if (rc != LSMKV_OK) return rc;
+    LaunchTimer timer(ctx, s, LSMKV_K_MERGE);
+    k_xrun_concat<<<merge_grid(ctx, n), 256, 0, s>>>(order_a, n_a, order_b, n_b, seq_off,
+                                                     ctx->geom.chunk_tokens, ws.idx[0],
+                                                     chunk_off_out, ctx->d_status);
+    k_scan_blocks<<<1, 1024, 0, s>>>(chunk_off_out, n, chunk_off_out + n);
+    k_xrun_merge_two<<<warp_grid(ctx, n, 256, 8), 256, 0, s>>>(tokens, seq_off, ws.idx[0],
+                                                               order_out, n, n_a);
+    ctx->launches += 3;
+    CU(ctx, cudaGetLastError());
+    return LSMKV_OK;
+}
+
 int lsmkv_xprobe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint32_t *tokens,
                        const uint64_t *seq_off, const uint64_t *qchunk_off, uint64_t n_qchunks,
                        const lsmkv_xrun_t *runs, uint32_t n_runs, uint32_t *hit_chunks_out,

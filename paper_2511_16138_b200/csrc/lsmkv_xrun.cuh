@@ -118,6 +118,48 @@ k_xrun_merge_level(const uint32_t *__restrict__ tokens, const uint64_t *__restri
     }
 }
 
+// Merge of two sorted runs that share one arena: src[0, mid) and src[mid, n) are each in token
+// order; one warp per element finds its rank in the other part, as in a merge level.
+__global__ void __launch_bounds__(256)
+k_xrun_merge_two(const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
+                 const uint32_t *__restrict__ src, uint32_t *__restrict__ dst, uint64_t n,
+                 uint64_t mid)
+{
+    const uint64_t warp0 = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    for (uint64_t i = warp0; i < n; i += n_warps) {
+        const uint32_t x = __ldg(src + i);
+        const SeqView vx = seq_view(tokens, seq_off, x);
+        uint64_t lo, hi;
+        if (i < mid) { lo = mid; hi = n; } else { lo = 0; hi = mid; }
+        const uint64_t below = warp_locate(vx, x, tokens, seq_off, src, lo, hi).pos - lo;
+        const uint64_t own = i < mid ? i : i - mid;
+        if (lane_id() == 0) dst[own + below] = x;
+    }
+}
+
+// src = order_a, then order_b with n_a added to every number (run B's sequences follow run A's
+// in the shared arena); chunk counts of all sequences as in k_xrun_init.
+__global__ void __launch_bounds__(256)
+k_xrun_concat(const uint32_t *__restrict__ order_a, uint32_t n_a,
+              const uint32_t *__restrict__ order_b, uint32_t n_b,
+              const uint64_t *__restrict__ seq_off, uint32_t C, uint32_t *__restrict__ src,
+              uint64_t *__restrict__ chunk_cnt, DevStatus *st)
+{
+    const uint64_t n = (uint64_t)n_a + n_b;
+    for (uint64_t s = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; s < n;
+         s += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t a = seq_off[s], b = seq_off[s + 1];
+        if (b < a) st_flag(st, LSMKV_ST_BAD_COUNT, s);
+        chunk_cnt[s] = b >= a ? (b - a) / C : 0;
+        uint32_t v = s < n_a ? order_a[s] : order_b[s - n_a] + n_a;
+        // a number outside its part would send the comparisons out of the arena
+        const bool ok = s < n_a ? v < n_a : (v >= n_a && v < n);
+        if (!ok) { st_flag(st, LSMKV_ST_BAD_COUNT, s); v = (uint32_t)s; }
+        src[s] = v;
+    }
+}
+
 constexpr int kMaxXRuns = LSMKV_MAX_RUNS;
 
 struct XRunTable {

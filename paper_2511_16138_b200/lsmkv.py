@@ -26,7 +26,7 @@ EXPORTS = (
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
     "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
-    "lsmkv_hindex_buckets", "lsmkv_hindex_build",
+    "lsmkv_hindex_buckets", "lsmkv_hindex_build", "lsmkv_xrun_merge",
     "lsmkv_relocate_records", "lsmkv_xrun_build", "lsmkv_xprobe_batch",
 )
 ST_OVERFLOW = 32
@@ -165,6 +165,8 @@ def lib() -> C.CDLL:
     L.lsmkv_relocate_records.argtypes = [vp, vp, vp, u64, C.POINTER(RelocStruct), u32, vp]
     L.lsmkv_xrun_build.restype = C.c_int
     L.lsmkv_xrun_build.argtypes = [vp, vp, vp, vp, u32, vp, vp]
+    L.lsmkv_xrun_merge.restype = C.c_int
+    L.lsmkv_xrun_merge.argtypes = [vp, vp, vp, vp, vp, u32, vp, u32, vp, vp]
     L.lsmkv_xprobe_batch.restype = C.c_int
     L.lsmkv_xprobe_batch.argtypes = [vp, vp, u32, vp, vp, vp, u64, C.POINTER(XRunStruct), u32,
                                      vp, vp]
@@ -367,6 +369,13 @@ def lsmkv_xrun_build(ctx, stream, tokens, seq_off, n_seq, order_out, chunk_off_o
     _check(ctx, rc, "lsmkv_xrun_build")
 
 
+def lsmkv_xrun_merge(ctx, stream, tokens, seq_off, order_a, n_a, order_b, n_b, order_out,
+                     chunk_off_out) -> None:
+    rc = lib().lsmkv_xrun_merge(ctx, _stream(stream), _ptr(tokens), _ptr(seq_off), _ptr(order_a),
+                                n_a, _ptr(order_b), n_b, _ptr(order_out), _ptr(chunk_off_out))
+    _check(ctx, rc, "lsmkv_xrun_merge")
+
+
 def lsmkv_xprobe_batch(ctx, stream, n_query, tokens, seq_off, qchunk_off, n_qchunks, xruns,
                        hit_chunks_out, recs_out) -> None:
     """xruns: sequence of (tokens, seq_off, vals, order, chunk_off, n_seq), newest first."""
@@ -535,6 +544,11 @@ class Context:
 
     def xrun_build(self, tokens, seq_off, n_seq, order_out, chunk_off_out, stream=None):
         lsmkv_xrun_build(self.handle, stream, tokens, seq_off, n_seq, order_out, chunk_off_out)
+
+    def xrun_merge(self, tokens, seq_off, order_a, n_a, order_b, n_b, order_out, chunk_off_out,
+                   stream=None):
+        lsmkv_xrun_merge(self.handle, stream, tokens, seq_off, order_a, n_a, order_b, n_b,
+                         order_out, chunk_off_out)
 
     def xprobe_batch(self, n_query, tokens, seq_off, qchunk_off, n_qchunks, xruns,
                      hit_chunks_out, recs_out, stream=None):

@@ -45,6 +45,9 @@ def test_start_chunk_and_base_offset():
     lsmkv.Geom(2, 1, 24, elem_bytes=2, page_tokens=3, chunk_tokens=3),   # 144-byte pages
     lsmkv.Geom(1, 1, 8, elem_bytes=1, page_tokens=2, chunk_tokens=2),    # 16-byte pages
     lsmkv.Geom(5, 2, 40, elem_bytes=2, page_tokens=1, chunk_tokens=1),   # one token per chunk
+    lsmkv.Geom(1, 2, 8, elem_bytes=2, page_tokens=24, chunk_tokens=24),  # a 16-token block + 8 tokens
+    lsmkv.Geom(2, 1, 16, elem_bytes=2, page_tokens=40, chunk_tokens=40), # two blocks + 8 tokens
+    lsmkv.Geom(1, 1, 8, elem_bytes=2, page_tokens=17, chunk_tokens=17),  # odd: no 16-byte token loads
 ])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_geometries_and_ragged_lengths(g, mode):

@@ -170,3 +170,65 @@ def test_bad_counts_are_flagged_not_read():
         hit, _, _ = gpu_xprobe(ctx, some, qoff, [x])
         assert hit[0] == 0
         assert ctx.last_status()["flags"] & lsmkv.ST_BAD_COUNT
+
+
+def random_store(rng, n_seq, alphabet, max_len, n_dup):
+    """Sequences over a small alphabet (many shared prefixes), a few of them repeated verbatim."""
+    seqs = [rng.integers(0, alphabet, int(rng.integers(0, max_len + 1)), dtype=np.uint32)
+            for _ in range(n_seq)]
+    for _ in range(n_dup):
+        seqs[int(rng.integers(0, n_seq))] = seqs[int(rng.integers(0, n_seq))].copy()
+    return seqs
+
+
+@pytest.mark.parametrize("n_a,n_b", [(0, 0), (0, 5), (7, 0), (1, 1), (40, 3), (300, 900), (1500, 700)])
+def test_merge_of_two_runs_equals_a_build_of_the_whole_arena(n_a, n_b):
+    g = geom(4)
+    rng = np.random.default_rng(1000 * n_a + n_b)
+    seqs = random_store(rng, n_a + n_b, 3, 40, (n_a + n_b) // 5) if n_a + n_b else []
+    whole = synth.make_batch(seqs)
+    part_a, part_b = synth.make_batch(seqs[:n_a]), synth.make_batch(seqs[n_a:])
+    want_order = oracle.xrun_order(whole.tokens, whole.seq_off)
+    want_coff = synth.offsets(synth.chunk_counts(whole.seq_off, g.chunk_tokens))
+    with lsmkv.Context(g, 0) as ctx:
+        def build(b):
+            d_order = torch.full((max(4, b.n),), -1, dtype=torch.int32, device=H.DEV)
+            d_coff = torch.full((b.n + 1,), -1, dtype=torch.int64, device=H.DEV)
+            ctx.xrun_build(H.dev(b.tokens), H.dev(b.seq_off), b.n, d_order, d_coff)
+            return d_order
+        order_a, order_b = build(part_a), build(part_b)       # B numbered within B
+        n = n_a + n_b
+        d_out = torch.full((max(4, n),), -1, dtype=torch.int32, device=H.DEV)
+        d_coff = torch.full((n + 1,), -1, dtype=torch.int64, device=H.DEV)
+        ctx.xrun_merge(H.dev(whole.tokens), H.dev(whole.seq_off), order_a, n_a, order_b, n_b,
+                       d_out, d_coff)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_out.cpu().numpy().view(np.uint32)[:n], want_order)
+        assert np.array_equal(d_coff.cpu().numpy().view(np.uint64), want_coff)
+        H.assert_status_clean(ctx)
+
+
+def test_probe_through_a_merged_run_equals_the_oracle_on_the_whole_store():
+    g = geom(4)
+    og = H.ogeom(g)
+    rng = np.random.default_rng(77)
+    seqs = random_store(rng, 600, 3, 64, 100)
+    whole = synth.make_batch(seqs)
+    vals = make_vals(g, whole, 5, rng)
+    n_a = 350
+    query = synth.make_batch(random_store(rng, 200, 3, 80, 0) + [s.copy() for s in seqs[::7]])
+    qoff = synth.offsets(synth.chunk_counts(query.seq_off, g.chunk_tokens))
+    o_hit, o_recs = oracle.xprobe_batch(og, query.tokens, query.seq_off, qoff,
+                                        [(whole.tokens, whole.seq_off, vals)])
+    with lsmkv.Context(g, 0) as ctx:
+        part_a, part_b = synth.make_batch(seqs[:n_a]), synth.make_batch(seqs[n_a:])
+        xa, _, _ = gpu_xrun(ctx, g, part_a, make_vals(g, part_a, 0))
+        xb, _, _ = gpu_xrun(ctx, g, part_b, make_vals(g, part_b, 0))
+        d_tok, d_off, d_vals = H.dev(whole.tokens), H.dev(whole.seq_off), H.dev(vals)
+        d_order = torch.full((whole.n,), -1, dtype=torch.int32, device=H.DEV)
+        d_coff = torch.full((whole.n + 1,), -1, dtype=torch.int64, device=H.DEV)
+        ctx.xrun_merge(d_tok, d_off, xa[3], n_a, xb[3], whole.n - n_a, d_order, d_coff)
+        hit, recs, _ = gpu_xprobe(ctx, query, qoff,
+                                  [(d_tok, d_off, d_vals, d_order, d_coff, whole.n)])
+        assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
+        H.assert_status_clean(ctx)
