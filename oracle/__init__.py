@@ -76,8 +76,12 @@ class Geom:
         return self.page_tokens * self.n_kv_heads * self.head_dim * self.elem_bytes
 
     @property
+    def pages_per_chunk(self) -> int:
+        return self.chunk_tokens // self.page_tokens
+
+    @property
     def chunk_bytes(self) -> int:
-        return 2 * self.n_layers * self.page_bytes
+        return self.pages_per_chunk * 2 * self.n_layers * self.page_bytes
 
 
 _lib = None
@@ -232,7 +236,7 @@ def encode_batch(g: Geom, tokens, seq_off, start_chunk, chunk_off, page_table, p
     num_pages = 0
     if with_blob:
         page_table = _arr(page_table, np.uint32)
-        assert len(page_table) == n_chunks
+        assert len(page_table) == n_chunks * g.pages_per_chunk
         blob = np.zeros(n_chunks * g.chunk_bytes, dtype=np.uint8)
         ptrs = _pool_ptrs(pool)
         num_pages = pool.shape[1]

@@ -26,7 +26,8 @@
  *   digest  = h <- 0; for every token t in order: h <- (h * BASE + (t + 1)) mod (2^61 - 1),
  *             always the canonical representative in [0, 2^61 - 1)
  *   record  = {u32 file_id, u32 reserved = 0, u64 offset}, offset = base + i * chunk_bytes
- *   blob    = for l in 0..L-1: K page slab of layer l, then V page slab of layer l
+ *   blob    = for every page of the chunk, in token order: for l in 0..L-1: K page slab of
+ *             layer l, then V page slab of layer l (chunk_tokens = m * page_tokens, m >= 1)
  *   pool    = 2L buffers (K of layers 0..L-1, then V of layers 0..L-1), each
  *             [num_pages][page_tokens][kv_heads][head_dim] elements, page slab contiguous
  *
@@ -60,15 +61,23 @@ uint64_t orc_page_bytes(const orc_geom *g)
     return (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
 }
 
+/* A chunk covers m = chunk_tokens / page_tokens whole pages (m = 1: a chunk is a page). Its
+ * blob is the m page blobs one after the other, each K0 V0 K1 V1 ...; page tables carry m
+ * entries per chunk, entry i*m + k for the k-th page of chunk i. */
+static uint64_t pages_per_chunk(const orc_geom *g)
+{
+    return g->chunk_tokens / g->page_tokens;
+}
+
 uint64_t orc_chunk_bytes(const orc_geom *g)
 {
-    return 2ull * g->n_layers * orc_page_bytes(g);
+    return pages_per_chunk(g) * 2ull * g->n_layers * orc_page_bytes(g);
 }
 
 static int geom_ok(const orc_geom *g)
 {
     return g && g->n_layers && g->n_kv_heads && g->head_dim && g->elem_bytes &&
-           g->page_tokens && g->chunk_tokens == g->page_tokens;
+           g->page_tokens && g->chunk_tokens && g->chunk_tokens % g->page_tokens == 0;
 }
 
 /* ---- digest: one Horner step of the polynomial hash over the Mersenne prime 2^61-1 -- */
@@ -140,7 +149,7 @@ int orc_encode_batch(const orc_geom *g, uint32_t n_req, const uint32_t *tokens,
                      uint8_t *blob_out, uint64_t blob_capacity)
 {
     if (!geom_ok(g)) return ORC_EINVAL;
-    const uint64_t C = g->chunk_tokens, L = g->n_layers;
+    const uint64_t C = g->chunk_tokens, L = g->n_layers, m = pages_per_chunk(g);
     const uint64_t pb = orc_page_bytes(g), cb = orc_chunk_bytes(g);
     if (blob_out && blob_capacity < n_chunks * cb) return ORC_ECAPACITY;
     if (n_req && chunk_off[n_req] != n_chunks) return ORC_EINVAL;
@@ -161,12 +170,14 @@ int orc_encode_batch(const orc_geom *g, uint32_t n_req, const uint32_t *tokens,
             vals_out[i].reserved = 0;
             vals_out[i].offset = base_offset + i * cb;
             if (!blob_out) continue;
-            const uint64_t page = page_table[i];
-            if (page >= num_pages) return ORC_EBADPAGE;
-            uint8_t *dst = blob_out + i * cb;
-            for (uint64_t l = 0; l < L; ++l) {
-                memcpy(dst + (2 * l) * pb, kv_ptrs[l] + page * pb, pb);         /* K, layer l */
-                memcpy(dst + (2 * l + 1) * pb, kv_ptrs[L + l] + page * pb, pb); /* V, layer l */
+            for (uint64_t k = 0; k < m; ++k) {           /* the chunk's pages, in token order */
+                const uint64_t page = page_table[i * m + k];
+                if (page >= num_pages) return ORC_EBADPAGE;
+                uint8_t *dst = blob_out + i * cb + k * 2 * L * pb;
+                for (uint64_t l = 0; l < L; ++l) {
+                    memcpy(dst + (2 * l) * pb, kv_ptrs[l] + page * pb, pb);         /* K, layer l */
+                    memcpy(dst + (2 * l + 1) * pb, kv_ptrs[L + l] + page * pb, pb); /* V, layer l */
+                }
             }
         }
     }
@@ -424,7 +435,7 @@ int orc_decode_batch(const orc_geom *g, uint32_t n_query, const uint64_t *qchunk
                      uint64_t num_pages)
 {
     if (!geom_ok(g)) return ORC_EINVAL;
-    const uint64_t L = g->n_layers;
+    const uint64_t L = g->n_layers, m = pages_per_chunk(g);
     const uint64_t pb = orc_page_bytes(g), cb = orc_chunk_bytes(g);
     for (uint32_t q = 0; q < n_query; ++q) {
         const uint64_t nch = qchunk_off[q + 1] - qchunk_off[q];
@@ -435,12 +446,14 @@ int orc_decode_batch(const orc_geom *g, uint32_t n_query, const uint64_t *qchunk
             if (rec.file_id >= n_arenas) return ORC_EBADREC;
             if (rec.offset > arena_bytes[rec.file_id] ||
                 arena_bytes[rec.file_id] - rec.offset < cb) return ORC_EBADREC;
-            const uint64_t page = dst_page_table[idx];
-            if (page >= num_pages) return ORC_EBADPAGE;
-            const uint8_t *src = arenas[rec.file_id] + rec.offset;
-            for (uint64_t l = 0; l < L; ++l) {
-                memcpy(kv_ptrs[l] + page * pb, src + (2 * l) * pb, pb);
-                memcpy(kv_ptrs[L + l] + page * pb, src + (2 * l + 1) * pb, pb);
+            for (uint64_t k = 0; k < m; ++k) {
+                const uint64_t page = dst_page_table[idx * m + k];
+                if (page >= num_pages) return ORC_EBADPAGE;
+                const uint8_t *src = arenas[rec.file_id] + rec.offset + k * 2 * L * pb;
+                for (uint64_t l = 0; l < L; ++l) {
+                    memcpy(kv_ptrs[l] + page * pb, src + (2 * l) * pb, pb);
+                    memcpy(kv_ptrs[L + l] + page * pb, src + (2 * l + 1) * pb, pb);
+                }
             }
         }
     }
@@ -473,7 +486,10 @@ static uint64_t round16(uint64_t x) { return (x + 15) & ~(uint64_t)15; }
 
 uint64_t orc_xp12_slab_bound(uint64_t n_elems) { return 16 + 2 * n_elems; }
 
-uint64_t orc_xp12_dir_bytes(const orc_geom *g) { return round16(4ull * (2ull * g->n_layers + 1)); }
+uint64_t orc_xp12_dir_bytes(const orc_geom *g)
+{
+    return round16(4ull * (g->chunk_tokens / g->page_tokens * 2ull * g->n_layers + 1));
+}
 
 /* Returns the encoded size; out needs orc_xp12_slab_bound(n) bytes. */
 uint64_t orc_xp12_slab_encode(const uint16_t *in, uint64_t n, uint8_t *out)
@@ -549,7 +565,8 @@ uint64_t orc_xp12_slab_decode(const uint8_t *in, uint64_t avail, uint64_t n, uin
  */
 uint64_t orc_xp12_chunk_bound(const orc_geom *g)
 {
-    return orc_xp12_dir_bytes(g) + 2ull * g->n_layers * orc_xp12_slab_bound(orc_page_bytes(g) / 2);
+    return orc_xp12_dir_bytes(g) +
+           pages_per_chunk(g) * 2ull * g->n_layers * orc_xp12_slab_bound(orc_page_bytes(g) / 2);
 }
 
 int orc_encode_batch_xp12(const orc_geom *g, uint32_t n_req, const uint32_t *tokens,
@@ -566,23 +583,24 @@ int orc_encode_batch_xp12(const orc_geom *g, uint32_t n_req, const uint32_t *tok
                               NULL, 0, file_id, base_offset, keys_out, vals_out, NULL, 0);
     if (rc != ORC_OK) return rc;
     const uint64_t L = g->n_layers, pb = orc_page_bytes(g), ne = pb / 2;
+    const uint64_t m = pages_per_chunk(g), slabs = m * 2 * L;
     const uint64_t dirb = orc_xp12_dir_bytes(g);
     uint64_t at = 0;
     for (uint64_t i = 0; i < n_chunks; ++i) {
         if (blob_capacity - at < orc_xp12_chunk_bound(g)) return ORC_ECAPACITY;
-        const uint64_t page = page_table[i];
-        if (page >= num_pages) return ORC_EBADPAGE;
         uint8_t *blob = blob_out + at;
         uint32_t *dir = (uint32_t *)blob;
         memset(blob, 0, dirb);
         uint64_t pos = dirb;
-        for (uint64_t b = 0; b < 2 * L; ++b) {          /* blob order: K0 V0 K1 V1 ... */
-            const uint64_t buf = (b & 1) * L + (b >> 1);
+        for (uint64_t b = 0; b < slabs; ++b) {      /* blob order: page by page, K0 V0 K1 V1 ... */
+            const uint64_t page = page_table[i * m + b / (2 * L)];
+            if (page >= num_pages) return ORC_EBADPAGE;
+            const uint64_t bb = b % (2 * L), buf = (bb & 1) * L + (bb >> 1);
             dir[b] = (uint32_t)pos;
             pos += orc_xp12_slab_encode((const uint16_t *)(kv_ptrs[buf] + page * pb), ne,
                                         blob + pos);
         }
-        dir[2 * L] = (uint32_t)pos;
+        dir[slabs] = (uint32_t)pos;
         vals_out[i].file_id = file_id;
         vals_out[i].reserved = (uint32_t)pos;
         vals_out[i].offset = base_offset + at;
@@ -600,6 +618,7 @@ int orc_decode_batch_xp12(const orc_geom *g, uint32_t n_query, const uint64_t *q
 {
     if (!geom_ok(g) || g->elem_bytes != 2) return ORC_EINVAL;
     const uint64_t L = g->n_layers, pb = orc_page_bytes(g), ne = pb / 2;
+    const uint64_t m = pages_per_chunk(g), slabs = m * 2 * L;
     const uint64_t dirb = orc_xp12_dir_bytes(g);
     for (uint32_t q = 0; q < n_query; ++q) {
         if (hit[q] > qchunk_off[q + 1] - qchunk_off[q]) return ORC_EINVAL;
@@ -609,13 +628,13 @@ int orc_decode_batch_xp12(const orc_geom *g, uint32_t n_query, const uint64_t *q
             if (rec.file_id >= n_arenas || rec.reserved < dirb) return ORC_EBADREC;
             if (rec.offset > arena_bytes[rec.file_id] ||
                 arena_bytes[rec.file_id] - rec.offset < rec.reserved) return ORC_EBADREC;
-            const uint64_t page = dst_page_table[idx];
-            if (page >= num_pages) return ORC_EBADPAGE;
             const uint8_t *blob = arenas[rec.file_id] + rec.offset;
             const uint32_t *dir = (const uint32_t *)blob;
-            if (dir[2 * L] != rec.reserved) return ORC_EBADREC;
-            for (uint64_t b = 0; b < 2 * L; ++b) {
-                const uint64_t buf = (b & 1) * L + (b >> 1);
+            if (dir[slabs] != rec.reserved) return ORC_EBADREC;
+            for (uint64_t b = 0; b < slabs; ++b) {
+                const uint64_t page = dst_page_table[idx * m + b / (2 * L)];
+                if (page >= num_pages) return ORC_EBADPAGE;
+                const uint64_t bb = b % (2 * L), buf = (bb & 1) * L + (bb >> 1);
                 if (dir[b] < dirb || dir[b] > dir[b + 1] || dir[b + 1] > rec.reserved)
                     return ORC_EBADREC;
                 if (!orc_xp12_slab_decode(blob + dir[b], dir[b + 1] - dir[b], ne,
