@@ -39,9 +39,12 @@
  *   pool    2L buffers: K of layers 0..L-1, then V of layers 0..L-1, each
  *             [num_pages][page_tokens][n_kv_heads][head_dim] elements (a page slab of
  *             page_bytes = page_tokens*n_kv_heads*head_dim*elem_bytes is contiguous)
- *   blob    for l in 0..L-1: K slab of layer l, V slab of layer l  (chunk_bytes = 2L*page_bytes)
- *   A chunk is C = chunk_tokens tokens; a sequence of len tokens has floor(len / C) chunks and
- *   a trailing partial chunk is never encoded, probed or decoded.
+ *   blob    for every page of the chunk, in token order: for l in 0..L-1: K slab of layer l,
+ *             V slab of layer l  (chunk_bytes = m*2L*page_bytes)
+ *   A chunk is C = chunk_tokens = m * page_tokens tokens (m >= 1 whole pages); a sequence of len
+ *   tokens has floor(len / C) chunks and a trailing partial chunk is never encoded, probed or
+ *   decoded. Page tables carry m entries per chunk: entry i*m + k names the pool page of the
+ *   k-th page of chunk i.
  */
 #ifndef LSMKV_H
 #define LSMKV_H
@@ -82,7 +85,7 @@ typedef struct { uint32_t file_id, reserved; uint64_t offset; } lsmkv_val_t; /* 
 
 typedef struct {
     uint32_t n_layers, n_kv_heads, head_dim, elem_bytes;
-    uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens must equal page_tokens; flags = LSMKV_CODEC_* */
+    uint32_t page_tokens, chunk_tokens, ns, flags; /* chunk_tokens = m * page_tokens, m >= 1; flags = LSMKV_CODEC_* */
 } lsmkv_geom_t;
 
 /* One immutable sorted run of the index: keys ascending and unique, vals[i] belongs to keys[i].
@@ -121,8 +124,9 @@ typedef struct {
 
 /*
  * Create a context on `device` for one KV geometry. Allocates the context, a small device
- * status block and the workspace. Errors: LSMKV_EINVAL for a zero field, chunk_tokens !=
- * page_tokens, or page_bytes not a multiple of 16; LSMKV_ECUDA / LSMKV_ENOMEM.
+ * status block and the workspace. Errors: LSMKV_EINVAL for a zero field, chunk_tokens not a
+ * multiple of page_tokens (or more than 4096 pages per chunk), or page_bytes not a multiple of
+ * 16; LSMKV_ECUDA / LSMKV_ENOMEM.
  */
 int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *geom, int device);
 
@@ -142,14 +146,15 @@ int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks);
  * request r has output index i = chunk_off[r] + c and produces
  *   keys_out[i]  the chunk key,
  *   vals_out[i]  {file_id, 0, base_offset + i*chunk_bytes},
- *   blob_out[i*chunk_bytes ..)  the 2L page slabs of pool page page_table[i].
+ *   blob_out[i*chunk_bytes ..)  the 2L page slabs of each of the pool pages
+ *                page_table[i*m .. i*m+m), page after page.
  *   tokens      [dev] u32, all sequences back to back
  *   seq_off     [dev] u64[n_req+1], ascending
  *   start_chunk [dev] u32[n_req] or NULL
  *   chunk_off   [dev] u64[n_req+1], exclusive prefix sums of max(0, n_r - start_r);
  *               chunk_off[n_req] must equal n_chunks (a mismatch sets LSMKV_ST_BAD_COUNT and
  *               the request is skipped)
- *   page_table  [dev] u32[n_chunks]; may be NULL together with pool and blob_out for an
+ *   page_table  [dev] u32[n_chunks * m]; may be NULL together with pool and blob_out for an
  *               index-only encode (keys and records, no payload)
  *   blob_out    [dev], 16-byte aligned, blob_capacity >= n_chunks*chunk_bytes else
  *               LSMKV_ECAPACITY
@@ -182,7 +187,8 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
 /*
  * get_batch, tensor half (App. B "Get Batch"; Sec. 3.4). For every query q and j < hit_chunks[q]
  * the blob at arenas[rec.file_id] + rec.offset (rec = recs[qchunk_off[q] + j]) is split into
- * its 2L page slabs, which are written to page dst_page_table[qchunk_off[q] + j] of the pool.
+ * its m*2L page slabs, which are written to pages dst_page_table[idx*m .. idx*m+m) of the pool
+ * (idx = qchunk_off[q] + j; dst_page_table has m entries per query chunk).
  * No other byte of the pool changes. Destination pages must be distinct within the call.
  *   arenas      [host] array of n_arenas [dev] base pointers (16-byte aligned), indexed by file_id
  *   arena_bytes [host] size of each arena; records must satisfy offset + chunk_bytes <= size
@@ -305,8 +311,8 @@ int lsmkv_relocate_records(lsmkv_ctx *ctx, void *stream, lsmkv_val_t *vals, uint
  *             element i in byte i/2, even i in the low nibble), n_exc raw exponent bytes of the
  *             code-15 elements in element order, zero padding to a multiple of 16
  *     mode 1 (n_exc >= N/2): the 2N raw bytes
- *   chunk blob: directory of 2L+1 u32 (byte offset of every slab, then the blob size; padded
- *     to 16 bytes) followed by the slabs in blob order (K0 V0 K1 V1 ...)
+ *   chunk blob: directory of m*2L+1 u32 (byte offset of every slab, then the blob size; padded
+ *     to 16 bytes) followed by the slabs in blob order (page by page, K0 V0 K1 V1 ...)
  *   records: {file_id, reserved = blob size, offset}; blobs are placed back to back, so
  *     offset = base_offset + sum of the sizes of the chunks before it. Data-dependent: size
  *     blob_out with lsmkv_encode_bound(); the bytes used are the last record's offset + size

@@ -48,6 +48,7 @@ struct lsmkv_ctx {
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
+    uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
     size_t io_cap[3];
@@ -277,7 +278,8 @@ int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &
                 uint64_t max_items)
 {
     LaunchTimer timer(ctx, s, job.unpack ? LSMKV_K_UNPACK : LSMKV_K_PACK);
-    const uint64_t slabs = 2ull * ctx->geom.n_layers;
+    const uint64_t slabs = 2ull * ctx->geom.n_layers * ctx->ppc;
+    job.pages_per_chunk = ctx->ppc;
     if (ctx->copy_mode == 1) {
         job.piece_bytes = (uint32_t)ctx->page_bytes;
         job.pieces_per_slab = 1;
@@ -323,7 +325,7 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
                 const lsmkv_pool_t *pool, uint32_t file_id, uint64_t base_offset,
                 lsmkv_val_t *vals_out, void *blob_out, uint64_t blob_capacity)
 {
-    const uint64_t slabs = 2ull * ctx->geom.n_layers;
+    const uint64_t slabs = 2ull * ctx->geom.n_layers * ctx->ppc;
     if (n_chunks > ctx->xp_cap || !ctx->d_xp) {
         void *p = nullptr;
         cudaError_t e = cudaMalloc(&p, (size_t)n_chunks * slabs * 12 + ((size_t)n_chunks + 2) * 8 + 256);
@@ -338,6 +340,7 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
     XpJob job;
     std::memset(&job, 0, sizeof(job));
     job.n_layers = ctx->geom.n_layers;
+    job.pages_per_chunk = ctx->ppc;
     job.page_bytes = (uint32_t)ctx->page_bytes;
     job.n_elems = (uint32_t)(ctx->page_bytes / 2);
     job.dir_bytes = ctx->xp_dir_bytes;
@@ -397,22 +400,27 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     if (!out || !g) return LSMKV_EINVAL;
     *out = nullptr;
     if (!g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes || !g->page_tokens ||
-        g->chunk_tokens != g->page_tokens || g->flags > LSMKV_CODEC_XP12)
+        !g->chunk_tokens || g->chunk_tokens % g->page_tokens != 0 || g->flags > LSMKV_CODEC_XP12)
         return LSMKV_EINVAL;
     const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
-    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
+    const uint64_t ppc = g->chunk_tokens / g->page_tokens;
+    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096 || ppc > 4096 ||
+        2ull * g->n_layers * ppc > 0x100000ull)
+        return LSMKV_EINVAL;
     if (g->flags == LSMKV_CODEC_XP12 &&
-        (g->elem_bytes != 2 || 2ull * g->n_layers * (pb + 16) + 8ull * g->n_layers + 16 > 0xFFFFFFF0ull))
+        (g->elem_bytes != 2 ||
+         ppc * (2ull * g->n_layers * (pb + 16) + 8ull * g->n_layers) + 16 > 0xFFFFFFF0ull))
         return LSMKV_EINVAL;
     lsmkv_ctx *ctx = new (std::nothrow) lsmkv_ctx();   // value-initialised: all fields zero
     if (!ctx) return LSMKV_ENOMEM;
     ctx->geom = *g;
     ctx->device = device;
     ctx->page_bytes = pb;
-    ctx->chunk_bytes = 2ull * g->n_layers * pb;
+    ctx->ppc = (uint32_t)ppc;
+    ctx->chunk_bytes = ppc * 2ull * g->n_layers * pb;
     fill_key_consts(ctx->kc, g->chunk_tokens);
     ctx->codec = g->flags;
-    ctx->xp_dir_bytes = (uint32_t)((4ull * (2ull * g->n_layers + 1) + 15) & ~15ull);
+    ctx->xp_dir_bytes = (uint32_t)((4ull * (ppc * 2ull * g->n_layers + 1) + 15) & ~15ull);
     ctx->copy_mode = 0;
     ctx->copy_stage_bytes = 16384;
     ctx->copy_stages = 12;
@@ -667,6 +675,7 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
         XpUnpackJob uj;
         std::memset(&uj, 0, sizeof(uj));
         uj.n_layers = ctx->geom.n_layers;
+        uj.pages_per_chunk = ctx->ppc;
         uj.page_bytes = (uint32_t)ctx->page_bytes;
         uj.n_elems = (uint32_t)(ctx->page_bytes / 2);
         uj.dir_bytes = ctx->xp_dir_bytes;
@@ -678,7 +687,7 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
         uj.recs = recs;
         uj.st = ctx->d_status;
         LaunchTimer timer(ctx, s, LSMKV_K_UNPACK);
-        uint64_t grid = n_qchunks * 2ull * ctx->geom.n_layers;
+        uint64_t grid = n_qchunks * 2ull * ctx->geom.n_layers * ctx->ppc;
         const uint64_t cap = (uint64_t)ctx->sm_count * 8;
         if (grid > cap) grid = cap;
         const uint32_t sweeps = uj.n_elems % 2048u == 0 && !ctx->xp_generic ? uj.n_elems / 2048u : 0;
@@ -929,7 +938,8 @@ uint64_t lsmkv_encode_bound(const lsmkv_ctx *ctx, uint64_t n_chunks)
 {
     if (!ctx) return 0;
     if (ctx->codec == LSMKV_CODEC_XP12)
-        return n_chunks * (ctx->xp_dir_bytes + 2ull * ctx->geom.n_layers * (16 + ctx->page_bytes));
+        return n_chunks * (ctx->xp_dir_bytes +
+                           2ull * ctx->geom.n_layers * ctx->ppc * (16 + ctx->page_bytes));
     return n_chunks * ctx->chunk_bytes;
 }
 
@@ -1168,11 +1178,15 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
                                          const lsmkv_pool_t *pool, lsmkv_status_t *status_out)
 {
     if (!g || !g->n_layers || !g->n_kv_heads || !g->head_dim || !g->elem_bytes ||
-        !g->page_tokens || g->chunk_tokens != g->page_tokens || g->flags != 0)
+        !g->page_tokens || !g->chunk_tokens || g->chunk_tokens % g->page_tokens != 0 ||
+        g->flags != 0)
         return LSMKV_EINVAL;
     const uint64_t pb = (uint64_t)g->page_tokens * g->n_kv_heads * g->head_dim * g->elem_bytes;
-    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096) return LSMKV_EINVAL;
-    const uint64_t cb = 2ull * g->n_layers * pb;
+    const uint64_t ppc = g->chunk_tokens / g->page_tokens;
+    if (pb % 16 != 0 || pb > 0x40000000ull || g->n_layers > 4096 || ppc > 4096 ||
+        2ull * g->n_layers * ppc > 0x100000ull)
+        return LSMKV_EINVAL;
+    const uint64_t cb = ppc * 2ull * g->n_layers * pb;
     if (n_query > kStaticMaxQueries || n_qchunks > kStaticMaxChunks) return LSMKV_ETOOBIG;
     if (!qchunk_off || !hit_chunks || !recs || !dst_page_table || !pool || !pool->kv_ptrs)
         return LSMKV_EINVAL;
@@ -1209,6 +1223,7 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
         std::memset(&job, 0, sizeof(job));
         job.unpack = 1;
         job.n_layers = g->n_layers;
+        job.pages_per_chunk = (uint32_t)ppc;
         job.page_bytes = (uint32_t)pb;
         job.num_pages = pool->num_pages;
         job.kv_ptrs = pool->kv_ptrs;
@@ -1225,7 +1240,7 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
         while (stages > 1 && (size_t)stages * stride + (size_t)stages * 8 + 1024 > (size_t)sd->max_smem_optin)
             --stages;
         const size_t smem = (size_t)stages * stride + (size_t)stages * 8;
-        const uint64_t pieces = n_qchunks * 2ull * g->n_layers * job.pieces_per_slab;
+        const uint64_t pieces = n_qchunks * ppc * 2ull * g->n_layers * job.pieces_per_slab;
         uint64_t grid = (uint64_t)sd->sm_count;
         const uint64_t need = (pieces + stages - 1) / stages;
         if (grid > need) grid = need;

@@ -20,12 +20,14 @@ struct ArenaTable {
     uint64_t bytes[kMaxArenas];
 };
 
-// What to copy. pack: item i = encoded chunk, pool page page_table[i] -> blob + i*chunk_bytes.
+// What to copy. pack: item i = encoded chunk, pool pages page_table[i*m .. i*m+m) -> blob +
+// i*chunk_bytes (m = pages_per_chunk; the blob is the m page blobs in token order).
 // unpack: item t = t-th hit chunk, idx = plan[t]; blob at arena[rec.file_id] + rec.offset ->
-// pool page page_table[idx].
+// pool pages page_table[idx*m .. idx*m+m).
 struct CopyJob {
     int unpack;                      // 0 = pack, 1 = unpack
     uint32_t n_layers;
+    uint32_t pages_per_chunk;        // m = chunk_tokens / page_tokens
     uint32_t page_bytes;
     uint32_t piece_bytes;            // bytes moved per step (<= page_bytes, multiple of 16)
     uint32_t pieces_per_slab;
@@ -46,12 +48,14 @@ struct Piece { const unsigned char *src; unsigned char *dst; uint32_t bytes; };
 __device__ __forceinline__ bool resolve_piece(const CopyJob &job, const ArenaTable &ar,
                                               uint64_t p, Piece &out)
 {
-    const uint32_t slabs = 2u * job.n_layers;
+    const uint32_t per_page = 2u * job.n_layers, slabs = per_page * job.pages_per_chunk;
     const uint64_t unit = p / job.pieces_per_slab;
     const uint32_t piece = (uint32_t)(p - unit * job.pieces_per_slab);
     const uint64_t item = unit / slabs;
-    const uint32_t b = (uint32_t)(unit - item * slabs);      // blob slab: 2*layer + (0=K, 1=V)
-    const uint32_t buf = (b & 1u) * job.n_layers + (b >> 1); // pool buffer: K layers, then V layers
+    const uint32_t b = (uint32_t)(unit - item * slabs);      // slab of the chunk's blob
+    const uint32_t pg = b / per_page;                        // which of the chunk's pages
+    const uint32_t bb = b - pg * per_page;                   // slab of that page: 2*layer + (0=K, 1=V)
+    const uint32_t buf = (bb & 1u) * job.n_layers + (bb >> 1);   // pool buffer: K layers, then V layers
     const uint32_t off = piece * job.piece_bytes;
     const uint32_t bytes = min(job.piece_bytes, job.page_bytes - off);
     uint64_t idx = item;
@@ -66,10 +70,10 @@ __device__ __forceinline__ bool resolve_piece(const CopyJob &job, const ArenaTab
     } else {
         blob_slab = job.blob + (item * slabs + b) * (uint64_t)job.page_bytes;
     }
-    const uint64_t page = __ldg(job.page_table + idx);
+    const uint64_t page = __ldg(job.page_table + idx * job.pages_per_chunk + pg);
     unsigned char *pool_buf = static_cast<unsigned char *>(job.kv_ptrs[buf]);
     if (page >= job.num_pages) {
-        if (piece == 0 && b == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
+        if (piece == 0 && bb == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
         return false;
     }
     if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) {
@@ -86,7 +90,7 @@ __device__ __forceinline__ bool resolve_piece(const CopyJob &job, const ArenaTab
 __device__ __forceinline__ uint64_t job_pieces(const CopyJob &job)
 {
     const uint64_t items = job.unpack ? *job.n_items_dev : job.n_items;
-    return items * (2ull * job.n_layers) * job.pieces_per_slab;
+    return items * (2ull * job.n_layers * job.pages_per_chunk) * job.pieces_per_slab;
 }
 
 // ---- bulk-async mover ----------------------------------------------------------------------

@@ -164,7 +164,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     // device scratch: every descriptor of the call (uploaded once, up front), one blob stage
     const size_t n_rel = (size_t)n_req + n_slices;        // sum over slices of (requests + 1)
     size_t need = pad256(nt * 4) + 2 * pad256(n_rel * 8) + pad256((size_t)n_req * 4) +
-                  pad256(n_chunks * 4) + pad256(m_max * 32) + pad256(m_max * 16) +
+                  pad256(n_chunks * ctx->ppc * 4) + pad256(m_max * 32) + pad256(m_max * 16) +
                   (with_blob ? pad256(m_max * slot) : 0) + 4096;
     int rc = ensure_io(ctx, 0, need);
     if (rc != LSMKV_OK) return rc;
@@ -173,7 +173,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     uint64_t *d_seq = io.take<uint64_t>(n_rel);
     uint64_t *d_coff = io.take<uint64_t>(n_rel);
     uint32_t *d_start = io.take<uint32_t>(n_req);
-    uint32_t *d_pages = io.take<uint32_t>(n_chunks);
+    uint32_t *d_pages = io.take<uint32_t>(n_chunks * ctx->ppc);      // ppc entries per chunk
     lsmkv_key_t *d_keys = io.take<lsmkv_key_t>(m_max);
     lsmkv_val_t *d_vals = io.take<lsmkv_val_t>(m_max);
     unsigned char *d_blob = with_blob ? io.take<unsigned char>(m_max * slot) : nullptr;
@@ -196,7 +196,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     if (start_chunk)
         CU(ctx, cudaMemcpyAsync(d_start, start_chunk, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
     if (with_blob)
-        CU(ctx, copy_pieces(d_pages, page_table, n_chunks * 4, cudaMemcpyHostToDevice, s));
+        CU(ctx, copy_pieces(d_pages, page_table, n_chunks * ctx->ppc * 4, cudaMemcpyHostToDevice, s));
 
     uint64_t host_used = 0;                          // compressing codec: bytes placed so far
     at = 0;
@@ -208,7 +208,8 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
         if (m == 0) continue;
         rc = lsmkv_encode_batch(ctx, stream, nr, d_tok + (seq_off[a] - t_first), d_seq + rel_at,
                                 start_chunk ? d_start + a : nullptr, d_coff + rel_at, m,
-                                with_blob ? d_pages + coff[a] : nullptr, with_blob ? pool : nullptr,
+                                with_blob ? d_pages + coff[a] * ctx->ppc : nullptr,
+                                with_blob ? pool : nullptr,
                                 file_id, base_offset + (coded ? host_used : coff[a] * cb), d_keys,
                                 d_vals, d_blob, with_blob ? m * slot : 0);
         if (rc != LSMKV_OK) return rc;
@@ -339,10 +340,11 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
     }
     first.push_back(total_hits);
     const size_t n_slices = first.size() - 1;
-    ScratchLease lease(ctx, 2, s, total_hits * 20 + n_slices * 24 + 4096);
+    const uint64_t ppc = ctx->ppc;                                   // page-table entries per chunk
+    ScratchLease lease(ctx, 2, s, total_hits * (16 + 4 * ppc) + n_slices * 24 + 4096);
     if (!lease.ok()) return LSMKV_ENOMEM;
     lsmkv_val_t *h_recs = lease.take<lsmkv_val_t>(total_hits);
-    uint32_t *h_pages = lease.take<uint32_t>(total_hits);
+    uint32_t *h_pages = lease.take<uint32_t>(total_hits * ppc);
     uint64_t *h_qoff = lease.take<uint64_t>(2 * n_slices);           // {0, m} per slice
     uint32_t *h_hit = lease.take<uint32_t>(n_slices);                // m per slice
     k = 0;
@@ -353,7 +355,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
             if (sl_at + 1 < first.size() && k == first[sl_at + 1]) ++sl_at;
             if (k == first[sl_at]) at = 0;
             h_recs[k] = lsmkv_val_t{0, coded ? recs[idx].reserved : 0u, at};
-            h_pages[k] = dst_page_table[idx];
+            for (uint64_t p = 0; p < ppc; ++p) h_pages[k * ppc + p] = dst_page_table[idx * ppc + p];
             at += coded ? recs[idx].reserved : cb;
         }
     }
@@ -365,20 +367,20 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
     }
     (void)m_max;
 
-    size_t need = pad256(blob_stage) + pad256(total_hits * 16) + pad256(total_hits * 4) +
+    size_t need = pad256(blob_stage) + pad256(total_hits * 16) + pad256(total_hits * ppc * 4) +
                   pad256(n_slices * 16) + pad256(n_slices * 4) + 4096;
     int rc = ensure_io(ctx, 2, need);
     if (rc != LSMKV_OK) return rc;
     IoLayout io(ctx->d_io[2]);
     unsigned char *d_blob = io.take<unsigned char>(blob_stage);
     lsmkv_val_t *d_recs = io.take<lsmkv_val_t>(total_hits);
-    uint32_t *d_pages = io.take<uint32_t>(total_hits);
+    uint32_t *d_pages = io.take<uint32_t>(total_hits * ppc);
     uint64_t *d_qoff = io.take<uint64_t>(2 * n_slices);
     uint32_t *d_hit = io.take<uint32_t>(n_slices);
     const void *stage_arena[1] = {d_blob};
     // every descriptor goes up first, so that nothing small queues behind the blob copies
     CU(ctx, copy_pieces(d_recs, h_recs, total_hits * 16, cudaMemcpyHostToDevice, s));
-    CU(ctx, copy_pieces(d_pages, h_pages, total_hits * 4, cudaMemcpyHostToDevice, s));
+    CU(ctx, copy_pieces(d_pages, h_pages, total_hits * ppc * 4, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_qoff, h_qoff, n_slices * 16, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_hit, h_hit, n_slices * 4, cudaMemcpyHostToDevice, s));
 
@@ -411,7 +413,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
         if (run_bytes)
             CU(ctx, copy_pieces(d_blob + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, s));
         rc = lsmkv_decode_batch(ctx, stream, 1, d_qoff + 2 * sl, m, d_hit + sl, d_recs + first[sl],
-                                stage_arena, &stage_used, 1, d_pages + first[sl], pool);
+                                stage_arena, &stage_used, 1, d_pages + first[sl] * ppc, pool);
         if (rc != LSMKV_OK) return rc;
     }
     return LSMKV_OK;

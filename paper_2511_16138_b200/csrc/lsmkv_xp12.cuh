@@ -20,9 +20,10 @@ constexpr int kXpThreads = 256;
 
 struct XpJob {
     uint32_t n_layers;
+    uint32_t pages_per_chunk;    // m = chunk_tokens / page_tokens; a chunk has 2L * m slabs
     uint32_t page_bytes;
     uint32_t n_elems;            // page_bytes / 2
-    uint32_t dir_bytes;          // round16(4 * (2L + 1))
+    uint32_t dir_bytes;          // round16(4 * (2L * m + 1))
     uint64_t num_pages;
     void *const *kv_ptrs;
     const uint32_t *page_table;
@@ -107,11 +108,12 @@ __device__ __forceinline__ void exps8(const uint4 &q, uint32_t e[8])
 __device__ __forceinline__ const unsigned char *xp_src(const XpJob &job, uint64_t i, uint32_t b,
                                                        bool report)
 {
-    const uint64_t page = __ldg(job.page_table + i);
-    const uint32_t buf = (b & 1u) * job.n_layers + (b >> 1);
+    const uint32_t per_page = 2u * job.n_layers, pg = b / per_page, bb = b - pg * per_page;
+    const uint64_t page = __ldg(job.page_table + i * job.pages_per_chunk + pg);
+    const uint32_t buf = (bb & 1u) * job.n_layers + (bb >> 1);
     const unsigned char *pool_buf = static_cast<const unsigned char *>(job.kv_ptrs[buf]);
     if (page >= job.num_pages) {
-        if (report && b == 0 && threadIdx.x == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, i);
+        if (report && bb == 0 && threadIdx.x == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, i);
         return nullptr;
     }
     if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) {
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(kXpThreads)
 k_xp_measure(const __grid_constant__ XpJob job)
 {
     __shared__ uint32_t sh[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers, n8 = job.n_elems >> 3;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, n8 = job.n_elems >> 3;
     const uint64_t total = job.n_chunks * slabs;
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
         const uint64_t i = u / slabs;
@@ -172,7 +174,7 @@ k_xp_measure(const __grid_constant__ XpJob job)
 __global__ void __launch_bounds__(256)
 k_xp_chunk_sizes(const __grid_constant__ XpJob job)
 {
-    const uint32_t slabs = 2u * job.n_layers;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < job.n_chunks;
          i += (uint64_t)gridDim.x * blockDim.x) {
         uint64_t sz = job.dir_bytes;
@@ -186,7 +188,7 @@ k_xp_chunk_sizes(const __grid_constant__ XpJob job)
 __global__ void __launch_bounds__(256)
 k_xp_layout(const __grid_constant__ XpJob job)
 {
-    const uint32_t slabs = 2u * job.n_layers;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk;
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < job.n_chunks;
          i += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t off = job.chunk_off[i], size = job.chunk_off[i + 1] - off;
@@ -219,7 +221,7 @@ __global__ void __launch_bounds__(kXpThreads)
 k_xp_pack(const __grid_constant__ XpJob job)
 {
     __shared__ uint32_t sh[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers, n8 = job.n_elems >> 3, N = job.n_elems;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, n8 = job.n_elems >> 3, N = job.n_elems;
     const uint64_t total = job.n_chunks * slabs;
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
         const uint64_t i = u / slabs;
@@ -287,6 +289,7 @@ k_xp_pack(const __grid_constant__ XpJob job)
 // decode: one CTA per (hit chunk, slab); every offset and header is checked before use
 struct XpUnpackJob {
     uint32_t n_layers;
+    uint32_t pages_per_chunk;
     uint32_t page_bytes;
     uint32_t n_elems;
     uint32_t dir_bytes;
@@ -303,7 +306,7 @@ __global__ void __launch_bounds__(kXpThreads)
 k_xp_unpack(const __grid_constant__ XpUnpackJob job, const __grid_constant__ ArenaTable ar)
 {
     __shared__ uint32_t sh[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers, n8 = job.n_elems >> 3, N = job.n_elems;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, n8 = job.n_elems >> 3, N = job.n_elems;
     const uint64_t total = *job.n_items_dev * slabs;
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
         const uint64_t item = u / slabs;
@@ -316,8 +319,9 @@ k_xp_unpack(const __grid_constant__ XpUnpackJob job, const __grid_constant__ Are
         const uint32_t csize = r.y;
         const uint32_t *dir = reinterpret_cast<const uint32_t *>(blob);
         const uint32_t d0 = __ldg(dir + b), d1 = __ldg(dir + b + 1);
-        const uint64_t page = __ldg(job.page_table + idx);
-        const uint32_t buf = (b & 1u) * job.n_layers + (b >> 1);
+        const uint32_t per_page = 2u * job.n_layers, pg = b / per_page, bb = b - pg * per_page;
+        const uint64_t page = __ldg(job.page_table + (uint64_t)idx * job.pages_per_chunk + pg);
+        const uint32_t buf = (bb & 1u) * job.n_layers + (bb >> 1);
         unsigned char *pool_buf = static_cast<unsigned char *>(job.kv_ptrs[buf]);
         bool ok = __ldg(dir + slabs) == csize && d0 >= job.dir_bytes && d0 <= d1 && d1 <= csize &&
                   (d0 & 15u) == 0 && d1 - d0 >= 16u;
@@ -332,7 +336,7 @@ k_xp_unpack(const __grid_constant__ XpUnpackJob job, const __grid_constant__ Are
             continue;
         }
         if (page >= job.num_pages) {
-            if (threadIdx.x == 0 && b == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
+            if (threadIdx.x == 0 && bb == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
             continue;
         }
         if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) {
@@ -448,7 +452,7 @@ __global__ void __launch_bounds__(kXpThreads)
 k_xp_measure_fast(const __grid_constant__ XpJob job)
 {
     __shared__ uint32_t sh[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk;
     const uint64_t total = job.n_chunks * slabs;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
@@ -507,7 +511,7 @@ k_xp_pack_fast(const __grid_constant__ XpJob job)
 {
     extern __shared__ __align__(16) unsigned char xp_smem[];
     __shared__ uint32_t warp_total[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers, N = job.n_elems, n8 = N >> 3;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, N = job.n_elems, n8 = N >> 3;
     const uint64_t total = job.n_chunks * slabs;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char *my_list = xp_smem + (size_t)warp * (N / 8);
@@ -590,7 +594,7 @@ __global__ void __launch_bounds__(kXpThreads)
 k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant__ ArenaTable ar)
 {
     __shared__ uint32_t warp_total[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers, n8 = job.n_elems >> 3, N = job.n_elems;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, n8 = job.n_elems >> 3, N = job.n_elems;
     const uint64_t total = *job.n_items_dev * slabs;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
@@ -604,8 +608,9 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
         const uint32_t csize = r.y;
         const uint32_t *dir = reinterpret_cast<const uint32_t *>(blob);
         const uint32_t d0 = __ldg(dir + b), d1 = __ldg(dir + b + 1);
-        const uint64_t page = __ldg(job.page_table + idx);
-        const uint32_t buf = (b & 1u) * job.n_layers + (b >> 1);
+        const uint32_t per_page = 2u * job.n_layers, pg = b / per_page, bb = b - pg * per_page;
+        const uint64_t page = __ldg(job.page_table + (uint64_t)idx * job.pages_per_chunk + pg);
+        const uint32_t buf = (bb & 1u) * job.n_layers + (bb >> 1);
         unsigned char *pool_buf = static_cast<unsigned char *>(job.kv_ptrs[buf]);
         bool ok = __ldg(dir + slabs) == csize && d0 >= job.dir_bytes && d0 <= d1 && d1 <= csize &&
                   (d0 & 15u) == 0 && d1 - d0 >= 16u;
@@ -620,7 +625,7 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
             continue;
         }
         if (page >= job.num_pages) {
-            if (threadIdx.x == 0 && b == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
+            if (threadIdx.x == 0 && bb == 0) st_flag(job.st, LSMKV_ST_BAD_PAGE, idx);
             continue;
         }
         if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) {

@@ -112,8 +112,12 @@ class Geom:
         return self.page_tokens * self.n_kv_heads * self.head_dim * self.elem_bytes
 
     @property
+    def pages_per_chunk(self) -> int:
+        return self.chunk_tokens // self.page_tokens
+
+    @property
     def chunk_bytes(self) -> int:
-        return 2 * self.n_layers * self.page_bytes
+        return self.pages_per_chunk * 2 * self.n_layers * self.page_bytes
 
     def c(self) -> GeomStruct:
         return GeomStruct(self.n_layers, self.n_kv_heads, self.head_dim, self.elem_bytes,

@@ -133,10 +133,11 @@ def roundtrip(g: lsmkv.Geom, store, query, start_chunk=None, n_runs=1, num_pages
     n = int(coff[-1])
     qoff = synth.offsets(synth.chunk_counts(query.seq_off, C))
     nq_chunks = int(qoff[-1])
-    num_pages = num_pages or max(n, nq_chunks, 1) + 3
+    m = g.pages_per_chunk                          # page-table entries per chunk
+    num_pages = num_pages or max(n, nq_chunks, 1) * m + 3
     pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
-    src_pages = synth.random_pages(rng, num_pages, n)
-    dst_pages = synth.random_pages(rng, num_pages, nq_chunks)
+    src_pages = synth.random_pages(rng, num_pages, n * m)
+    dst_pages = synth.random_pages(rng, num_pages, nq_chunks * m)
 
     # ---- oracle
     o_keys, o_vals, o_blob = oracle.encode_batch(og, store.tokens, store.seq_off,
@@ -291,7 +292,7 @@ def gpu_merge_runs(ctx, runs):
             host(ov, VAL_DTYPE, total * 16)[:m].copy())
 
 
-def roundtrip_xp12(g: lsmkv.Geom, store, query, seed=0):
+def roundtrip_xp12(g: lsmkv.Geom, store, query, seed=0, tuning=None):
     """Whole path with the compressing codec: encode, flush on the device, probe, decode into a
     zeroed pool; every output against the oracle's."""
     og = ogeom(g)
@@ -302,10 +303,11 @@ def roundtrip_xp12(g: lsmkv.Geom, store, query, seed=0):
     n = int(coff[-1])
     qoff = synth.offsets(synth.chunk_counts(query.seq_off, C))
     nq = int(qoff[-1])
-    num_pages = max(n, nq) + 3
+    m = g.pages_per_chunk
+    num_pages = max(n, nq) * m + 3
     pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
-    src_pages = synth.random_pages(rng, num_pages, n)
-    dst_pages = synth.random_pages(rng, num_pages, nq)
+    src_pages = synth.random_pages(rng, num_pages, n * m)
+    dst_pages = synth.random_pages(rng, num_pages, nq * m)
     o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, store.tokens, store.seq_off, None, coff,
                                                       src_pages, pool_np, 0, 0)
     o_run = oracle.flush(o_keys, o_vals)
@@ -313,6 +315,8 @@ def roundtrip_xp12(g: lsmkv.Geom, store, query, seed=0):
     o_dst = np.zeros_like(pool_np)
     oracle.decode_batch_xp12(og, qoff, o_hit, o_recs, [o_blob], dst_pages, o_dst)
     with lsmkv.Context(g, 0) as ctx:
+        for k, v in (tuning or {}).items():
+            ctx.set_tuning(k, v)
         pool = DevPool(g, num_pages, pool_np)
         bound = ctx.encode_bound(n)
         d_keys = torch.zeros(n * 32, dtype=torch.uint8, device=DEV)

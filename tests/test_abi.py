@@ -50,7 +50,7 @@ def test_host_argument_validation_needs_no_gpu():
     assert L.lsmkv_destroy(None) == 0
     assert L.lsmkv_create(None, None, 0) == lsmkv.EINVAL
     h = ctypes.c_void_p()
-    bad = lsmkv.Geom(4, 8, 128, page_tokens=16, chunk_tokens=32).c()     # C != P
+    bad = lsmkv.Geom(4, 8, 128, page_tokens=16, chunk_tokens=40).c()     # C not a multiple of P
     assert L.lsmkv_create(ctypes.byref(h), ctypes.byref(bad), 0) == lsmkv.EINVAL
     bad = lsmkv.Geom(4, 1, 3, elem_bytes=2, page_tokens=1, chunk_tokens=1).c()  # 6-byte pages
     assert L.lsmkv_create(ctypes.byref(h), ctypes.byref(bad), 0) == lsmkv.EINVAL

@@ -18,16 +18,22 @@ def pinned(a: np.ndarray) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a).view(np.uint8).reshape(-1).copy()).pin_memory()
 
 
+# the same 16 KiB chunks made of two 8-token pages each
+G2 = lsmkv.Geom(n_layers=2, n_kv_heads=2, head_dim=64, page_tokens=8, chunk_tokens=16)
+
+
 @pytest.mark.parametrize("use_pinned", [False, True])
 @pytest.mark.parametrize("stage", [1 << 20, 1 << 30])     # 1 MiB: many slices; 1 GiB: one slice
-def test_put_probe_decode_through_host_buffers(use_pinned, stage):
-    g, og = G, H.ogeom(G)
+@pytest.mark.parametrize("g", [G, G2], ids=["one-page-chunks", "two-page-chunks"])
+def test_put_probe_decode_through_host_buffers(use_pinned, stage, g):
+    og = H.ogeom(g)
     cb = g.chunk_bytes
+    m = g.pages_per_chunk
     rng = np.random.default_rng(11)
     w1 = synth.llama_requests(n_req=30, min_len=100, max_len=900, config_id=71)
     w2 = synth.llama_requests(n_req=17, min_len=100, max_len=900, config_id=72)
     start2 = rng.integers(0, 10, w2.batch.n).astype(np.uint32)
-    num_pages = 2500
+    num_pages = 2500 * m
     pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
 
     def sizes(b, start):
@@ -42,7 +48,7 @@ def test_put_probe_decode_through_host_buffers(use_pinned, stage):
         for fid, (b, start) in enumerate(((w1.batch, None), (w2.batch, start2))):
             coff = sizes(b, start)
             n = int(coff[-1])
-            pages = synth.random_pages(rng, num_pages, n)
+            pages = synth.random_pages(rng, num_pages, n * m)
             o_keys, o_vals, o_blob = oracle.encode_batch(og, b.tokens, b.seq_off, start, coff,
                                                          pages, pool_np, fid, 4096 * fid)
             keys = np.zeros((n, 4), np.uint64)
@@ -87,7 +93,7 @@ def test_put_probe_decode_through_host_buffers(use_pinned, stage):
         assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
         assert np.array_equal(qkeys, o_qkeys) and o_hit.sum() > 500
         # decode from the host arenas (two files) into a zeroed pool
-        dst_pages = synth.random_pages(rng, num_pages, total)
+        dst_pages = synth.random_pages(rng, num_pages, total * m)
         o_dst = np.zeros_like(pool_np)
         oracle.decode_batch(og, qoff, o_hit, o_recs, arenas_np, dst_pages, o_dst)
         dst = H.DevPool(g, num_pages)
