@@ -227,6 +227,33 @@ int lsmkv_merge_runs(lsmkv_ctx *ctx, void *stream, const lsmkv_run_t *runs, uint
                      lsmkv_key_t *keys_out, lsmkv_val_t *vals_out, uint64_t *n_out);
 
 /*
+ * Compaction policy (Sec. 2.2 "LSM-Tree Structure": levels whose capacities grow by a size ratio
+ * T, at most K sorted runs per level; K = 1 is leveling, K = T - 1 tiering; Sec. 3.3 and App. C:
+ * T and K change while the store runs and take effect lazily, as data is merged anyway). A pure
+ * host function: it looks at the shape of the index and names the next merge, which the caller
+ * carries out with lsmkv_merge_runs (or lsmkv_xrun_merge) and reports back by calling again.
+ *   level, entries [host, n_runs]: the runs newest first; level[r] >= 1, non-decreasing in r (a
+ *           flushed batch enters level 1); entries[r] = keys in run r
+ *   buffer_entries = M, keys in one flushed batch; level i holds M * T^i keys
+ *   size_ratio = T >= 2, runs_per_level = K >= 1
+ * Starting from the shallowest level, the first level that needs work decides:
+ *   - it holds M * T^i keys or more: all its runs are merged and the result moves to level
+ *     i + 1; if level i + 1 already holds K runs they join the same merge (with K = 1 this is
+ *     leveling's merge into the resident run);
+ *   - else it holds more than K runs: they are merged into one run that stays at level i.
+ * Returns 1 and fills *out (runs [first_run, first_run + n_runs) become one run of level
+ * to_level, at position first_run of the list; n_runs == 1 is a move without a merge), 0 when
+ * nothing is due, LSMKV_EINVAL for bad arguments. Because T and K come with every call, new
+ * values apply from the next merge on and never force a reorganisation by themselves. With
+ * K = T - 1, distinct keys and batches of M keys the run counts of the levels are the digits of
+ * the number of flushes written in base T.
+ */
+typedef struct { uint32_t first_run, n_runs, to_level, reserved; } lsmkv_compaction_t;
+int lsmkv_plan_compaction(const uint32_t *level, const uint64_t *entries, uint32_t n_runs,
+                          uint64_t buffer_entries, uint32_t size_ratio, uint32_t runs_per_level,
+                          lsmkv_compaction_t *out);
+
+/*
  * Exact prefix index (Sec. 3.1/3.2: keys that keep the structure of token prefixes, so that key
  * order is prefix order). An "xrun" indexes WHOLE stored sequences by their tokens themselves:
  * no digest takes part, so two different prefixes can never be confused. The caller keeps, on

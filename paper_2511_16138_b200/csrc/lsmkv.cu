@@ -1093,6 +1093,52 @@ const char *lsmkv_strerror(int code)
     }
 }
 
+int lsmkv_plan_compaction(const uint32_t *level, const uint64_t *entries, uint32_t n_runs,
+                          uint64_t buffer_entries, uint32_t size_ratio, uint32_t runs_per_level,
+                          lsmkv_compaction_t *out)
+{
+    if (!out || buffer_entries == 0 || size_ratio < 2 || runs_per_level == 0) return LSMKV_EINVAL;
+    if (n_runs && (!level || !entries)) return LSMKV_EINVAL;
+    for (uint32_t r = 0; r < n_runs; ++r)
+        if (level[r] == 0 || (r && level[r] < level[r - 1])) return LSMKV_EINVAL;
+    uint64_t cap = buffer_entries;                      // capacity of level i = M * T^i, saturating
+    uint32_t cap_level = 0;
+    for (uint32_t a = 0; a < n_runs;) {
+        const uint32_t i = level[a];
+        uint32_t b = a;
+        uint64_t sum = 0;
+        while (b < n_runs && level[b] == i) {
+            sum = sum + entries[b] < sum ? UINT64_MAX : sum + entries[b];
+            ++b;
+        }
+        while (cap_level < i) {
+            cap = cap > UINT64_MAX / size_ratio ? UINT64_MAX : cap * size_ratio;
+            ++cap_level;
+        }
+        const uint32_t count = b - a;
+        if (sum >= cap && cap != UINT64_MAX) {          // full: its runs leave for the next level
+            uint32_t c = b;                              // runs of level i + 1
+            while (c < n_runs && level[c] == i + 1) ++c;
+            const bool join = c - b >= runs_per_level;  // one more run would be too many there
+            out->first_run = a;
+            out->n_runs = (join ? c : b) - a;
+            out->to_level = i + 1;
+            return 1;
+        }
+        if (count > runs_per_level) {                   // too many runs: they become one, in place
+            out->first_run = a;
+            out->n_runs = count;
+            out->to_level = i;
+            return 1;
+        }
+        a = b;
+    }
+    out->first_run = 0;
+    out->n_runs = 0;
+    out->to_level = 0;
+    return 0;
+}
+
 int lsmkv_format_version(void) { return LSMKV_FORMAT_VERSION; }
 
 }  // extern "C"

@@ -461,8 +461,8 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
         uint4 *recs = reinterpret_cast<uint4 *>(recs_out + o0);
         uint64_t hit = nch, base = 0;
         bool done = false;
-        // Round 0 is one warp's 32 chunks -- four queries in ten never get past it -- the
-        // later rounds take 32 chunks per warp of the CTA.
+        // Round 0 is one warp's 32 chunks -- a query without a cached prefix never gets past
+        // it -- the later rounds take 32 chunks per warp of the CTA.
         for (unsigned rnd = 0; base < nch; ++rnd) {
             const unsigned wact = (rnd == 0 && !keys_out) ? 1u : W;
             const uint64_t span = 32ull * wact;

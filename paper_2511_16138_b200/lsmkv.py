@@ -26,7 +26,7 @@ EXPORTS = (
     "lsmkv_decode_batch_static", "lsmkv_flush_batch", "lsmkv_merge_runs",
     "lsmkv_put_batch_host", "lsmkv_probe_batch_host", "lsmkv_decode_batch_host",
     "lsmkv_bloom_blocks", "lsmkv_bloom_build", "lsmkv_encode_bound", "lsmkv_last_cuda_line",
-    "lsmkv_hindex_buckets", "lsmkv_hindex_build", "lsmkv_xrun_merge",
+    "lsmkv_hindex_buckets", "lsmkv_hindex_build", "lsmkv_xrun_merge", "lsmkv_plan_compaction",
     "lsmkv_relocate_records", "lsmkv_xrun_build", "lsmkv_xprobe_batch",
 )
 ST_OVERFLOW = 32
@@ -75,6 +75,11 @@ def _run_array(runs):
         if len(r) > 5 and r[5] is not None:
             arr[i].hindex, arr[i].hindex_buckets = _ptr(r[5]), r[6]
     return arr
+
+
+class CompactionStruct(C.Structure):
+    _fields_ = [("first_run", C.c_uint32), ("n_runs", C.c_uint32), ("to_level", C.c_uint32),
+                ("reserved", C.c_uint32)]
 
 
 class PoolStruct(C.Structure):
@@ -169,6 +174,8 @@ def lib() -> C.CDLL:
     L.lsmkv_relocate_records.argtypes = [vp, vp, vp, u64, C.POINTER(RelocStruct), u32, vp]
     L.lsmkv_xrun_build.restype = C.c_int
     L.lsmkv_xrun_build.argtypes = [vp, vp, vp, vp, u32, vp, vp]
+    L.lsmkv_plan_compaction.restype = C.c_int
+    L.lsmkv_plan_compaction.argtypes = [vp, vp, u32, u64, u32, u32, vp]
     L.lsmkv_xrun_merge.restype = C.c_int
     L.lsmkv_xrun_merge.argtypes = [vp, vp, vp, vp, vp, u32, vp, u32, vp, vp]
     L.lsmkv_xprobe_batch.restype = C.c_int
@@ -398,6 +405,21 @@ def lsmkv_encode_bound(ctx, n_chunks: int) -> int:
 
 def lsmkv_bloom_blocks(n: int) -> int:
     return int(lib().lsmkv_bloom_blocks(n))
+
+
+def lsmkv_plan_compaction(levels, entries, buffer_entries: int, size_ratio: int,
+                          runs_per_level: int):
+    """Next merge the (T, K) policy asks for: (first_run, n_runs, to_level), or None when the
+    index is in shape. levels / entries describe the runs newest first (host sequences)."""
+    n = len(levels)
+    lv = (C.c_uint32 * max(1, n))(*[int(x) for x in levels])
+    en = (C.c_uint64 * max(1, n))(*[int(x) for x in entries])
+    out = CompactionStruct()
+    rc = lib().lsmkv_plan_compaction(lv, en, n, buffer_entries, size_ratio, runs_per_level,
+                                     C.byref(out))
+    if rc < 0:
+        raise LsmkvError(rc, "lsmkv_plan_compaction")
+    return (out.first_run, out.n_runs, out.to_level) if rc == 1 else None
 
 
 def lsmkv_hindex_buckets(n: int) -> int:
