@@ -471,28 +471,29 @@ k_xp_measure_fast(const __grid_constant__ XpJob job)
         uint4 q[SWEEPS];
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) q[s] = __ldcs(s4 + s * 32);
+        // exponent fields stay where they are (bits 7..14 of each half); the largest per half
+        // comes from the two-halves maximum instruction
         uint32_t m = 0;
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
-            const uint32_t w[4] = {q[s].x, q[s].y, q[s].z, q[s].w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const uint32_t a = w[k] & 0x7F807F80u;
-                m = max(m, max(a & 0xFFFFu, a >> 16));
-            }
+            m = __vimax3_u16x2(m, q[s].x & 0x7F807F80u, q[s].y & 0x7F807F80u);
+            m = __vimax3_u16x2(m, q[s].z & 0x7F807F80u, q[s].w & 0x7F807F80u);
         }
+        m = max(m & 0xFFFFu, m >> 16);
         const uint32_t emax = block_max(m, sh) >> 7;
         const uint32_t base = emax > 14u ? emax - 14u : 0u;
-        const uint32_t base2 = base | (base << 16);
-        uint32_t in_win = 0;
+        // per half: field + 0x8000 - (base << 7) has bit 15 set exactly when e >= base, and never
+        // carries into the other half (field <= 0x7F80); the bits are summed per half
+        const uint32_t lift = 0x80008000u - ((base | (base << 16)) << 7);
+        uint32_t acc = 0;
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
-            uint32_t d;
-            in_win += __popc(xpfast::in_window2(q[s].x, base2, d)) +
-                      __popc(xpfast::in_window2(q[s].y, base2, d)) +
-                      __popc(xpfast::in_window2(q[s].z, base2, d)) +
-                      __popc(xpfast::in_window2(q[s].w, base2, d));
+            acc += (((q[s].x & 0x7F807F80u) + lift) & 0x80008000u) >> 15;
+            acc += (((q[s].y & 0x7F807F80u) + lift) & 0x80008000u) >> 15;
+            acc += (((q[s].z & 0x7F807F80u) + lift) & 0x80008000u) >> 15;
+            acc += (((q[s].w & 0x7F807F80u) + lift) & 0x80008000u) >> 15;
         }
+        const uint32_t in_win = (acc & 0xFFFFu) + (acc >> 16);
         const uint32_t cnt = block_sum(8u * SWEEPS - in_win, sh);
         if (threadIdx.x == 0) {
             const bool packed = cnt < job.n_elems / 2;
@@ -506,7 +507,7 @@ k_xp_measure_fast(const __grid_constant__ XpJob job)
 
 // dynamic shared memory: n_elems bytes (per-warp exception lists) 
 template <int SWEEPS>
-__global__ void __launch_bounds__(kXpThreads)
+__global__ void __launch_bounds__(kXpThreads, SWEEPS <= 8 ? 4 : 2)
 k_xp_pack_fast(const __grid_constant__ XpJob job)
 {
     extern __shared__ __align__(16) unsigned char xp_smem[];
@@ -518,35 +519,40 @@ k_xp_pack_fast(const __grid_constant__ XpJob job)
     for (uint64_t u = blockIdx.x; u < total; u += gridDim.x) {
         const uint64_t i = u / slabs;
         const uint32_t b = (uint32_t)(u - i * slabs);
+        // The slab's loads go out first: where it lands (offsets, directory) is a chain of small
+        // dependent loads of its own, which then overlaps with the data on its way.
+        const unsigned char *src = xp_src(job, i, b, false);
+        const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+        const uint32_t k_first = warp * SWEEPS * 32 + lane;       // this lane's first uint4
+        uint4 qs[SWEEPS];                                         // all loads in flight at once
+        if (src) {
+#pragma unroll
+            for (int s = 0; s < SWEEPS; ++s) qs[s] = __ldcs(s4 + k_first + s * 32);
+        }
         const uint64_t off = job.chunk_off[i], csize = job.chunk_off[i + 1] - off;
-        if (off + csize > job.blob_capacity || csize > 0xFFFFFFFFull) continue;
         const uint32_t info = job.slab_info[u], size = job.slab_size[u];
+        if (off + csize > job.blob_capacity || csize > 0xFFFFFFFFull) continue;
         const uint32_t *dir = reinterpret_cast<const uint32_t *>(job.blob + off);
         unsigned char *out = job.blob + off + dir[b];
-        const unsigned char *src = info == 0xFFFFu ? nullptr : xp_src(job, i, b, false);
-        if (!src) {
+        if (!src || info == 0xFFFFu) {
             uint4 *o4 = reinterpret_cast<uint4 *>(out);
             for (uint32_t k = threadIdx.x; k < size / 16; k += kXpThreads)
                 o4[k] = k == 0 ? make_uint4(kXpMagic, 0, 1u << 8, size) : make_uint4(0, 0, 0, 0);
             continue;
         }
-        const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
         const uint32_t mode = (info >> 8) & 0xFFu, base = info & 0xFFu;
         if (threadIdx.x == 0)
             *reinterpret_cast<uint4 *>(out) =
                 make_uint4(kXpMagic, job.slab_nexc[u], base | (mode << 8), size);
         if (mode == 1) {
-            uint4 *o4 = reinterpret_cast<uint4 *>(out + 16);
-            for (uint32_t k = threadIdx.x; k < n8; k += kXpThreads) __stcs(o4 + k, __ldcs(s4 + k));
+            uint4 *o4 = reinterpret_cast<uint4 *>(out + 16) + k_first;
+#pragma unroll
+            for (int s = 0; s < SWEEPS; ++s) __stcs(o4 + s * 32, qs[s]);
             continue;
         }
         unsigned char *sm = out + 16, *codes = sm + N, *exc = codes + N / 2;
         const uint32_t base2 = base | (base << 16);
-        const uint32_t k_first = warp * SWEEPS * 32 + lane;       // this lane's first uint4
         uint32_t warp_count = 0;
-        uint4 qs[SWEEPS];                                         // all loads in flight at once
-#pragma unroll
-        for (int s = 0; s < SWEEPS; ++s) qs[s] = __ldcs(s4 + k_first + s * 32);
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
             const uint32_t k = k_first + s * 32;
