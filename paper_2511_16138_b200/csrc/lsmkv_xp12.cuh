@@ -512,7 +512,7 @@ k_xp_pack_fast(const __grid_constant__ XpJob job)
 {
     extern __shared__ __align__(16) unsigned char xp_smem[];
     __shared__ uint32_t warp_total[kXpThreads / 32];
-    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, N = job.n_elems, n8 = N >> 3;
+    const uint32_t slabs = 2u * job.n_layers * job.pages_per_chunk, N = job.n_elems;
     const uint64_t total = job.n_chunks * slabs;
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char *my_list = xp_smem + (size_t)warp * (N / 8);
@@ -622,6 +622,21 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
                   (d0 & 15u) == 0 && d1 - d0 >= 16u;
         uint4 h = make_uint4(0, 0, 0, 0);
         if (ok) h = __ldg(reinterpret_cast<const uint4 *>(blob + d0));
+        // The packed planes are fetched together with the header rather than after it: every
+        // well-formed slab is at least 16 + 1.5 N bytes long, so whenever the directory grants
+        // that much the loads stay inside the slab, whatever the header turns out to say.
+        const unsigned char *in = blob + d0 + 16;
+        const uint32_t k_first = warp * SWEEPS * 32 + lane;
+        uint2 sms[SWEEPS];                                       // all loads in flight at once
+        uint32_t cds[SWEEPS];
+        const bool early = ok && d1 - d0 >= 16u + N + N / 2;
+        if (early) {
+#pragma unroll
+            for (int s = 0; s < SWEEPS; ++s) {
+                sms[s] = __ldcs(reinterpret_cast<const uint2 *>(in + 8ull * (k_first + s * 32)));
+                cds[s] = __ldcs(reinterpret_cast<const uint32_t *>(in + N + 4ull * (k_first + s * 32)));
+            }
+        }
         const uint32_t mode = (h.z >> 8) & 0xFFu, base = h.z & 0xFFu, n_exc = h.y;
         ok = ok && h.x == kXpMagic && h.w == d1 - d0 &&
              ((mode == 1 && h.w == 16u + 2u * N) ||
@@ -639,22 +654,14 @@ k_xp_unpack_fast(const __grid_constant__ XpUnpackJob job, const __grid_constant_
             continue;
         }
         uint4 *dst = reinterpret_cast<uint4 *>(pool_buf + page * (uint64_t)job.page_bytes);
-        const unsigned char *in = blob + d0 + 16;
+        if (mode == 0 && !early) continue;                       // cannot happen: see above
         if (mode == 1) {
             const uint4 *s4 = reinterpret_cast<const uint4 *>(in);
             for (uint32_t k = threadIdx.x; k < n8; k += kXpThreads) __stcs(dst + k, __ldcs(s4 + k));
             continue;
         }
-        const unsigned char *sm = in, *codes = in + N, *exc = codes + N / 2;
-        const uint32_t k_first = warp * SWEEPS * 32 + lane;
+        const unsigned char *exc = in + N + N / 2;
         const uint32_t base2 = base | (base << 16);
-        uint2 sms[SWEEPS];                                       // all loads in flight at once
-        uint32_t cds[SWEEPS];
-#pragma unroll
-        for (int s = 0; s < SWEEPS; ++s) {
-            sms[s] = __ldcs(reinterpret_cast<const uint2 *>(sm + 8ull * (k_first + s * 32)));
-            cds[s] = __ldcs(reinterpret_cast<const uint32_t *>(codes + 4ull * (k_first + s * 32)));
-        }
         // exceptions before this warp's segment (only when the slab has any)
         uint32_t at_warp = 0;
         if (n_exc) {                                             // uniform over the CTA
