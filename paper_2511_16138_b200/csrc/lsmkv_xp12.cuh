@@ -398,30 +398,30 @@ namespace xpfast {
 
 constexpr uint32_t kOnes2 = 0x00010001u;
 
-// per 32-bit word (two elements): bit 0 / bit 16 set where the element's exponent is >= base
-__device__ __forceinline__ uint32_t in_window2(uint32_t w, uint32_t base2, uint32_t &d)
+// The exponent fields are tested and rebased where they sit (bits 7..14 of each half of a word):
+// with lift = 0x8000 - (base << 7) per half, field + lift has bit 15 set exactly when e >= base,
+// carries e - base in bits 7..10 then, and never spills into the other half (field <= 0x7F80).
+__device__ __forceinline__ uint32_t window_lift(uint32_t base)
 {
-    d = ((w >> 7) & 0x00FF00FFu) + 0x01000100u - base2;      // per half: 256 + e - base, no borrow
-    return (d >> 8) & kOnes2;
+    return 0x80008000u - ((base | (base << 16)) << 7);
 }
 
-// sign+mantissa bytes of four words -> two packed words
+// sign+mantissa bytes of four words -> two packed words (only bytes 0 and 2 of a t survive)
 __device__ __forceinline__ uint2 sm_bytes(const uint4 &q)
 {
-    const uint32_t t0 = ((q.x >> 8) & 0x00800080u) | (q.x & 0x007F007Fu);
-    const uint32_t t1 = ((q.y >> 8) & 0x00800080u) | (q.y & 0x007F007Fu);
-    const uint32_t t2 = ((q.z >> 8) & 0x00800080u) | (q.z & 0x007F007Fu);
-    const uint32_t t3 = ((q.w >> 8) & 0x00800080u) | (q.w & 0x007F007Fu);
+    const uint32_t t0 = (q.x & 0x007F007Fu) | ((q.x >> 8) & 0xFF80FF80u);
+    const uint32_t t1 = (q.y & 0x007F007Fu) | ((q.y >> 8) & 0xFF80FF80u);
+    const uint32_t t2 = (q.z & 0x007F007Fu) | ((q.z >> 8) & 0xFF80FF80u);
+    const uint32_t t3 = (q.w & 0x007F007Fu) | ((q.w >> 8) & 0xFF80FF80u);
     return make_uint2(__byte_perm(t0, t1, 0x6420), __byte_perm(t2, t3, 0x6420));
 }
 
 // code byte (two nibbles) of one word; exc gets bit 0 / bit 16 for elements below the window
-__device__ __forceinline__ uint32_t code_byte(uint32_t w, uint32_t base2, uint32_t &exc)
+__device__ __forceinline__ uint32_t code_byte(uint32_t w, uint32_t lift, uint32_t &exc)
 {
-    uint32_t d;
-    const uint32_t ok = in_window2(w, base2, d);
-    exc = ok ^ kOnes2;
-    const uint32_t c2 = (d & (ok * 15u)) | (exc * 15u);
+    const uint32_t t = (w & 0x7F807F80u) + lift;
+    exc = ((t >> 15) & kOnes2) ^ kOnes2;
+    const uint32_t c2 = ((t >> 7) & 0x000F000Fu) | (exc * 15u);   // e - base (< 15), or 15
     return (c2 | (c2 >> 12)) & 0xFFu;
 }
 
@@ -482,9 +482,8 @@ k_xp_measure_fast(const __grid_constant__ XpJob job)
         m = max(m & 0xFFFFu, m >> 16);
         const uint32_t emax = block_max(m, sh) >> 7;
         const uint32_t base = emax > 14u ? emax - 14u : 0u;
-        // per half: field + 0x8000 - (base << 7) has bit 15 set exactly when e >= base, and never
-        // carries into the other half (field <= 0x7F80); the bits are summed per half
-        const uint32_t lift = 0x80008000u - ((base | (base << 16)) << 7);
+        // bit 15 of field + lift says "in the window"; the bits are summed per half
+        const uint32_t lift = xpfast::window_lift(base);
         uint32_t acc = 0;
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
@@ -551,17 +550,17 @@ k_xp_pack_fast(const __grid_constant__ XpJob job)
             continue;
         }
         unsigned char *sm = out + 16, *codes = sm + N, *exc = codes + N / 2;
-        const uint32_t base2 = base | (base << 16);
+        const uint32_t lift = xpfast::window_lift(base);
         uint32_t warp_count = 0;
 #pragma unroll
         for (int s = 0; s < SWEEPS; ++s) {
             const uint32_t k = k_first + s * 32;
             const uint4 q = qs[s];
             uint32_t x0, x1, x2, x3;
-            const uint32_t c32 = xpfast::code_byte(q.x, base2, x0) |
-                                 (xpfast::code_byte(q.y, base2, x1) << 8) |
-                                 (xpfast::code_byte(q.z, base2, x2) << 16) |
-                                 (xpfast::code_byte(q.w, base2, x3) << 24);
+            const uint32_t c32 = xpfast::code_byte(q.x, lift, x0) |
+                                 (xpfast::code_byte(q.y, lift, x1) << 8) |
+                                 (xpfast::code_byte(q.z, lift, x2) << 16) |
+                                 (xpfast::code_byte(q.w, lift, x3) << 24);
             __stcs(reinterpret_cast<uint2 *>(sm + 8ull * k), xpfast::sm_bytes(q));
             __stcs(reinterpret_cast<uint32_t *>(codes + 4ull * k), c32);
             const uint32_t any = x0 | x1 | x2 | x3;
