@@ -171,3 +171,33 @@ def test_launch_shapes_do_not_change_results(tuning):
     w = synth.long_context(n_req=5, seq_len=16 * 530 + 7, shared=16 * 200, n_mutate=16 * 40 + 3)
     start = np.array([0, 3, 200, 529, 600], dtype=np.uint32)
     H.roundtrip(g, w.store, w.query, start_chunk=start, n_runs=3, tuning=tuning, seed=17)
+
+
+def test_more_queries_than_the_hand_out_order_covers():
+    """Batches beyond 65 536 queries are handed out in their given order (no length sort): the
+    answers must not depend on which of the two the probe does."""
+    g = lsmkv.Geom(1, 1, 8, elem_bytes=2, page_tokens=4, chunk_tokens=4)
+    og = H.ogeom(g)
+    rng = np.random.default_rng(21)
+    stored = [rng.integers(0, 3, int(rng.integers(4, 40)), dtype=np.uint32) for _ in range(300)]
+    store = synth.make_batch(stored)
+    coff = synth.offsets(synth.chunk_counts(store.seq_off, 4))
+    n_q = 70_000
+    lens = rng.integers(0, 30, n_q)
+    toks = rng.integers(0, 3, int(lens.sum()), dtype=np.uint32)
+    q_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.uint64)
+    # every third query starts with a stored sequence
+    for i in range(0, n_q, 3):
+        s = stored[i % len(stored)]
+        m = min(len(s), int(lens[i]))
+        toks[int(q_off[i]):int(q_off[i]) + m] = s[:m]
+    query = synth.Batch(toks, q_off)
+    qoff = synth.offsets(synth.chunk_counts(query.seq_off, 4))
+    with lsmkv.Context(g, 0) as ctx:
+        keys, vals, _, _ = H.gpu_encode(ctx, g, store, None, coff, None, None)
+        run = H.gpu_flush_run(ctx, keys, vals)
+        o_hit, o_recs, _, _ = oracle.probe_batch(og, query.tokens, query.seq_off, qoff, [run])
+        hit, recs, _, _ = H.gpu_probe(ctx, query, qoff, [run], want_keys=False)
+        assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
+        assert 10_000 < int((o_hit > 0).sum()) < n_q
+        assert ctx.last_status()["flags"] == 0
