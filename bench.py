@@ -874,9 +874,12 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
         tv = torch.empty(n * 16, dtype=torch.uint8, device=dev)
         tn = torch.zeros(1, dtype=torch.int64, device=dev)
         ctx.flush_batch(dk, dv, n, tk, tv, tn, stream=stream)
+        nb = lsmkv.lsmkv_hindex_buckets(n)
+        hx = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+        ctx.hindex_build(tk, n, hx, stream=stream)
         torch.cuda.synchronize()
-        p["run_t"] = (tk, tv, tn)
-        p["runs"] = [(tk, tv, n)]
+        p["run_t"] = (tk, tv, tn, hx)
+        p["runs"] = [(tk, tv, n, None, 0, hx, nb)]
     h2d = d2h = moved = 0
     put_done = [torch.cuda.Event() for _ in range(NS)]
     slot_free = [torch.cuda.Event() for _ in range(NS)]
