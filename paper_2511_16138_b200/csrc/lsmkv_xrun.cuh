@@ -23,24 +23,46 @@ __device__ __forceinline__ SeqView seq_view(const uint32_t *__restrict__ tokens,
     return SeqView{tokens + a, b >= a ? b - a : 0};
 }
 
+// One comparison step of warp_lcp: tokens [i, i + 32 * kUnroll) of a and b, all loads in flight at
+// once. Returns the position of the first difference, or ~0 if there is none below n.
+template <int kUnroll>
+__device__ __forceinline__ uint64_t lcp_step(const SeqView &a, const SeqView &b, uint64_t i,
+                                             uint64_t n)
+{
+    const unsigned lane = lane_id();
+    bool differ[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const uint64_t k = i + 32u * u + lane;
+        differ[u] = k < n && __ldg(a.tok + k) != __ldg(b.tok + k);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, differ[u]);
+        if (m) return i + 32u * u + (unsigned)__ffs(m) - 1u;
+    }
+    return ~0ull;
+}
+
 // Warp-cooperative: length of the common token prefix of a and b, starting the comparison at
 // `from` (the caller knows the first `from` tokens agree). Every lane returns the same value.
+// Steps of 128 tokens; with kWiden, a comparison that is still running after two of them goes on
+// in steps of 512 (a step costs one memory round trip whatever its width, most comparisons end
+// in their first step, and the few long ones are what the probe waits for).
+template <bool kWiden>
 __device__ __forceinline__ uint64_t warp_lcp(const SeqView &a, const SeqView &b, uint64_t from)
 {
-    constexpr int kUnroll = 4;                   // 128 tokens per step, all loads in flight at once
     const uint64_t n = a.len < b.len ? a.len : b.len;
-    const unsigned lane = lane_id();
-    for (uint64_t i = from; i < n; i += 32 * kUnroll) {
-        bool differ[kUnroll];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const uint64_t k = i + 32u * u + lane;
-            differ[u] = k < n && __ldg(a.tok + k) != __ldg(b.tok + k);
-        }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, differ[u]);
-            if (m) return i + 32u * u + (unsigned)__ffs(m) - 1u;
+    uint64_t i = from;
+    for (int step = 0; i < n; ++step) {
+        if (kWiden && step >= 2) {
+            const uint64_t r = lcp_step<16>(a, b, i, n);
+            if (r != ~0ull) return r;
+            i += 512;
+        } else {
+            const uint64_t r = lcp_step<4>(a, b, i, n);
+            if (r != ~0ull) return r;
+            i += 128;
         }
     }
     return n;
@@ -71,7 +93,7 @@ __device__ __forceinline__ Located warp_locate(const SeqView &x, uint32_t x_id,
         const uint32_t y = __ldg(order + m);
         const SeqView vy = seq_view(tokens, seq_off, y);
         const uint64_t from = r.have_lo && r.have_hi ? (r.l_lo < r.l_hi ? r.l_lo : r.l_hi) : 0;
-        const uint64_t l = warp_lcp(vy, x, from);
+        const uint64_t l = warp_lcp<false>(vy, x, from);
         // y ends at l: a prefix of x (below) or the same tokens (the numbers decide)
         const bool above = l < vy.len ? (l >= x.len || __ldg(vy.tok + l) > __ldg(x.tok + l))
                                       : (vy.len == x.len && y > x_id);
@@ -174,7 +196,7 @@ struct XRunTable {
 // One warp per query. Per run, newest first: the position of the query among the sorted stored
 // sequences; the longer of the prefixes shared with the two neighbours is the longest prefix
 // shared with anything in the run, and that neighbour (the lower one on a tie) lends its records.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint32_t n_query,
          const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
          const uint64_t *__restrict__ qchunk_off, uint64_t n_qchunks,
@@ -210,7 +232,7 @@ k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint
                 const SeqView vy = seq_view(rt.tokens[r], rt.seq_off[r], y);
                 // everything between the bounds shares at least min(l_lo, l_hi) tokens with Q
                 const uint64_t from = have_lo && have_hi ? (l_lo < l_hi ? l_lo : l_hi) : 0;
-                const uint64_t l = warp_lcp(vy, Q, from);
+                const uint64_t l = warp_lcp<true>(vy, Q, from);
                 const bool above = l < vy.len && (l >= Q.len || __ldg(vy.tok + l) > __ldg(Q.tok + l));
                 if (above) { hi = m; l_hi = l; s_hi = y; have_hi = true; }
                 else { lo = m + 1; l_lo = l; s_lo = y; have_lo = true; }
