@@ -93,7 +93,7 @@ __device__ __forceinline__ Located warp_locate(const SeqView &x, uint32_t x_id,
         const uint32_t y = __ldg(order + m);
         const SeqView vy = seq_view(tokens, seq_off, y);
         const uint64_t from = r.have_lo && r.have_hi ? (r.l_lo < r.l_hi ? r.l_lo : r.l_hi) : 0;
-        const uint64_t l = warp_lcp<false>(vy, x, from);
+        const uint64_t l = warp_lcp<true>(vy, x, from);
         // y ends at l: a prefix of x (below) or the same tokens (the numbers decide)
         const bool above = l < vy.len ? (l >= x.len || __ldg(vy.tok + l) > __ldg(x.tok + l))
                                       : (vy.len == x.len && y > x_id);
@@ -120,7 +120,7 @@ k_xrun_init(const uint64_t *__restrict__ seq_off, uint32_t n_seq, uint32_t C,
 // One merge level over sequence ids, one warp per element: its rank among the sibling segment
 // comes from a binary search with the token comparison. The order is total (ties by id), so the
 // two halves never hold equal elements.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_xrun_merge_level(const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
                    const uint32_t *__restrict__ src, uint32_t *__restrict__ dst, uint64_t n,
                    uint64_t width)
@@ -142,7 +142,7 @@ k_xrun_merge_level(const uint32_t *__restrict__ tokens, const uint64_t *__restri
 
 // Merge of two sorted runs that share one arena: src[0, mid) and src[mid, n) are each in token
 // order; one warp per element finds its rank in the other part, as in a merge level.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_xrun_merge_two(const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
                  const uint32_t *__restrict__ src, uint32_t *__restrict__ dst, uint64_t n,
                  uint64_t mid)
