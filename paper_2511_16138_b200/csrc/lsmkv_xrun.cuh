@@ -46,16 +46,16 @@ __device__ __forceinline__ uint64_t lcp_step(const SeqView &a, const SeqView &b,
 
 // Warp-cooperative: length of the common token prefix of a and b, starting the comparison at
 // `from` (the caller knows the first `from` tokens agree). Every lane returns the same value.
-// Steps of 128 tokens; with kWiden, a comparison that is still running after two of them goes on
-// in steps of 512 (a step costs one memory round trip whatever its width, most comparisons end
-// in their first step, and the few long ones are what the probe waits for).
-template <bool kWiden>
+// Steps of 128 tokens; a comparison that is still running after two of them goes on in steps of
+// 512 (a step costs one memory round trip whatever its width, most comparisons end in their
+// first step, and the few long ones are what the sort and the probe wait for). The wide step
+// needs registers: the kernels that call this allow themselves 128.
 __device__ __forceinline__ uint64_t warp_lcp(const SeqView &a, const SeqView &b, uint64_t from)
 {
     const uint64_t n = a.len < b.len ? a.len : b.len;
     uint64_t i = from;
     for (int step = 0; i < n; ++step) {
-        if (kWiden && step >= 2) {
+        if (step >= 2) {
             const uint64_t r = lcp_step<16>(a, b, i, n);
             if (r != ~0ull) return r;
             i += 512;
@@ -93,7 +93,7 @@ __device__ __forceinline__ Located warp_locate(const SeqView &x, uint32_t x_id,
         const uint32_t y = __ldg(order + m);
         const SeqView vy = seq_view(tokens, seq_off, y);
         const uint64_t from = r.have_lo && r.have_hi ? (r.l_lo < r.l_hi ? r.l_lo : r.l_hi) : 0;
-        const uint64_t l = warp_lcp<true>(vy, x, from);
+        const uint64_t l = warp_lcp(vy, x, from);
         // y ends at l: a prefix of x (below) or the same tokens (the numbers decide)
         const bool above = l < vy.len ? (l >= x.len || __ldg(vy.tok + l) > __ldg(x.tok + l))
                                       : (vy.len == x.len && y > x_id);
@@ -232,7 +232,7 @@ k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint
                 const SeqView vy = seq_view(rt.tokens[r], rt.seq_off[r], y);
                 // everything between the bounds shares at least min(l_lo, l_hi) tokens with Q
                 const uint64_t from = have_lo && have_hi ? (l_lo < l_hi ? l_lo : l_hi) : 0;
-                const uint64_t l = warp_lcp<true>(vy, Q, from);
+                const uint64_t l = warp_lcp(vy, Q, from);
                 const bool above = l < vy.len && (l >= Q.len || __ldg(vy.tok + l) > __ldg(Q.tok + l));
                 if (above) { hi = m; l_hi = l; s_hi = y; have_hi = true; }
                 else { lo = m + 1; l_lo = l; s_lo = y; have_lo = true; }
