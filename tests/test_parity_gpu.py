@@ -201,3 +201,13 @@ def test_more_queries_than_the_hand_out_order_covers():
         assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
         assert 10_000 < int((o_hit > 0).sum()) < n_q
         assert ctx.last_status()["flags"] == 0
+
+
+@pytest.mark.parametrize("n_runs", [5, 11, 64])
+def test_many_runs_are_searched_in_groups_newest_first(n_runs):
+    """More runs than one lock-step group holds (4), up to the most a probe accepts; keys are
+    dealt to the runs at random, so a query's chunks are answered by many different runs."""
+    g = lsmkv.Geom(1, 2, 32, elem_bytes=2, page_tokens=8, chunk_tokens=8)
+    w = synth.tiny_codec(n_req=10, seq_len=8 * 50 + 3, max_shared=200, n_mutate=40, config_id=60)
+    out = H.roundtrip(g, w.store, w.query, n_runs=n_runs, seed=n_runs)
+    assert np.array_equal(out["hit"], w.expected_hit_tokens // 8)
