@@ -900,11 +900,25 @@ int lsmkv_xprobe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uin
     }
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the probe's scratch: [0] = work counter, then the hand-out order (longest query first)
+    const bool ordered = n_query > 1 && n_query <= kOrderMaxQueries;
+    {
+        int rc = ensure_dir(ctx, 2 + (ordered ? ((uint64_t)n_query + 1) / 2 : 0));
+        if (rc != LSMKV_OK) return rc;
+    }
+    unsigned long long *next_query = reinterpret_cast<unsigned long long *>(ctx->d_dir);
+    uint32_t *order = ordered ? reinterpret_cast<uint32_t *>(ctx->d_dir + 2) : nullptr;
     LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
-    k_xprobe<<<warp_grid(ctx, n_query, 256, 8), 256, 0, s>>>(
+    {
+        RunTable none;
+        std::memset(&none, 0, sizeof(none));
+        k_run_dir<<<1, 256, 0, s>>>(none, 0, ctx->geom.ns, 0, ctx->d_dir + 2, next_query, n_query,
+                                    seq_off, ctx->geom.chunk_tokens, order);
+    }
+    k_xprobe<<<warp_grid(ctx, n_query, 256, 2), 256, 0, s>>>(
         rt, n_runs, ctx->geom.chunk_tokens, n_query, tokens, seq_off, qchunk_off, n_qchunks,
-        hit_chunks_out, recs_out, ctx->d_status);
-    ++ctx->launches;
+        hit_chunks_out, recs_out, ctx->d_status, next_query, order);
+    ctx->launches += 2;
     CU(ctx, cudaGetLastError());
     return LSMKV_OK;
 }

@@ -193,20 +193,26 @@ struct XRunTable {
     uint32_t n_seq[kMaxXRuns];
 };
 
-// One warp per query. Per run, newest first: the position of the query among the sorted stored
+// One warp per query at a time, queries drawn from a counter in the order given (longest first
+// when `order` is set, so that the long comparisons start early and the short queries fill in
+// behind them). Per run, newest first: the position of the query among the sorted stored
 // sequences; the longer of the prefixes shared with the two neighbours is the longest prefix
 // shared with anything in the run, and that neighbour (the lower one on a tie) lends its records.
 __global__ void __launch_bounds__(256, 2)
 k_xprobe(const __grid_constant__ XRunTable rt, uint32_t n_runs, uint32_t C, uint32_t n_query,
          const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
          const uint64_t *__restrict__ qchunk_off, uint64_t n_qchunks,
-         uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out, DevStatus *st)
+         uint32_t *__restrict__ hit_out, lsmkv_val_t *__restrict__ recs_out, DevStatus *st,
+         unsigned long long *next_query, const uint32_t *__restrict__ order)
 {
     const unsigned lane = lane_id();
-    const uint64_t warp0 = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint4 zero = make_uint4(0, 0, 0, 0);
-    for (uint64_t q = warp0; q < n_query; q += n_warps) {
+    for (;;) {
+        unsigned long long t = 0;
+        if (lane == 0) t = atomicAdd(next_query, 1ull);
+        t = __shfl_sync(0xFFFFFFFFu, t, 0);
+        if (t >= n_query) break;
+        const uint64_t q = order ? order[t] : t;
         const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
         const uint64_t nch = s1 >= s0 ? (s1 - s0) / C : 0;
         const uint64_t o0 = qchunk_off[q], o1 = qchunk_off[q + 1];
