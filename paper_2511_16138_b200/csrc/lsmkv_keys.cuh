@@ -2,11 +2,12 @@
 // token prefix, evaluated warp-cooperatively.
 //
 // The digest is defined sequentially (h <- h*B + t + 1 mod p per token). Because
-// H(XY) = H(X) * B^|Y| + H(Y), a warp hashes 32 consecutive chunks at once: every lane runs
-// the recurrence over its own chunk from h = 0, then an inclusive warp scan with the fixed
-// multiplier M = B^C stitches the chunk hashes into prefix hashes, and the running prefix of
-// the previous 32 chunks enters through M^(lane+1). All arithmetic is exact, so the result is
-// bit-identical to the sequential definition.
+// H(XY) = H(X) * B^|Y| + H(Y), a warp hashes 32 consecutive chunks at once: every lane digests
+// its own chunk from h = 0 (16 tokens at a time as one dot product with the powers of B, see
+// block16_dot), then an inclusive warp scan with the fixed multiplier M = B^C stitches the
+// chunk hashes into prefix hashes, and the running prefix of the chunks before enters through
+// M^(lane+1). All arithmetic is exact, so the result is bit-identical to the sequential
+// definition.
 #pragma once
 #include "lsmkv_common.cuh"
 

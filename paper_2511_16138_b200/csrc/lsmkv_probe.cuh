@@ -1,7 +1,8 @@
 // Batched longest-cached-prefix probe.
 //
-// A CTA takes one query at a time. Its W warps hash 32*W consecutive chunks per round (each
-// warp one 32-chunk block; the block digests are chained through shared memory), every lane
+// A CTA takes one query at a time, longest queries first. Its W warps hash 32*W consecutive
+// chunks per round (each warp one 32-chunk block; the block digests are chained through shared
+// memory; the very first round is one warp's 32 chunks), every lane
 // looks its key up in the runs newest -> oldest, a warp ballot finds each warp's first miss and
 // a shared-memory minimum gives the query's. The hit length is the number of leading chunks
 // that were all found (first-miss rule); hashing stops at the round of the first miss unless
@@ -12,7 +13,10 @@
 // runs up front (one binary search per boundary). Inside a bucket keys are ordered by the
 // digest w1, which is uniform on [0, 2^61), so the position is interpolated and pinned by a
 // branch-free binary search over a small window around the guess: ~6 dependent 8-byte loads
-// per run instead of ~20 32-byte ones, with identical control flow across the lanes of a warp.
+// per run instead of ~20 32-byte ones, with identical control flow across the lanes of a warp,
+// the searches of four runs advancing together so that their loads overlap. When every run
+// brings a hash index (k_hidx_build) no search happens at all: one 32-byte bucket per run says
+// where the key is, if anywhere.
 #pragma once
 #include "lsmkv_keys.cuh"
 
