@@ -265,6 +265,22 @@ unsigned merge_grid(const lsmkv_ctx *ctx, uint64_t n)
     return g ? (unsigned)g : 1u;
 }
 
+// Grid of a kernel that strides over its work: no more CTAs than the GPU holds at once (those
+// beyond would only start when others have finished their whole share, and run under-occupied).
+template <typename Kernel>
+unsigned resident_grid(const lsmkv_ctx *ctx, Kernel kern, int threads, size_t smem, uint64_t want)
+{
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem) != cudaSuccess ||
+        per_sm < 1) {
+        cudaGetLastError();
+        per_sm = 1;
+    }
+    const uint64_t cap = (uint64_t)ctx->sm_count * (uint64_t)per_sm;
+    const uint64_t g = want < cap ? want : cap;
+    return g ? (unsigned)g : 1u;
+}
+
 constexpr uint64_t kDirMaxJ = 65536;   // chunk indices covered by the probe's directory
 constexpr uint64_t kOrderMaxQueries = 65536;   // batches up to this size are handed out longest first
 
@@ -359,23 +375,23 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
     job.vals_out = vals_out;
     job.st = ctx->d_status;
     LaunchTimer timer(ctx, s, LSMKV_K_PACK);
-    uint64_t grid = n_chunks * slabs;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 8;
-    if (grid > cap) grid = cap;
+    const uint64_t units = n_chunks * slabs;
     // common slab sizes take the fast kernels (2048 * {4, 8, 16} elements), the rest the generic
     const uint32_t sweeps = job.n_elems % 2048u == 0 && !ctx->xp_generic ? job.n_elems / 2048u : 0;
     const size_t list_bytes = job.n_elems;
-    if (sweeps == 4) k_xp_measure_fast<4><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
-    else if (sweeps == 8) k_xp_measure_fast<8><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
-    else if (sweeps == 16) k_xp_measure_fast<16><<<(unsigned)grid, kXpThreads, 0, s>>>(job);
-    else k_xp_measure<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    void (*measure)(XpJob) = sweeps == 4 ? k_xp_measure_fast<4>
+                           : sweeps == 8 ? k_xp_measure_fast<8>
+                           : sweeps == 16 ? k_xp_measure_fast<16> : k_xp_measure;
+    void (*pack)(XpJob) = sweeps == 4 ? k_xp_pack_fast<4>
+                        : sweeps == 8 ? k_xp_pack_fast<8>
+                        : sweeps == 16 ? k_xp_pack_fast<16> : k_xp_pack;
+    const bool fast = sweeps == 4 || sweeps == 8 || sweeps == 16;
+    const size_t pack_smem = fast ? list_bytes : 0;
+    measure<<<resident_grid(ctx, measure, kXpThreads, 0, units), kXpThreads, 0, s>>>(job);
     k_xp_chunk_sizes<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
     k_scan_blocks<<<1, 1024, 0, s>>>(job.chunk_off, n_chunks, job.chunk_off + n_chunks);
     k_xp_layout<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(job);
-    if (sweeps == 4) k_xp_pack_fast<4><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
-    else if (sweeps == 8) k_xp_pack_fast<8><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
-    else if (sweeps == 16) k_xp_pack_fast<16><<<(unsigned)grid, kXpThreads, list_bytes, s>>>(job);
-    else k_xp_pack<<<(unsigned)grid, kXpThreads, 0, s>>>(job);
+    pack<<<resident_grid(ctx, pack, kXpThreads, pack_smem, units), kXpThreads, pack_smem, s>>>(job);
     ctx->launches += 5;
     CU(ctx, cudaGetLastError());
     return LSMKV_OK;
@@ -687,14 +703,12 @@ int lsmkv_decode_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query,
         uj.recs = recs;
         uj.st = ctx->d_status;
         LaunchTimer timer(ctx, s, LSMKV_K_UNPACK);
-        uint64_t grid = n_qchunks * 2ull * ctx->geom.n_layers * ctx->ppc;
-        const uint64_t cap = (uint64_t)ctx->sm_count * 8;
-        if (grid > cap) grid = cap;
+        const uint64_t units = n_qchunks * 2ull * ctx->geom.n_layers * ctx->ppc;
         const uint32_t sweeps = uj.n_elems % 2048u == 0 && !ctx->xp_generic ? uj.n_elems / 2048u : 0;
-        if (sweeps == 4) k_xp_unpack_fast<4><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
-        else if (sweeps == 8) k_xp_unpack_fast<8><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
-        else if (sweeps == 16) k_xp_unpack_fast<16><<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
-        else k_xp_unpack<<<(unsigned)grid, kXpThreads, 0, s>>>(uj, ar);
+        void (*unpack)(XpUnpackJob, ArenaTable) = sweeps == 4 ? k_xp_unpack_fast<4>
+                                                : sweeps == 8 ? k_xp_unpack_fast<8>
+                                                : sweeps == 16 ? k_xp_unpack_fast<16> : k_xp_unpack;
+        unpack<<<resident_grid(ctx, unpack, kXpThreads, 0, units), kXpThreads, 0, s>>>(uj, ar);
         ++ctx->launches;
         CU(ctx, cudaGetLastError());
         return LSMKV_OK;
