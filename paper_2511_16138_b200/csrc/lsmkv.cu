@@ -110,15 +110,21 @@ uint64_t host_powmod(uint64_t b, uint64_t e)
     return r;
 }
 
-void fill_key_consts(KeyConsts &kc, uint32_t C)
+// tab [host, 4 * kKeyTab]: powers and inverse powers of M = BASE ^ C (layout: see KeyConsts)
+void fill_key_consts(KeyConsts &kc, uint32_t C, uint64_t *tab)
 {
     const uint64_t mA = host_powmod(kBaseA, C), mB = host_powmod(kBaseB, C);
-    uint64_t a = mA, b = mB;
-    for (int i = 0; i < 32; ++i) {
-        kc.pwA[i] = a;
-        kc.pwB[i] = b;
+    const uint64_t iA = host_powmod(mA, kP - 2), iB = host_powmod(mB, kP - 2);   // p is prime
+    uint64_t a = mA, b = mB, ia = 1, ib = 1;
+    for (int i = 0; i < kKeyTab; ++i) {
+        tab[i] = a;
+        tab[kKeyTab + i] = b;
+        tab[2 * kKeyTab + i] = ia;
+        tab[3 * kKeyTab + i] = ib;
         a = host_mulmod(a, mA);
         b = host_mulmod(b, mB);
+        ia = host_mulmod(ia, iA);
+        ib = host_mulmod(ib, iB);
     }
     // weights of the 16 tokens of a block, BASE^(15-i), in limbs of 21 + 21 + 19 bits
     a = 1;
@@ -434,7 +440,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->page_bytes = pb;
     ctx->ppc = (uint32_t)ppc;
     ctx->chunk_bytes = ppc * 2ull * g->n_layers * pb;
-    fill_key_consts(ctx->kc, g->chunk_tokens);
+    uint64_t key_tab[4 * kKeyTab];
+    fill_key_consts(ctx->kc, g->chunk_tokens, key_tab);
     ctx->codec = g->flags;
     ctx->xp_dir_bytes = (uint32_t)((4ull * (ppc * 2ull * g->n_layers + 1) + 15) & ~15ull);
     ctx->copy_mode = 0;
@@ -450,12 +457,18 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(DevStatus));
+    // one small block: the status words, then (256 bytes in) the key tables
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256 + sizeof(key_tab));
     if (e == cudaSuccess) {
         DevStatus z;
         std::memset(&z, 0, sizeof(z));
         z.first_bad = ~0ull;
         e = cudaMemcpy(ctx->d_status, &z, sizeof(z), cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) {
+        uint64_t *d_tab = reinterpret_cast<uint64_t *>(reinterpret_cast<char *>(ctx->d_status) + 256);
+        e = cudaMemcpy(d_tab, key_tab, sizeof(key_tab), cudaMemcpyHostToDevice);
+        ctx->kc.tab = d_tab;
     }
     if (e != cudaSuccess) {
         cudaGetLastError();

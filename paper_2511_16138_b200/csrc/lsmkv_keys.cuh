@@ -2,12 +2,15 @@
 // token prefix, evaluated warp-cooperatively.
 //
 // The digest is defined sequentially (h <- h*B + t + 1 mod p per token). Because
-// H(XY) = H(X) * B^|Y| + H(Y), a warp hashes 32 consecutive chunks at once: every lane digests
-// its own chunk from h = 0 (16 tokens at a time as one dot product with the powers of B, see
-// block16_dot), then an inclusive warp scan with the fixed multiplier M = B^C stitches the
-// chunk hashes into prefix hashes, and the running prefix of the chunks before enters through
-// M^(lane+1). All arithmetic is exact, so the result is bit-identical to the sequential
-// definition.
+// H(XY) = H(X) * B^|Y| + H(Y), a CTA hashes 32 chunks per warp at once: every lane digests its
+// own chunk from h = 0 (16 tokens at a time as one dot product with the powers of B, see
+// block16_dot). With M = B^C the digest of the prefix that ends with chunk j of a round is
+//     P_j = c * M^(j+1) + sum_{i<=j} d_i * M^(j-i) = c * M^(j+1) + M^j * sum_{i<=j} d_i * M^(-i)
+// (c = digest before the round, d_i = chunk digests; M is invertible because p is prime), so the
+// chunk digests are scaled by M^(-i), summed with a plain additive scan, and scaled back: three
+// independent modular multiplications per lane and digest instead of a chain of them through
+// the scan. All arithmetic is exact in the field, so the canonical result is bit-identical to
+// the sequential definition.
 #pragma once
 #include "lsmkv_common.cuh"
 
@@ -17,21 +20,22 @@ constexpr uint64_t kP = 0x1FFFFFFFFFFFFFFFull;  // 2^61 - 1
 constexpr uint64_t kBaseA = 0x0B4E0EF37BC32127ull;
 constexpr uint64_t kBaseB = 0x16A09E667F3BCC90ull;
 
-// pw[x][i] = (BASE_x ^ C) ^ (i+1) mod p for i = 0..31; entries 0,1,3,7,15 are the scan
-// multipliers M^1, M^2, M^4, M^8, M^16.
 // d[x][i] = BASE_x ^ (15 - i) mod p cut into limbs of 21, 21 and 19 bits: the weights of the 16
 // tokens of a block (see block16_dot). sum[x] = BASE^0 + ... + BASE^15, b16[x] = BASE^16 (mod p).
+// tab [dev]: four tables of kKeyTab entries, M = BASE ^ C:
+//   tab[i] = M_A^(i+1), tab[kKeyTab + i] = M_B^(i+1), tab[2 kKeyTab + i] = M_A^(-i),
+//   tab[3 kKeyTab + i] = M_B^(-i)   (i = position of a chunk inside a round, < 32 * warps)
+constexpr int kKeyTab = 256;
 struct KeyConsts {
-    uint64_t pwA[32];
-    uint64_t pwB[32];
+    const uint64_t *tab;
     uint32_t dA[16][3];
     uint32_t dB[16][3];
     uint64_t sumA, sumB;
     uint64_t b16A, b16B;
 };
 
-// a, b < 2^61  ->  a*b mod p, canonical
-__host__ __device__ __forceinline__ uint64_t fold61(uint64_t s)  // s < 2^62
+// the canonical representative of s < 2^63
+__host__ __device__ __forceinline__ uint64_t fold61(uint64_t s)
 {
     s = (s & kP) + (s >> 61);
     return s >= kP ? s - kP : s;
@@ -51,8 +55,8 @@ __device__ __forceinline__ uint64_t addmod61(uint64_t a, uint64_t b)  // a, b < 
     return s >= kP ? s - kP : s;
 }
 
-// The scans below keep their intermediate values only partly reduced -- any representative below
-// 2^62 -- and take the canonical one (fold61) once at the end; the value mod p is the same.
+// The exchange below keeps its intermediate values only partly reduced -- any representative
+// below 2^62 -- and takes the canonical one (fold61) once at the end; the value mod p is the same.
 // a, b < 2^62  ->  a*b mod p, below 2^61 + 8
 __device__ __forceinline__ uint64_t mulmod61_lazy(uint64_t a, uint64_t b)
 {
@@ -62,10 +66,10 @@ __device__ __forceinline__ uint64_t mulmod61_lazy(uint64_t a, uint64_t b)
     return (s & kP) + (s >> 61);
 }
 
-// a*m + b mod p for a, m, b < 2^62, below 2^61 + 8
-__device__ __forceinline__ uint64_t muladd61_lazy(uint64_t a, uint64_t m, uint64_t b)
+// a + b mod p for a, b < 2^62, below 2^61 + 4
+__device__ __forceinline__ uint64_t add61_lazy(uint64_t a, uint64_t b)
 {
-    const uint64_t s = mulmod61_lazy(a, m) + b;         // < 2^63
+    const uint64_t s = a + b;                           // < 2^63
     return (s & kP) + (s >> 61);
 }
 
@@ -157,38 +161,11 @@ __device__ __forceinline__ void chunk_hash(const KeyConsts &kc, const uint32_t *
     }
 }
 
-// One warp, 32 consecutive chunks j = base_j + lane of the sequence starting at `seq`: every
-// lane gets the digests of tokens [base_j*C, (j+1)*C), i.e. relative to the start of this
-// 32-chunk block (no carry yet), partly reduced. Lanes with j >= nch hold garbage. All 32 lanes
-// must call.
-__device__ __forceinline__ void warp_block_scan(const KeyConsts &kc, const uint32_t *seq,
-                                                uint32_t C, uint64_t base_j, uint64_t nch,
-                                                uint64_t &hA, uint64_t &hB, uint32_t &first,
-                                                uint32_t &last)
-{
-    const unsigned lane = lane_id();
-    const uint64_t j = base_j + lane;
-    hA = 0; hB = 0; first = 0; last = 0;
-    if (j < nch) {
-        const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
-        chunk_hash(kc, seq + j * C, C, vec_ok, hA, hB, first, last);
-    }
-    // inclusive scan: x_i <- x_{i-d} * M^d + x_i
-#pragma unroll
-    for (unsigned d = 1; d < 32; d <<= 1) {
-        const uint64_t uA = shfl_up64(hA, d), uB = shfl_up64(hB, d);
-        if (lane >= d) {
-            hA = muladd61_lazy(uA, kc.pwA[d - 1], hA);
-            hB = muladd61_lazy(uB, kc.pwB[d - 1], hB);
-        }
-    }
-}
-
 constexpr int kKeyMaxWarps = 16;
 
 // Shared-memory exchange of a CTA that hashes one sequence round by round.
 struct KeyShared {
-    uint64_t aggA[kKeyMaxWarps], aggB[kKeyMaxWarps];   // digest of each warp's 32-chunk block
+    uint64_t aggA[kKeyMaxWarps], aggB[kKeyMaxWarps];   // scaled sum of each warp's 32-chunk block
     uint64_t carryA[2], carryB[2];                     // prefix before the round, by round parity
 };
 
@@ -199,40 +176,63 @@ __device__ __forceinline__ void key_rounds_begin(KeyShared &sh)
 }
 
 // One round of a CTA: its first `wact` warps hash 32*wact consecutive chunks starting at `base`
-// (warp w the 32-chunk block base + 32*w). The block digests are exchanged through shared
-// memory; warp w chains the w blocks before its own onto the prefix the previous round left, so
-// every thread of an active warp ends up with the key of chunk base + 32*warp + lane. The last
+// (warp w the 32-chunk block base + 32*w), as laid out at the top of this file: chunk digests
+// scaled by M^(-i), an additive scan inside every warp, the warps' totals exchanged through
+// shared memory, and the sum scaled back and joined with the prefix the previous round left.
+// Every thread of an active warp ends up with the key of chunk base + 32*warp + lane; the last
 // active warp leaves the prefix behind the round for round `rnd + 1`. Warps >= wact get an
 // unspecified key. Contains one __syncthreads(); the caller must put another one between two
-// calls (the exchange is rewritten).
+// calls (the exchange is rewritten). 32 * wact <= kKeyTab.
 __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
                                                    uint32_t C, uint32_t ns, uint64_t base,
                                                    uint64_t nch, unsigned rnd, unsigned wact,
                                                    KeyShared &sh)
 {
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
-    uint64_t hA = 0, hB = 0;
+    const unsigned idx = 32u * warp + lane;                // position inside the round
+    const uint64_t j = base + idx;
+    uint64_t zA = 0, zB = 0;
     uint32_t first = 0, last = 0;
     if (warp < wact) {
-        warp_block_scan(kc, seq, C, base + 32ull * warp, nch, hA, hB, first, last);
-        if (lane == 31) { sh.aggA[warp] = hA; sh.aggB[warp] = hB; }
+        uint64_t dA = 0, dB = 0;
+        if (j < nch) {
+            const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
+            chunk_hash(kc, seq + j * C, C, vec_ok, dA, dB, first, last);
+        }
+        zA = mulmod61_lazy(dA, __ldg(kc.tab + 2 * kKeyTab + idx));
+        zB = mulmod61_lazy(dB, __ldg(kc.tab + 3 * kKeyTab + idx));
+#pragma unroll
+        for (unsigned d = 1; d < 32; d <<= 1) {            // inclusive sums inside the warp
+            const uint64_t uA = shfl_up64(zA, d), uB = shfl_up64(zB, d);
+            if (lane >= d) {
+                zA = add61_lazy(uA, zA);
+                zB = add61_lazy(uB, zB);
+            }
+        }
+        if (lane == 31) { sh.aggA[warp] = zA; sh.aggB[warp] = zB; }
     }
     __syncthreads();
+    uint64_t hA = 0, hB = 0;
     if (warp < wact) {
-        uint64_t pA = sh.carryA[rnd & 1u], pB = sh.carryB[rnd & 1u];   // prefix before block 0
-        for (unsigned v = 0; v < warp; ++v) {                          // ... before block `warp`
-            pA = muladd61_lazy(pA, kc.pwA[31], sh.aggA[v]);
-            pB = muladd61_lazy(pB, kc.pwB[31], sh.aggB[v]);
+        for (unsigned v = 0; v < warp; ++v) {              // the warps before this one
+            zA = add61_lazy(zA, sh.aggA[v]);
+            zB = add61_lazy(zB, sh.aggB[v]);
         }
-        hA = fold61(muladd61_lazy(pA, kc.pwA[lane], hA));
-        hB = fold61(muladd61_lazy(pB, kc.pwB[lane], hB));
-        if (warp == wact - 1 && lane == 31) {          // meaningful when the round was full
+        const uint64_t cA = mulmod61_lazy(sh.carryA[rnd & 1u], __ldg(kc.tab + idx));
+        const uint64_t cB = mulmod61_lazy(sh.carryB[rnd & 1u], __ldg(kc.tab + kKeyTab + idx));
+        if (idx) {                                         // scale the sum back by M^idx
+            zA = mulmod61_lazy(zA, __ldg(kc.tab + idx - 1));
+            zB = mulmod61_lazy(zB, __ldg(kc.tab + kKeyTab + idx - 1));
+        }
+        hA = fold61(cA + zA);
+        hB = fold61(cB + zB);
+        if (warp == wact - 1 && lane == 31) {              // meaningful when the round was full
             sh.carryA[(rnd + 1u) & 1u] = hA;
             sh.carryB[(rnd + 1u) & 1u] = hB;
         }
     }
     ChunkKey k;
-    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)(base + 32ull * warp + lane);
+    k.w0 = ((uint64_t)ns << 32) | (uint64_t)(uint32_t)j;
     k.w1 = hA;
     k.w2 = hB;
     k.w3 = ((uint64_t)first << 32) | (uint64_t)last;
