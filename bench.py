@@ -699,7 +699,7 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
 # Warp instructions of one k_probe<true> launch on this workload: ncu smsp__inst_executed.sum of
 # the capture summarised under profiles/ (k_probe, probe-heavy workload). Set to None whenever the
 # kernel changes until the counter has been taken again.
-PROBE_WARP_INSTRUCTIONS = 69272798
+PROBE_WARP_INSTRUCTIONS = 64280836
 
 
 def probe_roofline(torch, device_index, ms):
