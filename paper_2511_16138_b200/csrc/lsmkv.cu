@@ -51,7 +51,7 @@ struct lsmkv_ctx {
     uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
-    size_t io_cap[3];
+    uint64_t io_cap[3];
     std::vector<uint64_t> h_off_a;
     std::vector<uint32_t> h_cuts;
     struct HostScratch { void *p; size_t cap; cudaEvent_t done; bool used; };
@@ -180,34 +180,78 @@ struct LaunchTimer {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The bulk copy kernels take their stages as dynamic shared memory beyond the default limit.
+// The limit is a per-device attribute of the function: it is raised once per device, to the
+// device's maximum, with that device current -- never per call with a call-specific size, so
+// that callers on different host threads (regular and allocation-free decodes alike) cannot
+// lower it under one another between setting it and launching.
+constexpr int kMaxDevices = 64;
+std::mutex g_smem_limit_mu;
+bool g_smem_limit_set[kMaxDevices];
+
+cudaError_t set_copy_smem_limit(int max_smem_optin)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_smem_limit_mu);
+    if (g_smem_limit_set[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(k_copy_slabs_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             max_smem_optin);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem_optin);
+    if (e == cudaSuccess) g_smem_limit_set[dev] = true;
+    return e;
+}
+
+// Every scratch buffer of a context has exactly one owner (a pointer field and its capacity
+// field) and goes through the two helpers below: nothing else frees or replaces one.
+// release_scratch: free, null the pointer and zero the capacity in one step, so that a stale
+// pointer can never be used or freed again; the result of cudaFree is reported.
+template <typename T>
+int release_scratch(lsmkv_ctx *ctx, T **slot, uint64_t *cap, int line)
+{
+    if (!*slot) { *cap = 0; return LSMKV_OK; }
+    void *old = *slot;
+    *slot = nullptr;
+    *cap = 0;
+    const cudaError_t e = cudaFree(old);   // waits for work that may still use the buffer
+    return e == cudaSuccess ? LSMKV_OK : cuda_fail(ctx, e, line);
+}
+
+// grow_scratch: a fresh allocation of `bytes` replaces the slot's buffer; `cap` receives
+// `new_cap` (in whatever unit the owner counts). On failure the old buffer stays in place.
+template <typename T>
+int grow_scratch(lsmkv_ctx *ctx, T **slot, uint64_t *cap, size_t bytes, uint64_t new_cap, int line)
+{
+    void *p = nullptr;
+    const cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { cuda_fail(ctx, e, line); return LSMKV_ENOMEM; }
+    const int rc = release_scratch(ctx, slot, cap, line);
+    if (rc != LSMKV_OK) { cudaFree(p); return rc; }
+    *slot = static_cast<T *>(p);
+    *cap = new_cap;
+    return LSMKV_OK;
+}
+
 int ensure_workspace(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
 {
     if (n_seq <= ctx->ws_seq && n_chunks <= ctx->ws_chunks && ctx->d_ws) return LSMKV_OK;
     const uint64_t ns = n_seq > ctx->ws_seq ? n_seq : ctx->ws_seq;
     const uint64_t nc = n_chunks > ctx->ws_chunks ? n_chunks : ctx->ws_chunks;
-    void *p = nullptr;
     const size_t bytes = (size_t)(ns + 2) * 8 + (size_t)(nc + 4) * 4;
-    cudaError_t e = cudaMalloc(&p, bytes);
-    if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
-    if (ctx->d_ws) cudaFree(ctx->d_ws);   // waits for work that may still use the old one
-    ctx->d_ws = p;
-    cudaGetLastError();   // drop any stale last-error left by the allocation calls
-    ctx->ws_seq = ns;
-    ctx->ws_chunks = nc;
-    return LSMKV_OK;
+    const int rc = grow_scratch(ctx, &ctx->d_ws, &ctx->ws_seq, bytes, ns, __LINE__);
+    ctx->ws_chunks = rc == LSMKV_OK ? nc : (ctx->d_ws ? ctx->ws_chunks : 0);
+    return rc;
 }
 
 int ensure_dir(lsmkv_ctx *ctx, uint64_t entries)
 {
     if (entries <= ctx->dir_cap && ctx->d_dir) return LSMKV_OK;
-    void *p = nullptr;
-    cudaError_t e = cudaMalloc(&p, (size_t)entries * sizeof(uint64_t));
-    if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
-    if (ctx->d_dir) cudaFree(ctx->d_dir);   // waits for work that may still use the old one
-    ctx->d_dir = static_cast<uint64_t *>(p);
-    cudaGetLastError();   // drop any stale last-error left by the allocation calls
-    ctx->dir_cap = entries;
-    return LSMKV_OK;
+    return grow_scratch(ctx, &ctx->d_dir, &ctx->dir_cap, (size_t)entries * sizeof(uint64_t),
+                        entries, __LINE__);
 }
 
 struct SortWs {
@@ -225,14 +269,8 @@ size_t sort_ws_bytes(uint64_t n)
 int ensure_sort(lsmkv_ctx *ctx, uint64_t n, SortWs *ws)
 {
     if (n > ctx->sort_cap || !ctx->d_sort) {
-        void *p = nullptr;
-        cudaError_t e = cudaMalloc(&p, sort_ws_bytes(n));
-        if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
-        if (ctx->d_sort) cudaFree(ctx->d_sort);
-    if (ctx->d_xp) cudaFree(ctx->d_xp);
-        ctx->d_sort = p;
-    cudaGetLastError();   // drop any stale last-error left by the allocation calls
-        ctx->sort_cap = n;
+        const int rc = grow_scratch(ctx, &ctx->d_sort, &ctx->sort_cap, sort_ws_bytes(n), n, __LINE__);
+        if (rc != LSMKV_OK) return rc;
     }
     const uint64_t cap = ctx->sort_cap;
     unsigned char *b = static_cast<unsigned char *>(ctx->d_sort);
@@ -327,15 +365,11 @@ int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &
         const uint64_t need = (pieces + stages - 1) / stages;
         if (grid > need) grid = need;
         if (grid == 0) return LSMKV_OK;
-        if (ctx->copy_l2_hint) {
-            CU(ctx, cudaFuncSetAttribute(k_copy_slabs_bulk<true>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        // (the shared-memory limit of both instantiations was raised at lsmkv_create)
+        if (ctx->copy_l2_hint)
             k_copy_slabs_bulk<true><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
-        } else {
-            CU(ctx, cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else
             k_copy_slabs_bulk<false><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
-        }
     }
     ++ctx->launches;
     CU(ctx, cudaGetLastError());
@@ -349,15 +383,10 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
 {
     const uint64_t slabs = 2ull * ctx->geom.n_layers * ctx->ppc;
     if (n_chunks > ctx->xp_cap || !ctx->d_xp) {
-        void *p = nullptr;
-        cudaError_t e = cudaMalloc(&p, (size_t)n_chunks * slabs * 12 + ((size_t)n_chunks + 2) * 8 + 256);
-        if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
-        if (ctx->d_xp) cudaFree(ctx->d_xp);
-        ctx->d_xp = p;
-        ctx->xp_cap = n_chunks;
-        // A successful allocation can still leave a stale entry in the runtime's last-error
-        // slot (seen on this driver); drop it so the launch checks below report only launches.
-        cudaGetLastError();
+        const int rc = grow_scratch(ctx, &ctx->d_xp, &ctx->xp_cap,
+                                    (size_t)n_chunks * slabs * 12 + ((size_t)n_chunks + 2) * 8 + 256,
+                                    n_chunks, __LINE__);
+        if (rc != LSMKV_OK) return rc;
     }
     XpJob job;
     std::memset(&job, 0, sizeof(job));
@@ -472,16 +501,15 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     }
     if (e != cudaSuccess) {
         cudaGetLastError();
-        if (ctx->d_status) cudaFree(ctx->d_status);
-        delete ctx;
+        lsmkv_destroy(ctx);
         return LSMKV_ECUDA;
     }
     int rc = ensure_workspace(ctx, 1024, 65536);
     if (rc == LSMKV_OK) rc = ensure_dir(ctx, 2 + 8 * (kDirMaxJ + 1) + kOrderMaxQueries / 2);
+    if (rc == LSMKV_OK) rc = set_copy_smem_limit(ctx->max_smem_optin) == cudaSuccess ? LSMKV_OK : LSMKV_ECUDA;
     if (rc != LSMKV_OK) {
-        if (ctx->d_ws) cudaFree(ctx->d_ws);
-        cudaFree(ctx->d_status);
-        delete ctx;
+        cudaGetLastError();
+        lsmkv_destroy(ctx);
         return rc;
     }
     *out = ctx;
@@ -492,23 +520,30 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
 {
     if (!ctx) return LSMKV_OK;
     DeviceGuard guard(ctx->device);
-    cudaDeviceSynchronize();
-    if (ctx->d_ws) cudaFree(ctx->d_ws);
-    if (ctx->d_dir) cudaFree(ctx->d_dir);
-    if (ctx->d_sort) cudaFree(ctx->d_sort);
-    if (ctx->d_xp) cudaFree(ctx->d_xp);
-    for (void *p : ctx->d_io) if (p) cudaFree(p);
+    // Everything is released even when one step fails; the first failure is what is reported.
+    cudaError_t first = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
+    auto note = [&first](cudaError_t e) { if (first == cudaSuccess && e != cudaSuccess) first = e; };
+    note(cudaDeviceSynchronize());
+    uint64_t cap = 0;
+    if (release_scratch(ctx, &ctx->d_ws, &ctx->ws_seq, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
+    ctx->ws_chunks = 0;
+    if (release_scratch(ctx, &ctx->d_dir, &ctx->dir_cap, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
+    if (release_scratch(ctx, &ctx->d_sort, &ctx->sort_cap, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
+    if (release_scratch(ctx, &ctx->d_xp, &ctx->xp_cap, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
+    for (int k = 0; k < 3; ++k)
+        if (release_scratch(ctx, &ctx->d_io[k], &ctx->io_cap[k], __LINE__) != LSMKV_OK)
+            note((cudaError_t)ctx->last_cuda);
     for (auto &kind : ctx->hs)
         for (auto &h : kind) {
-            if (h.p) cudaFreeHost(h.p);
-            if (h.done) cudaEventDestroy(h.done);
+            if (h.p) note(cudaFreeHost(h.p));
+            if (h.done) note(cudaEventDestroy(h.done));
         }
-    if (ctx->d_status) cudaFree(ctx->d_status);
-    for (auto &t : ctx->pending) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
-    for (auto e : ctx->free_events) cudaEventDestroy(e);
-    cudaGetLastError();
+    if (release_scratch(ctx, &ctx->d_status, &cap, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
+    for (auto &t : ctx->pending) { note(cudaEventDestroy(t.a)); note(cudaEventDestroy(t.b)); }
+    for (auto e : ctx->free_events) note(cudaEventDestroy(e));
+    if (first != cudaSuccess) cudaGetLastError();
     delete ctx;
-    return LSMKV_OK;
+    return first == cudaSuccess ? LSMKV_OK : LSMKV_ECUDA;
 }
 
 int lsmkv_reserve(lsmkv_ctx *ctx, uint64_t n_seq, uint64_t n_chunks)
@@ -1222,7 +1257,7 @@ __global__ void k_static_reset()
     }
 }
 
-constexpr int kStaticMaxDevices = 64;
+constexpr int kStaticMaxDevices = kMaxDevices;
 struct StaticDev {
     bool ready;
     unsigned char *scratch;   // device address of g_static_scratch on this device
@@ -1243,6 +1278,7 @@ int static_setup(int device, StaticDev **out)
         cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        if (e == cudaSuccess) e = set_copy_smem_limit(d.max_smem_optin);
         if (e != cudaSuccess || !ptr) {
             cudaGetLastError();
             return LSMKV_ECUDA;
@@ -1331,9 +1367,7 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
         uint64_t grid = (uint64_t)sd->sm_count;
         const uint64_t need = (pieces + stages - 1) / stages;
         if (grid > need) grid = need;
-        cudaError_t e = cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) { cudaGetLastError(); return LSMKV_ECUDA; }
+        // (the kernel's shared-memory limit was raised to the device maximum by the set-up)
         k_copy_slabs_bulk<false><<<(unsigned)grid, stages * 32, smem, s>>>(job, ar);
     }
     if (status_out) {

@@ -25,14 +25,7 @@ struct IoLayout {
 int ensure_io(lsmkv_ctx *ctx, int kind, size_t bytes)
 {
     if (bytes <= ctx->io_cap[kind] && ctx->d_io[kind]) return LSMKV_OK;
-    void *p = nullptr;
-    cudaError_t e = cudaMalloc(&p, bytes);
-    if (e != cudaSuccess) { cuda_fail(ctx, e); return LSMKV_ENOMEM; }
-    if (ctx->d_io[kind]) cudaFree(ctx->d_io[kind]);   // waits for work that may still use it
-    ctx->d_io[kind] = p;
-    cudaGetLastError();   // drop any stale last-error left by the allocation calls
-    ctx->io_cap[kind] = bytes;
-    return LSMKV_OK;
+    return grow_scratch(ctx, &ctx->d_io[kind], &ctx->io_cap[kind], bytes, bytes, __LINE__);
 }
 
 size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }

@@ -161,7 +161,8 @@ __device__ __forceinline__ void chunk_hash(const KeyConsts &kc, const uint32_t *
     }
 }
 
-constexpr int kKeyMaxWarps = 16;
+constexpr int kKeyMaxWarps = 8;   // one table entry per chunk of a round: 32 chunks per warp
+static_assert(32 * kKeyMaxWarps <= kKeyTab, "a CTA's round must fit the power tables");
 
 // Shared-memory exchange of a CTA that hashes one sequence round by round.
 struct KeyShared {
@@ -248,7 +249,7 @@ __device__ __forceinline__ void store_key(lsmkv_key_t *dst, const ChunkKey &k)
 
 // put_batch keys + records: one CTA per request at a time (requests handed out round-robin),
 // 32 * W chunks per round.
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(32 * kKeyMaxWarps)
 k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uint32_t n_req,
               const uint32_t *__restrict__ tokens, const uint64_t *__restrict__ seq_off,
               const uint32_t *__restrict__ start_chunk, const uint64_t *__restrict__ chunk_off,

@@ -611,6 +611,10 @@ class Context:
     def launch_count(self) -> int:
         return lsmkv_launch_count(self.handle)
 
+    def last_cuda_error(self) -> int:
+        """The cudaError_t behind the context's last LSMKV_ECUDA (0 if there was none)."""
+        return lib().lsmkv_last_cuda_error(self.handle)
+
     def set_tuning(self, name, value):
         lsmkv_set_tuning(self.handle, name, value)
 

@@ -1,6 +1,7 @@
-"""Host-side index maintenance: turning a write batch into a sorted run (flush) and merging
-runs (compaction). These are the LSM steps between put_batch and probe (paper Sec. 2.2); they
-sit outside the timed device path and run on the host with numpy.
+"""Test utility: flush (a write batch becomes a sorted run) and compaction (runs are merged) with
+numpy on the host -- the LSM steps between put_batch and probe (paper Sec. 2.2). The library does
+both on the GPU (lsmkv_flush_batch, lsmkv_merge_runs); the tests use this form to build runs
+without going through the code under test.
 
 Keys are uint64 [n, 4] ordered lexicographically as unsigned words; records are 16-byte
 entries kept as a numpy structured array or as raw uint8 [n, 16].

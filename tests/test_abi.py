@@ -8,7 +8,8 @@ import numpy as np
 
 import oracle
 from oracle import VAL_DTYPE
-from paper_2511_16138_b200 import build, hostindex, lsmkv
+import hostindex
+from paper_2511_16138_b200 import build, lsmkv
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 

@@ -9,7 +9,8 @@ import torch
 
 import oracle
 from oracle import VAL_DTYPE
-from paper_2511_16138_b200 import hostindex, lsmkv, synth
+import hostindex
+from paper_2511_16138_b200 import lsmkv, synth
 
 import gpu_harness as H
 

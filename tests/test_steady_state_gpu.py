@@ -63,3 +63,6 @@ def test_repeated_calls_do_not_allocate(flags):
         assert free_after == free_before
         assert np.array_equal(t["hit"].cpu().numpy(), (w.expected_hit_tokens // 16).astype(np.int32))
         assert ctx.last_status()["flags"] == 0
+        assert ctx.last_cuda_error() == 0
+        ctx.close()                                # raises unless lsmkv_destroy returned LSMKV_OK
+        assert ctx.handle is None

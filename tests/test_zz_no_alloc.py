@@ -15,7 +15,8 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2511_16138_b200 import hostindex, lsmkv, synth
+import hostindex
+from paper_2511_16138_b200 import lsmkv, synth
 
 import gpu_harness as H
 
