@@ -1,8 +1,12 @@
 """Full-size parity on the named workloads, in the launch configuration the benchmark times
 (default tuning, waves sized for HBM). Metadata (keys, records, hit lengths, hit records) is
-compared with the oracle in full; payload (blobs, restored pages) on sampled chunk ranges the
-oracle recomputes from host copies, plus device-side identities that hold at any size
-(decode(encode(x)) == x on every page, untouched pages stay zero)."""
+compared with the oracle in full. Payload: every blob of every wave is checked on the device,
+slab by slab, against the pool pages it must hold (a statement of the blob layout in tensor
+indexing, independent of the library); one whole wave of the Llama-shaped workload and the whole
+long-context workload are also streamed through the oracle's encoder in slices and compared byte
+for byte; the other waves on sampled chunk ranges. Restored pages: sampled against the oracle's
+decode, plus device-side identities that hold at any size (decode(encode(x)) == x on every
+page, untouched pages stay zero)."""
 import numpy as np
 import pytest
 import torch
@@ -40,6 +44,66 @@ def sample_ranges(rng, nch, n_samples, width):
     return out
 
 
+def blobs_hold_their_pages_on_gpu(g, arena, n, src, src_pages, slice_chunks=2048) -> bool:
+    """The blob layout written out with tensor indexing: blob i is 2L slabs, slab 2l + kv is page
+    src_pages[i] of buffer kv * L + l (K of layer l, then V of layer l). One page per chunk."""
+    assert g.pages_per_chunk == 1
+    L = g.n_layers
+    blobs = arena[:n * g.chunk_bytes].view(n, 2 * L, g.page_bytes)
+    sp = torch.as_tensor(np.asarray(src_pages, dtype=np.int64), device=H.DEV)
+    for kv in range(2):
+        for l in range(L):
+            buf = src.bufs[kv * L + l]
+            for a in range(0, n, slice_chunks):
+                if not torch.equal(blobs[a:a + slice_chunks, 2 * l + kv], buf[sp[a:a + slice_chunks]]):
+                    return False
+    return True
+
+
+class PinnedFetch:
+    """Device -> host copies through one reusable pinned buffer."""
+
+    def __init__(self, nbytes):
+        self.t = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+
+    def __call__(self, d):
+        d = d.reshape(-1)
+        out = self.t[:d.numel()]
+        out.copy_(d)
+        torch.cuda.synchronize()
+        return out.numpy()
+
+
+def whole_wave_against_oracle(g, batch, nch, coff, src, src_pages, arena, keys, vals,
+                              slice_bytes=1 << 30):
+    """Every blob of the wave from the oracle's encoder, in slices of whole chunk ranges of one
+    request (host copies of that range's pages in, blob bytes out), against the arena."""
+    og = H.ogeom(g)
+    cb, C, L2 = g.chunk_bytes, g.chunk_tokens, 2 * g.n_layers
+    per = max(1, slice_bytes // cb)
+    fetch_pool, fetch_blob = PinnedFetch(per * cb), PinnedFetch(per * cb)
+    checked = 0
+    for r in range(batch.n):
+        toks = batch.seq(r)
+        for a in range(0, int(nch[r]), per):
+            b = min(int(nch[r]), a + per)
+            i0 = int(coff[r]) + a
+            idx = torch.as_tensor(src_pages[i0:i0 + b - a].astype(np.int64), device=H.DEV)
+            host_pool = fetch_pool(torch.stack([buf[idx] for buf in src.bufs])).reshape(
+                L2, b - a, g.page_bytes)
+            t = np.ascontiguousarray(toks[:b * C])
+            k, v, blob = oracle.encode_batch(og, t, np.array([0, len(t)], np.uint64),
+                                             np.array([a], np.uint32),
+                                             np.array([0, b - a], np.uint64),
+                                             np.arange(b - a, dtype=np.uint32), host_pool, 0,
+                                             i0 * cb)
+            assert np.array_equal(k, keys[i0:i0 + b - a]) and np.array_equal(v, vals[i0:i0 + b - a])
+            got = fetch_blob(arena[i0 * cb:(i0 + b - a) * cb])
+            assert np.array_equal(got, blob), f"blob of request {r} chunks [{a},{b}) differs"
+            checked += b - a
+    assert checked == int(coff[-1])
+
+
 def check_restored_sample(g, rng, sel, recs, arena, dst, dst_pages, n_sample):
     """Sampled restored pages against the oracle's decode of the blob their record names."""
     cb = g.chunk_bytes
@@ -50,7 +114,8 @@ def check_restored_sample(g, rng, sel, recs, arena, dst, dst_pages, n_sample):
         assert np.array_equal(dst.gather(dst_pages[i:i + 1]), want)
 
 
-def encode_probe_decode_wave(ctx, g, batch, nch, src, dst, arena, rng, n_sample=4, width=8):
+def encode_probe_decode_wave(ctx, g, batch, nch, src, dst, arena, rng, n_sample=4, width=8,
+                             whole_wave=False):
     """One wave of 'full encode, probe, decode' with every check. Returns (keys, vals)."""
     og = H.ogeom(g)
     cb = g.chunk_bytes
@@ -94,7 +159,11 @@ def encode_probe_decode_wave(ctx, g, batch, nch, src, dst, arena, rng, n_sample=
     dst.zero_()
     ctx.decode_batch(batch.n, d_coff, n, d_hit, d_recs, [(arena, n * cb)], up(dst_pages), dst.table)
     torch.cuda.synchronize()
-    # payload: sampled ranges against the oracle
+    # payload: every blob against the pages it must hold (device side), the whole wave or
+    # sampled ranges against the oracle
+    assert blobs_hold_their_pages_on_gpu(g, arena, n, src, src_pages), "a blob differs from its pages"
+    if whole_wave:
+        whole_wave_against_oracle(g, batch, nch, coff, src, src_pages, arena, keys, vals)
     for r, a, b in sample_ranges(rng, nch, n_sample, width):
         i0 = int(coff[r]) + a
         k, v, blob = H.oracle_blob_range(g, batch.seq(r), a, b, src, src_pages[i0:i0 + b - a], 0,
@@ -129,10 +198,10 @@ def test_config2_llama8b_full_encode_probe_decode():
     arena = torch.empty(cap * g.chunk_bytes, dtype=torch.uint8, device=H.DEV)
     rng = synth.rng_for(2, 5)
     with lsmkv.Context(g, 0) as ctx:
-        for a, b in zip(bounds[:-1], bounds[1:]):
+        for k, (a, b) in enumerate(zip(bounds[:-1], bounds[1:])):
             t0, t1 = int(w.batch.seq_off[a]), int(w.batch.seq_off[b])
             wb = synth.Batch(w.batch.tokens[t0:t1], w.batch.seq_off[a:b + 1] - w.batch.seq_off[a])
-            encode_probe_decode_wave(ctx, g, wb, nch[a:b], src, dst, arena, rng)
+            encode_probe_decode_wave(ctx, g, wb, nch[a:b], src, dst, arena, rng, whole_wave=k == 1)
 
 
 def test_config5_long_context_encode_probe_decode():
@@ -150,7 +219,8 @@ def test_config5_long_context_encode_probe_decode():
     arena = torch.empty(n * cb, dtype=torch.uint8, device=H.DEV)
     rng = synth.rng_for(5, 5)
     with lsmkv.Context(g, 0) as ctx:
-        keys, vals = encode_probe_decode_wave(ctx, g, w.store, nch, src, dst, arena, rng, width=4)
+        keys, vals = encode_probe_decode_wave(ctx, g, w.store, nch, src, dst, arena, rng, width=4,
+                                              whole_wave=True)
         run = H.gpu_flush_run(ctx, keys, vals)
         qn = synth.chunk_counts(w.query.seq_off, 16)
         qoff = synth.offsets(qn)
@@ -329,6 +399,7 @@ def test_config4_gqa_multi_turn():
                                                         None, None, 0, used * cb, with_blob=False)
                 assert np.array_equal(keys, o_keys) and np.array_equal(vals, o_vals)
                 blob_page[used:used + n] = src_pages
+                assert blobs_hold_their_pages_on_gpu(g, arena[used * cb:], n, src, src_pages)
                 for _ in range(2):                 # sampled blob ranges against the oracle
                     k = int(rng.integers(0, hist.n))
                     if nch[k] == stored[k]:

@@ -128,3 +128,83 @@ def test_order_is_pythons_tuple_order():
     b = synth.make_batch(seqs)
     want = sorted(range(b.n), key=lambda i: (tuple(int(t) for t in b.seq(i)), i))
     assert list(oracle.xrun_order(b.tokens, b.seq_off)) == want
+
+
+def _shared_len(a, b):
+    n = 0
+    while n < min(len(a), len(b)) and a[n] == b[n]:
+        n += 1
+    return n
+
+
+def _store_with_copied_records(C, seqs, file_id):
+    """Records as a put after a probe writes them: chunk j of sequence s takes a copy of the record
+    of the earliest stored sequence whose first (j + 1) * C tokens are the same, else a fresh one."""
+    vals, fresh = [], 0
+    rows = []
+    for s, seq in enumerate(seqs):
+        row = []
+        for j in range(len(seq) // C):
+            src = next((t for t in range(s) if _shared_len(seqs[t], seq) >= (j + 1) * C), None)
+            if src is None:
+                fresh += 1
+                row.append((file_id, 16 * fresh))
+            else:
+                row.append(rows[src][j])
+        rows.append(row)
+        vals += row
+    v = np.zeros(len(vals), dtype=VAL_DTYPE)
+    v["file_id"] = [a for a, _ in vals]
+    v["offset"] = [b for _, b in vals]
+    return v, rows
+
+
+def _brute_force_any_owner(C, Q, stores, pick):
+    """Longest shared prefix per run, records from the holder chosen by ``pick`` (min = the first
+    sequence put that reaches it, max = the last); no ordering of the stored sequences is used."""
+    nq = len(Q) // C
+    rec, hit = [(0, 0)] * nq, 0
+    for seqs, rows in stores:                                # newest first
+        lens = [_shared_len(s, Q) for s in seqs]
+        m = max(lens + [0]) // C
+        if m <= hit:
+            continue
+        owner = pick(i for i, n in enumerate(lens) if n == max(lens))
+        rec[hit:m] = rows[owner][hit:m]
+        hit = m
+    return hit, rec
+
+
+def test_records_do_not_depend_on_which_holder_is_taken():
+    """With records of shared chunks copied from their first owner (the state every put after a
+    probe leaves), whichever stored sequence reaches the longest shared prefix supplies the same
+    records: the oracle's answer must equal a brute force that takes the first holder and one that
+    takes the last, neither of which knows the neighbour rule."""
+    C = 2
+    g = G(C)
+    rng = np.random.default_rng(11)
+    stores, xruns = [], []
+    for r in range(3):
+        seqs = [tuple(int(t) for t in rng.integers(0, 2, rng.integers(0, 15))) for _ in range(40)]
+        seqs += [(0, 1, 0, 1, 1, 1)] * 2 + [(0, 1, 0, 1)]
+        v, rows = _store_with_copied_records(C, seqs, file_id=r + 1)
+        b = synth.make_batch([np.array(s, np.uint32) for s in seqs])
+        stores.append((seqs, rows))
+        xruns.append((b.tokens, b.seq_off, v))
+    queries = [tuple(int(t) for t in rng.integers(0, 2, rng.integers(0, 18))) for _ in range(200)]
+    queries += [(0, 1, 0, 1, 1, 1, 0, 0), (0, 1, 0, 1, 2), ()]
+    qb = synth.make_batch([np.array(q, np.uint32) for q in queries])
+    qoff = synth.offsets(synth.chunk_counts(qb.seq_off, C))
+    hit, recs = oracle.xprobe_batch(g, qb.tokens, qb.seq_off, qoff, xruns)
+    n_multi = 0
+    for q, Q in enumerate(queries):
+        h_first, r_first = _brute_force_any_owner(C, Q, stores, min)
+        h_last, r_last = _brute_force_any_owner(C, Q, stores, max)
+        assert h_first == h_last == int(hit[q])
+        assert r_first == r_last
+        a = int(qoff[q])
+        got = [(int(recs[a + j]["file_id"]), int(recs[a + j]["offset"])) for j in range(len(Q) // C)]
+        assert got == r_first
+        lens = [_shared_len(s, Q) for s in stores[0][0]]
+        n_multi += sum(1 for n in lens if n == max(lens)) > 1 and max(lens) >= C
+    assert n_multi > 50                       # the choice of holder was a real one in many queries

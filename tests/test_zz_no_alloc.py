@@ -6,9 +6,10 @@ driver allocations from then on. They cannot create a context (that allocates), 
 offers one context-free decode whose scratch is a fixed array inside the library itself.
 
 The test drives that entry point through the C ABI and requires the restored pool to be
-byte-identical to what the regular lsmkv_decode_batch produces -- on two calls in a row, the
-second with shorter hits and other destination pages, so that anything the shared scratch kept
-from the first call would show up. This file sorts last on purpose: a run that stops at the
+byte-identical to what the regular lsmkv_decode_batch produces and to what the CPU oracle
+restores from its own blobs and records -- on two calls in a row, the second with shorter hits
+and other destination pages, so that anything the shared scratch kept from the first call would
+show up. This file sorts last on purpose: a run that stops at the
 first failure has then already executed every other test.
 """
 import numpy as np
@@ -16,6 +17,7 @@ import pytest
 import torch
 
 import hostindex
+import oracle
 from paper_2511_16138_b200 import lsmkv, synth
 
 import gpu_harness as H
@@ -36,20 +38,30 @@ def _prepare(ctx, g, seed):
     num_pages = n + 5
     pool_np = synth.random_pool_bytes(rng, 2 * g.n_layers, num_pages, g.page_bytes)
     pool = H.DevPool(g, num_pages, pool_np)
-    keys, vals, blob, d_blob = H.gpu_encode(ctx, g, w.store, None, coff,
-                                            synth.random_pages(rng, num_pages, n), pool)
+    src_pages = synth.random_pages(rng, num_pages, n)
+    keys, vals, blob, d_blob = H.gpu_encode(ctx, g, w.store, None, coff, src_pages, pool)
     runs = [hostindex.flush(keys, vals)]
     qoff = synth.offsets(synth.chunk_counts(w.query.seq_off, g.chunk_tokens))
     hit, recs, _, (d_qoff, d_hit, d_recs) = H.gpu_probe(ctx, w.query, qoff, runs, want_keys=False)
     assert hit.sum() > 0
+    # the oracle's own chain on the same inputs: its blobs and records feed its decode below
+    og = H.ogeom(g)
+    o_keys, o_vals, o_blob = oracle.encode_batch(og, w.store.tokens, w.store.seq_off, None, coff,
+                                                 src_pages, pool_np, 0, 0)
+    o_hit, o_recs, _, _ = oracle.probe_batch(og, w.query.tokens, w.query.seq_off, qoff,
+                                             [oracle.flush(o_keys, o_vals)])
+    assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
     return dict(n_query=w.query.n, qoff=qoff, total=int(qoff[-1]), d_qoff=d_qoff, hit=hit,
-                d_recs=d_recs, d_blob=d_blob, blob_bytes=blob.size, num_pages=num_pages, rng=rng)
+                d_recs=d_recs, d_blob=d_blob, blob_bytes=blob.size, num_pages=num_pages, rng=rng,
+                og=og, o_recs=o_recs, o_blob=o_blob, pool_shape=pool_np.shape)
 
 
 def _decode_both(ctx, g, p, hit):
     """Decode once through each entry point into its own zeroed pool; return both pools and the
-    status block of the allocation-free call."""
-    dst_pages = H.dev(synth.random_pages(p["rng"], p["num_pages"], p["total"]))
+    status block of the allocation-free call. The allocation-free call's pool must also equal
+    the oracle's decode of the oracle's blobs."""
+    dst_np = synth.random_pages(p["rng"], p["num_pages"], p["total"])
+    dst_pages = H.dev(dst_np)
     d_hit = H.dev(hit.astype(np.uint32))
     arenas = [(p["d_blob"], p["blob_bytes"])]
     ref = H.DevPool(g, p["num_pages"])
@@ -63,6 +75,10 @@ def _decode_both(ctx, g, p, hit):
     st = d_status.cpu().numpy()
     flags = int(st[:4].view(np.uint32)[0])
     decoded = int(st[48:56].view(np.uint64)[0])
+    want = np.zeros(p["pool_shape"], dtype=np.uint8)
+    oracle.decode_batch(p["og"], p["qoff"], hit.astype(np.uint32), p["o_recs"], [p["o_blob"]],
+                        dst_np, want)
+    assert np.array_equal(out.numpy(), want), "allocation-free decode differs from the oracle"
     return ref.numpy(), out.numpy(), flags, decoded
 
 
