@@ -16,6 +16,7 @@
 #include "lsmkv_probe.cuh"
 #include "lsmkv_sort.cuh"
 #include "lsmkv_xp12.cuh"
+#include "lsmkv_xp12_fused.cuh"
 #include "lsmkv_xrun.cuh"
 
 using namespace lsmkv;
@@ -48,6 +49,7 @@ struct lsmkv_ctx {
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
+    int64_t xp_one_pass, wait_cycles;
     uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
@@ -180,11 +182,16 @@ struct LaunchTimer {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// The bulk copy kernels take their stages as dynamic shared memory beyond the default limit.
+// The bulk copy kernels and the one-pass encoder take their stages as dynamic shared memory
+// beyond the default limit.
 // The limit is a per-device attribute of the function: it is raised once per device, to the
 // device's maximum, with that device current -- never per call with a call-specific size, so
 // that callers on different host threads (regular and allocation-free decodes alike) cannot
 // lower it under one another between setting it and launching.
+// one-pass encoder of the compressing codec: slabs of 8192 and 16384 elements
+using XpfShape8k = xpf::Shape<4, 8, 2, 4, 4>;
+using XpfShape16k = xpf::Shape<4, 16, 1, 3, 3>;
+
 constexpr int kMaxDevices = 64;
 std::mutex g_smem_limit_mu;
 bool g_smem_limit_set[kMaxDevices];
@@ -202,6 +209,12 @@ cudaError_t set_copy_smem_limit(int max_smem_optin)
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_copy_slabs_bulk<false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem_optin);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_xpf_encode<XpfShape8k>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XpfShape8k::kSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_xpf_encode<XpfShape16k>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XpfShape16k::kSmem);
     if (e == cudaSuccess) g_smem_limit_set[dev] = true;
     return e;
 }
@@ -411,6 +424,29 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
     job.st = ctx->d_status;
     LaunchTimer timer(ctx, s, LSMKV_K_PACK);
     const uint64_t units = n_chunks * slabs;
+    // One pass over the pool when the slab size has a pipeline shape, the blob buffer takes the
+    // worst case (so no chunk can overflow half-written) and the pipeline fits the device.
+    if (ctx->xp_one_pass && !ctx->xp_generic && (job.n_elems == 8192u || job.n_elems == 16384u) &&
+        blob_capacity >= lsmkv_encode_bound(ctx, n_chunks) &&
+        (size_t)ctx->max_smem_optin >= (job.n_elems == 8192u ? XpfShape8k::kSmem : XpfShape16k::kSmem)) {
+        unsigned char *scratch = static_cast<unsigned char *>(ctx->d_xp);
+        xpf::Job fj;
+        fj.x = job;
+        fj.ticket = reinterpret_cast<unsigned long long *>(scratch);
+        fj.abort = reinterpret_cast<unsigned int *>(scratch + 8);
+        fj.state = reinterpret_cast<unsigned long long *>(scratch + 256);
+        fj.wait_cycles = ctx->wait_cycles;
+        CU(ctx, cudaMemsetAsync(scratch, 0, 256 + (size_t)units * 8, s));
+        const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)ctx->sm_count, units);
+        if (job.n_elems == 8192u)
+            k_xpf_encode<XpfShape8k><<<grid, XpfShape8k::kThreads, XpfShape8k::kSmem, s>>>(fj);
+        else
+            k_xpf_encode<XpfShape16k><<<grid, XpfShape16k::kThreads, XpfShape16k::kSmem, s>>>(fj);
+        k_xpf_layout<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(fj);
+        ctx->launches += 2;
+        CU(ctx, cudaGetLastError());
+        return LSMKV_OK;
+    }
     // common slab sizes take the fast kernels (2048 * {4, 8, 16} elements), the rest the generic
     const uint32_t sweeps = job.n_elems % 2048u == 0 && !ctx->xp_generic ? job.n_elems / 2048u : 0;
     const size_t list_bytes = job.n_elems;
@@ -481,6 +517,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->probe_warps_per_cta = 4;
     ctx->simt_ctas_per_sm = 8;
     ctx->host_stage_bytes = 1ll << 30;
+    ctx->xp_one_pass = 1;
+    ctx->wait_cycles = 2000000000ll;
 
     DeviceGuard guard(device);
     cudaError_t e = guard.ok ? cudaSuccess : cudaErrorInvalidDevice;
@@ -1131,6 +1169,8 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"simt_ctas_per_sm", &ctx->simt_ctas_per_sm, 1, 32},
         {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
         {"xp_generic", &ctx->xp_generic, 0, 1},
+        {"xp_one_pass", &ctx->xp_one_pass, 0, 1},
+        {"wait_cycles", &ctx->wait_cycles, 100000, 100000000000ll},
     };
     for (auto &t : tab)
         if (std::strcmp(t.n, name) == 0) { *lo = t.lo; *hi = t.hi; return t.p; }

@@ -40,13 +40,14 @@ def mixed_pool(rng, g, num_pages):
     return pool
 
 
-@pytest.mark.parametrize("g,generic", [(geom(3, 2, 16, 4), 0), (geom(2, 8, 128, 16), 0),
-                                       (geom(2, 8, 128, 16), 1), (geom(2, 1, 24, 3), 0),
-                                       (geom(1, 4, 128, 64), 0), (geom(1, 4, 128, 64), 1),
-                                       (geom(2, 8, 64, 16), 0)])
-def test_encode_and_decode_equal_the_oracle(g, generic):
-    """Slabs of 128, 16384, 72, 32768 and 8192 elements: fast kernels where they apply (and the
-    generic ones forced on the same shapes)."""
+@pytest.mark.parametrize("g,generic,one_pass", [
+    (geom(3, 2, 16, 4), 0, 1), (geom(2, 8, 128, 16), 0, 1), (geom(2, 8, 128, 16), 0, 0),
+    (geom(2, 8, 128, 16), 1, 1), (geom(2, 1, 24, 3), 0, 1), (geom(1, 4, 128, 64), 0, 1),
+    (geom(1, 4, 128, 64), 1, 1), (geom(2, 8, 64, 16), 0, 1), (geom(2, 8, 64, 16), 0, 0)])
+def test_encode_and_decode_equal_the_oracle(g, generic, one_pass):
+    """Slabs of 128, 16384, 72, 32768 and 8192 elements: the one-pass encoder where it applies
+    (16384 and 8192 elements), the three-step fast kernels on the same shapes and on 32768, and
+    the generic ones forced on the same shapes."""
     og = H.ogeom(g)
     rng = np.random.default_rng(g.page_bytes)
     C = g.chunk_tokens
@@ -62,6 +63,7 @@ def test_encode_and_decode_equal_the_oracle(g, generic):
                                                       pool_np, 5, 1024)
     with lsmkv.Context(g, 0) as ctx:
         ctx.set_tuning("xp_generic", generic)
+        ctx.set_tuning("xp_one_pass", one_pass)
         bound = ctx.encode_bound(n)
         assert bound == n * oracle.xp12_chunk_bound(og)
         pool = H.DevPool(g, num_pages, pool_np)
@@ -159,3 +161,60 @@ def test_codec_needs_16_bit_elements():
         lsmkv.Context(lsmkv.Geom(2, 2, 64, elem_bytes=1, flags=lsmkv.CODEC_XP12), 0)
     with pytest.raises(lsmkv.LsmkvError):
         lsmkv.Context(lsmkv.Geom(2, 2, 64, flags=2), 0)
+
+
+@pytest.mark.parametrize("L,Hh,D", [(16, 8, 128), (12, 8, 64)])
+def test_one_pass_encoder_over_many_slabs_equals_the_three_step_one_and_the_oracle(L, Hh, D):
+    """Enough slabs that every CTA of the one-pass encoder takes many turns (a few thousand
+    slabs of 16384 / 8192 elements, N(0,1) payload with planted special pages): blobs and records
+    must equal the three-step encoder's byte for byte, and the oracle's."""
+    g = geom(L, Hh, D, 16)
+    og = H.ogeom(g)
+    rng = np.random.default_rng(L)
+    C = 16
+    b = synth.make_batch([rng.integers(0, 32000, n * C + 1, dtype=np.uint32)
+                          for n in (37, 1, 64, 5, 90)])
+    nch = synth.chunk_counts(b.seq_off, C)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    assert n * 2 * L > 4000
+    num_pages = n + 3
+    pool_np = synth.random_pool_bytes(rng, 2 * L, num_pages, g.page_bytes)
+    v = pool_np.view(np.uint16)
+    v[3, 5] = 0                                                       # an all-zero slab
+    v[0, 7] = rng.integers(0, 65536, v.shape[2], dtype=np.uint16)     # an incompressible one
+    v[1, 9][::3] = 0x0001                                             # many exceptions
+    pages = synth.random_pages(rng, num_pages, n)
+    pages[11] = num_pages + 100                                       # an unusable page id
+    outs = []
+    with lsmkv.Context(g, 0) as ctx:
+        bound = ctx.encode_bound(n)
+        pool = H.DevPool(g, num_pages, pool_np)
+        for one_pass in (1, 0):
+            ctx.set_tuning("xp_one_pass", one_pass)
+            d_keys = torch.zeros(n * 32, dtype=torch.uint8, device=H.DEV)
+            d_vals = torch.zeros(n * 16, dtype=torch.uint8, device=H.DEV)
+            d_blob = torch.full((bound,), 0xEE, dtype=torch.uint8, device=H.DEV)
+            ctx.encode_batch(b.n, H.dev(b.tokens), H.dev(b.seq_off), None, H.dev(coff), n,
+                             H.dev(pages), pool.table, 2, 0, d_keys, d_vals, d_blob, bound)
+            torch.cuda.synchronize()
+            st = ctx.last_status()
+            assert st["flags"] == lsmkv.ST_BAD_PAGE and st["first_bad"] == 11
+            outs.append((H.host(d_vals, VAL_DTYPE, n * 16).copy(), d_blob.cpu().numpy()))
+    (v1, b1), (v0, b0) = outs
+    assert np.array_equal(v1, v0), "records differ between the two encoders"
+    assert np.array_equal(b1, b0), "blobs differ between the two encoders"
+    # the oracle refuses an unusable page id, so it encodes the batch with that page readable and
+    # the comparison leaves that one chunk out
+    good = pages.copy()
+    good[11] = 0
+    o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, b.tokens, b.seq_off, None, coff, good,
+                                                      pool_np, 2, 0)
+    a, e = int(o_vals["offset"][11]), int(o_vals["offset"][12])
+    assert np.array_equal(v1[:11], o_vals[:11]) and np.array_equal(b1[:a], o_blob[:a])
+    shift = int(v1["offset"][12]) - e                                 # the raw-zero chunk's size differs
+    assert np.array_equal(v1["reserved"][12:], o_vals["reserved"][12:])
+    assert np.array_equal(v1["offset"][12:] - shift, o_vals["offset"][12:])
+    used = int(v1["offset"][-1]) + int(v1["reserved"][-1])
+    assert np.array_equal(b1[e + shift:used], o_blob[e:])
+    assert np.all(b1[used:] == 0xEE)
