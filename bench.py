@@ -52,12 +52,15 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--requests", type=int, default=256, help="requests in the batch (256 = the named workload)")
-    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU baseline budget (0 = skip)")
     ap.add_argument("--only-probe-block", action="store_true",
                     help="run just the probe-heavy measurement (a small case for profiling)")
     ap.add_argument("--no-shapes-block", action="store_true",
-                    help="skip the pack/unpack rates on the other workloads' KV shapes")
+                    help="skip the other named workloads (their KV shapes, and the workloads "
+                         "themselves: long context, multi-turn, decode of the probe-heavy hits)")
+    ap.add_argument("--only-workloads-block", action="store_true",
+                    help="run just the other named workloads as workloads")
     ap.add_argument("--no-xp12-block", action="store_true",
                     help="skip the compressing-codec measurement")
     ap.add_argument("--no-probe-block", action="store_true",
@@ -186,6 +189,58 @@ def time_oracle(og, sample, budget_s):
             return moved / el / 1e9, passes, el
 
 
+def _oracle_worker(job):
+    """One process of the all-cores baseline: a plain parallel-for over requests -- this worker
+    takes requests i, i + P, ... of the batch (up to its share of chunks) and runs the oracle's
+    encode / probe / decode passes over them for the given time."""
+    i, n_workers, n_req_total, chunks_per_worker, budget_s = job
+    import oracle
+    og = oracle.Geom(**GEOM)
+    w = synth.llama_requests(n_req=n_req_total)
+    nch_all = synth.chunk_counts(w.batch.seq_off, og.chunk_tokens)
+    seqs, acc = [], 0
+    for r in range(i, w.batch.n, n_workers):           # whole requests, the last one cut to fit
+        take = min(int(nch_all[r]), chunks_per_worker - acc)
+        if take <= 0:
+            break
+        seqs.append(w.batch.seq(r)[:take * og.chunk_tokens])
+        acc += take
+    b = synth.make_batch(seqs)
+    nch = synth.chunk_counts(b.seq_off, og.chunk_tokens)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    rng = synth.rng_for(2, 500 + i)
+    pages, dst_pages = synth.random_pages(rng, n, n), synth.random_pages(rng, n, n)
+    pool = synth.random_pool_bytes(rng, 2 * og.n_layers, n, og.page_bytes)
+    keys, vals, _ = oracle.encode_batch(og, b.tokens, b.seq_off, None, coff, None, None, 0, 0,
+                                        with_blob=False)
+    sample = (b, coff, pages, pool, [oracle.flush(keys, vals)], dst_pages, np.zeros_like(pool))
+    oracle_sample_pass(og, sample)                           # warm (pages everything in)
+    v, passes, el = time_oracle(og, sample, budget_s)
+    return v * el * 1e9, el, passes, n
+
+
+def time_oracle_all_cores(n_req_total, max_chunks_total, budget_s):
+    """The oracle on every host core the process may use: spawned workers (never forked: the
+    parent may hold a CUDA context), each timing its own share; the rate is all bytes moved over
+    the longest worker's time."""
+    import multiprocessing as mp
+    try:
+        n_workers = len(os.sched_getaffinity(0))
+    except AttributeError:
+        n_workers = os.cpu_count() or 1
+    n_workers = max(1, min(n_workers, 64))
+    per = max(4, max_chunks_total // n_workers)
+    jobs = [(i, n_workers, n_req_total, per, budget_s) for i in range(n_workers)]
+    with mp.get_context("spawn").Pool(n_workers) as pool:
+        res = pool.map(_oracle_worker, jobs)
+    moved = sum(r[0] for r in res)
+    el = max(r[1] for r in res)
+    return {"value": moved / el / 1e9, "unit": UNIT, "cores": n_workers, "kind": "oracle",
+            "sample": f"{n_workers} workers, parallel-for over requests: {sum(r[3] for r in res)} chunks "
+                      f"in all, {sum(r[2] for r in res)} passes, longest worker {el:.1f} s"}
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle, as it stands, on the host cores; one step = one pass
     over a bounded sample of the same workload."""
@@ -254,6 +309,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.only_workloads_block:
+        if rank == 0:
+            peak, _ = hbm_peak()
+            print(json.dumps({"other_workloads": [f(torch, lsmkv, dev, local_rank, peak)
+                                                  for f in (long_context_block, multi_turn_block,
+                                                            probe_heavy_decode_block)]}))
+        return
     if args.only_probe_block:
         if rank == 0:
             print(json.dumps({"probe": probe_heavy_block(torch, lsmkv, dev, local_rank,
@@ -415,13 +477,14 @@ def main():
     if args.e2e_steps > 0:
         del arena                                    # the host-buffer calls stage on their own
         torch.cuda.empty_cache()
+        link = link_ceiling(torch, dev)                  # same run, same box: the e2e ceiling
         e2e = run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barrier,
-                      world, "identity")
+                      world, "identity", link)
         if not args.no_xp12_block:
             ctx_xp = lsmkv.Context(lsmkv.Geom(**dict(GEOM, flags=lsmkv.CODEC_XP12)), local_rank)
             try:
                 e2e_xp = run_e2e(args, torch, lsmkv, ctx_xp, g, W, src_pool, dst_pool, dev, stream,
-                                 barrier, world, "xp12")
+                                 barrier, world, "xp12", link)
             finally:
                 ctx_xp.close()
 
@@ -443,8 +506,14 @@ def main():
         cpu = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {s_req} requests = {s_n} chunks ({s_n * cb / 2**30:.2f} GiB per "
                          f"direction), {passes} passes in {el:.1f} s; host cpus={os.cpu_count()}"}
+        del sample
+        try:
+            cpu["all_cores"] = time_oracle_all_cores(args.requests, max_chunks,
+                                                     min(5.0, args.cpu_seconds))
+        except Exception as exc:                           # e.g. no room for the workers' pools
+            cpu["all_cores"] = {"unavailable": repr(exc)}
 
-    shapes_block = None
+    shapes_block = workloads_block = None
     if rank == 0:
         n_waves_used = len(W)
         if not args.no_shapes_block:
@@ -454,6 +523,9 @@ def main():
                 del arena
             torch.cuda.empty_cache()
             shapes_block = other_shapes_block(torch, lsmkv, dev, local_rank, peak)
+            workloads_block = [f(torch, lsmkv, dev, local_rank, peak)
+                               for f in (long_context_block, multi_turn_block,
+                                         probe_heavy_decode_block)]
         copy_ms = prof["pack"][0] + prof["unpack"][0]
         copy_launches = prof["pack"][1] + prof["unpack"][1]
         algo_bytes_per_launch = 2.0 * (2 * payload * args.steps) / max(1, copy_launches)
@@ -470,7 +542,8 @@ def main():
                        "tuning": {k: ctx.get_tuning(k) for k in
                                   ("copy_mode", "copy_stage_bytes", "copy_stages",
                                    "copy_ctas_per_sm", "copy_l2_hint")}},
-            "e2e": e2e, "e2e_codec_xp12": e2e_xp, "gpu_launches": int(launches), "clocks": clocks,
+            "e2e": e2e, "e2e_codec_xp12": e2e_xp, "host_link": link if args.e2e_steps > 0 else None,
+            "gpu_launches": int(launches), "clocks": clocks,
             "roofline": {"bound": "hbm", "kernel": "k_copy_slabs (pack + unpack launches)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_source": peak_src,
@@ -486,6 +559,7 @@ def main():
             "probe": probe_block,
             "codec_xp12": xp_block,
             "other_shapes": shapes_block,
+            "other_workloads": workloads_block,
             "phases": {
                 "pack_GBps_payload": payload * args.steps / (prof["pack"][0] * 1e-3) / 1e9,
                 "unpack_GBps_payload": payload * args.steps / (prof["unpack"][0] * 1e-3) / 1e9,
@@ -581,7 +655,342 @@ def other_shapes_block(torch, lsmkv, dev, device_index, peak):
     return out
 
 
+# ---- the other named workloads, run as workloads (identity codec) ---------------------------
+
+def _up(torch, dev, a):
+    b = np.ascontiguousarray(a).view(np.uint8).reshape(-1)
+    t = torch.empty(max(16, b.size), dtype=torch.uint8, device=dev)
+    if b.size:
+        t[:b.size] = torch.from_numpy(b.copy())
+    return t
+
+
+def _filled_pool(torch, lsmkv, dev, g, num_pages, seed):
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    bufs = [torch.randn(num_pages * g.page_bytes // 2, dtype=torch.bfloat16, device=dev,
+                        generator=gen).view(torch.uint8).view(num_pages, g.page_bytes)
+            for _ in range(2 * g.n_layers)]
+    return bufs, lsmkv.pool_table(bufs)
+
+
+def _zero_pool(torch, lsmkv, dev, g, num_pages):
+    bufs = [torch.zeros((num_pages, g.page_bytes), dtype=torch.uint8, device=dev)
+            for _ in range(2 * g.n_layers)]
+    return bufs, lsmkv.pool_table(bufs)
+
+
+def _class_ms(prof, reps=1):
+    return {k: v[0] / reps for k, v in prof.items() if v[1]}
+
+
+def long_context_block(torch, lsmkv, dev, device_index, peak, reps=3):
+    """configs[4] as a workload: 4 requests x 32768 tokens (two share 16k), 80x8x128 bf16, page 16:
+    encode all (40 GiB), flush, probe with the last 1k tokens changed, decode the 1984-chunk hits.
+    Device time per kernel class from the library's own events, on the launching stream."""
+    g = lsmkv.Geom(80, 8, 128, page_tokens=16, chunk_tokens=16)
+    cb = g.chunk_bytes
+    w = synth.long_context()
+    nch = synth.chunk_counts(w.store.seq_off, 16)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    free, _ = torch.cuda.mem_get_info()
+    if 3 * n * cb > free * 0.92:
+        return {"workload": "configs[4] long-context", "unavailable": "not enough free device memory"}
+    qoff = synth.offsets(synth.chunk_counts(w.query.seq_off, 16))
+    nq = int(qoff[-1])
+    rng = synth.rng_for(5, 77)
+    ctx = lsmkv.Context(g, device_index)
+    src = dst = arena = None
+    try:
+        src, sp = _filled_pool(torch, lsmkv, dev, g, n, 5)
+        dst, dp = _zero_pool(torch, lsmkv, dev, g, n)
+        arena = torch.empty(n * cb, dtype=torch.uint8, device=dev)
+        d_tok, d_off, d_coff = (_up(torch, dev, a) for a in (w.store.tokens, w.store.seq_off, coff))
+        d_src = _up(torch, dev, synth.random_pages(rng, n, n))
+        q_tok, q_off, q_qoff = (_up(torch, dev, a) for a in (w.query.tokens, w.query.seq_off, qoff))
+        d_dst = _up(torch, dev, synth.random_pages(rng, n, nq))
+        keys = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+        vals = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        rk, rv = torch.empty_like(keys), torch.empty_like(vals)
+        rn = torch.zeros(1, dtype=torch.int64, device=dev)
+        nb = lsmkv.lsmkv_hindex_buckets(n)
+        hx = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+        hit = torch.zeros(w.query.n, dtype=torch.int32, device=dev)
+        recs = torch.empty(nq * 16, dtype=torch.uint8, device=dev)
+        runs = [(rk, rv, n, None, 0, hx, nb)]
+
+        def once():
+            ctx.encode_batch(w.store.n, d_tok, d_off, None, d_coff, n, d_src, sp, 0, 0, keys, vals,
+                             arena, n * cb)
+            ctx.flush_batch(keys, vals, n, rk, rv, rn)
+            ctx.hindex_build(rk, n, hx)
+            ctx.probe_batch(w.query.n, q_tok, q_off, q_qoff, nq, runs, hit, recs, None)
+            ctx.decode_batch(w.query.n, q_qoff, nq, hit, recs, [(arena, n * cb)], d_dst, dp)
+
+        once()
+        torch.cuda.synchronize()
+        hits = hit.cpu().numpy()
+        assert np.array_equal(hits, (w.expected_hit_tokens // 16).astype(np.int32)), hits
+        assert ctx.last_status()["flags"] == 0
+        ctx.profile_enable(True)
+        ctx.profile_read()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            once()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = _class_ms(ctx.profile_read(), reps)
+        n_hit = int(hits.sum())
+        return {"workload": "configs[4]: 4 x 32768 tokens, 80x8x128 bf16, page 16; encode, flush, "
+                            "probe with the last 1k tokens changed, decode the hits",
+                "chunks_encoded": n, "chunks_decoded": n_hit, "chunk_MiB": cb / 2**20,
+                "payload_GiB_encoded": n * cb / 2**30, "payload_GiB_decoded": n_hit * cb / 2**30,
+                "ms_per_pass": e0.elapsed_time(e1) / reps, "kernel_ms": ms,
+                "pack_GBps_payload": n * cb / ms["pack"] / 1e6,
+                "unpack_GBps_payload": n_hit * cb / ms["unpack"] / 1e6,
+                "round_trip_GBps_payload": (n + n_hit) * cb / (ms["pack"] + ms["unpack"]) / 1e6,
+                "pack_hbm_frac_of_peak": 2 * n * cb / ms["pack"] / 1e6 / peak,
+                "unpack_hbm_frac_of_peak": 2 * n_hit * cb / ms["unpack"] / 1e6 / peak,
+                "probe_keys_per_s": nq / ms["probe"] * 1e3,
+                "flush_share_of_pass": (ms.get("flush", 0.0)) / (e0.elapsed_time(e1) / reps)}
+    finally:
+        ctx.close()
+        del src, dst, arena
+        torch.cuda.empty_cache()
+
+def multi_turn_block(torch, lsmkv, dev, device_index, peak, max_groups=8):
+    """configs[3] as a workload: 512 conversations x 8 turns of 256-1024 new tokens, 28x4x128
+    bf16, page 64. Per turn: probe and decode the stored history, encode the new chunks
+    (start_chunk), flush them as the newest run with its hash index, merge the two oldest runs
+    when more than four pile up. Conversations in groups of 64 (pool and arena reused)."""
+    g = lsmkv.Geom(28, 4, 128, page_tokens=64, chunk_tokens=64)
+    cb, C = g.chunk_bytes, 64
+    w = synth.multi_turn()
+    n_conv, n_turns, group = w.full.n, w.turn_end.shape[1], 64
+    final_nch = synth.chunk_counts(w.full.seq_off, C)
+    groups = [list(range(a, min(n_conv, a + group))) for a in range(0, n_conv, group)][:max_groups]
+    cap = int(max(final_nch[c].sum() for c in groups))
+    free, _ = torch.cuda.mem_get_info()
+    if 3 * cap * cb > free * 0.92:
+        return {"workload": "configs[3] GQA multi-turn", "unavailable": "not enough free device memory"}
+    rng = synth.rng_for(4, 77)
+    # host side of every turn, prepared before anything is timed
+    plan = []
+    for convs in groups:
+        perm = synth.random_pages(rng, cap, int(final_nch[convs].sum()))
+        page_of, at = {}, 0
+        for c in convs:
+            page_of[c] = perm[at:at + int(final_nch[c])]
+            at += int(final_nch[c])
+        stored = np.zeros(len(convs), dtype=np.int64)
+        turns = []
+        for t in range(n_turns):
+            hist = synth.make_batch([w.full.seq(c)[:int(w.turn_end[c, t])] for c in convs])
+            nch = synth.chunk_counts(hist.seq_off, C)
+            qoff = synth.offsets(nch)
+            coff = synth.offsets(nch - stored)
+            src_pages = np.concatenate([page_of[c][int(stored[k]):int(nch[k])]
+                                        for k, c in enumerate(convs)]).astype(np.uint32)
+            turns.append(dict(n_req=hist.n, tokens=hist.tokens, seq_off=hist.seq_off, qoff=qoff,
+                              total=int(qoff[-1]), start=stored.astype(np.uint32), coff=coff,
+                              n=int(coff[-1]), src_pages=src_pages, hist_chunks=int(stored.sum()),
+                              dst_pages=synth.random_pages(rng, cap, int(qoff[-1]))))
+            stored = nch.copy()
+        plan.append(turns)
+    ctx = lsmkv.Context(g, device_index)
+    src = dst = arena = None
+    try:
+        src, sp = _filled_pool(torch, lsmkv, dev, g, cap, 4)
+        dst, dp = _zero_pool(torch, lsmkv, dev, g, cap)
+        arena = torch.empty(cap * cb, dtype=torch.uint8, device=dev)
+        up = lambda a: _up(torch, dev, a)
+        enc_chunks = dec_chunks = merges = 0
+
+        def run_groups(which):
+            nonlocal enc_chunks, dec_chunks, merges
+            for turns in which:
+                runs, used, keep = [], 0, []
+                for t in turns:
+                    d_tok, d_off = up(t["tokens"]), up(t["seq_off"])
+                    if runs:                           # the stored history: probe, then decode
+                        d_qoff = up(t["qoff"])
+                        hit = torch.zeros(t["n_req"], dtype=torch.int32, device=dev)
+                        recs = torch.empty(max(1, t["total"]) * 16, dtype=torch.uint8, device=dev)
+                        ctx.probe_batch(t["n_req"], d_tok, d_off, d_qoff, t["total"], runs, hit, recs,
+                                        None)
+                        ctx.decode_batch(t["n_req"], d_qoff, t["total"], hit, recs,
+                                         [(arena, used * cb)], up(t["dst_pages"]), dp)
+                        dec_chunks += t["hist_chunks"]
+                        keep.append((hit, recs))
+                    n = t["n"]
+                    keys = torch.empty(max(1, n) * 32, dtype=torch.uint8, device=dev)
+                    vals = torch.empty(max(1, n) * 16, dtype=torch.uint8, device=dev)
+                    ctx.encode_batch(t["n_req"], d_tok, d_off, up(t["start"]), up(t["coff"]), n,
+                                     up(t["src_pages"]), sp, 0, used * cb, keys, vals,
+                                     arena[used * cb:], (cap - used) * cb)
+                    rk, rv = torch.empty_like(keys), torch.empty_like(vals)
+                    rn = torch.zeros(1, dtype=torch.int64, device=dev)
+                    ctx.flush_batch(keys, vals, n, rk, rv, rn)
+                    nb = lsmkv.lsmkv_hindex_buckets(n)
+                    hx = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+                    ctx.hindex_build(rk, n, hx)
+                    runs.insert(0, (rk, rv, n, None, 0, hx, nb))
+                    used += n
+                    enc_chunks += n
+                    if len(runs) > 4:                  # compaction of the two oldest runs
+                        m = runs[-1][2] + runs[-2][2]
+                        mk = torch.empty(m * 32, dtype=torch.uint8, device=dev)
+                        mv = torch.empty(m * 16, dtype=torch.uint8, device=dev)
+                        mn = torch.zeros(1, dtype=torch.int64, device=dev)
+                        ctx.merge_runs([r[:3] for r in runs[-2:]], mk, mv, mn)
+                        mb = lsmkv.lsmkv_hindex_buckets(m)
+                        mh = torch.empty(mb * 32, dtype=torch.uint8, device=dev)
+                        ctx.hindex_build(mk, m, mh)
+                        runs[-2:] = [(mk, mv, m, None, 0, mh, mb)]
+                        merges += 1
+                torch.cuda.synchronize()
+                last_hit = keep[-1][0].cpu().numpy()
+                want = turns[-1]["qoff"][1:] - turns[-1]["qoff"][:-1] - (turns[-1]["coff"][1:] - turns[-1]["coff"][:-1])
+                assert np.array_equal(last_hit, want.astype(np.int32)), "multi-turn probe missed"
+
+        run_groups(plan[:1])                           # warm-up: scratch reaches its size
+        assert ctx.last_status()["flags"] == 0
+        enc_chunks = dec_chunks = merges = 0
+        ctx.profile_enable(True)
+        ctx.profile_read()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run_groups(plan)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = _class_ms(ctx.profile_read())
+        assert ctx.last_status()["flags"] == 0
+        dev_ms = sum(ms.values())
+        return {"workload": "configs[3]: %d conversations x %d turns, 28x4x128 bf16, page 64; per turn "
+                            "probe + decode of the history, encode of the new chunks, flush, "
+                            "compaction" % (sum(len(t[0]["start"]) for t in plan), n_turns),
+                "chunks_encoded": enc_chunks, "chunks_decoded": dec_chunks, "chunk_MiB": cb / 2**20,
+                "payload_GiB_encoded": enc_chunks * cb / 2**30,
+                "payload_GiB_decoded": dec_chunks * cb / 2**30, "compactions": merges,
+                "elapsed_ms_with_host_work": e0.elapsed_time(e1), "kernel_ms": ms,
+                "pack_GBps_payload": enc_chunks * cb / ms["pack"] / 1e6,
+                "unpack_GBps_payload": dec_chunks * cb / ms["unpack"] / 1e6,
+                "round_trip_GBps_payload": (enc_chunks + dec_chunks) * cb / (ms["pack"] + ms["unpack"]) / 1e6,
+                "pack_hbm_frac_of_peak": 2 * enc_chunks * cb / ms["pack"] / 1e6 / peak,
+                "unpack_hbm_frac_of_peak": 2 * dec_chunks * cb / ms["unpack"] / 1e6 / peak,
+                "flush_and_merge_share_of_kernel_time": (ms.get("flush", 0) + ms.get("merge", 0)) / dev_ms,
+                "probe_share_of_kernel_time": ms.get("probe", 0) / dev_ms}
+    finally:
+        ctx.close()
+        del src, dst, arena
+        torch.cuda.empty_cache()
+
+def probe_heavy_decode_block(torch, lsmkv, dev, device_index, peak, n_blobs=32768, num_pages=131072):
+    """configs[2], the decode half: the hits of the 4096 queries (1M stored keys in 4 runs) are
+    scattered into an 8x8x128 bf16 pool of 64 GiB from an arena of 32768 blobs that the million
+    records alias (offset = (i mod 32768) * chunk_bytes), in waves of queries that fit the pool."""
+    g = lsmkv.Geom(8, 8, 128, page_tokens=16, chunk_tokens=16)
+    cb = g.chunk_bytes
+    free, _ = torch.cuda.mem_get_info()
+    if (n_blobs + num_pages) * cb > free * 0.92:
+        return {"workload": "configs[2] decode", "unavailable": "not enough free device memory"}
+    w = synth.probe_heavy()
+    nch = synth.chunk_counts(w.store.seq_off, 16)
+    coff = synth.offsets(nch - w.store_start_chunk)
+    up = lambda a: _up(torch, dev, a)
+    ctx = lsmkv.Context(g, device_index)
+    dst = arena = None
+    try:
+        n = w.n_stored
+        d_keys = torch.empty(n * 32, dtype=torch.uint8, device=dev)
+        d_vals = torch.empty(n * 16, dtype=torch.uint8, device=dev)
+        ctx.encode_batch(w.store.n, up(w.store.tokens), up(w.store.seq_off), up(w.store_start_chunk),
+                         up(coff), n, None, None, 0, 0, d_keys, d_vals, None, 0)
+        torch.cuda.synchronize()
+        keys = d_keys.cpu().numpy().view(np.uint64).reshape(-1, 4)
+        vals = d_vals.cpu().numpy().reshape(-1, 16).copy()
+        off = vals[:, 8:16].view(np.uint64).reshape(-1)           # records alias the arena
+        off[:] = (np.arange(n, dtype=np.uint64) % np.uint64(n_blobs)) * np.uint64(cb)
+        runs, keep = [], []
+        for r in range(4):
+            sel = w.run_of_key == r
+            dup = w.dup_idx[w.dup_run == r]
+            m = int(sel.sum()) + len(dup)
+            tk = torch.empty(m * 32, dtype=torch.uint8, device=dev)
+            tv = torch.empty(m * 16, dtype=torch.uint8, device=dev)
+            tn = torch.zeros(1, dtype=torch.int64, device=dev)
+            ctx.flush_batch(up(np.concatenate([keys[sel], keys[dup]])),
+                            up(np.concatenate([vals[sel], vals[(dup + 7919) % n]])), m, tk, tv, tn)
+            nb = lsmkv.lsmkv_hindex_buckets(m)
+            hx = torch.empty(nb * 32, dtype=torch.uint8, device=dev)
+            ctx.hindex_build(tk, m, hx)
+            keep.append(tn)
+            runs.append((tk, tv, m, None, 0, hx, nb))
+        qoff = synth.offsets(synth.chunk_counts(w.query.seq_off, 16))
+        total = int(qoff[-1])
+        d_qoff = up(qoff)
+        d_hit = torch.zeros(w.query.n, dtype=torch.int32, device=dev)
+        d_recs = torch.empty(total * 16, dtype=torch.uint8, device=dev)
+        ctx.probe_batch(w.query.n, up(w.query.tokens), up(w.query.seq_off), d_qoff, total, runs,
+                        d_hit, d_recs, None)
+        torch.cuda.synchronize()
+        hit = d_hit.cpu().numpy().astype(np.int64)
+        assert np.array_equal(hit, w.expected_hit.astype(np.int64))
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(3)
+        arena = torch.randn(n_blobs * cb // 2, dtype=torch.bfloat16, device=dev,
+                            generator=gen).view(torch.uint8)
+        dst, dp = _zero_pool(torch, lsmkv, dev, g, num_pages)
+        rng = synth.rng_for(3, 77)
+        waves, q0 = [], 0
+        while q0 < w.query.n:                            # waves of queries that fit the pool
+            q1, acc = q0, 0
+            while q1 < w.query.n and acc + int(hit[q1]) <= num_pages:
+                acc += int(hit[q1])
+                q1 += 1
+            hit_w = np.zeros(w.query.n, dtype=np.uint32)
+            hit_w[q0:q1] = hit[q0:q1]
+            pages = np.zeros(total, dtype=np.uint32)
+            sel = np.concatenate([np.arange(int(qoff[q]), int(qoff[q]) + int(hit[q]))
+                                  for q in range(q0, q1)] + [np.zeros(0, np.int64)]).astype(np.int64)
+            pages[sel] = synth.random_pages(rng, num_pages, len(sel))
+            waves.append((up(hit_w), up(pages), acc))
+            q0 = q1
+
+        def all_waves():
+            for d_hw, d_pg, _ in waves:
+                ctx.decode_batch(w.query.n, d_qoff, total, d_hw, d_recs, [(arena, n_blobs * cb)],
+                                 d_pg, dp)
+
+        all_waves()
+        torch.cuda.synchronize()
+        st = ctx.last_status()
+        assert st["flags"] == 0 and st["chunks_decoded"] == int(hit.sum()), st
+        ctx.profile_enable(True)
+        ctx.profile_read()
+        all_waves()
+        torch.cuda.synchronize()
+        ms = _class_ms(ctx.profile_read())
+        n_hit = int(hit.sum())
+        return {"workload": "configs[2], decode of the hits: %d hit chunks of 512 KiB from an arena of "
+                            "%d aliased blobs into a %d-page pool, %d waves"
+                            % (n_hit, n_blobs, num_pages, len(waves)),
+                "chunks_decoded": n_hit, "payload_GiB_decoded": n_hit * cb / 2**30,
+                "kernel_ms": ms, "unpack_GBps_payload": n_hit * cb / ms["unpack"] / 1e6,
+                "unpack_hbm_frac_of_peak": 2 * n_hit * cb / ms["unpack"] / 1e6 / peak,
+                "note": "the arena (16 GiB) is re-read about %.0f times, so its reads partly hit L2; "
+                        "the fraction counts read + write bytes as if all came from HBM"
+                        % (n_hit / n_blobs)}
+    finally:
+        ctx.close()
+        del dst, arena
+        torch.cuda.empty_cache()
+
+
 def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
+    peak, peak_src = hbm_peak()
     """Probe throughput on the probe-heavy workload (configs[2]): 1M stored chunk keys in four
     sorted runs (900 / 9000 / 90000 / 900100 keys, 1% newer duplicates), 4096 queries of 2k-32k
     tokens, 60% with a cached prefix. Keys come from the library's own encoder and the runs from
@@ -694,41 +1103,17 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
                 "algorithmic_GBps": algo_bytes / ms / 1e6,
                 "flush_ms_for_%d_keys" % big: flush_big_ms,
                 "exact_index": exact,
-                "roofline": probe_roofline(torch, device_index, ms),
-                "bound": "instruction issue and dependent L2 loads (not HBM)"}
+                # the probe's least traffic (tokens up to the first miss, a record per query chunk,
+                # a hit length per query) against the measured copy bandwidth: small by nature --
+                # the kernel is bound by integer issue and dependent L2 loads, not by HBM
+                "roofline": {"bound": "hbm", "kernel": "k_probe<true>",
+                             "achieved": algo_bytes / ms / 1e6, "peak": peak, "unit": "GB/s",
+                             "frac": algo_bytes / ms / 1e6 / peak, "peak_source": peak_src,
+                             "algorithmic_bytes_per_launch": algo_bytes, "traffic": None},
+                "bound": "instruction issue and dependent L2 loads (issue-slot counters: see the "
+                         "committed ncu summary of k_probe on this workload)"}
     finally:
         ctx.close()
-
-
-# Warp instructions of one k_probe<true> launch on this workload: ncu smsp__inst_executed.sum of
-# the capture summarised under profiles/ (k_probe, probe-heavy workload). Set to None whenever the
-# kernel changes until the counter has been taken again.
-PROBE_WARP_INSTRUCTIONS = 64280836
-
-
-def probe_roofline(torch, device_index, ms):
-    """The probe is integer arithmetic plus dependent loads, so its ceiling is the rate at which
-    the SMs can issue instructions: SMs x 4 schedulers x 1 warp instruction per cycle x the
-    maximum SM clock."""
-    props = torch.cuda.get_device_properties(device_index)
-    try:
-        import pynvml
-        pynvml.nvmlInit()
-        h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
-        mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
-    except Exception:
-        mhz = 1965.0
-    peak = props.multi_processor_count * 4 * mhz * 1e6 / 1e9          # G warp instructions / s
-    if PROBE_WARP_INSTRUCTIONS is None:
-        return {"bound": "alu", "kernel": "k_probe<true>", "achieved": None, "peak": peak,
-                "unit": "G warp instructions/s", "frac": None}
-    achieved = PROBE_WARP_INSTRUCTIONS / ms / 1e6
-    return {"bound": "alu", "kernel": "k_probe<true>", "achieved": achieved, "peak": peak,
-            "unit": "G warp instructions/s", "frac": achieved / peak,
-            "peak_source": "SMs x 4 warp schedulers x max SM clock (%d x 4 x %.0f MHz)"
-                           % (props.multi_processor_count, mhz),
-            "instructions_per_launch": PROBE_WARP_INSTRUCTIONS,
-            "instructions_source": "ncu smsp__inst_executed.sum of one launch on this workload"}
 
 
 def exact_index_numbers(torch, ctx, w, up, d_tok, d_off, d_qoff, total, d_hit, d_recs, warm, reps):
@@ -824,8 +1209,43 @@ def xp12_block(torch, lsmkv, dev, device_index, d, src_bufs, src_pool, dst_bufs,
         ctx.close()
 
 
+def link_ceiling(torch, dev, nbytes=1 << 30, reps=3):
+    """What the host link gives in this run: pinned cudaMemcpyAsync of `nbytes` host->device and
+    device->host at the same time on two streams (GB/s, summed over both directions), and each
+    direction alone."""
+    hp_in = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    hp_out = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    d_in = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    d_out = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+    hp_in.zero_()
+    s_a, s_b = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+
+    def run(up, down):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        s_a.wait_event(e0)
+        s_b.wait_event(e0)
+        for _ in range(reps):
+            if up:
+                with torch.cuda.stream(s_a):
+                    d_in.copy_(hp_in, non_blocking=True)
+            if down:
+                with torch.cuda.stream(s_b):
+                    hp_out.copy_(d_out, non_blocking=True)
+        torch.cuda.current_stream().wait_stream(s_a)
+        torch.cuda.current_stream().wait_stream(s_b)
+        e1.record()
+        torch.cuda.synchronize()
+        return (int(up) + int(down)) * reps * nbytes / e0.elapsed_time(e1) / 1e6
+
+    run(True, True)                                      # warm-up (pages the pinned buffers in)
+    return {"h2d_GBps": run(True, False), "d2h_GBps": run(False, True),
+            "both_directions_GBps": run(True, True), "bytes_per_copy": nbytes}
+
+
 def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barrier, world,
-            label):
+            label, link=None):
     """Same path through the host-buffer entry points of the C ABI: per sub-batch the token
     sequences and page tables are HOST arrays, the packed blobs, keys and records come back to
     pinned host memory (where a tensor-log writer would take them), the probe returns hit
@@ -971,9 +1391,13 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
     moved = ranks.sum_over_ranks(moved, dev)
     steps = max(1, args.e2e_steps)
     ctx.last_status()
+    pcie = (h2d + d2h) / (e0.elapsed_time(e1) * 1e-3) / 1e9          # this rank's link traffic
     return {"value": ranks.whole_job_rate(moved, ms) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
             "steps": steps, "ms_per_step": ms / steps, "codec": label,
+            "link_GBps_both_directions": link["both_directions_GBps"] if link else None,
+            "link_traffic_GBps": pcie,
+            "frac_of_link": pcie / link["both_directions_GBps"] if link else None,
             "api": "lsmkv_put_batch_host / lsmkv_probe_batch_host / lsmkv_decode_batch_host",
             "note": "host buffers in and out through the C ABI: blobs, keys and records land in "
                     "pinned host memory, hit blobs are copied back from it before the scatter; "

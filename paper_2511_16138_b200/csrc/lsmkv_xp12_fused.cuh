@@ -1,24 +1,28 @@
 // One-pass encoder of the compressing codec "xp12": every page slab is read from the pool once.
 //
 // The three-step encoder (lsmkv_xp12.cuh) reads the pool twice, because where a slab lands
-// depends on the sizes of all slabs before it. Here a slab stays on the SM between being
-// measured and being written: a persistent CTA per SM runs a pipeline of
-//   producer warp   draws the next slab number from a counter, fetches the slab into a ring of
-//                   shared-memory stages with one bulk copy (cp.async.bulk, mbarrier-completed);
-//   compute groups  (8 or 16 warps) take the slab into registers, find its exponent window and
-//                   exception count, publish its encoded size, and build the encoded slab in a
-//                   ring of shared-memory output buffers;
-//   commit warps    one per output buffer: sum the sizes of all earlier slabs (decoupled
-//                   look-back over a per-slab state word: empty / size known / prefix known),
-//                   publish the prefix, and send the buffer to its place with one bulk copy.
-// Slab numbers are handed out in order by the counter, so every slab a look-back waits for is
-// held by a CTA that is already running. A small kernel afterwards (k_xpf_layout) turns the
-// prefixes into chunk directories and records. Bytes out are those of the three-step encoder.
+// depends on the sizes of all slabs before it. Here a slab stays on the SM, in a ring of
+// shared-memory stages, between being measured and being written. A persistent CTA per SM runs
+//   producer warp    draws the next slab number from a counter and fetches the slab into the
+//                    ring with one bulk copy (cp.async.bulk, mbarrier-completed);
+//   measuring warps  take each slab as it lands: exponent window and exception count give its
+//                    encoded size, which is published at once;
+//   look-back warps  sum the sizes of all earlier slabs (decoupled look-back over a per-slab
+//                    state word: empty / size known / prefix known), publish the prefix and
+//                    hand the slab's place on;
+//   packing warps    encode the slab straight into its final place in the blob, then free the
+//                    stage.
+// The three run side by side on different slabs of the ring, so each one's chain of short
+// dependent steps (waits, shuffles, barriers) hides behind the others' arithmetic, and a slab's
+// size is known well before its turn to be packed, which absorbs the differences in pace
+// between the SMs. Slab numbers are handed out in order by the counter, so
+// every slab a look-back waits for is held by a CTA that is already running. A small kernel
+// afterwards (k_xpf_layout) turns the prefixes into chunk directories and records. Bytes out
+// are those of the three-step encoder.
 //
 // Every wait is bounded (the mbarrier waits and the look-back polls give up after `wait_cycles`
 // clock cycles, set LSMKV_ST_WAIT_EXPIRED and an abort word that makes every other wait of the
-// launch return at its next poll); a CTA leaves only after the bulk copies it issued have
-// finished with its shared memory.
+// launch return at its next poll); the producer leaves only after its fetches have landed.
 #pragma once
 #include "lsmkv_common.cuh"
 #include "lsmkv_copy.cuh"
@@ -32,24 +36,22 @@ constexpr uint64_t kFlagIncl = 2ull << 62;     // low 62 bits: bytes of all slab
 constexpr uint64_t kValueMask = (1ull << 62) - 1;
 constexpr uint64_t kEnd = ~0ull;               // slab number that tells a role to stop
 
-// Shape of the pipeline for a slab of kWpg * kSweeps * 256 elements.
-template <int SWEEPS, int WPG, int GROUPS, int RAW, int OUT>
+// Shape of the pipeline for a slab of WARPS * SWEEPS * 256 elements: WARPS packing warps, each
+// owning a contiguous part of SWEEPS * 256 elements; WARPS / SPLIT measuring warps, each covering
+// SPLIT such parts; RING stages; LB look-back warps that share the slabs round-robin.
+template <int SWEEPS, int WARPS, int SPLIT, int RING, int LB>
 struct Shape {
-    static constexpr int kSweeps = SWEEPS, kWpg = WPG, kGroups = GROUPS, kRaw = RAW, kOut = OUT;
-    static constexpr int kElems = WPG * SWEEPS * 256;
+    static constexpr int kSweeps = SWEEPS, kWarps = WARPS, kSplit = SPLIT, kRing = RING, kLb = LB;
+    static constexpr int kMeasureWarps = WARPS / SPLIT, kMeasureSweeps = SWEEPS * SPLIT;
+    static constexpr int kElems = WARPS * SWEEPS * 256;
     static constexpr int kPageBytes = 2 * kElems;
-    static constexpr int kOutStride = kPageBytes + 128;              // header + raw slab, padded
-    static constexpr int kComputeWarps = WPG * GROUPS;
-    static constexpr int kProducerWarp = kComputeWarps;
-    static constexpr int kFirstCommitWarp = kComputeWarps + 1;
-    static constexpr int kWarps = kComputeWarps + 1 + OUT;
-    static constexpr int kThreads = kWarps * 32;
-    static constexpr size_t kSmem = (size_t)RAW * kPageBytes + (size_t)OUT * kOutStride + 1024;
-    // A ring position must always come back to the same group: a waiter tells phases apart by
-    // their parity only, which is safe as long as it cannot be two phases ahead of the barrier --
-    // true when the group that waits for use n of a stage is the one that finished use n - 1
-    // of it, false when another group, running behind, still owes that use.
-    static_assert(RAW % GROUPS == 0 && OUT % GROUPS == 0, "rings must divide among the groups");
+    static constexpr int kFirstPackWarp = kMeasureWarps;
+    static constexpr int kProducerWarp = kMeasureWarps + WARPS;
+    static constexpr int kFirstLbWarp = kProducerWarp + 1;
+    static constexpr int kThreads = (kMeasureWarps + WARPS + 1 + LB) * 32;
+    static constexpr size_t kSmem = (size_t)RING * kPageBytes + 2048;
+    static_assert(RING >= 3 && LB >= 1 && WARPS <= 16 && WARPS % SPLIT == 0 && kMeasureSweeps <= 32,
+                  "shape out of range");
 };
 
 struct Job {
@@ -178,6 +180,7 @@ __device__ __forceinline__ bool look_back(const Job &job, uint64_t u, uint64_t *
             if (first < 32u) done = true; else pos -= 32;
         }
         if (done) break;
+        if (stalled) __nanosleep(256);                    // a size is on its way: do not hammer L2
         if (stalled && (++polls & 15u) == 0) {
             const bool give_up = ld_abort(job.abort) != 0u || clock64() - t0 > job.wait_cycles;
             if (__any_sync(0xFFFFFFFFu, give_up)) return false;
@@ -189,50 +192,42 @@ __device__ __forceinline__ bool look_back(const Job &job, uint64_t u, uint64_t *
 
 }  // namespace xpf
 
-// Dynamic shared memory: kRaw stages of page_bytes, kOut output buffers, barriers and mailboxes.
+// Dynamic shared memory: kRing stages of page_bytes, then barriers and per-stage mailboxes.
 template <class S>
 __global__ void __launch_bounds__(S::kThreads, 1)
 k_xpf_encode(const __grid_constant__ xpf::Job job)
 {
     using namespace xpf;
     extern __shared__ __align__(128) unsigned char xpf_smem[];
-    constexpr int N = S::kElems;
-    unsigned char *raw = xpf_smem;
-    unsigned char *outb = xpf_smem + (size_t)S::kRaw * S::kPageBytes;
-    unsigned char *tail = outb + (size_t)S::kOut * S::kOutStride;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);             // 2 * kRaw + 4 * kOut
-    uint64_t *raw_slab = bars + 2 * S::kRaw + 4 * S::kOut;           // [kRaw] slab number or kEnd
-    uint32_t *raw_ok = reinterpret_cast<uint32_t *>(raw_slab + S::kRaw);   // [kRaw] page usable
-    // per output buffer, by parity of its use: the slab it will hold (or kEnd) and its size
-    uint64_t *out_slab = reinterpret_cast<uint64_t *>(raw_ok + S::kRaw + (S::kRaw & 1));
-    uint32_t *out_size = reinterpret_cast<uint32_t *>(out_slab + 2 * S::kOut);  // [kOut][2]
-    uint32_t *red = out_size + 2 * S::kOut;                          // [kGroups][2][kWpg]
-    uint32_t *n_real = red + S::kGroups * 2 * S::kWpg;               // slabs this CTA was handed
+    constexpr int N = S::kElems, R = S::kRing, W = S::kWarps, WM = S::kMeasureWarps,
+                  SM = S::kMeasureSweeps;
+    unsigned char *ring = xpf_smem;
+    unsigned char *tail = xpf_smem + (size_t)R * S::kPageBytes;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);             // 4 per stage
+    uint64_t *slot_u = bars + 4 * R;                                 // producer: slab number / kEnd
+    uint64_t *m_u = slot_u + R;                                      // measure: the same, for the look-back
+    uint64_t *m_prefix = m_u + R;                                    // look-back: bytes before the slab
+    uint32_t *slot_ok = reinterpret_cast<uint32_t *>(m_prefix + R);  // producer: page usable
+    uint32_t *m_size = slot_ok + R;                                  // measure: encoded size
+    uint32_t *m_info = m_size + R;                                   // measure: base | packed << 8
+    uint32_t *m_nexc = m_info + R;                                   // measure: exceptions of the slab
+    uint32_t *m_wcnt = m_nexc + R;                                   // measure: [R][W] exceptions per part
+    uint32_t *m_wsweeps = m_wcnt + R * W;                            // measure: [R][W] sweeps that have any
+    uint32_t *red_max = m_wsweeps + R * W;                           // [WM]
 
     const uint32_t bar0 = smem_addr(bars);
-    auto raw_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    auto raw_empty = [&](int s) { return bar0 + 8u * (uint32_t)(S::kRaw + s); };
-    auto out_full = [&](int s) { return bar0 + 8u * (uint32_t)(2 * S::kRaw + s); };
-    auto out_empty = [&](int s) { return bar0 + 8u * (uint32_t)(2 * S::kRaw + S::kOut + s); };
-    // "the size of the slab that buffer s will hold in its use n is known", one barrier per
-    // parity of n: the commit warp starts its look-back there, while the slab is still being
-    // packed. Two barriers, because the group announces use n + 1 before the commit warp is
-    // known to have seen the announcement of use n; use n + 2 it cannot reach before that.
-    auto size_known = [&](int s, uint32_t n) {
-        return bar0 + 8u * (uint32_t)(2 * S::kRaw + 2 * S::kOut + 2 * s + (int)(n & 1u));
-    };
+    auto raw_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };              // fetch landed
+    auto raw_empty = [&](int s) { return bar0 + 8u * (uint32_t)(R + s); };       // packing warps done with it
+    auto measured = [&](int s) { return bar0 + 8u * (uint32_t)(2 * R + s); };    // size known
+    auto placed = [&](int s) { return bar0 + 8u * (uint32_t)(3 * R + s); };      // prefix known
 
     const unsigned warp = threadIdx.x >> 5, lane = lane_id();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S::kRaw; ++s) {
+        for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);                    // the producer's arrive (+ copy bytes)
-            mbar_init(raw_empty(s), S::kWpg);             // one arrive per warp of the group
-        }
-        for (int s = 0; s < S::kOut; ++s) {
-            mbar_init(out_full(s), S::kWpg * 32);         // every thread of the group
-            mbar_init(out_empty(s), 1);                   // the commit warp
-            mbar_init(size_known(s, 0), 1);               // one thread of the group
-            mbar_init(size_known(s, 1), 1);
+            mbar_init(raw_empty(s), W);                   // one arrive per packing warp
+            mbar_init(measured(s), 1);                    // one measuring thread
+            mbar_init(placed(s), 1);                      // one look-back lane
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -270,49 +265,46 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         bool ended = false;
         uint64_t u_a = draw(false), u_b = draw(false), u_c = draw(false);
         Where w_a = locate(u_a);
-        int ends = 0;
         uint32_t fetch_mask = 0, fetch_parity = 0;        // per stage: last arm was a fetch / its phase
         for (uint32_t k = 0;; ++k) {
             const uint64_t u_d = draw(ended);             // three slabs ahead
             const Where w_b = locate(u_b);                // one slab ahead
             ended = ended || u_b >= total;
-            const int s = (int)(k % S::kRaw);
-            const uint32_t ph = (k / S::kRaw) & 1u;
+            const int s = (int)(k % R);
+            const uint32_t ph = (k / R) & 1u;
             if (!mbar_wait(raw_empty(s), ph ^ 1u, job)) { raise_abort(job, 0); break; }
-            if (u_a >= total) {                           // every group gets its own stop mark
-                if (ends == 0) *n_real = k;
-                raw_slab[s] = kEnd;
+            if (u_a >= total) {                           // the stop mark
+                slot_u[s] = kEnd;
                 fetch_mask &= ~(1u << s);
                 mbar_arrive(raw_full(s));
-                if (++ends == S::kGroups) break;
+                break;
+            }
+            if (w_a.ok == 2u && w_a.first_of_page) st_flag(job.x.st, LSMKV_ST_BAD_PAGE, w_a.chunk);
+            if (w_a.ok == 3u) st_flag(job.x.st, LSMKV_ST_MISALIGNED, w_a.chunk);
+            slot_u[s] = u_a;
+            slot_ok[s] = w_a.ok == 1u ? 1u : 0u;
+            if (w_a.ok == 1u) {
+                mbar_arrive_expect(raw_full(s), (uint32_t)S::kPageBytes);
+                asm volatile(
+                    "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes"
+                    " [%0], [%1], %2, [%3];"
+                    :: "r"(smem_addr(ring + (size_t)s * S::kPageBytes)), "l"(w_a.src),
+                       "r"((uint32_t)S::kPageBytes), "r"(raw_full(s)) : "memory");
+                fetch_mask |= 1u << s;
+                fetch_parity = (fetch_parity & ~(1u << s)) | (ph << s);
             } else {
-                if (w_a.ok == 2u && w_a.first_of_page) st_flag(job.x.st, LSMKV_ST_BAD_PAGE, w_a.chunk);
-                if (w_a.ok == 3u) st_flag(job.x.st, LSMKV_ST_MISALIGNED, w_a.chunk);
-                raw_slab[s] = u_a;
-                raw_ok[s] = w_a.ok == 1u ? 1u : 0u;
-                if (w_a.ok == 1u) {
-                    mbar_arrive_expect(raw_full(s), (uint32_t)S::kPageBytes);
-                    asm volatile(
-                        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes"
-                        " [%0], [%1], %2, [%3];"
-                        :: "r"(smem_addr(raw + (size_t)s * S::kPageBytes)), "l"(w_a.src),
-                           "r"((uint32_t)S::kPageBytes), "r"(raw_full(s)) : "memory");
-                    fetch_mask |= 1u << s;
-                    fetch_parity = (fetch_parity & ~(1u << s)) | (ph << s);
-                } else {
-                    fetch_mask &= ~(1u << s);
-                    mbar_arrive(raw_full(s));
-                }
+                fetch_mask &= ~(1u << s);
+                mbar_arrive(raw_full(s));
             }
             u_a = u_b; w_a = w_b;
             u_b = u_c;
             u_c = u_d;
         }
         // Do not leave while a fetch may still be writing this CTA's shared memory. A stage
-        // whose last arm was a fetch is waited for here (its group normally did so long ago); a
-        // stage armed again since (stop mark, unusable page) had its earlier fetch consumed
+        // whose last arm was a fetch is waited for here (the compute warps normally did so long
+        // ago); a stage armed again since (stop mark, unusable page) had its earlier fetch read
         // before the producer was let back in.
-        for (int s = 0; s < S::kRaw; ++s) {
+        for (int s = 0; s < R; ++s) {
             if (!(fetch_mask >> s & 1u)) continue;
             const long long t0 = clock64();
             while (!mbar_try(raw_full(s), (fetch_parity >> s) & 1u))
@@ -321,223 +313,244 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         return;
     }
 
-    if (warp >= (unsigned)S::kFirstCommitWarp) {
-        // ---- commit warp c: slabs k = c, c + kOut, ... of this CTA, buffer c
-        const int c = (int)warp - S::kFirstCommitWarp;
-        const uint32_t obuf = smem_addr(outb + (size_t)c * S::kOutStride);
-        for (uint32_t n = 0;; ++n) {
+    if (warp >= (unsigned)S::kFirstLbWarp) {
+        // ---- look-back warp c: slabs k = c, c + kLb, ... of this CTA, as soon as they are measured
+        const uint32_t c = warp - (unsigned)S::kFirstLbWarp;
+        for (uint32_t k = c;; k += S::kLb) {
+            const int s = (int)(k % R);
             bool ok = true;
-            if (lane == 0) ok = mbar_wait(size_known(c, n), (n >> 1) & 1u, job);
+            if (lane == 0) ok = mbar_wait(measured(s), (k / R) & 1u, job);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok) { if (lane == 0) raise_abort(job, 0); break; }
-            uint64_t u = lane == 0 ? out_slab[2 * c + (n & 1u)] : 0;   // read by the lane that waited
-            uint32_t size = lane == 0 ? out_size[2 * c + (n & 1u)] : 0;
+            uint64_t u = lane == 0 ? m_u[s] : 0;          // read by the lane that waited
+            uint32_t size = 0;
+            if (lane == 0) size = m_size[s] + (u != kEnd && (m_info[s] & 0x200u) ? job.x.dir_bytes : 0u);
             u = __shfl_sync(0xFFFFFFFFu, u, 0);
             size = __shfl_sync(0xFFFFFFFFu, size, 0);
-            if (u == kEnd) break;
-            const bool first = u % slabs == 0;            // the chunk's directory goes before it
-            const uint64_t add = (uint64_t)size + (first ? job.x.dir_bytes : 0u);
+            if (u == kEnd) {
+                if (size != 0 && lane == 0) mbar_arrive(placed(s));   // the packing warps stop too
+                break;
+            }
+            const uint64_t add = size;                    // bytes the slab adds to the blob
             uint64_t before = 0;
             if (!look_back(job, u, &before)) { if (lane == 0) raise_abort(job, u); break; }
             if (lane == 0) {
+                m_prefix[s] = before;
+                mbar_arrive(placed(s));                   // the compute warps may pack it
                 st_state(job.state + u, kFlagIncl | (before + add));
-                ok = mbar_wait(out_full(c), n & 1u, job);             // the packed slab is there
-                if (ok) {
-                    if (before + add <= job.x.blob_capacity) {
-                        unsigned char *dst = job.x.blob + before + (first ? job.x.dir_bytes : 0u);
-                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                                     :: "l"(dst), "r"(obuf), "r"(size) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    } else {
-                        st_flag(job.x.st, LSMKV_ST_OVERFLOW, u / slabs);
-                    }
-                    mbar_arrive(out_empty(c));
-                }
             }
-            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-            if (!ok) { if (lane == 0) raise_abort(job, u); break; }
+            __syncwarp();
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         return;
     }
 
-    // ---- compute group g: slabs k = g, g + kGroups, ... of this CTA
-    const int g = (int)warp / S::kWpg;
-    const unsigned gw = warp - (unsigned)g * S::kWpg;     // warp within the group
-    const unsigned gt = threadIdx.x - (unsigned)g * S::kWpg * 32u;
-    uint32_t *red_max = red + (size_t)g * 2 * S::kWpg, *red_cnt = red_max + S::kWpg;
-    const uint32_t k_first = gw * S::kSweeps * 32 + lane; // this lane's first 16 bytes of the slab
-    bool dead = false;                                    // a wait gave up: skip the rest
-    for (uint32_t k = (uint32_t)g;; k += S::kGroups) {
-        const int rs = (int)(k % S::kRaw), os = (int)(k % S::kOut);
-        if (!dead && !mbar_wait(raw_full(rs), (k / S::kRaw) & 1u, job)) dead = true;
-        uint64_t u = kEnd;
-        bool page_ok = false;
-        uint4 q[S::kSweeps];
-        if (!dead) {
-            u = raw_slab[rs];
-            page_ok = u != kEnd && raw_ok[rs] != 0u;
-        }
-        if (page_ok) {
-            const uint4 *s4 = reinterpret_cast<const uint4 *>(raw + (size_t)rs * S::kPageBytes);
+    if (warp < (unsigned)S::kFirstPackWarp) {
+        // ---- measuring warps: slab j of this CTA as soon as it has landed
+        const unsigned gt = threadIdx.x;                  // thread within the measuring group
+        const uint32_t k_first = warp * SM * 32 + lane;   // this lane's first 16 bytes of a slab
+        bool dead = false;                                // a wait gave up: do nothing but leave
+        for (uint32_t j = 0;; ++j) {
+            const int s = (int)(j % R);
+            if (!dead && !mbar_wait(raw_full(s), (j / R) & 1u, job)) dead = true;
+            uint64_t u = kEnd;
+            bool page_ok = false;
+            if (!dead) {
+                u = slot_u[s];
+                page_ok = u != kEnd && slot_ok[s] != 0u;
+            }
+            // the largest exponent field of the slab, and the smallest of every sweep (an
+            // unusable page measures as zeros)
+            uint32_t least[SM];
+            uint32_t m = 0;
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(ring + (size_t)s * S::kPageBytes);
 #pragma unroll
-            for (int s = 0; s < S::kSweeps; ++s) q[s] = s4[k_first + s * 32];
-        } else {
+            for (int e = 0; e < SM; ++e) {
+                const uint4 v = page_ok ? s4[k_first + e * 32] : make_uint4(0, 0, 0, 0);
+                const uint32_t f0 = v.x & 0x7F807F80u, f1 = v.y & 0x7F807F80u,
+                               f2 = v.z & 0x7F807F80u, f3 = v.w & 0x7F807F80u;
+                m = __vimax3_u16x2(m, f0, f1);
+                m = __vimax3_u16x2(m, f2, f3);
+                least[e] = __vimin3_u16x2(__vimin3_u16x2(f0, f1, f2), f3, f3);
+            }
+            m = max(m & 0xFFFFu, m >> 16);
 #pragma unroll
-            for (int s = 0; s < S::kSweeps; ++s) q[s] = make_uint4(0, 0, 0, 0);
-        }
-        __syncwarp();
-        if (!dead && lane == 0) mbar_arrive(raw_empty(rs));   // the stage may be refilled
-        // exponent fields of the slab's words (kept: the window test and the codes start from
-        // them) and the largest of them
-        uint32_t t[4 * S::kSweeps], least[S::kSweeps];    // least: smallest fields of a sweep
-        uint32_t m = 0;
+            for (int d = 16; d; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
+            if (lane == 0) red_max[warp] = m;
+            // group barrier; it also tells every thread whether any of them gave up on a wait
+            int any_dead;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "barrier.cta.red.or.pred p, 1, %2, q;\n\t"
+                "selp.s32 %0, 1, 0, p;\n\t}"
+                : "=r"(any_dead) : "r"(dead ? 1u : 0u), "r"(WM * 32) : "memory");
+            if (any_dead) {
+                if (gt == 0) raise_abort(job, u == kEnd ? 0 : u);
+                break;
+            }
+            if (u == kEnd) {
+                // No more slabs. Every look-back warp gets a stop mark at its next position, and
+                // passes it on to the packing warps. The stages of positions j + 1 .. are only
+                // borrowed for their mailboxes and barriers: the producer has stopped, and a
+                // stage's earlier slab is always handed on before the stage is used again.
+                if (gt == 0) {
+                    for (uint32_t k2 = j; k2 < j + (uint32_t)S::kLb; ++k2) {
+                        const int s2 = (int)(k2 % R);
+                        if (k2 != j && !mbar_wait(raw_empty(s2), ((k2 / R) & 1u) ^ 1u, job)) {
+                            raise_abort(job, 0);
+                            break;
+                        }
+                        m_u[s2] = kEnd;
+                        m_size[s2] = k2 == j ? 1u : 0u;   // the first mark goes on to the packing warps
+                        mbar_arrive(measured(s2));
+                    }
+                }
+                break;
+            }
+            uint32_t emax = 0;
 #pragma unroll
-        for (int s = 0; s < S::kSweeps; ++s) {
-            t[4 * s] = q[s].x & 0x7F807F80u; t[4 * s + 1] = q[s].y & 0x7F807F80u;
-            t[4 * s + 2] = q[s].z & 0x7F807F80u; t[4 * s + 3] = q[s].w & 0x7F807F80u;
-            m = __vimax3_u16x2(m, t[4 * s], t[4 * s + 1]);
-            m = __vimax3_u16x2(m, t[4 * s + 2], t[4 * s + 3]);
-            least[s] = __vimin3_u16x2(__vimin3_u16x2(t[4 * s], t[4 * s + 1], t[4 * s + 2]),
-                                      t[4 * s + 3], t[4 * s + 3]);
-        }
-        m = max(m & 0xFFFFu, m >> 16);
+            for (int w = 0; w < WM; ++w) emax = max(emax, red_max[w]);
+            emax >>= 7;
+            const uint32_t base = emax > 14u ? emax - 14u : 0u;
+            const uint32_t lift = xpfast::window_lift(base);
+            // A field plus `lift` has bit 15 of its half set exactly when the element is in the
+            // window. Elements below it are rare: a sweep is only looked at closely (and its
+            // count taken) when its smallest fields say the warp has one.
+            // (the sweep is then read again from the stage, which stays as it is until packed).
+            // Counts and sweep masks are kept per part of the slab, one part per packing warp.
+            uint32_t my_exc[S::kSplit], exc_sweeps[S::kSplit];
 #pragma unroll
-        for (int d = 16; d; d >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, d));
-        if (lane == 0) red_max[gw] = m;
-        // group barrier; it also tells every thread whether any of them gave up on a wait
-        int any_dead;
-        asm volatile(
-            "{\n\t.reg .pred p, q;\n\t"
-            "setp.ne.u32 q, %1, 0;\n\t"
-            "barrier.cta.red.or.pred p, %2, %3, q;\n\t"
-            "selp.s32 %0, 1, 0, p;\n\t}"
-            : "=r"(any_dead) : "r"(dead ? 1u : 0u), "r"(1 + g), "r"(S::kWpg * 32) : "memory");
-        if (any_dead) {
-            if (gt == 0) raise_abort(job, u == kEnd ? 0 : u);
-            break;
-        }
-        if (u == kEnd) {
-            // Stop marks for the commit warps: the buffers of the kOut slab positions that follow
-            // the CTA's last real slab each get one, from the group whose turn that position is.
-            const uint32_t K = *n_real;
-            if (gt == 0) {
-                for (uint32_t k2 = K; k2 < K + (uint32_t)S::kOut; ++k2) {
-                    if (k2 % S::kGroups != (uint32_t)g) continue;
-                    const int o2 = (int)(k2 % S::kOut);
-                    const uint32_t n2 = k2 / S::kOut;
-                    // (the mailbox of this parity was last used two uses ago, and this group
-                    // packed the use between them only after the commit warp was done with that)
-                    out_slab[2 * o2 + (n2 & 1u)] = kEnd;
-                    mbar_arrive(size_known(o2, n2));
+            for (int p = 0; p < S::kSplit; ++p) my_exc[p] = exc_sweeps[p] = 0;
+#pragma unroll
+            for (int e = 0; e < SM; ++e) {
+                const uint32_t below = ~(least[e] + lift) & 0x80008000u;
+                if (__any_sync(0xFFFFFFFFu, below != 0)) {
+                    const uint4 v = page_ok ? s4[k_first + e * 32] : make_uint4(0, 0, 0, 0);
+                    my_exc[e / S::kSweeps] +=
+                        8u - (__popc(((v.x & 0x7F807F80u) + lift) & 0x80008000u) +
+                              __popc(((v.y & 0x7F807F80u) + lift) & 0x80008000u) +
+                              __popc(((v.z & 0x7F807F80u) + lift) & 0x80008000u) +
+                              __popc(((v.w & 0x7F807F80u) + lift) & 0x80008000u));
+                    exc_sweeps[e / S::kSweeps] |= 1u << (e % S::kSweeps);
                 }
             }
-            break;
-        }
-        uint32_t emax = 0;
 #pragma unroll
-        for (int w = 0; w < S::kWpg; ++w) emax = max(emax, red_max[w]);
-        emax >>= 7;
-        const uint32_t base = emax > 14u ? emax - 14u : 0u;
-        const uint32_t lift = xpfast::window_lift(base);
-        // A field plus `lift` has bit 15 of its half set exactly when the element is in the
-        // window, and then bits 7..10 of the half hold e - base with zeros up to bit 14. Elements
-        // below the window are rare: a sweep is only looked at closely (and its count taken) when
-        // its smallest fields say the warp has one.
-        uint32_t my_exc = 0, exc_sweeps = 0;              // this lane's count; sweeps that had any
+            for (int p = 0; p < S::kSplit; ++p) {
+                uint32_t part_exc = 0;
+                if (exc_sweeps[p]) {                      // the same in every lane of the warp
+                    part_exc = my_exc[p];
 #pragma unroll
-        for (int s = 0; s < S::kSweeps; ++s) {
-            const uint32_t below = ~(least[s] + lift) & 0x80008000u;
-            if (__any_sync(0xFFFFFFFFu, below != 0)) {
-                my_exc += 8u - (__popc((t[4 * s] + lift) & 0x80008000u) +
-                                __popc((t[4 * s + 1] + lift) & 0x80008000u) +
-                                __popc((t[4 * s + 2] + lift) & 0x80008000u) +
-                                __popc((t[4 * s + 3] + lift) & 0x80008000u));
-                exc_sweeps |= 1u << s;
+                    for (int d = 16; d; d >>= 1) part_exc += __shfl_xor_sync(0xFFFFFFFFu, part_exc, d);
+                }
+                if (lane == 0) {
+                    m_wcnt[s * W + warp * S::kSplit + p] = part_exc;
+                    m_wsweeps[s * W + warp * S::kSplit + p] = exc_sweeps[p];
+                }
+            }
+            asm volatile("barrier.cta.sync 1, %0;" :: "r"(WM * 32) : "memory");
+            if (gt == 0) {
+                uint32_t n_exc = 0;
+#pragma unroll
+                for (int w = 0; w < W; ++w) {             // counts become "exceptions before the part"
+                    const uint32_t c = m_wcnt[s * W + w];
+                    m_wcnt[s * W + w] = n_exc;
+                    n_exc += c;
+                }
+                const bool packed = page_ok && n_exc < (uint32_t)N / 2;
+                const uint32_t size = packed ? round16u(16u + N + N / 2 + n_exc) : 16u + 2u * N;
+                const bool first = u % slabs == 0;        // the chunk's directory goes before it
+                m_u[s] = u;
+                m_size[s] = size;
+                m_info[s] = base | (packed ? 0x100u : 0u) | (first ? 0x200u : 0u);
+                m_nexc[s] = n_exc;
+                mbar_arrive(measured(s));                 // a look-back warp takes it from here
+                // (after the arrive: an arrive orders the stores before it, and would sit out
+                // this one's trip to L2)
+                st_state(job.state + u, kFlagAgg | ((uint64_t)size + (first ? job.x.dir_bytes : 0u)));
             }
         }
-        // The fields are kept as f * 4097 = f + (f << 12) with f = field + lift: for a word whose
-        // two elements are in the window that sets the low element's code right below the high
-        // one's (bits 19..22 and 23..26: one byte's worth), and nothing overlaps or carries.
-        const uint32_t lift4097 = lift * 4097u;
+        return;
+    }
+
+    // ---- packing warps: slab k of this CTA once its place is known, straight into the blob.
+    // Each warp runs on its own: no barrier, only the stage's mbarriers.
+    const unsigned pw = warp - (unsigned)S::kFirstPackWarp;   // which part of a slab is this warp's
+    const unsigned pt = threadIdx.x - (unsigned)S::kFirstPackWarp * 32u;
+    const uint32_t k_first = pw * S::kSweeps * 32 + lane;     // this lane's first 16 bytes of a slab
+    for (uint32_t k = 0;; ++k) {
+        const int s = (int)(k % R);
+        if (!mbar_wait(placed(s), (k / R) & 1u, job)) { raise_abort(job, 0); break; }
+        const uint64_t u = m_u[s];
+        if (u == kEnd) break;
+        const uint64_t before_bytes = m_prefix[s];
+        const uint32_t size = m_size[s], info = m_info[s], n_exc = m_nexc[s];
+        const bool packed = (info & 0x100u) != 0u, page_ok = slot_ok[s] != 0u;
+        const uint32_t my_sweeps = m_wsweeps[s * W + pw];
+        const uint32_t exc_before = m_wcnt[s * W + pw];   // exceptions of the parts before this one
+        uint4 q[S::kSweeps];
+        {
+            const uint4 *s4 = reinterpret_cast<const uint4 *>(ring + (size_t)s * S::kPageBytes);
 #pragma unroll
-        for (int e = 0; e < 4 * S::kSweeps; ++e) t[e] = mad_u32(t[e], 4097u, lift4097);
-        uint32_t warp_exc = 0;
-        if (exc_sweeps) {                                 // the same in every lane of the warp
-            warp_exc = my_exc;
-#pragma unroll
-            for (int d = 16; d; d >>= 1) warp_exc += __shfl_xor_sync(0xFFFFFFFFu, warp_exc, d);
+            for (int e = 0; e < S::kSweeps; ++e)
+                q[e] = page_ok ? s4[k_first + e * 32] : make_uint4(0, 0, 0, 0);
         }
-        if (lane == 0) red_cnt[gw] = warp_exc;
-        asm volatile("barrier.cta.sync %0, %1;" :: "r"(1 + g), "r"(S::kWpg * 32) : "memory");
-        uint32_t before = 0, n_exc = 0;
-#pragma unroll
-        for (int w = 0; w < S::kWpg; ++w) {
-            const uint32_t c = red_cnt[w];
-            if ((unsigned)w < gw) before += c;
-            n_exc += c;
-        }
-        const bool packed = page_ok && n_exc < (uint32_t)N / 2;
-        const uint32_t size = packed ? round16u(16u + N + N / 2 + n_exc) : 16u + 2u * N;
-        const bool first = u % slabs == 0;
-        // the size goes out before anything that may wait: later slabs' look-backs need it
-        if (gt == 0) {
-            const uint32_t n = k / S::kOut;               // which use of the buffer this is
-            out_slab[2 * os + (n & 1u)] = u;
-            out_size[2 * os + (n & 1u)] = size;
-            mbar_arrive(size_known(os, n));               // the commit warp may start looking back
-            // (after the arrive: an arrive orders the stores before it, and would sit out this
-            // one's trip to L2)
-            st_state(job.state + u, kFlagAgg | ((uint64_t)size + (first ? job.x.dir_bytes : 0u)));
-        }
-        if (!mbar_wait(out_empty(os), ((k / S::kOut) & 1u) ^ 1u, job)) {
-            dead = true;                                  // reported at the next group barrier
+        __syncwarp();
+        if (lane == 0) mbar_arrive(raw_empty(s));         // this warp is done with the stage
+        const bool first = (info & 0x200u) != 0u;         // the chunk's directory goes before it
+        const uint64_t add = (uint64_t)size + (first ? job.x.dir_bytes : 0u);
+        if (before_bytes + add > job.x.blob_capacity) {   // cannot happen with a worst-case buffer
+            if (pt == 0) st_flag(job.x.st, LSMKV_ST_OVERFLOW, u / slabs);
             continue;
         }
-        unsigned char *out = outb + (size_t)os * S::kOutStride;
-        if (gt == 0)
-            *reinterpret_cast<uint4 *>(out) =
-                packed ? make_uint4(kXpMagic, n_exc, base, size) : make_uint4(kXpMagic, 0, 1u << 8, size);
+        unsigned char *out = job.x.blob + before_bytes + (first ? job.x.dir_bytes : 0u);
+        if (pt == 0)
+            __stcs(reinterpret_cast<uint4 *>(out),
+                   packed ? make_uint4(kXpMagic, n_exc, info & 0xFFu, size)
+                          : make_uint4(kXpMagic, 0, 1u << 8, size));
         if (!packed) {                                    // raw slab (zeros for an unusable page)
             uint4 *o4 = reinterpret_cast<uint4 *>(out + 16) + k_first;
 #pragma unroll
-            for (int s = 0; s < S::kSweeps; ++s) o4[s * 32] = q[s];
-        } else {
-            unsigned char *sm = out + 16, *codes = sm + N, *exc = codes + N / 2;
-            uint32_t at_warp = before;                    // exceptions before this warp's next one
-#pragma unroll
-            for (int s = 0; s < S::kSweeps; ++s) {
-                const uint32_t kk = k_first + s * 32;
-                const uint4 v = q[s];
-                uint32_t c32;
-                if (exc_sweeps >> s & 1u) {               // rare: a sweep with elements below
-                    uint32_t x0, x1, x2, x3;
-                    c32 = xpfast::code_byte(v.x, lift, x0) | (xpfast::code_byte(v.y, lift, x1) << 8) |
-                          (xpfast::code_byte(v.z, lift, x2) << 16) | (xpfast::code_byte(v.w, lift, x3) << 24);
-                    const uint32_t cnt = __popc(x0) + __popc(x1) + __popc(x2) + __popc(x3);
-                    const uint32_t incl = xpfast::warp_incl_scan(cnt);
-                    uint32_t at = at_warp + incl - cnt;
-                    const uint32_t w[4] = {v.x, v.y, v.z, v.w}, x[4] = {x0, x1, x2, x3};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        if (x[e] & 1u) exc[at++] = (unsigned char)((w[e] >> 7) & 0xFFu);
-                        if (x[e] >> 16) exc[at++] = (unsigned char)((w[e] >> 23) & 0xFFu);
-                    }
-                    at_warp += __shfl_sync(0xFFFFFFFFu, incl, 31);
-                } else {
-                    // both codes of a word are the byte at bits 19..26 of its kept product
-                    c32 = __byte_perm(__byte_perm(t[4 * s] >> 19, t[4 * s + 1] >> 19, 0x0040),
-                                      __byte_perm(t[4 * s + 2] >> 19, t[4 * s + 3] >> 19, 0x0040), 0x5410);
-                }
-                *reinterpret_cast<uint2 *>(sm + 8ull * kk) = sm_bytes_mul(v);
-                *reinterpret_cast<uint32_t *>(codes + 4ull * kk) = c32;
-            }
-            const uint32_t used = 16u + N + N / 2 + n_exc;
-            if (gt < size - used) out[used + gt] = 0;     // padding up to the slab's size
+            for (int e = 0; e < S::kSweeps; ++e) __stcs(o4 + e * 32, q[e]);
+            continue;
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the bulk copy reads it
-        mbar_arrive(out_full(os));
+        unsigned char *sm = out + 16, *codes = sm + N, *exc = codes + N / 2;
+        const uint32_t lift = xpfast::window_lift(info & 0xFFu), lift4097 = lift * 4097u;
+        uint32_t at_warp = exc_before;                    // exceptions before this warp's next one
+#pragma unroll
+        for (int e = 0; e < S::kSweeps; ++e) {
+            const uint32_t kk = k_first + e * 32;
+            const uint4 v = q[e];
+            uint32_t c32;
+            if (my_sweeps >> e & 1u) {                    // rare: a sweep with elements below
+                uint32_t x0, x1, x2, x3;
+                c32 = xpfast::code_byte(v.x, lift, x0) | (xpfast::code_byte(v.y, lift, x1) << 8) |
+                      (xpfast::code_byte(v.z, lift, x2) << 16) | (xpfast::code_byte(v.w, lift, x3) << 24);
+                const uint32_t cnt = __popc(x0) + __popc(x1) + __popc(x2) + __popc(x3);
+                const uint32_t incl = xpfast::warp_incl_scan(cnt);
+                uint32_t at = at_warp + incl - cnt;
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w}, x[4] = {x0, x1, x2, x3};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (x[i] & 1u) exc[at++] = (unsigned char)((w[i] >> 7) & 0xFFu);
+                    if (x[i] >> 16) exc[at++] = (unsigned char)((w[i] >> 23) & 0xFFu);
+                }
+                at_warp += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            } else {
+                // With f = field + lift, f * 4097 = f + (f << 12) sets the low element's code
+                // right below the high one's (bits 19..22 and 23..26); for a word whose elements
+                // are both in the window nothing overlaps or carries, and the byte at bits
+                // 19..26 is the word's code byte.
+                const uint32_t y0 = mad_u32(v.x & 0x7F807F80u, 4097u, lift4097) >> 19,
+                               y1 = mad_u32(v.y & 0x7F807F80u, 4097u, lift4097) >> 19,
+                               y2 = mad_u32(v.z & 0x7F807F80u, 4097u, lift4097) >> 19,
+                               y3 = mad_u32(v.w & 0x7F807F80u, 4097u, lift4097) >> 19;
+                c32 = __byte_perm(__byte_perm(y0, y1, 0x0040), __byte_perm(y2, y3, 0x0040), 0x5410);
+            }
+            __stcs(reinterpret_cast<uint2 *>(sm + 8ull * kk), sm_bytes_mul(v));
+            __stcs(reinterpret_cast<uint32_t *>(codes + 4ull * kk), c32);
+        }
+        const uint32_t used = 16u + N + N / 2 + n_exc;
+        if (pt < size - used) out[used + pt] = 0;         // padding up to the slab's size
     }
 }
 
