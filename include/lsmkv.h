@@ -345,6 +345,9 @@ int lsmkv_relocate_records(lsmkv_ctx *ctx, void *stream, lsmkv_val_t *vals, uint
  *     blob_out with lsmkv_encode_bound(); the bytes used are the last record's offset + size
  *     - base_offset. A chunk that does not fit blob_capacity sets LSMKV_ST_OVERFLOW and gets
  *     an all-zero-size record.
+ *   Encoding reads the pool once when blob_capacity >= lsmkv_encode_bound(n_chunks) and the slab
+ *   has 8192 or 16384 elements (see "xp_one_pass" below), twice otherwise; the bytes are the same.
+ *   The encoder's scratch (12 bytes per slab) belongs to the context and grows with the batch.
  * lsmkv_decode_batch validates every directory entry and slab header (LSMKV_ST_BAD_RECORD).
  * lsmkv_decode_batch_static supports the identity codec only.
  */
@@ -511,6 +514,12 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "host_stage_bytes"  blob bytes staged per slice by the host-buffer calls, 1 MiB..64 GiB
  *   "xp_generic"        1 = compressing codec always uses its generic kernels (0 = fast kernels
  *                       for slabs of 8192 / 16384 / 32768 elements)
+ *   "xp_one_pass"       1 (default) = the compressing codec encodes slabs of 8192 / 16384 elements
+ *                       in one pass over the pool whenever blob_capacity >= lsmkv_encode_bound()
+ *                       (a persistent pipeline per SM; same bytes out); 0 = always three steps
+ *   "wait_cycles"       limit, in GPU clock cycles, of every bounded wait inside a kernel (the bulk
+ *                       copies' completion, the one-pass encoder's hand-offs); default 2e9, about
+ *                       a second; 1e5..1e11. A wait that runs out sets LSMKV_ST_WAIT_EXPIRED
  */
 int lsmkv_set_tuning(lsmkv_ctx *ctx, const char *name, int64_t value);
 int64_t lsmkv_get_tuning(const lsmkv_ctx *ctx, const char *name);

@@ -49,7 +49,7 @@ struct lsmkv_ctx {
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
-    int64_t xp_one_pass, wait_cycles, xp_shape;
+    int64_t xp_one_pass, wait_cycles;
     uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
@@ -190,9 +190,7 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // lower it under one another between setting it and launching.
 // one-pass encoder of the compressing codec: slabs of 8192 and 16384 elements
 using XpfShape8k = xpf::Shape<2, 16, 2, 8, 1>;
-using XpfShape16k = xpf::Shape<4, 16, 2, 6, 1>;
-using XpfShape16kB = xpf::Shape<4, 16, 2, 7, 1>;
-using XpfShape16kC = xpf::Shape<8, 8, 1, 7, 1>;
+using XpfShape16k = xpf::Shape<4, 16, 2, 7, 1>;
 
 constexpr int kMaxDevices = 64;
 std::mutex g_smem_limit_mu;
@@ -217,12 +215,6 @@ cudaError_t set_copy_smem_limit(int max_smem_optin)
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_xpf_encode<XpfShape16k>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XpfShape16k::kSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_xpf_encode<XpfShape16kB>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XpfShape16kB::kSmem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_xpf_encode<XpfShape16kC>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)XpfShape16kC::kSmem);
     if (e == cudaSuccess) g_smem_limit_set[dev] = true;
     return e;
 }
@@ -448,10 +440,6 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
         const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)ctx->sm_count, units);
         if (job.n_elems == 8192u)
             k_xpf_encode<XpfShape8k><<<grid, XpfShape8k::kThreads, XpfShape8k::kSmem, s>>>(fj);
-        else if (ctx->xp_shape == 1)
-            k_xpf_encode<XpfShape16kB><<<grid, XpfShape16kB::kThreads, XpfShape16kB::kSmem, s>>>(fj);
-        else if (ctx->xp_shape == 2)
-            k_xpf_encode<XpfShape16kC><<<grid, XpfShape16kC::kThreads, XpfShape16kC::kSmem, s>>>(fj);
         else
             k_xpf_encode<XpfShape16k><<<grid, XpfShape16k::kThreads, XpfShape16k::kSmem, s>>>(fj);
         k_xpf_layout<<<merge_grid(ctx, n_chunks), 256, 0, s>>>(fj);
@@ -1182,7 +1170,6 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
         {"xp_generic", &ctx->xp_generic, 0, 1},
         {"xp_one_pass", &ctx->xp_one_pass, 0, 1},
-        {"xp_shape", &ctx->xp_shape, 0, 2},
         {"wait_cycles", &ctx->wait_cycles, 100000, 100000000000ll},
     };
     for (auto &t : tab)
