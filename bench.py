@@ -1251,8 +1251,9 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
     pinned host memory (where a tensor-log writer would take them), the probe returns hit
     lengths and records to the host, and the decode copies the hit blobs from the host arena
     back to the device and scatters them. The KV pool itself lives on the GPU by nature. Two
-    slots on two streams: the get of sub-batch i is enqueued, then the put of sub-batch i+1,
-    so both PCIe directions are busy. `ctx` decides the codec (identity or compressing)."""
+    slots, two streams, two host threads: one thread puts sub-batch i+1 while the other gets
+    sub-batch i, so both PCIe directions are busy. `ctx` decides the codec (identity or
+    compressing)."""
     cb = g.chunk_bytes
     sub_cap = 2048 if world == 1 else 1024           # chunks per sub-batch (4 or 2 GiB of raw blobs)
     subs = []
@@ -1315,82 +1316,118 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
         torch.cuda.synchronize()
         p["run_t"] = (tk, tv, tn, hx)
         p["runs"] = [(tk, tv, n, None, 0, hx, nb)]
-    h2d = d2h = moved = 0
+    # Two host threads, as a serving process would have them: one issues the puts, the other the
+    # gets (probe, then decode) of the sub-batches already put, each with a context and a stream
+    # of its own (a context is not thread-safe), two sub-batches in flight. A thread that has to
+    # wait -- the get for the probe's answer, the compressing put for a slice's records -- then
+    # never keeps the other direction of the link idle.
+    import threading
+    ctx_get = lsmkv.Context(ctx.geom, ctx.device)
+    for k_ in ("host_stage_bytes",):
+        ctx_get.set_tuning(k_, ctx.get_tuning(k_))
     put_done = [torch.cuda.Event() for _ in range(NS)]
     slot_free = [torch.cuda.Event() for _ in range(NS)]
+    count = {"h2d": 0, "d2h": 0, "moved": 0}
+    errors = []
 
     def put(i):
-        nonlocal h2d, d2h
         p, k_ = prepared[i], i % NS
-        s_put.wait_event(slot_free[k_])
         ctx.put_batch_host(p["n_req"], p["tokens"], p["seq_off"], None, p["src"], src_pool, 0, 0,
                            pin_keys[k_], pin_vals[k_], pin_blob[k_], blob_cap, stream=s_put)
-        put_done[k_].record(s_put)
-        h2d += p["tokens"].numel() + p["seq_off"].numel() * 2 + p["src"].numel()
-        d2h += p["blob_bytes"] + p["n"] * 48
+        return (p["tokens"].numel() + p["seq_off"].numel() * 2 + p["src"].numel(),
+                p["blob_bytes"] + p["n"] * 48)
 
-    def probe(i):
-        nonlocal h2d, d2h
+    def get(i, check):
         p, k_ = prepared[i], i % NS
-        s_get.wait_event(put_done[k_])
-        ctx.probe_batch_host(p["n_req"], p["tokens"], p["seq_off"], p["runs"], pin_hit[k_],
-                             pin_recs[k_], None, stream=s_get)
+        ctx_get.probe_batch_host(p["n_req"], p["tokens"], p["seq_off"], p["runs"], pin_hit[k_],
+                                 pin_recs[k_], None, stream=s_get)
         s_get.synchronize()                 # the host reads hit lengths and records
-        h2d += p["tokens"].numel() + p["seq_off"].numel()
-        d2h += p["n_req"] * 4 + p["n"] * 16
+        if check:
+            hits = pin_hit[k_][:p["n_req"] * 4].numpy().view(np.uint32)
+            assert np.array_equal(hits, p["nch"].astype(np.uint32)), "e2e probe missed"
+        ctx_get.decode_batch_host(p["n_req"], p["qoff"], pin_hit[k_], pin_recs[k_],
+                                  [(pin_blob[k_], p["blob_bytes"])], p["dst"], dst_pool, stream=s_get)
+        return (p["tokens"].numel() + p["seq_off"].numel() + p["blob_bytes"] + p["n"] * 20 + 20,
+                p["n_req"] * 4 + p["n"] * 16)
 
-    def decode(i):
-        nonlocal h2d, moved
-        p, k_ = prepared[i], i % NS
-        ctx.decode_batch_host(p["n_req"], p["qoff"], pin_hit[k_], pin_recs[k_],
-                              [(pin_blob[k_], p["blob_bytes"])], p["dst"], dst_pool, stream=s_get)
-        slot_free[k_].record(s_get)
-        h2d += p["blob_bytes"] + p["n"] * 20 + 20
-        moved += 2 * p["n"] * cb
+    def run_steps(n_steps, check=False):
+        total = n_steps * len(prepared)
+        ready = [threading.Semaphore(0) for _ in range(NS)]      # slot holds a finished put
+        free = [threading.Semaphore(1) for _ in range(NS)]       # slot may be written again
+        first_use = [True] * NS
 
-    # Transfers of one direction are served in the order they were issued, across streams. With
-    # the identity codec a put never blocks the host, so the next put is issued first (its
-    # small uploads then sit in front of the get's large one); with the compressing codec a
-    # put synchronises per slice, so the get is issued first and runs under it.
-    put_first = label == "identity"
+        def put_side():
+            try:
+                torch.cuda.set_device(dev)
+                for t in range(total):
+                    k_ = t % NS
+                    free[k_].acquire()
+                    if not first_use[k_]:
+                        s_put.wait_event(slot_free[k_])          # recorded before the release
+                    first_use[k_] = False
+                    a_, b_ = put(t % len(prepared))
+                    put_done[k_].record(s_put)
+                    count["h2d"] += a_
+                    count["d2h"] += b_
+                    ready[k_].release()
+            except Exception as exc:                             # noqa: BLE001
+                errors.append(exc)
+                for sem in ready:
+                    sem.release()
 
-    def one_step(check=False):
-        put(0)
-        for i in range(len(prepared)):
-            probe(i)
-            nxt = i + 1 < len(prepared)
-            if put_first and nxt:
-                put(i + 1)
-            decode(i)
-            if not put_first and nxt:
-                put(i + 1)
-            if check:
-                hits = pin_hit[i % NS][:prepared[i]["n_req"] * 4].numpy().view(np.uint32)
-                assert np.array_equal(hits, prepared[i]["nch"].astype(np.uint32)), "e2e probe missed"
+        def get_side():
+            try:
+                torch.cuda.set_device(dev)
+                for t in range(total):
+                    k_ = t % NS
+                    ready[k_].acquire()
+                    if errors:
+                        return
+                    s_get.wait_event(put_done[k_])
+                    a_, b_ = get(t % len(prepared), check)
+                    slot_free[k_].record(s_get)
+                    count["h2d"] += a_
+                    count["d2h"] += b_
+                    count["moved"] += 2 * prepared[t % len(prepared)]["n"] * cb
+                    free[k_].release()
+            except Exception as exc:                             # noqa: BLE001
+                errors.append(exc)
+                for sem in free:
+                    sem.release()
+
+        ths = [threading.Thread(target=put_side), threading.Thread(target=get_side)]
+        for th in ths:
+            th.start()
+        for th in ths:
+            th.join()
+        if errors:
+            raise errors[0]
 
     s_put.wait_stream(stream)
     s_get.wait_stream(stream)
     ctx.last_status()
-    one_step(check=True)                    # warm-up (also faults in the pinned pages)
+    run_steps(1, check=True)                # warm-up (also faults in the pinned pages)
     barrier()
-    st = ctx.last_status()
-    assert st["flags"] == 0 and st["chunks_decoded"] == sum(p["n"] for p in prepared), st
-    h2d = d2h = moved = 0
+    st, st_get = ctx.last_status(), ctx_get.last_status()
+    assert st["flags"] == 0 and st_get["flags"] == 0, (st, st_get)
+    assert st_get["chunks_decoded"] == sum(p["n"] for p in prepared), st_get
+    count.update(h2d=0, d2h=0, moved=0)
+    steps = max(1, args.e2e_steps)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     s_put.wait_stream(stream)
     s_get.wait_stream(stream)
-    for _ in range(max(1, args.e2e_steps)):
-        one_step()
+    run_steps(steps)
     stream.wait_stream(s_put)
     stream.wait_stream(s_get)
     e1.record(stream)
     barrier()
     from paper_2511_16138_b200 import ranks
     ms = ranks.max_over_ranks(e0.elapsed_time(e1), dev)
-    moved = ranks.sum_over_ranks(moved, dev)
-    steps = max(1, args.e2e_steps)
+    h2d, d2h = count["h2d"], count["d2h"]
+    moved = ranks.sum_over_ranks(count["moved"], dev)
     ctx.last_status()
+    ctx_get.close()
     pcie = (h2d + d2h) / (e0.elapsed_time(e1) * 1e-3) / 1e9          # this rank's link traffic
     return {"value": ranks.whole_job_rate(moved, ms) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
@@ -1401,7 +1438,8 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
             "api": "lsmkv_put_batch_host / lsmkv_probe_batch_host / lsmkv_decode_batch_host",
             "note": "host buffers in and out through the C ABI: blobs, keys and records land in "
                     "pinned host memory, hit blobs are copied back from it before the scatter; "
-                    "put and get sides run on two streams so both PCIe directions are busy; "
+                    "puts and gets are issued by two host threads on two streams (a context each) "
+                    "so both PCIe directions stay busy; "
                     "value counts raw (uncompressed) payload bytes; PCIe-bound"}
 
 

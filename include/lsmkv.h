@@ -11,7 +11,8 @@
  *     stream reaches the point following the call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Every
  *     batch call only enqueues work and returns; none of them synchronises (one documented
- *     exception: lsmkv_put_batch_host with the compressing codec).
+ *     exception: lsmkv_put_batch_host with the compressing codec, which waits briefly for the
+ *     records of each slice unless asked to place the bytes from the device).
  *   - Return value: 0 = enqueued, negative = LSMKV_E* and nothing was enqueued.
  *   - Problems only the GPU can see (a page id beyond the pool, a record that points outside
  *     its arena, a misaligned buffer, a wait that ran out) never fault: the offending item is
@@ -402,9 +403,17 @@ int lsmkv_hindex_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, ui
  *   lsmkv_encode_batch produces; *n_chunks_out (optional) is set before returning. blob_out
  *   may be NULL together with page_table and pool (index-only). *blob_bytes_out (optional) =
  *   bytes placed in blob_out. With the compressing codec blob sizes depend on the data: the
- *   call then synchronises `stream` once per slice, copies back exactly the bytes produced
- *   (blobs stay back to back across slices) and returns LSMKV_ECAPACITY if blob_out is too
- *   small; with the identity codec it never synchronises.
+ *   call then waits, once per slice, for that slice's records (a short wait: only the slice's
+ *   encode is ahead of it; the slice before is meanwhile on its way to the host on a stream of
+ *   the context's own, from the other of two stages), copies exactly the bytes produced behind
+ *   those of the slices before, sets *blob_bytes_out and returns LSMKV_ECAPACITY if blob_out is
+ *   too small; the caller's stream reaches the end of the call's work only when those copies
+ *   have landed. With the knob "host_put_device_placed", pinned 16-byte aligned blob_out and
+ *   blob_bytes_out == NULL the call never waits instead: kernels place every slice's bytes in
+ *   blob_out themselves (at about four fifths of the copy engines' rate); the bytes used are
+ *   then the last record's offset + size - base_offset, and a blob_out that is too small sets
+ *   LSMKV_ST_OVERFLOW (the slice is left out) instead of an error code. With the identity codec
+ *   the call never waits.
  * lsmkv_probe_batch_host: probe. hit_chunks_out [host n_query], recs_out [host, sum of
  *   floor(len/C)], optional keys_out; *n_qchunks_out (optional) is set before returning.
  * lsmkv_decode_batch_host: get_batch, tensor half. qchunk_off, hit_chunks, recs and
@@ -517,6 +526,14 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "xp_one_pass"       1 (default) = the compressing codec encodes slabs of 8192 / 16384 elements
  *                       in one pass over the pool whenever blob_capacity >= lsmkv_encode_bound()
  *                       (a persistent pipeline per SM; same bytes out); 0 = always three steps
+ *   "host_put_device_placed"  1 = lsmkv_put_batch_host with the compressing codec never waits
+ *                       (see there); "host_copy_ctas" = CTAs of the kernel that then writes the
+ *                       host blob, 1..4096 (default 32: posted writes need little parallelism)
+ *   "test_drop_piece"   test hook, -1 = off (default): the bulk copy kernel arms the completion
+ *                       barrier of the piece with this number (pieces are numbered over the
+ *                       whole launch) but starts no copy for it, so that wait runs out: the
+ *                       kernel records LSMKV_ST_WAIT_EXPIRED with first_bad = the piece and
+ *                       returns; the warp that owned the piece copies nothing further
  *   "wait_cycles"       limit, in GPU clock cycles, of every bounded wait inside a kernel (the bulk
  *                       copies' completion, the one-pass encoder's hand-offs); default 2e9, about
  *                       a second; 1e5..1e11. A wait that runs out sets LSMKV_ST_WAIT_EXPIRED

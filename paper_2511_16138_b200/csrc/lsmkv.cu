@@ -40,6 +40,7 @@ struct lsmkv_ctx {
     uint32_t xp_dir_bytes;
     void *d_xp;
     uint64_t xp_cap;     // chunks
+    const uint64_t *xp_base_add;   // set by the host-buffer put for its next encode, else NULL
     // fence-pointer directory of the probe: u64[n_runs * (jcap + 1)]
     uint64_t *d_dir;
     uint64_t dir_cap;
@@ -49,11 +50,13 @@ struct lsmkv_ctx {
     // tuning
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
-    int64_t xp_one_pass, wait_cycles;
+    int64_t xp_one_pass, wait_cycles, host_copy_ctas, host_put_device_placed, test_drop_piece;
     uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
     uint64_t io_cap[3];
+    cudaStream_t io_stream;          // second stream + events of the compressing host-buffer put
+    cudaEvent_t io_ev_enc, io_ev_free[2];
     std::vector<uint64_t> h_off_a;
     std::vector<uint32_t> h_cuts;
     struct HostScratch { void *p; size_t cap; cudaEvent_t done; bool used; };
@@ -353,6 +356,8 @@ int launch_copy(lsmkv_ctx *ctx, cudaStream_t s, CopyJob &job, const ArenaTable &
     LaunchTimer timer(ctx, s, job.unpack ? LSMKV_K_UNPACK : LSMKV_K_PACK);
     const uint64_t slabs = 2ull * ctx->geom.n_layers * ctx->ppc;
     job.pages_per_chunk = ctx->ppc;
+    job.wait_cycles = ctx->wait_cycles;
+    job.test_drop_piece = ctx->test_drop_piece < 0 ? ~0ull : (uint64_t)ctx->test_drop_piece;
     if (ctx->copy_mode == 1) {
         job.piece_bytes = (uint32_t)ctx->page_bytes;
         job.pieces_per_slab = 1;
@@ -420,6 +425,8 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
     job.blob_capacity = blob_capacity;
     job.file_id = file_id;
     job.base_offset = base_offset;
+    job.base_add = ctx->xp_base_add;
+    ctx->xp_base_add = nullptr;
     job.vals_out = vals_out;
     job.st = ctx->d_status;
     LaunchTimer timer(ctx, s, LSMKV_K_PACK);
@@ -518,6 +525,8 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->simt_ctas_per_sm = 8;
     ctx->host_stage_bytes = 1ll << 30;
     ctx->xp_one_pass = 1;
+    ctx->host_copy_ctas = 32;
+    ctx->test_drop_piece = -1;
     ctx->wait_cycles = 2000000000ll;
 
     DeviceGuard guard(device);
@@ -576,6 +585,12 @@ int lsmkv_destroy(lsmkv_ctx *ctx)
             if (h.p) note(cudaFreeHost(h.p));
             if (h.done) note(cudaEventDestroy(h.done));
         }
+    if (ctx->io_stream) {
+        note(cudaStreamDestroy(ctx->io_stream));
+        note(cudaEventDestroy(ctx->io_ev_enc));
+        note(cudaEventDestroy(ctx->io_ev_free[0]));
+        note(cudaEventDestroy(ctx->io_ev_free[1]));
+    }
     if (release_scratch(ctx, &ctx->d_status, &cap, __LINE__) != LSMKV_OK) note((cudaError_t)ctx->last_cuda);
     for (auto &t : ctx->pending) { note(cudaEventDestroy(t.a)); note(cudaEventDestroy(t.b)); }
     for (auto e : ctx->free_events) note(cudaEventDestroy(e));
@@ -1170,6 +1185,9 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"host_stage_bytes", &ctx->host_stage_bytes, 1 << 20, 1ll << 36},
         {"xp_generic", &ctx->xp_generic, 0, 1},
         {"xp_one_pass", &ctx->xp_one_pass, 0, 1},
+        {"host_copy_ctas", &ctx->host_copy_ctas, 1, 4096},
+        {"host_put_device_placed", &ctx->host_put_device_placed, 0, 1},
+        {"test_drop_piece", &ctx->test_drop_piece, -1, 1ll << 40},
         {"wait_cycles", &ctx->wait_cycles, 100000, 100000000000ll},
     };
     for (auto &t : tab)
@@ -1395,6 +1413,8 @@ extern "C" int lsmkv_decode_batch_static(const lsmkv_geom_t *g, int device, void
         job.plan = plan;
         job.recs = recs;
         job.st = st;
+        job.wait_cycles = 2000000000ll;
+        job.test_drop_piece = ~0ull;
         const uint64_t piece = pb < 32768 ? pb : 32768;
         job.piece_bytes = (uint32_t)piece;
         job.pieces_per_slab = (uint32_t)((pb + piece - 1) / piece);

@@ -40,6 +40,9 @@ struct CopyJob {
     const uint32_t *plan;            // unpack: [dev] hit chunk -> query-chunk index, or kSkip
     const lsmkv_val_t *recs;         // unpack
     DevStatus *st;
+    long long wait_cycles;           // limit of the wait for a bulk copy's completion
+    uint64_t test_drop_piece;        // test hook: this piece arms its barrier but starts no copy,
+                                     // so its wait runs out (~0 = none)
 };
 
 struct Piece { const unsigned char *src; unsigned char *dst; uint32_t bytes; };
@@ -100,8 +103,8 @@ __device__ __forceinline__ uint32_t smem_addr(const void *p)
     return (uint32_t)__cvta_generic_to_shared(p);
 }
 
-// Wait for phase `parity` of an mbarrier with a time limit (about a second); false = gave up.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Wait for phase `parity` of an mbarrier for at most `limit` clock cycles; false = gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit)
 {
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
@@ -112,7 +115,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
-        if ((it & 1023u) == 1023u && clock64() - t0 > 2000000000ll) return false;
+        if ((it & 63u) == 63u && clock64() - t0 > limit) return false;
     }
 }
 
@@ -146,7 +149,9 @@ k_copy_slabs_bulk(const __grid_constant__ CopyJob job, const __grid_constant__ A
         if (!resolve_piece(job, ar, p, pc)) continue;
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                      :: "r"(bar), "r"(pc.bytes) : "memory");
-        if (kHint)
+        if (p == job.test_drop_piece) {
+            // (test hook) nothing is started, so nothing is in flight when the wait gives up
+        } else if (kHint)
             asm volatile(
                 "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
                 " [%0], [%1], %2, [%3], %4;"
@@ -156,9 +161,12 @@ k_copy_slabs_bulk(const __grid_constant__ CopyJob job, const __grid_constant__ A
                 "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes"
                 " [%0], [%1], %2, [%3];"
                 :: "r"(sbuf), "l"(pc.src), "r"(pc.bytes), "r"(bar) : "memory");
-        if (!mbar_wait_bounded(bar, parity)) {
+        if (!mbar_wait_bounded(bar, parity, job.wait_cycles)) {
+            // The copy did not report completion in time: record it and stop using this stage.
+            // A copy that was started gets one more bounded wait before the warp leaves, so
+            // that it is not still writing this CTA's shared memory then.
             st_flag(job.st, LSMKV_ST_WAIT_EXPIRED, p);
-            mbar_wait_bounded(bar, parity);      // give the copy in flight one more bounded chance
+            mbar_wait_bounded(bar, parity, job.wait_cycles);
             break;
         }
         parity ^= 1u;

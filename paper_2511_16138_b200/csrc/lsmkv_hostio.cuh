@@ -28,6 +28,17 @@ int ensure_io(lsmkv_ctx *ctx, int kind, size_t bytes)
     return grow_scratch(ctx, &ctx->d_io[kind], &ctx->io_cap[kind], bytes, bytes, __LINE__);
 }
 
+// Second stream and events of the host-buffer put with the compressing codec.
+int ensure_io_stream(lsmkv_ctx *ctx)
+{
+    if (ctx->io_stream) return LSMKV_OK;
+    CU(ctx, cudaStreamCreateWithFlags(&ctx->io_stream, cudaStreamNonBlocking));
+    CU(ctx, cudaEventCreateWithFlags(&ctx->io_ev_enc, cudaEventDisableTiming));
+    CU(ctx, cudaEventCreateWithFlags(&ctx->io_ev_free[0], cudaEventDisableTiming));
+    CU(ctx, cudaEventCreateWithFlags(&ctx->io_ev_free[1], cudaEventDisableTiming));
+    return LSMKV_OK;
+}
+
 size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 
 // Large transfers go out in pieces: copies of one direction are served in issue order even
@@ -99,6 +110,47 @@ struct ScratchLease {
     }
 };
 
+// put with the compressing codec, without a stop per slice: how many bytes a slice's encode
+// produced is only known on the device, so the device itself moves them from the stage to the
+// caller's host blob (pinned memory is visible to kernels), behind the bytes of the slices
+// before, and keeps the running total. `last` is the slice's last record: its end, less the
+// call's base offset and the total so far, is the slice's size.
+__device__ __forceinline__ bool slice_extent(const uint64_t *total, const lsmkv_val_t *last,
+                                             uint64_t base_offset, uint64_t capacity,
+                                             uint64_t stage_bytes, uint64_t *start, uint64_t *used)
+{
+    const uint4 r = *reinterpret_cast<const uint4 *>(last);
+    *start = *total;
+    if (r.y == 0) return false;                          // the encode overflowed its stage (flagged)
+    *used = (((uint64_t)r.z | ((uint64_t)r.w << 32)) + r.y) - base_offset - *start;
+    return *used <= stage_bytes && (*used & 15u) == 0 && *start <= capacity && *used <= capacity - *start;
+}
+
+__global__ void __launch_bounds__(256)
+k_blob_to_host(const unsigned char *__restrict__ stage, unsigned char *__restrict__ host_blob,
+               const uint64_t *total, const lsmkv_val_t *last, uint64_t base_offset,
+               uint64_t capacity, uint64_t stage_bytes, lsmkv::DevStatus *st)
+{
+    uint64_t start, used;
+    if (!slice_extent(total, last, base_offset, capacity, stage_bytes, &start, &used)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) lsmkv::st_flag(st, LSMKV_ST_OVERFLOW, 0);
+        return;
+    }
+    const uint4 *src = reinterpret_cast<const uint4 *>(stage);
+    uint4 *dst = reinterpret_cast<uint4 *>(host_blob + start);
+    const uint64_t n = used >> 4, step = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step)
+        dst[i] = __ldcs(src + i);
+}
+
+__global__ void k_blob_advance(uint64_t *total, const lsmkv_val_t *last, uint64_t base_offset,
+                               uint64_t capacity, uint64_t stage_bytes)
+{
+    uint64_t start, used;
+    if (slice_extent(total, last, base_offset, capacity, stage_bytes, &start, &used))
+        *total = start + used;
+}
+
 }  // namespace
 
 extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req,
@@ -158,7 +210,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     const size_t n_rel = (size_t)n_req + n_slices;        // sum over slices of (requests + 1)
     size_t need = pad256(nt * 4) + 2 * pad256(n_rel * 8) + pad256((size_t)n_req * 4) +
                   pad256(n_chunks * ctx->ppc * 4) + pad256(m_max * 32) + pad256(m_max * 16) +
-                  (with_blob ? pad256(m_max * slot) : 0) + 4096;
+                  (with_blob ? pad256(m_max * slot) : 0) + (coded ? pad256(m_max * slot) : 0) + 4096;
     int rc = ensure_io(ctx, 0, need);
     if (rc != LSMKV_OK) return rc;
     IoLayout io(ctx->d_io[0]);
@@ -170,6 +222,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     lsmkv_key_t *d_keys = io.take<lsmkv_key_t>(m_max);
     lsmkv_val_t *d_vals = io.take<lsmkv_val_t>(m_max);
     unsigned char *d_blob = with_blob ? io.take<unsigned char>(m_max * slot) : nullptr;
+    unsigned char *d_blob2 = coded ? io.take<unsigned char>(m_max * slot) : nullptr;   // second stage
 
     ScratchLease lease(ctx, 0, s, 2 * n_rel * 8 + 256);
     if (!lease.ok()) return LSMKV_ENOMEM;
@@ -191,7 +244,29 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
     if (with_blob)
         CU(ctx, copy_pieces(d_pages, page_table, n_chunks * ctx->ppc * 4, cudaMemcpyHostToDevice, s));
 
-    uint64_t host_used = 0;                          // compressing codec: bytes placed so far
+    // Compressing codec: how many bytes a slice produced is only known on the device. Either
+    // the device places the slices in the host blob itself and nothing ever stops (on request:
+    // "host_put_device_placed", needs pinned memory and no byte count at return), or -- the
+    // default, which moves the bytes with the copy engines at the link's full rate -- the host
+    // waits for each slice's records only (a short wait: the slice before it is still on its way
+    // to the host on a second stream and from the other of two stages).
+    unsigned char *host_blob_dev = nullptr;
+    uint64_t *d_total = reinterpret_cast<uint64_t *>(reinterpret_cast<char *>(ctx->d_status) + 128);
+    if (coded && !blob_bytes_out && ctx->host_put_device_placed) {
+        void *dp = nullptr;
+        if (cudaHostGetDevicePointer(&dp, blob_out, 0) == cudaSuccess && dp && aligned16(dp))
+            host_blob_dev = static_cast<unsigned char *>(dp);
+        else
+            cudaGetLastError();                      // pageable memory: the waiting path below
+    }
+    if (host_blob_dev) CU(ctx, cudaMemsetAsync(d_total, 0, sizeof(uint64_t), s));
+    uint64_t host_used = 0;                          // waiting path: bytes placed so far
+    bool stage_used[2] = {false, false};
+    if (coded && !host_blob_dev) {
+        rc = ensure_io_stream(ctx);
+        if (rc != LSMKV_OK) return rc;
+    }
+    size_t coded_slices = 0;
     at = 0;
     for (size_t k = 0; k < n_slices; ++k) {
         const uint32_t a = cuts[k], b = cuts[k + 1], nr = b - a;
@@ -199,25 +274,48 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
         const size_t rel_at = at;
         at += (size_t)nr + 1;
         if (m == 0) continue;
+        // waiting path: slices alternate between two stages; a stage is free again once the
+        // copy of the slice it held two slices ago has left on the second stream
+        const int sg = coded && !host_blob_dev ? (int)(coded_slices & 1) : 0;
+        unsigned char *stage = sg ? d_blob2 : d_blob;
+        if (coded && !host_blob_dev && stage_used[sg])
+            CU(ctx, cudaStreamWaitEvent(s, ctx->io_ev_free[sg], 0));
+        ctx->xp_base_add = host_blob_dev ? d_total : nullptr;   // records count from the device's total
         rc = lsmkv_encode_batch(ctx, stream, nr, d_tok + (seq_off[a] - t_first), d_seq + rel_at,
                                 start_chunk ? d_start + a : nullptr, d_coff + rel_at, m,
                                 with_blob ? d_pages + coff[a] * ctx->ppc : nullptr,
                                 with_blob ? pool : nullptr,
                                 file_id, base_offset + (coded ? host_used : coff[a] * cb), d_keys,
-                                d_vals, d_blob, with_blob ? m * slot : 0);
+                                d_vals, stage, with_blob ? m * slot : 0);
+        ctx->xp_base_add = nullptr;
         if (rc != LSMKV_OK) return rc;
         CU(ctx, cudaMemcpyAsync(keys_out + coff[a], d_keys, m * 32, cudaMemcpyDeviceToHost, s));
         CU(ctx, cudaMemcpyAsync(vals_out + coff[a], d_vals, m * 16, cudaMemcpyDeviceToHost, s));
-        if (coded) {
-            // blob sizes depend on the data: wait for this slice's records, then copy exactly
-            // the bytes it produced behind the previous slice's
-            CU(ctx, cudaStreamSynchronize(s));
+        if (host_blob_dev) {
+            // posted writes over the host link need little parallelism: a few CTAs saturate it
+            // and leave the other SMs to whatever runs beside the put
+            k_blob_to_host<<<(unsigned)ctx->host_copy_ctas, 256, 0, s>>>(
+                stage, host_blob_dev, d_total, d_vals + (m - 1), base_offset, blob_capacity,
+                m * slot, ctx->d_status);
+            k_blob_advance<<<1, 1, 0, s>>>(d_total, d_vals + (m - 1), base_offset, blob_capacity,
+                                           m * slot);
+            ctx->launches += 2;
+            CU(ctx, cudaGetLastError());
+        } else if (coded) {
+            // wait for this slice's records (only the encode and two small copies are ahead of
+            // the event), then send exactly the bytes it produced, behind the previous slice's
+            CU(ctx, cudaEventRecord(ctx->io_ev_enc, s));
+            CU(ctx, cudaEventSynchronize(ctx->io_ev_enc));
             const lsmkv_val_t &last = vals_out[coff[b] - 1];
             if (last.reserved == 0) return LSMKV_ECAPACITY;   // stage overflow (flagged on device)
             const uint64_t used = last.offset + last.reserved - (base_offset + host_used);
             if (blob_capacity - host_used < used) return LSMKV_ECAPACITY;
-            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + host_used, d_blob, used,
-                                cudaMemcpyDeviceToHost, s));
+            CU(ctx, cudaStreamWaitEvent(ctx->io_stream, ctx->io_ev_enc, 0));
+            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + host_used, stage, used,
+                                cudaMemcpyDeviceToHost, ctx->io_stream));
+            CU(ctx, cudaEventRecord(ctx->io_ev_free[sg], ctx->io_stream));
+            stage_used[sg] = true;
+            ++coded_slices;
             host_used += used;
             if (blob_bytes_out) *blob_bytes_out = host_used;
         } else if (with_blob) {
@@ -225,6 +323,8 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
                                 cudaMemcpyDeviceToHost, s));
         }
     }
+    for (int sg = 0; sg < 2; ++sg)                   // the call's work ends when its copies have
+        if (stage_used[sg]) CU(ctx, cudaStreamWaitEvent(s, ctx->io_ev_free[sg], 0));
     return LSMKV_OK;
 }
 

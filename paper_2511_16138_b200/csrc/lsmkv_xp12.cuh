@@ -36,6 +36,8 @@ struct XpJob {
     uint64_t blob_capacity;
     uint32_t file_id;
     uint64_t base_offset;
+    const uint64_t *base_add;    // [dev] or NULL: added to base_offset in the records (a running
+                                 // total kept on the device by the host-buffer put)
     lsmkv_val_t *vals_out;
     DevStatus *st;
 };
@@ -200,7 +202,7 @@ k_xp_layout(const __grid_constant__ XpJob job)
             *reinterpret_cast<uint4 *>(job.vals_out + i) = v;
             continue;
         }
-        const uint64_t o = job.base_offset + off;
+        const uint64_t o = job.base_offset + off + (job.base_add ? *job.base_add : 0ull);
         v.y = (uint32_t)size;
         v.z = (uint32_t)o;
         v.w = (uint32_t)(o >> 32);

@@ -579,7 +579,7 @@ k_xpf_layout(const __grid_constant__ xpf::Job job)
             *reinterpret_cast<uint4 *>(job.x.vals_out + i) = v;
             continue;
         }
-        const uint64_t o = job.x.base_offset + off;
+        const uint64_t o = job.x.base_offset + off + (job.x.base_add ? *job.x.base_add : 0ull);
         v.y = (uint32_t)(end - off);
         v.z = (uint32_t)o;
         v.w = (uint32_t)(o >> 32);

@@ -333,7 +333,7 @@ def lsmkv_put_batch_host(ctx, stream, n_req, tokens, seq_off, start_chunk, page_
                                     _hptr(start_chunk), _hptr(page_table),
                                     C.byref(p) if p is not None else None, file_id, base_offset,
                                     _hptr(keys_out), _hptr(vals_out), _hptr(blob_out),
-                                    blob_capacity, C.byref(n), C.byref(nb))
+                                    blob_capacity, C.byref(n), C.byref(nb) if want_bytes else None)
     _check(ctx, rc, "lsmkv_put_batch_host")
     return (int(n.value), int(nb.value)) if want_bytes else int(n.value)
 

@@ -191,3 +191,52 @@ def test_host_buffers_with_the_compressing_codec(stage):
         assert np.array_equal(dst.numpy(), o_dst)
         st = ctx.last_status()
         assert st["flags"] == 0 and st["chunks_decoded"] == n
+
+
+def test_xp12_put_placed_by_the_device_equals_the_oracle():
+    """On request, with a pinned host blob and no byte count wanted at return, the device places
+    the slices itself (several slices here): keys, records and blob bytes are the oracle's; a
+    host blob that is too small is flagged, not overrun."""
+    g = lsmkv.Geom(2, 8, 64, elem_bytes=2, page_tokens=16, chunk_tokens=16, flags=lsmkv.CODEC_XP12)
+    og = H.ogeom(g)                                             # 16 KiB slabs, 64 KiB chunks
+    rng = np.random.default_rng(21)
+    b = synth.make_batch([rng.integers(0, 5000, 16 * k + 3, dtype=np.uint32) for k in (7, 1, 12, 4, 9)])
+    nch = synth.chunk_counts(b.seq_off, 16)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    num_pages = n + 5
+    pool_np = synth.random_pool_bytes(rng, 4, num_pages, g.page_bytes)
+    pool_np.view(np.uint16)[:, ::5, ::9] = 0x0001               # sprinkle exceptions
+    pages = synth.random_pages(rng, num_pages, n)
+    o_keys, o_vals, o_blob = oracle.encode_batch_xp12(og, b.tokens, b.seq_off, None, coff, pages,
+                                                      pool_np, 1, 4096)
+    with lsmkv.Context(g, 0) as ctx:
+        ctx.set_tuning("host_stage_bytes", 1 << 20)            # 1 MiB stage: several slices
+        ctx.set_tuning("host_put_device_placed", 1)
+        pool = H.DevPool(g, num_pages, pool_np)
+        keys = torch.zeros(n * 32, dtype=torch.uint8).pin_memory()
+        vals = torch.zeros(n * 16, dtype=torch.uint8).pin_memory()
+        blob = torch.full((ctx.encode_bound(n),), 0xEE, dtype=torch.uint8).pin_memory()
+        got_n = ctx.put_batch_host(b.n, b.tokens, b.seq_off, None, pages, pool.table, 1, 4096,
+                                   keys, vals, blob, blob.numel())
+        torch.cuda.synchronize()
+        assert got_n == n
+        assert np.array_equal(keys.numpy().view(np.uint64).reshape(-1, 4), o_keys)
+        v = vals.numpy().view(VAL_DTYPE)
+        assert np.array_equal(v, o_vals)
+        used = int(v["offset"][-1]) + int(v["reserved"][-1]) - 4096
+        assert used == o_blob.size
+        assert np.array_equal(blob.numpy()[:used], o_blob)
+        assert np.all(blob.numpy()[used:] == 0xEE)
+        assert ctx.last_status()["flags"] == 0
+        # a host blob with room for the first slices only: the rest is flagged and left out
+        blob.fill_(0xEE)
+        cap = o_blob.size // 2 // 16 * 16
+        ctx.put_batch_host(b.n, b.tokens, b.seq_off, None, pages, pool.table, 1, 4096, keys, vals,
+                           blob, cap)
+        torch.cuda.synchronize()
+        assert ctx.last_status()["flags"] == lsmkv.ST_OVERFLOW
+        got = blob.numpy()
+        placed = int(np.flatnonzero(got != 0xEE).max()) + 1 if (got != 0xEE).any() else 0
+        assert placed <= cap and np.array_equal(got[:placed], o_blob[:placed])
+        assert np.all(got[cap:] == 0xEE)
