@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 from paper_2511_16138_b200 import synth  # noqa: E402
 
-NCU_TRAFFIC_RATIO = 0.9868   # measured DRAM traffic / algorithmic bytes of the slab copy kernel
+NCU_TRAFFIC_RATIO = 0.9867   # measured DRAM traffic / algorithmic bytes of the slab copy kernel
 METRIC = "codec_GBps_pack_plus_unpack"
 UNIT = "GB/s"
 WORKLOAD = ("configs[1]: Llama-3-8B KV shape, 32 layers x 8 KV heads x 128 head_dim bf16, page 16; "
@@ -549,7 +549,7 @@ def main():
                          "frac": achieved / peak, "peak_source": peak_src,
                          "frac_of_8TBps_nominal": achieved / 8000.0,
                          # DRAM read+write bytes per launch: ncu counters of a 774-chunk capture
-                         # (traffic / algorithmic bytes = 0.9868), scaled by chunk count
+                         # (traffic / algorithmic bytes = 0.9867), scaled by chunk count
                          "traffic": NCU_TRAFFIC_RATIO * algo_bytes_per_launch,
                          "traffic_source": "ncu dram__bytes_read+write on a 774-chunk launch, "
                                            "scaled by chunks (ncu summary committed with the repository)",

@@ -192,8 +192,8 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // that callers on different host threads (regular and allocation-free decodes alike) cannot
 // lower it under one another between setting it and launching.
 // one-pass encoder of the compressing codec: slabs of 8192 and 16384 elements
-using XpfShape8k = xpf::Shape<2, 16, 2, 8, 1>;
-using XpfShape16k = xpf::Shape<4, 16, 2, 7, 1>;
+using XpfShape8k = xpf::Shape<2, 16, 2, 1, 12, 1>;
+using XpfShape16k = xpf::Shape<4, 16, 2, 1, 7, 1>;
 
 constexpr int kMaxDevices = 64;
 std::mutex g_smem_limit_mu;

@@ -10,15 +10,15 @@
 //   look-back warps  sum the sizes of all earlier slabs (decoupled look-back over a per-slab
 //                    state word: empty / size known / prefix known), publish the prefix and
 //                    hand the slab's place on;
-//   packing warps    encode the slab straight into its final place in the blob, then free the
-//                    stage.
-// The three run side by side on different slabs of the ring, so each one's chain of short
-// dependent steps (waits, shuffles, barriers) hides behind the others' arithmetic, and a slab's
-// size is known well before its turn to be packed, which absorbs the differences in pace
-// between the SMs. Slab numbers are handed out in order by the counter, so
-// every slab a look-back waits for is held by a CTA that is already running. A small kernel
-// afterwards (k_xpf_layout) turns the prefixes into chunk directories and records. Bytes out
-// are those of the three-step encoder.
+//   packing warps    take a measured slab into registers, which frees its stage, wait for the
+//                    slab's place, and encode it straight into the blob.
+// The three run side by side on different slabs, so each one's chain of short dependent steps
+// (waits, shuffles, barriers) hides behind the others' arithmetic; a slab's size is known well
+// before its place is, and the stages plus the packing warps' registers are what absorbs the
+// differences in pace between the SMs while a look-back waits for its slowest predecessor.
+// Slab numbers are handed out in order by the counter, so every slab a look-back waits for is
+// held by a CTA that is already running. A small kernel afterwards (k_xpf_layout) turns the
+// prefixes into chunk directories and records. Bytes out are those of the three-step encoder.
 //
 // Every wait is bounded (the mbarrier waits and the look-back polls give up after `wait_cycles`
 // clock cycles, set LSMKV_ST_WAIT_EXPIRED and an abort word that makes every other wait of the
@@ -36,22 +36,32 @@ constexpr uint64_t kFlagIncl = 2ull << 62;     // low 62 bits: bytes of all slab
 constexpr uint64_t kValueMask = (1ull << 62) - 1;
 constexpr uint64_t kEnd = ~0ull;               // slab number that tells a role to stop
 
-// Shape of the pipeline for a slab of WARPS * SWEEPS * 256 elements: WARPS packing warps, each
-// owning a contiguous part of SWEEPS * 256 elements; WARPS / SPLIT measuring warps, each covering
-// SPLIT such parts; RING stages; LB look-back warps that share the slabs round-robin.
-template <int SWEEPS, int WARPS, int SPLIT, int RING, int LB>
+// Shape of the pipeline for a slab of WARPS * SWEEPS * 256 elements. Packing: GROUPS groups of
+// WARPS warps, each warp owning a contiguous part of SWEEPS * 256 elements, a group per slab
+// (group g takes slabs g, g + GROUPS, ...). Measuring: WARPS / SPLIT warps, each covering SPLIT
+// such parts. RING stages; LB look-back warps that share the slabs round-robin. What one role
+// tells the next about a slab travels in kQ mailboxes (with their barriers), more than there
+// are stages: a packing group takes its slab into registers as soon as it is measured, frees
+// the stage, and only then waits for the slab's place.
+template <int SWEEPS, int WARPS, int SPLIT, int GROUPS, int RING, int LB>
 struct Shape {
-    static constexpr int kSweeps = SWEEPS, kWarps = WARPS, kSplit = SPLIT, kRing = RING, kLb = LB;
+    static constexpr int kSweeps = SWEEPS, kWarps = WARPS, kSplit = SPLIT, kGroups = GROUPS,
+                         kRing = RING, kLb = LB, kQ = RING + GROUPS <= 8 ? 8 : 16;
     static constexpr int kMeasureWarps = WARPS / SPLIT, kMeasureSweeps = SWEEPS * SPLIT;
     static constexpr int kElems = WARPS * SWEEPS * 256;
     static constexpr int kPageBytes = 2 * kElems;
     static constexpr int kFirstPackWarp = kMeasureWarps;
-    static constexpr int kProducerWarp = kMeasureWarps + WARPS;
+    static constexpr int kProducerWarp = kMeasureWarps + GROUPS * WARPS;
     static constexpr int kFirstLbWarp = kProducerWarp + 1;
-    static constexpr int kThreads = (kMeasureWarps + WARPS + 1 + LB) * 32;
-    static constexpr size_t kSmem = (size_t)RING * kPageBytes + 2048;
-    static_assert(RING >= 3 && LB >= 1 && WARPS <= 16 && WARPS % SPLIT == 0 && kMeasureSweeps <= 32,
-                  "shape out of range");
+    static constexpr int kThreads = (kMeasureWarps + GROUPS * WARPS + 1 + LB) * 32;
+    static constexpr size_t kTail = 1536 + (size_t)kQ * WARPS * 8;   // barriers and mailboxes
+    static constexpr size_t kSmem = (size_t)RING * kPageBytes + kTail;
+    static_assert(RING >= 3 && LB >= 1 && WARPS <= 16 && WARPS % SPLIT == 0 && kMeasureSweeps <= 32 &&
+                  kThreads <= 1024, "shape out of range");
+    // a mailbox is used again kQ slabs later; by then the slab it served must be packed: a stage
+    // is only refilled once its slab is in a group's registers, and a group takes one slab at a
+    // time, so when slab k + kQ is fetched the slabs up to k + kQ - RING - GROUPS are packed
+    static_assert(kQ >= RING + GROUPS && kQ >= LB + GROUPS, "too few mailboxes");
 };
 
 struct Job {
@@ -200,34 +210,39 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
     using namespace xpf;
     extern __shared__ __align__(128) unsigned char xpf_smem[];
     constexpr int N = S::kElems, R = S::kRing, W = S::kWarps, WM = S::kMeasureWarps,
-                  SM = S::kMeasureSweeps;
+                  SM = S::kMeasureSweeps, Q = S::kQ;
     unsigned char *ring = xpf_smem;
     unsigned char *tail = xpf_smem + (size_t)R * S::kPageBytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);             // 4 per stage
-    uint64_t *slot_u = bars + 4 * R;                                 // producer: slab number / kEnd
-    uint64_t *m_u = slot_u + R;                                      // measure: the same, for the look-back
-    uint64_t *m_prefix = m_u + R;                                    // look-back: bytes before the slab
-    uint32_t *slot_ok = reinterpret_cast<uint32_t *>(m_prefix + R);  // producer: page usable
-    uint32_t *m_size = slot_ok + R;                                  // measure: encoded size
-    uint32_t *m_info = m_size + R;                                   // measure: base | packed << 8
-    uint32_t *m_nexc = m_info + R;                                   // measure: exceptions of the slab
-    uint32_t *m_wcnt = m_nexc + R;                                   // measure: [R][W] exceptions per part
-    uint32_t *m_wsweeps = m_wcnt + R * W;                            // measure: [R][W] sweeps that have any
-    uint32_t *red_max = m_wsweeps + R * W;                           // [WM]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);             // 2 per stage, 2 per mailbox
+    uint64_t *slot_u = bars + 2 * R + 2 * Q;                         // producer: slab number / kEnd
+    uint64_t *m_u = slot_u + R;                                      // measure: the same, per mailbox
+    uint64_t *m_prefix = m_u + Q;                                    // look-back: bytes before the slab
+    uint32_t *slot_ok = reinterpret_cast<uint32_t *>(m_prefix + Q);  // producer: page usable
+    uint32_t *m_ok = slot_ok + R + (R & 1);                          // measure: the same, per mailbox
+    uint32_t *m_size = m_ok + Q;                                     // measure: encoded size
+    uint32_t *m_info = m_size + Q;                                   // measure: base | packed << 8 | first << 9
+    uint32_t *m_nexc = m_info + Q;                                   // measure: exceptions of the slab
+    uint32_t *m_wcnt = m_nexc + Q;                                   // measure: [Q][W] exceptions before a part
+    uint32_t *m_wsweeps = m_wcnt + Q * W;                            // measure: [Q][W] sweeps that have any
+    uint32_t *red_max = m_wsweeps + Q * W;                           // [WM]
+    static_assert((2 * R + 2 * Q + R + 2 * Q) * 8 + (R + 1 + 4 * Q + 2 * Q * W + WM) * 4 <= S::kTail,
+                  "mailboxes do not fit");
 
     const uint32_t bar0 = smem_addr(bars);
     auto raw_full = [&](int s) { return bar0 + 8u * (uint32_t)s; };              // fetch landed
-    auto raw_empty = [&](int s) { return bar0 + 8u * (uint32_t)(R + s); };       // packing warps done with it
-    auto measured = [&](int s) { return bar0 + 8u * (uint32_t)(2 * R + s); };    // size known
-    auto placed = [&](int s) { return bar0 + 8u * (uint32_t)(3 * R + s); };      // prefix known
+    auto raw_empty = [&](int s) { return bar0 + 8u * (uint32_t)(R + s); };       // slab taken into registers
+    auto measured = [&](int q) { return bar0 + 8u * (uint32_t)(2 * R + q); };    // size known
+    auto placed = [&](int q) { return bar0 + 8u * (uint32_t)(2 * R + Q + q); };  // prefix known
 
     const unsigned warp = threadIdx.x >> 5, lane = lane_id();
     if (threadIdx.x == 0) {
         for (int s = 0; s < R; ++s) {
             mbar_init(raw_full(s), 1);                    // the producer's arrive (+ copy bytes)
-            mbar_init(raw_empty(s), W);                   // one arrive per packing warp
-            mbar_init(measured(s), 1);                    // one measuring thread
-            mbar_init(placed(s), 1);                      // one look-back lane
+            mbar_init(raw_empty(s), W);                   // one arrive per warp of a packing group
+        }
+        for (int q = 0; q < Q; ++q) {
+            mbar_init(measured(q), 1);                    // one measuring thread
+            mbar_init(placed(q), 1);                      // one look-back lane
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -242,12 +257,12 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         // and looking up its page are two dependent round trips to L2; they run three and one
         // slab ahead of the fetch, so the loop turns at the pace of one round trip, not three.
         if (lane != 0) return;
-        struct Where { const unsigned char *src; uint64_t chunk; uint32_t ok, first_of_page; };
+        struct Where { const unsigned char *src; uint64_t chunk; uint32_t ok, first_of_page, first_of_chunk; };
         auto draw = [&](bool ended) -> uint64_t {
             return ended ? total : (uint64_t)atomicAdd(job.ticket, 1ull);
         };
         auto locate = [&](uint64_t u) -> Where {
-            Where w{nullptr, 0, 0u, 0u};
+            Where w{nullptr, 0, 0u, 0u, 0u};
             if (u >= total) return w;
             const uint64_t i = u / slabs;
             const uint32_t b = (uint32_t)(u - i * slabs);
@@ -257,6 +272,7 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                 job.x.kv_ptrs[(bb & 1u) * job.x.n_layers + (bb >> 1)]);
             w.chunk = i;
             w.first_of_page = bb == 0 ? 1u : 0u;
+            w.first_of_chunk = b == 0 ? 2u : 0u;
             if (page >= job.x.num_pages) w.ok = 2u;                       // unusable page id
             else if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) w.ok = 3u;   // misaligned
             else { w.ok = 1u; w.src = pool_buf + page * (uint64_t)S::kPageBytes; }
@@ -282,7 +298,7 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
             if (w_a.ok == 2u && w_a.first_of_page) st_flag(job.x.st, LSMKV_ST_BAD_PAGE, w_a.chunk);
             if (w_a.ok == 3u) st_flag(job.x.st, LSMKV_ST_MISALIGNED, w_a.chunk);
             slot_u[s] = u_a;
-            slot_ok[s] = w_a.ok == 1u ? 1u : 0u;
+            slot_ok[s] = (w_a.ok == 1u ? 1u : 0u) | w_a.first_of_chunk;   // bit 1: the chunk's first slab
             if (w_a.ok == 1u) {
                 mbar_arrive_expect(raw_full(s), (uint32_t)S::kPageBytes);
                 asm volatile(
@@ -317,20 +333,17 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         // ---- look-back warp c: slabs k = c, c + kLb, ... of this CTA, as soon as they are measured
         const uint32_t c = warp - (unsigned)S::kFirstLbWarp;
         for (uint32_t k = c;; k += S::kLb) {
-            const int s = (int)(k % R);
+            const int s = (int)(k % Q);                   // the slab's mailbox
             bool ok = true;
-            if (lane == 0) ok = mbar_wait(measured(s), (k / R) & 1u, job);
+            if (lane == 0) ok = mbar_wait(measured(s), (k / Q) & 1u, job);
             ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
             if (!ok) { if (lane == 0) raise_abort(job, 0); break; }
             uint64_t u = lane == 0 ? m_u[s] : 0;          // read by the lane that waited
             uint32_t size = 0;
-            if (lane == 0) size = m_size[s] + (u != kEnd && (m_info[s] & 0x200u) ? job.x.dir_bytes : 0u);
+            if (lane == 0 && u != kEnd) size = m_size[s] + ((m_info[s] & 0x200u) ? job.x.dir_bytes : 0u);
             u = __shfl_sync(0xFFFFFFFFu, u, 0);
             size = __shfl_sync(0xFFFFFFFFu, size, 0);
-            if (u == kEnd) {
-                if (size != 0 && lane == 0) mbar_arrive(placed(s));   // the packing warps stop too
-                break;
-            }
+            if (u == kEnd) break;
             const uint64_t add = size;                    // bytes the slab adds to the blob
             uint64_t before = 0;
             if (!look_back(job, u, &before)) { if (lane == 0) raise_abort(job, u); break; }
@@ -350,13 +363,13 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         const uint32_t k_first = warp * SM * 32 + lane;   // this lane's first 16 bytes of a slab
         bool dead = false;                                // a wait gave up: do nothing but leave
         for (uint32_t j = 0;; ++j) {
-            const int s = (int)(j % R);
+            const int s = (int)(j % R), qs = (int)(j % Q);    // the slab's stage and mailbox
             if (!dead && !mbar_wait(raw_full(s), (j / R) & 1u, job)) dead = true;
             uint64_t u = kEnd;
             bool page_ok = false;
             if (!dead) {
                 u = slot_u[s];
-                page_ok = u != kEnd && slot_ok[s] != 0u;
+                page_ok = u != kEnd && (slot_ok[s] & 1u) != 0u;
             }
             // the largest exponent field of the slab, and the smallest of every sweep (an
             // unusable page measures as zeros)
@@ -389,20 +402,13 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                 break;
             }
             if (u == kEnd) {
-                // No more slabs. Every look-back warp gets a stop mark at its next position, and
-                // passes it on to the packing warps. The stages of positions j + 1 .. are only
-                // borrowed for their mailboxes and barriers: the producer has stopped, and a
-                // stage's earlier slab is always handed on before the stage is used again.
+                // No more slabs. Every look-back warp and every packing group finds a stop mark
+                // at its next position (mailboxes are free that far ahead: see the shape).
                 if (gt == 0) {
-                    for (uint32_t k2 = j; k2 < j + (uint32_t)S::kLb; ++k2) {
-                        const int s2 = (int)(k2 % R);
-                        if (k2 != j && !mbar_wait(raw_empty(s2), ((k2 / R) & 1u) ^ 1u, job)) {
-                            raise_abort(job, 0);
-                            break;
-                        }
-                        m_u[s2] = kEnd;
-                        m_size[s2] = k2 == j ? 1u : 0u;   // the first mark goes on to the packing warps
-                        mbar_arrive(measured(s2));
+                    constexpr uint32_t kMarks = S::kLb > S::kGroups ? S::kLb : S::kGroups;
+                    for (uint32_t k2 = j; k2 < j + kMarks; ++k2) {
+                        m_u[k2 % Q] = kEnd;
+                        mbar_arrive(measured((int)(k2 % Q)));
                     }
                 }
                 break;
@@ -443,8 +449,8 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                     for (int d = 16; d; d >>= 1) part_exc += __shfl_xor_sync(0xFFFFFFFFu, part_exc, d);
                 }
                 if (lane == 0) {
-                    m_wcnt[s * W + warp * S::kSplit + p] = part_exc;
-                    m_wsweeps[s * W + warp * S::kSplit + p] = exc_sweeps[p];
+                    m_wcnt[qs * W + warp * S::kSplit + p] = part_exc;
+                    m_wsweeps[qs * W + warp * S::kSplit + p] = exc_sweeps[p];
                 }
             }
             asm volatile("barrier.cta.sync 1, %0;" :: "r"(WM * 32) : "memory");
@@ -452,18 +458,19 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                 uint32_t n_exc = 0;
 #pragma unroll
                 for (int w = 0; w < W; ++w) {             // counts become "exceptions before the part"
-                    const uint32_t c = m_wcnt[s * W + w];
-                    m_wcnt[s * W + w] = n_exc;
+                    const uint32_t c = m_wcnt[qs * W + w];
+                    m_wcnt[qs * W + w] = n_exc;
                     n_exc += c;
                 }
                 const bool packed = page_ok && n_exc < (uint32_t)N / 2;
                 const uint32_t size = packed ? round16u(16u + N + N / 2 + n_exc) : 16u + 2u * N;
-                const bool first = u % slabs == 0;        // the chunk's directory goes before it
-                m_u[s] = u;
-                m_size[s] = size;
-                m_info[s] = base | (packed ? 0x100u : 0u) | (first ? 0x200u : 0u);
-                m_nexc[s] = n_exc;
-                mbar_arrive(measured(s));                 // a look-back warp takes it from here
+                const bool first = (slot_ok[s] & 2u) != 0u;   // the chunk's directory goes before it
+                m_u[qs] = u;
+                m_ok[qs] = page_ok ? 1u : 0u;
+                m_size[qs] = size;
+                m_info[qs] = base | (packed ? 0x100u : 0u) | (first ? 0x200u : 0u);
+                m_nexc[qs] = n_exc;
+                mbar_arrive(measured(qs));                // look-back and packing take it from here
                 // (after the arrive: an arrive orders the stores before it, and would sit out
                 // this one's trip to L2)
                 st_state(job.state + u, kFlagAgg | ((uint64_t)size + (first ? job.x.dir_bytes : 0u)));
@@ -472,21 +479,20 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         return;
     }
 
-    // ---- packing warps: slab k of this CTA once its place is known, straight into the blob.
-    // Each warp runs on its own: no barrier, only the stage's mbarriers.
-    const unsigned pw = warp - (unsigned)S::kFirstPackWarp;   // which part of a slab is this warp's
-    const unsigned pt = threadIdx.x - (unsigned)S::kFirstPackWarp * 32u;
+    // ---- packing groups: group g takes slabs g, g + kGroups, ... of this CTA. A slab goes into
+    // the group's registers as soon as it is measured, which frees its stage; the group then
+    // waits for the slab's place and encodes it straight into the blob. Each warp runs on its
+    // own: no barrier, only the mbarriers of the stage and of the mailbox.
+    const unsigned pg = (warp - (unsigned)S::kFirstPackWarp) / W;      // this warp's group
+    const unsigned pw = (warp - (unsigned)S::kFirstPackWarp) % W;      // its part of a slab
+    const unsigned pt = pw * 32u + lane;                                // thread within the group
     const uint32_t k_first = pw * S::kSweeps * 32 + lane;     // this lane's first 16 bytes of a slab
-    for (uint32_t k = 0;; ++k) {
-        const int s = (int)(k % R);
-        if (!mbar_wait(placed(s), (k / R) & 1u, job)) { raise_abort(job, 0); break; }
-        const uint64_t u = m_u[s];
+    for (uint32_t k = pg;; k += S::kGroups) {
+        const int s = (int)(k % R), qs = (int)(k % Q);
+        if (!mbar_wait(measured(qs), (k / Q) & 1u, job)) { raise_abort(job, 0); break; }
+        const uint64_t u = m_u[qs];
         if (u == kEnd) break;
-        const uint64_t before_bytes = m_prefix[s];
-        const uint32_t size = m_size[s], info = m_info[s], n_exc = m_nexc[s];
-        const bool packed = (info & 0x100u) != 0u, page_ok = slot_ok[s] != 0u;
-        const uint32_t my_sweeps = m_wsweeps[s * W + pw];
-        const uint32_t exc_before = m_wcnt[s * W + pw];   // exceptions of the parts before this one
+        const bool page_ok = m_ok[qs] != 0u;
         uint4 q[S::kSweeps];
         {
             const uint4 *s4 = reinterpret_cast<const uint4 *>(ring + (size_t)s * S::kPageBytes);
@@ -496,6 +502,12 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(raw_empty(s));         // this warp is done with the stage
+        if (!mbar_wait(placed(qs), (k / Q) & 1u, job)) { raise_abort(job, u); break; }
+        const uint64_t before_bytes = m_prefix[qs];
+        const uint32_t size = m_size[qs], info = m_info[qs], n_exc = m_nexc[qs];
+        const bool packed = (info & 0x100u) != 0u;
+        const uint32_t my_sweeps = m_wsweeps[qs * W + pw];
+        const uint32_t exc_before = m_wcnt[qs * W + pw];  // exceptions of the parts before this one
         const bool first = (info & 0x200u) != 0u;         // the chunk's directory goes before it
         const uint64_t add = (uint64_t)size + (first ? job.x.dir_bytes : 0u);
         if (before_bytes + add > job.x.blob_capacity) {   // cannot happen with a worst-case buffer
