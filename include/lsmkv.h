@@ -24,7 +24,8 @@
  *   - No call allocates device memory except lsmkv_create(), lsmkv_reserve() and a call whose
  *     batch is larger than any before it (the internal scratch of that kind of call grows;
  *     lsmkv_reserve() pre-sizes the scratch of probe and decode, a first full-size call that
- *     of flush, merge, the compressing codec and the host-buffer calls).
+ *     of flush, merge, the compressing codec and the host-buffer calls; the first host-buffer
+ *     put with the compressing codec also creates a stream and three events of the context's).
  *
  * Formats (version 1). The paper states properties (key order follows token-prefix order;
  * index values are a file identifier plus a byte offset; a batch's tensors are stored
