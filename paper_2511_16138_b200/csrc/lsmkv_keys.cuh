@@ -193,8 +193,15 @@ __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const ui
     const unsigned idx = 32u * warp + lane;                // position inside the round
     const uint64_t j = base + idx;
     uint64_t zA = 0, zB = 0;
+    uint64_t upA = 0, upB = 0, backA = 0, backB = 0;      // M^(idx+1) and M^idx, asked for early
     uint32_t first = 0, last = 0;
     if (warp < wact) {
+        upA = __ldg(kc.tab + idx);
+        upB = __ldg(kc.tab + kKeyTab + idx);
+        if (idx) {
+            backA = __ldg(kc.tab + idx - 1);
+            backB = __ldg(kc.tab + kKeyTab + idx - 1);
+        }
         uint64_t dA = 0, dB = 0;
         if (j < nch) {
             const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
@@ -219,11 +226,11 @@ __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const ui
             zA = add61_lazy(zA, sh.aggA[v]);
             zB = add61_lazy(zB, sh.aggB[v]);
         }
-        const uint64_t cA = mulmod61_lazy(sh.carryA[rnd & 1u], __ldg(kc.tab + idx));
-        const uint64_t cB = mulmod61_lazy(sh.carryB[rnd & 1u], __ldg(kc.tab + kKeyTab + idx));
+        const uint64_t cA = mulmod61_lazy(sh.carryA[rnd & 1u], upA);
+        const uint64_t cB = mulmod61_lazy(sh.carryB[rnd & 1u], upB);
         if (idx) {                                         // scale the sum back by M^idx
-            zA = mulmod61_lazy(zA, __ldg(kc.tab + idx - 1));
-            zB = mulmod61_lazy(zB, __ldg(kc.tab + kKeyTab + idx - 1));
+            zA = mulmod61_lazy(zA, backA);
+            zB = mulmod61_lazy(zB, backB);
         }
         hA = fold61(cA + zA);
         hB = fold61(cB + zB);

@@ -352,10 +352,31 @@ __device__ __noinline__ uint64_t hidx_find(const uint32_t *hidx, uint64_t n_buck
     return ~0ull;
 }
 
+// What a bucket says about a key from slot `from` on: the first slot that is empty or carries the
+// key's tag. Returns the position + 1 a tag match names (0: none) and sets `slot` to where the
+// scan stopped (kHidxSlots: every slot from `from` on holds another tag).
+__device__ __forceinline__ uint32_t bucket_stop(const uint4 &lo, const uint4 &hi, uint32_t tag,
+                                                uint32_t from, uint32_t &slot)
+{
+    const uint32_t w[kHidxSlots] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    uint32_t cand = 0;
+    slot = kHidxSlots;
+#pragma unroll
+    for (int t = (int)kHidxSlots - 1; t >= 0; --t) {       // the lowest slot wins
+        if ((uint32_t)t >= from && (w[t] == 0 || (w[t] >> 24) == tag)) {
+            cand = w[t] & 0xFFFFFFu;
+            slot = (uint32_t)t;
+        }
+    }
+    return cand;
+}
+
 // Point lookup through the hash indexes, newest run first. The home buckets of kLookupGroup
-// runs are fetched together, then the key and record of each candidate in age order, so a group
-// costs two dependent loads as a rule; the rare cases the home bucket cannot settle go slot by
-// slot.
+// runs are fetched together; then every lane fetches key and record of its newest candidate,
+// whichever run that is in, so the lanes of a warp advance together: as a rule two dependent
+// loads per group. A lane whose candidate is another key with the same tag (one lookup in a
+// hundred) goes on behind it in the same bucket, read again from L1, and from there to its next
+// run; a bucket without any answer (every slot taken by other tags) goes slot by slot.
 __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_runs,
                                                  const ChunkKey &k, uint4 &val)
 {
@@ -374,51 +395,55 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
                 hi[g] = __ldg(bkt + 1);
             }
         }
-        // first slot that is empty or carries the key's tag: cand = position + 1 of a tag match,
-        // 0 if an empty slot came first; open = neither in this bucket
-        uint32_t cand[kLookupGroup];
-        bool open[kLookupGroup];
+        // per run: cand = position + 1 of the first tag match (0: none); todo bit g = the run may
+        // still hold the key (a candidate, or a bucket that cannot say); slots = 4 bits per run,
+        // where the scan stopped
+        uint32_t cand[kLookupGroup], todo = 0, slots = 0;
 #pragma unroll
         for (int g = 0; g < kLookupGroup; ++g) {
-            const uint32_t w[8] = {lo[g].x, lo[g].y, lo[g].z, lo[g].w,
-                                   hi[g].x, hi[g].y, hi[g].z, hi[g].w};
-            cand[g] = 0;
-            open[g] = true;
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const bool stop = open[g] && (w[t] == 0 || (w[t] >> 24) == tag);
-                if (stop) {
-                    cand[g] = w[t] & 0xFFFFFFu;
-                    open[g] = false;
-                }
-            }
-            if (r0 + g < n_runs && cand[g] > rt.n[r0 + g]) {   // not a position of this run
+            uint32_t slot;
+            cand[g] = bucket_stop(lo[g], hi[g], tag, 0, slot);
+            const bool live = r0 + g < n_runs && rt.n[r0 + g] != 0;
+            if (live && cand[g] > rt.n[r0 + g]) {           // not a position of this run
                 cand[g] = 0;
-                open[g] = true;
+                slot = kHidxSlots;
             }
+            if (live && (cand[g] != 0 || slot == kHidxSlots)) todo |= 1u << g;
+            slots |= slot << (4 * g);
         }
-        // answers in age order; a candidate's key and record are fetched together (as a rule
-        // one run of the group has a candidate, so this is one more dependent load)
-#pragma unroll
-        for (int g = 0; g < kLookupGroup; ++g) {
-            const uint32_t r = r0 + g;
-            if (r >= n_runs || rt.n[r] == 0) continue;
-            if (cand[g]) {
-                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (cand[g] - 1));
+        while (todo) {                                       // newest run first
+            const int g = __ffs((int)todo) - 1;
+            const uint32_t r = r0 + (uint32_t)g;
+            const uint32_t c = g == 0 ? cand[0] : g == 1 ? cand[1] : g == 2 ? cand[2] : cand[3];
+            if (c) {
+                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (c - 1));
                 const ulonglong2 ka = __ldg(p), kb = __ldg(p + 1);
-                const uint4 rec = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (cand[g] - 1)));
+                const uint4 rec = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (c - 1)));
                 if (ka.x == k.w0 && ka.y == k.w1 && kb.x == k.w2 && kb.y == k.w3) {
                     val = rec;
                     return true;
                 }
-                open[g] = true;                            // another key with the same tag
-            }
-            if (open[g]) {
+                // another key with the same tag: what does the rest of the bucket say
+                const uint4 *bkt = reinterpret_cast<const uint4 *>(
+                    rt.hidx[r] + kHidxSlots * hidx_home(k.w1, rt.hidx_buckets[r]));
+                const uint4 l2 = __ldg(bkt), h2 = __ldg(bkt + 1);
+                uint32_t slot;
+                uint32_t c2 = bucket_stop(l2, h2, tag, ((slots >> (4 * g)) & 15u) + 1u, slot);
+                if (c2 > rt.n[r]) {
+                    c2 = 0;
+                    slot = kHidxSlots;
+                }
+                if (g == 0) cand[0] = c2; else if (g == 1) cand[1] = c2;
+                else if (g == 2) cand[2] = c2; else cand[3] = c2;
+                slots = (slots & ~(15u << (4 * g))) | (slot << (4 * g));
+                if (c2 == 0 && slot != kHidxSlots) todo &= ~(1u << g);   // an empty slot: not here
+            } else {
                 const uint64_t at = hidx_find(rt.hidx[r], rt.hidx_buckets[r], rt.keys[r], rt.n[r], k);
                 if (at != ~0ull) {
                     val = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + at));
                     return true;
                 }
+                todo &= ~(1u << g);
             }
         }
     }
