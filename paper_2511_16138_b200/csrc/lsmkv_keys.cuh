@@ -95,63 +95,82 @@ __device__ __forceinline__ uint64_t limbs_mod61(uint64_t a0, uint64_t a1, uint64
     return s >= kP ? s - kP : s;
 }
 
-__device__ __forceinline__ uint4 load_tokens4(const uint32_t *t, bool vec_ok)
-{
-    if (vec_ok) return __ldg(reinterpret_cast<const uint4 *>(t));
-    return make_uint4(__ldg(t), __ldg(t + 1), __ldg(t + 2), __ldg(t + 3));
-}
-
-// Digest of 16 tokens from h = 0 (both lanes). Sixteen Horner steps from zero give
-// sum_i (t_i + 1) * BASE^(15-i); with the weights cut into limbs of at most 21 bits every
+// Digest of the 16 tokens w[M .. M+15] from h = 0 (both lanes). Sixteen Horner steps from zero
+// give sum_i (t_i + 1) * BASE^(15-i); with the weights cut into limbs of at most 21 bits every
 // product t_i * limb is below 2^53, sixteen of them add up without overflow, and one reduction
 // at the end replaces sixteen modular multiplications. Exact, hence the same value.
-__device__ __forceinline__ void block16_dot(const KeyConsts &kc, const uint4 (&v)[4], uint64_t &dA,
-                                            uint64_t &dB)
+template <int M>
+__device__ __forceinline__ void block16_dot(const KeyConsts &kc, const uint32_t (&w)[20],
+                                            uint64_t &dA, uint64_t &dB, uint32_t &first,
+                                            uint32_t &last)
 {
     uint64_t a0 = 0, a1 = 0, a2 = 0, b0 = 0, b1 = 0, b2 = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int i = 4 * q + e;
-            a0 += (uint64_t)w[e] * kc.dA[i][0];
-            a1 += (uint64_t)w[e] * kc.dA[i][1];
-            a2 += (uint64_t)w[e] * kc.dA[i][2];
-            b0 += (uint64_t)w[e] * kc.dB[i][0];
-            b1 += (uint64_t)w[e] * kc.dB[i][1];
-            b2 += (uint64_t)w[e] * kc.dB[i][2];
-        }
+    for (int i = 0; i < 16; ++i) {
+        a0 += (uint64_t)w[i + M] * kc.dA[i][0];
+        a1 += (uint64_t)w[i + M] * kc.dA[i][1];
+        a2 += (uint64_t)w[i + M] * kc.dA[i][2];
+        b0 += (uint64_t)w[i + M] * kc.dB[i][0];
+        b1 += (uint64_t)w[i + M] * kc.dB[i][1];
+        b2 += (uint64_t)w[i + M] * kc.dB[i][2];
     }
     dA = limbs_mod61(a0, a1, a2, kc.sumA);
     dB = limbs_mod61(b0, b1, b2, kc.sumB);
+    first = w[M];
+    last = w[M + 15];
 }
 
 // Hash of one chunk from h = 0 (both lanes), plus its first and last token: whole blocks of 16
 // tokens by block16_dot, chained with BASE^16, the remaining tokens by the recurrence itself.
-// 16-byte loads when the chunk start is 16-byte aligned.
+// A block is fetched with 16-byte loads: four when it starts on a 16-byte boundary, else the
+// five aligned ones that cover it, as long as those stay inside [lim_lo, lim_hi) -- the token
+// array up to the end of this sequence -- and token by token otherwise. Sequences are packed
+// back to back, so three in four start off a boundary.
 __device__ __forceinline__ void chunk_hash(const KeyConsts &kc, const uint32_t *t, uint32_t C,
-                                           bool vec_ok, uint64_t &hA, uint64_t &hB,
-                                           uint32_t &first, uint32_t &last)
+                                           const uint32_t *lim_lo, const uint32_t *lim_hi,
+                                           uint64_t &hA, uint64_t &hB, uint32_t &first,
+                                           uint32_t &last)
 {
     hA = 0;
     hB = 0;
     uint32_t i = 0;
     for (; i + 16 <= C; i += 16) {
-        uint4 v[4];
+        const uint32_t *blk = t + i;
+        unsigned m = (unsigned)(reinterpret_cast<uintptr_t>(blk) >> 2) & 3u;   // words past a boundary
+        const uint32_t *al = blk - m;
+        uint32_t w[20];
+        if (m == 0 || (al >= lim_lo && al + 20 <= lim_hi)) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) v[q] = load_tokens4(t + i + 4 * q, vec_ok);
+            for (int q = 0; q < 4; ++q) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(al) + q);
+                w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+            }
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (m) v = __ldg(reinterpret_cast<const uint4 *>(al) + 4);
+            w[16] = v.x; w[17] = v.y; w[18] = v.z; w[19] = v.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) w[e] = __ldg(blk + e);
+            w[16] = w[17] = w[18] = w[19] = 0;
+            m = 0;
+        }
         uint64_t dA, dB;
-        block16_dot(kc, v, dA, dB);
+        uint32_t f, l;
+        switch (m) {
+        case 0: block16_dot<0>(kc, w, dA, dB, f, l); break;
+        case 1: block16_dot<1>(kc, w, dA, dB, f, l); break;
+        case 2: block16_dot<2>(kc, w, dA, dB, f, l); break;
+        default: block16_dot<3>(kc, w, dA, dB, f, l); break;
+        }
         if (i == 0) {
-            first = v[0].x;
+            first = f;
             hA = dA;
             hB = dB;
         } else {
             hA = addmod61(mulmod61(hA, kc.b16A), dA);
             hB = addmod61(mulmod61(hB, kc.b16B), dB);
         }
-        last = v[3].w;
+        last = l;
     }
     for (; i < C; ++i) {
         last = __ldg(t + i);
@@ -183,11 +202,13 @@ __device__ __forceinline__ void key_rounds_begin(KeyShared &sh)
 // Every thread of an active warp ends up with the key of chunk base + 32*warp + lane; the last
 // active warp leaves the prefix behind the round for round `rnd + 1`. Warps >= wact get an
 // unspecified key. Contains one __syncthreads(); the caller must put another one between two
-// calls (the exchange is rewritten). 32 * wact <= kKeyTab.
+// calls (the exchange is rewritten). 32 * wact <= kKeyTab. [lim_lo, lim_hi) is the part of the
+// token array that may be read: from its start to the end of this sequence.
 __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const uint32_t *seq,
                                                    uint32_t C, uint32_t ns, uint64_t base,
                                                    uint64_t nch, unsigned rnd, unsigned wact,
-                                                   KeyShared &sh)
+                                                   KeyShared &sh, const uint32_t *lim_lo,
+                                                   const uint32_t *lim_hi)
 {
     const unsigned lane = lane_id(), warp = threadIdx.x >> 5;
     const unsigned idx = 32u * warp + lane;                // position inside the round
@@ -204,8 +225,7 @@ __device__ __forceinline__ ChunkKey cta_chunk_keys(const KeyConsts &kc, const ui
         }
         uint64_t dA = 0, dB = 0;
         if (j < nch) {
-            const bool vec_ok = ((reinterpret_cast<uintptr_t>(seq) & 15u) == 0) && ((C & 3u) == 0);
-            chunk_hash(kc, seq + j * C, C, vec_ok, dA, dB, first, last);
+            chunk_hash(kc, seq + j * C, C, lim_lo, lim_hi, dA, dB, first, last);
         }
         zA = mulmod61_lazy(dA, __ldg(kc.tab + 2 * kKeyTab + idx));
         zB = mulmod61_lazy(dB, __ldg(kc.tab + 3 * kKeyTab + idx));
@@ -282,7 +302,8 @@ k_encode_keys(const __grid_constant__ KeyConsts kc, uint32_t C, uint32_t ns, uin
         __syncthreads();
         unsigned rnd = 0;
         for (uint64_t base = 0; base < nch; base += round_chunks, ++rnd) {
-            const ChunkKey k = cta_chunk_keys(kc, tokens + s0, C, ns, base, nch, rnd, W, sh);
+            const ChunkKey k = cta_chunk_keys(kc, tokens + s0, C, ns, base, nch, rnd, W, sh,
+                                              tokens, tokens + s1);
             const uint64_t j = base + threadIdx.x;           // = base + 32 * warp + lane
             if (j >= start && j < nch) {
                 const uint64_t i = o0 + (j - start);

@@ -505,7 +505,8 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(nx + b));
                 }
             }
-            const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, rnd, wact, sh);
+            const ChunkKey k = cta_chunk_keys(kc, seq, C, ns, base, nch, rnd, wact, sh, tokens,
+                                              tokens + s1);
             if (threadIdx.x == 0) s_first_miss[(rnd + 1u) % 3u] = ~0ull;
             if (keys_out && valid) store_key(keys_out + o0 + j, k);
             if (done) {                                      // only the keys were wanted
