@@ -685,6 +685,7 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     RunTable rt;
     std::memset(&rt, 0, sizeof(rt));
     bool hashed = true;   // every non-empty run brings its hash index: no directory, no searches
+    bool wide = true;     // ... and index and keys start on 32-byte boundaries: 32-byte loads
     for (uint32_t r = 0; r < n_runs; ++r) {
         if (runs[r].n && (!runs[r].keys || !runs[r].vals || !aligned16(runs[r].keys) ||
                           !aligned16(runs[r].vals)))
@@ -702,6 +703,9 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
         rt.hidx[r] = static_cast<const uint32_t *>(runs[r].hindex);
         rt.hidx_buckets[r] = runs[r].hindex_buckets;
         if (runs[r].n && !runs[r].hindex) hashed = false;
+        if (runs[r].n && ((reinterpret_cast<uintptr_t>(runs[r].hindex) & 31u) ||
+                          (reinterpret_cast<uintptr_t>(runs[r].keys) & 31u)))
+            wide = false;
     }
     if (n_runs == 0) hashed = false;
     DeviceGuard guard(ctx->device);
@@ -721,21 +725,26 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     {
         LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
         {
-            uint64_t dgrid = (dir_entries + 255) / 256;
-            const uint64_t dcap = (uint64_t)ctx->sm_count * 8;
+            // blocks of 1024: the last one also orders the queries, a few per thread (without a
+            // directory to fill it is the only block)
+            uint64_t dgrid = (dir_entries + 1023) / 1024;
+            const uint64_t dcap = (uint64_t)ctx->sm_count * 2;
             if (dgrid > dcap) dgrid = dcap;
             if (dgrid == 0) dgrid = 1;
-            k_run_dir<<<(unsigned)dgrid, 256, 0, s>>>(rt, dir_runs, ctx->geom.ns, jcap, dir,
-                                                      next_query, n_query, seq_off,
-                                                      ctx->geom.chunk_tokens, order);
+            k_run_dir<<<(unsigned)dgrid, 1024, 0, s>>>(rt, dir_runs, ctx->geom.ns, jcap, dir,
+                                                       next_query, n_query, seq_off,
+                                                       ctx->geom.chunk_tokens, order);
             ++ctx->launches;
         }
         const unsigned warps = (unsigned)ctx->probe_warps_per_cta;
         const unsigned threads = warps * 32u;
         uint64_t grid = n_query;
-        const uint64_t cap = (uint64_t)ctx->sm_count * (2048u / threads);
+        // six CTAs of four warps per SM: with more of them every round takes longer, and the
+        // rounds of the longest query, one after another, are what the launch waits for
+        const uint64_t cap = (uint64_t)ctx->sm_count * (threads <= 768u ? 768u / threads : 1u);
         if (grid > cap) grid = cap;
-        auto kern = hashed ? k_probe<true> : k_probe<false>;
+        auto kern = !hashed ? k_probe<false, false>
+                            : (wide ? k_probe<true, true> : k_probe<true, false>);
         kern<<<(unsigned)grid, threads, 0, s>>>(ctx->kc, rt, n_runs, dir, jcap,
                                                 ctx->geom.chunk_tokens, ctx->geom.ns, n_query,
                                                 tokens, seq_off, qchunk_off, n_qchunks,

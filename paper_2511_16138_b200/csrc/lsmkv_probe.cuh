@@ -103,23 +103,63 @@ __device__ __forceinline__ void order_queries(uint32_t n_query, const uint64_t *
     __shared__ uint32_t s_cnt[kLenClasses];
     for (uint32_t t = threadIdx.x; t < kLenClasses; t += blockDim.x) s_cnt[t] = 0;
     __syncthreads();
-    for (uint32_t q = threadIdx.x; q < n_query; q += blockDim.x) {
-        const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
-        atomicAdd(&s_cnt[len_class(s1 >= s0 ? (s1 - s0) / C : 0)], 1u);
+    // four queries per thread at a time, their offsets asked for together: an atomic between
+    // two loads would make every load wait for the one before it
+    constexpr int kPer = 4;
+    for (uint32_t q0 = 0; q0 < n_query; q0 += kPer * blockDim.x) {
+        uint32_t cls[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const uint32_t q = q0 + (uint32_t)u * blockDim.x + threadIdx.x;
+            cls[u] = ~0u;
+            if (q < n_query) {
+                const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
+                cls[u] = len_class(s1 >= s0 ? (s1 - s0) / C : 0);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kPer; ++u)
+            if (cls[u] != ~0u) atomicAdd(&s_cnt[cls[u]], 1u);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {                                // counts -> first slot of every class
-        uint32_t at = 0;
-        for (int c = kLenClasses - 1; c >= 0; --c) {
-            const uint32_t n = s_cnt[c];
-            s_cnt[c] = at;
-            at += n;
+    if (threadIdx.x < 32) {              // counts -> first slot of every class, longest class first
+        static_assert(kLenClasses == 4 * 32, "four classes per lane");
+        const unsigned lane = threadIdx.x;
+        uint32_t n[4], tot = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            n[u] = s_cnt[kLenClasses - 1 - (4 * (int)lane + u)];
+            tot += n[u];
+        }
+        uint32_t incl = tot;
+#pragma unroll
+        for (unsigned d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        uint32_t at = incl - tot;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            s_cnt[kLenClasses - 1 - (4 * (int)lane + u)] = at;
+            at += n[u];
         }
     }
     __syncthreads();
-    for (uint32_t q = threadIdx.x; q < n_query; q += blockDim.x) {
-        const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
-        order[atomicAdd(&s_cnt[len_class(s1 >= s0 ? (s1 - s0) / C : 0)], 1u)] = q;
+    for (uint32_t q0 = 0; q0 < n_query; q0 += kPer * blockDim.x) {
+        uint32_t cls[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const uint32_t q = q0 + (uint32_t)u * blockDim.x + threadIdx.x;
+            cls[u] = ~0u;
+            if (q < n_query) {
+                const uint64_t s0 = seq_off[q], s1 = seq_off[q + 1];
+                cls[u] = len_class(s1 >= s0 ? (s1 - s0) / C : 0);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kPer; ++u)
+            if (cls[u] != ~0u)
+                order[atomicAdd(&s_cnt[cls[u]], 1u)] = q0 + (uint32_t)u * blockDim.x + threadIdx.x;
     }
 }
 
@@ -127,7 +167,7 @@ __device__ __forceinline__ void order_queries(uint32_t n_query, const uint64_t *
 // for j = 0..jcap (stride = jcap + 1).
 // Also resets the probe's work counter (*next_query) for the launch that follows, and its last
 // block writes the hand-out order of the queries when `order` is given.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 k_run_dir(const __grid_constant__ RunTable rt, uint32_t n_runs, uint32_t ns, uint32_t jcap,
           uint64_t *__restrict__ dir, unsigned long long *next_query, uint32_t n_query,
           const uint64_t *__restrict__ seq_off, uint32_t C, uint32_t *__restrict__ order)
@@ -352,6 +392,27 @@ __device__ __noinline__ uint64_t hidx_find(const uint32_t *hidx, uint64_t n_buck
     return ~0ull;
 }
 
+// One 32-byte load (the address must be 32-byte aligned): a whole bucket, or a whole key.
+__device__ __forceinline__ void ldg256(const void *p, uint4 &lo, uint4 &hi)
+{
+    asm("ld.global.nc.v8.u32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z),
+          "=r"(hi.w)
+        : "l"(p));
+}
+
+// A bucket or a key: one load when the caller vouches for 32-byte alignment (WIDE), else two.
+template <bool WIDE>
+__device__ __forceinline__ void load32(const void *p, uint4 &lo, uint4 &hi)
+{
+    if (WIDE) {
+        ldg256(p, lo, hi);
+    } else {
+        lo = __ldg(reinterpret_cast<const uint4 *>(p));
+        hi = __ldg(reinterpret_cast<const uint4 *>(p) + 1);
+    }
+}
+
 // What a bucket says about a key from slot `from` on: the first slot that is empty or carries the
 // key's tag. Returns the position + 1 a tag match names (0: none) and sets `slot` to where the
 // scan stopped (kHidxSlots: every slot from `from` on holds another tag).
@@ -377,6 +438,8 @@ __device__ __forceinline__ uint32_t bucket_stop(const uint4 &lo, const uint4 &hi
 // loads per group. A lane whose candidate is another key with the same tag (one lookup in a
 // hundred) goes on behind it in the same bucket, read again from L1, and from there to its next
 // run; a bucket without any answer (every slot taken by other tags) goes slot by slot.
+// WIDE: every run's index and key array start on a 32-byte boundary.
+template <bool WIDE>
 __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_runs,
                                                  const ChunkKey &k, uint4 &val)
 {
@@ -391,8 +454,7 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
             if (r < n_runs && rt.n[r]) {
                 const uint4 *bkt = reinterpret_cast<const uint4 *>(
                     rt.hidx[r] + kHidxSlots * hidx_home(k.w1, rt.hidx_buckets[r]));
-                lo[g] = __ldg(bkt);
-                hi[g] = __ldg(bkt + 1);
+                load32<WIDE>(bkt, lo[g], hi[g]);
             }
         }
         // per run: cand = position + 1 of the first tag match (0: none); todo bit g = the run may
@@ -416,17 +478,21 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
             const uint32_t r = r0 + (uint32_t)g;
             const uint32_t c = g == 0 ? cand[0] : g == 1 ? cand[1] : g == 2 ? cand[2] : cand[3];
             if (c) {
-                const ulonglong2 *p = reinterpret_cast<const ulonglong2 *>(rt.keys[r] + (c - 1));
-                const ulonglong2 ka = __ldg(p), kb = __ldg(p + 1);
+                uint4 k0, k1;
+                load32<WIDE>(rt.keys[r] + (c - 1), k0, k1);
                 const uint4 rec = __ldg(reinterpret_cast<const uint4 *>(rt.vals[r] + (c - 1)));
-                if (ka.x == k.w0 && ka.y == k.w1 && kb.x == k.w2 && kb.y == k.w3) {
+                if (k0.x == (uint32_t)k.w0 && k0.y == (uint32_t)(k.w0 >> 32) &&
+                    k0.z == (uint32_t)k.w1 && k0.w == (uint32_t)(k.w1 >> 32) &&
+                    k1.x == (uint32_t)k.w2 && k1.y == (uint32_t)(k.w2 >> 32) &&
+                    k1.z == (uint32_t)k.w3 && k1.w == (uint32_t)(k.w3 >> 32)) {
                     val = rec;
                     return true;
                 }
                 // another key with the same tag: what does the rest of the bucket say
                 const uint4 *bkt = reinterpret_cast<const uint4 *>(
                     rt.hidx[r] + kHidxSlots * hidx_home(k.w1, rt.hidx_buckets[r]));
-                const uint4 l2 = __ldg(bkt), h2 = __ldg(bkt + 1);
+                uint4 l2, h2;
+                load32<WIDE>(bkt, l2, h2);
                 uint32_t slot;
                 uint32_t c2 = bucket_stop(l2, h2, tag, ((slots >> (4 * g)) & 15u) + 1u, slot);
                 if (c2 > rt.n[r]) {
@@ -450,7 +516,7 @@ __device__ __forceinline__ bool lookup_runs_hash(const RunTable &rt, uint32_t n_
     return false;
 }
 
-template <bool HASHED>
+template <bool HASHED, bool WIDE>
 __global__ void __launch_bounds__(256, 3)
 k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable rt,
         uint32_t n_runs, const uint64_t *__restrict__ dir, uint32_t jcap, uint32_t C,
@@ -516,7 +582,7 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
                 continue;
             }
             uint4 val = zero;
-            const bool found = valid && (HASHED ? lookup_runs_hash(rt, n_runs, k, val)
+            const bool found = valid && (HASHED ? lookup_runs_hash<WIDE>(rt, n_runs, k, val)
                                                 : lookup_runs(rt, n_runs, dir, jcap, k, val));
             n_lookups += valid ? 1ull : 0ull;
             const unsigned miss = __ballot_sync(0xFFFFFFFFu, valid && !found);

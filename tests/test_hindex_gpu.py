@@ -62,6 +62,15 @@ def test_build_refuses_runs_beyond_24_bit_positions():
         assert rc == lsmkv.EINVAL
 
 
+def off16(t):
+    """A copy of a device byte tensor that starts 16 bytes past a 32-byte boundary."""
+    buf = torch.empty(t.numel() + 48, dtype=torch.uint8, device=t.device)
+    at = 16 + (-buf.data_ptr()) % 32
+    out = buf[at:at + t.numel()]
+    out.copy_(t.view(torch.uint8).reshape(-1))
+    return out
+
+
 def build_runs(ctx, w, g):
     nch = synth.chunk_counts(w.store.seq_off, 16)
     coff = synth.offsets(nch - w.store_start_chunk)
@@ -110,8 +119,11 @@ def test_probe_through_hash_indexes_equals_the_searching_probe_and_the_oracle(wh
             tables.append(t)
             hashed.append((dk, dv, n, None, 0, t, nb))
         mixed = hashed[:2] + [druns[2]] + hashed[3:]       # one run without a table: all searched
+        # keys and tables 16 bytes off a 32-byte boundary: the probe may not use 32-byte loads
+        odd = [(off16(dk), dv, n, None, 0, off16(t), nb) for (dk, dv, n, _, _, t, nb) in hashed]
+        assert all(r[0].data_ptr() % 32 == 16 and r[5].data_ptr() % 32 == 16 for r in odd)
         ctx.last_status()
-        for rr in (druns, hashed, mixed):
+        for rr in (druns, hashed, mixed, odd):
             hit, recs, st = probe(ctx, w, qoff, total, rr, batch)
             assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
             assert st["chunks_hit"] == int(o_hit.sum())
