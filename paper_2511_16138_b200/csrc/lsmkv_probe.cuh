@@ -198,7 +198,7 @@ __device__ __forceinline__ int bucket_cmp(const lsmkv_key_t *e, const ChunkKey &
 
 // Plain exact binary search over [a, b) of a bucket with the full key (slow path).
 __device__ __noinline__ uint64_t bucket_find_exact(const lsmkv_key_t *keys, uint64_t a, uint64_t b,
-                                                   const ChunkKey &k)
+                                                   const ChunkKey k)   // by value: in registers
 {
     while (a < b) {
         const uint64_t mid = a + ((b - a) >> 1);
@@ -376,8 +376,8 @@ __device__ __forceinline__ bool key_equals(const lsmkv_key_t *e, const ChunkKey 
 
 // The lookup rule, slot by slot (any table, any fill). Returns the position or ~0.
 __device__ __noinline__ uint64_t hidx_find(const uint32_t *hidx, uint64_t n_buckets,
-                                           const lsmkv_key_t *keys, uint64_t n, const ChunkKey &k)
-{
+                                           const lsmkv_key_t *keys, uint64_t n, const ChunkKey k)
+{                                                          // (the key by value: in registers)
     const uint32_t tag = (uint32_t)k.w2 & 0xFFu;
     uint64_t b = hidx_home(k.w1, n_buckets);
     for (uint64_t it = 0; it < n_buckets; ++it) {
