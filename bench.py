@@ -1105,13 +1105,14 @@ def probe_heavy_block(torch, lsmkv, dev, device_index, steps, warmup):
                 "exact_index": exact,
                 # the probe's least traffic (tokens up to the first miss, a record per query chunk,
                 # a hit length per query) against the measured copy bandwidth: small by nature --
-                # the kernel is bound by integer issue and dependent L2 loads, not by HBM
+                # the kernel is bound by a chain of dependent steps per round, not by HBM
                 "roofline": {"bound": "hbm", "kernel": "k_probe<true>",
                              "achieved": algo_bytes / ms / 1e6, "peak": peak, "unit": "GB/s",
                              "frac": algo_bytes / ms / 1e6 / peak, "peak_source": peak_src,
                              "algorithmic_bytes_per_launch": algo_bytes, "traffic": None},
-                "bound": "instruction issue and dependent L2 loads (issue-slot counters: see the "
-                         "committed ncu summary of k_probe on this workload)"}
+                "bound": "latency chain: a query's rounds run one after another, each a chain of "
+                         "dependent loads and digest arithmetic; the longest query's rounds last "
+                         "as long as the launch (committed ncu summary of k_probe on this workload)"}
     finally:
         ctx.close()
 
