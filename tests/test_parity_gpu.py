@@ -212,3 +212,52 @@ def test_many_runs_are_searched_in_groups_newest_first(n_runs):
     w = synth.tiny_codec(n_req=10, seq_len=8 * 50 + 3, max_shared=200, n_mutate=40, config_id=60)
     out = H.roundtrip(g, w.store, w.query, n_runs=n_runs, seed=n_runs)
     assert np.array_equal(out["hit"], w.expected_hit_tokens // 8)
+
+
+@pytest.mark.parametrize("shift", [0, 1, 2, 3])
+@pytest.mark.parametrize("C", [16, 32, 20])
+def test_keys_do_not_depend_on_where_the_token_array_starts(shift, C):
+    """The token array starts `shift` tokens past a 16-byte boundary and ends with the last token
+    of the last chunk. A block of 16 tokens is fetched with the aligned 16-byte loads that cover
+    it where those stay inside the array up to the end of its sequence, and token by token at the
+    edges; sequences of odd lengths packed back to back give every misalignment in one batch.
+    Keys from the encoder and from both probes equal the oracle's, and every stored chunk hits."""
+    g = lsmkv.Geom(2, 1, 32, page_tokens=C, chunk_tokens=C)
+    og = H.ogeom(g)
+    rng = np.random.default_rng(100 + 4 * C + shift)
+    lens = [3 * C, 2 * C + 5, 7, 40 * C + 1, 33 * C + 2, C + 3, 5 * C]
+    batch = synth.make_batch([rng.integers(0, 2**32, n, dtype=np.uint64).astype(np.uint32)
+                              for n in lens])
+    want = np.concatenate([oracle.chunk_keys(og, batch.seq(i)) for i in range(batch.n)])
+    nch = synth.chunk_counts(batch.seq_off, C)
+    coff = synth.offsets(nch)
+    n = int(coff[-1])
+    assert int(batch.seq_off[-1]) == sum(lens) and lens[-1] % C == 0   # the array ends with a chunk
+    raw = torch.zeros(4 * (shift + len(batch.tokens)), dtype=torch.uint8, device=H.DEV)
+    assert raw.data_ptr() % 16 == 0
+    d_tok = raw[4 * shift:]
+    d_tok.copy_(torch.from_numpy(batch.tokens.view(np.uint8).copy()))
+    assert d_tok.data_ptr() % 16 == 4 * shift
+    with lsmkv.Context(g, 0) as ctx:
+        d_off, d_coff = H.dev(batch.seq_off), H.dev(coff)
+        d_keys = torch.zeros(n * 32, dtype=torch.uint8, device=H.DEV)
+        d_vals = torch.zeros(n * 16, dtype=torch.uint8, device=H.DEV)
+        ctx.encode_batch(batch.n, d_tok, d_off, None, d_coff, n, None, None, 0, 0, d_keys, d_vals,
+                         None, 0)
+        torch.cuda.synchronize()
+        keys = H.host(d_keys, np.uint64, n * 32).reshape(-1, 4)
+        assert np.array_equal(keys, want)
+        vals = H.host(d_vals, VAL_DTYPE, n * 16)
+        run = H.gpu_flush_run(ctx, keys, vals)
+        druns, keep = H.dev_runs([run])
+        hruns, hkeep = H.with_hindex(ctx, druns)
+        for rr in (druns, hruns):
+            d_hit = torch.full((batch.n,), -1, dtype=torch.int32, device=H.DEV)
+            d_recs = torch.full((n * 16,), 0xAB, dtype=torch.uint8, device=H.DEV)
+            d_qk = torch.zeros(n * 32, dtype=torch.uint8, device=H.DEV)
+            ctx.probe_batch(batch.n, d_tok, d_off, d_coff, n, rr, d_hit, d_recs, d_qk)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_hit.cpu().numpy().view(np.uint32), nch.astype(np.uint32))
+            assert np.array_equal(H.host(d_qk, np.uint64, n * 32).reshape(-1, 4), want)
+            assert np.array_equal(H.host(d_recs, VAL_DTYPE, n * 16), vals)
+        H.assert_status_clean(ctx)
