@@ -488,6 +488,10 @@ int lsmkv_last_status(lsmkv_ctx *ctx, void *stream, lsmkv_status_t *out);
  * the recorded events, returns the summed device time and launch count per kernel class since
  * the previous read, and clears them. Class LSMKV_K_PLAN covers the two small kernels that
  * turn hit lengths into the list of chunks to copy.
+ * Independently of that switch the launches of every call of a context sit inside an NVTX
+ * range named after their class ("lsmkv:keys", "lsmkv:pack", "lsmkv:probe", "lsmkv:plan",
+ * "lsmkv:unpack", "lsmkv:flush", "lsmkv:merge"): a timeline tool that collects NVTX shows
+ * them, without such a tool the ranges do nothing. lsmkv_decode_batch_static opens none.
  */
 #define LSMKV_K_KEYS 0
 #define LSMKV_K_PACK 1

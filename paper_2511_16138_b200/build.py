@@ -36,7 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo",
            "-std=c++17", "-Xcompiler", "-fPIC", "-shared", "--use_fast_math",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp]
+           "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp, "-ldl"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]

@@ -9,6 +9,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "lsmkv.h"
 #include "lsmkv_common.cuh"
 #include "lsmkv_copy.cuh"
@@ -154,11 +156,20 @@ void fill_key_consts(KeyConsts &kc, uint32_t C, uint64_t *tab)
 }
 
 // Brackets one kernel launch with events when profiling is on.
+// Around the launches of one ABI call: an NVTX range named after the kernel class (a no-op
+// unless a tool that collects NVTX is attached) and, when profiling is on, a pair of events.
 struct LaunchTimer {
     lsmkv_ctx *ctx;
     cudaStream_t s;
     lsmkv_ctx::Timed t{};
     bool on;
+    static const char *range_name(int cls)
+    {
+        static const char *const names[LSMKV_K_CLASSES] = {
+            "lsmkv:keys", "lsmkv:pack", "lsmkv:probe", "lsmkv:plan",
+            "lsmkv:unpack", "lsmkv:flush", "lsmkv:merge", "lsmkv:other"};
+        return names[cls >= 0 && cls < LSMKV_K_CLASSES ? cls : LSMKV_K_CLASSES - 1];
+    }
     static cudaEvent_t get(lsmkv_ctx *c)
     {
         cudaEvent_t e = nullptr;
@@ -168,6 +179,7 @@ struct LaunchTimer {
     }
     LaunchTimer(lsmkv_ctx *c, cudaStream_t st, int cls) : ctx(c), s(st), on(c->profiling)
     {
+        nvtxRangePushA(range_name(cls));
         if (!on) return;
         t.a = get(c);
         t.b = get(c);
@@ -177,6 +189,7 @@ struct LaunchTimer {
     }
     ~LaunchTimer()
     {
+        nvtxRangePop();
         if (!on) return;
         cudaEventRecord(t.b, s);
         ctx->pending.push_back(t);
