@@ -96,7 +96,10 @@ typedef struct {
  * hindex (optional, NULL = none): the run's hash index as built by lsmkv_hindex_build, with
  * hindex_buckets 32-byte buckets. When every non-empty run of a probe brings one, point lookups
  * go through the hash indexes instead of searching the sorted keys (and ignore the Bloom
- * filters, which the tables make redundant); otherwise the probe ignores the hash indexes. */
+ * filters, which the tables make redundant); otherwise the probe ignores the hash indexes.
+ * Alignment: keys, vals, bloom and hindex on 16-byte boundaries (LSMKV_EINVAL otherwise); when
+ * keys and hindex of every non-empty run also start on 32-byte boundaries the probe fetches a
+ * bucket or a key with one 32-byte load instead of two 16-byte ones (same answers). */
 typedef struct {
     const lsmkv_key_t *keys; /* [dev] */
     const lsmkv_val_t *vals; /* [dev] */
