@@ -259,47 +259,74 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
     const uint64_t total = job.x.n_chunks * slabs;
 
     if (warp == (unsigned)S::kProducerWarp) {
-        // ---- producer: one lane hands out slab numbers and starts the fetches. Drawing a number
-        // and looking up its page are two dependent round trips to L2; they run three and one
-        // slab ahead of the fetch, so the loop turns at the pace of one round trip, not three.
+        // ---- producer: one lane hands out slab numbers and starts the fetches. Drawing a number,
+        // reading its page id and its layer's pool pointer are dependent round trips to L2; the
+        // number is drawn three slabs ahead, the two loads are started one slab ahead and their
+        // values first looked at after the wait for the stage, so none of them holds the loop.
         if (lane != 0) return;
         struct Where { const unsigned char *src; uint64_t chunk; uint32_t ok, first_of_page, first_of_chunk; };
+        // loads on their way, and where the slab sits: chunk, slab of the chunk, slab of the page
+        struct Asked { uint64_t page; const unsigned char *pool_buf; uint64_t chunk; uint32_t b, bb; };
+        // One lane divides on its own here, and a 64-bit division is a chain of some eighty
+        // dependent instructions: slab number / slabs per chunk is taken from the reciprocal
+        // (at most one too small for any 63-bit number, put right by one comparison), slab of
+        // the chunk / slabs per page likewise in 32 bits.
+        const uint32_t per_page = 2u * job.x.n_layers;
+        const uint64_t inv_slabs = ~0ull / slabs;
+        const uint32_t inv_per_page = 0xFFFFFFFFu / per_page;
         auto draw = [&](bool ended) -> uint64_t {
             return ended ? total : (uint64_t)atomicAdd(job.ticket, 1ull);
         };
-        auto locate = [&](uint64_t u) -> Where {
+        auto ask = [&](uint64_t u) -> Asked {
+            Asked a{0, nullptr, 0, 0u, 0u};
+            if (u >= total) return a;
+            uint64_t i = __umul64hi(u, inv_slabs);
+            uint64_t b64 = u - i * slabs;
+            if (b64 >= slabs) { ++i; b64 -= slabs; }
+            const uint32_t b = (uint32_t)b64;
+            uint32_t pg = __umulhi(b, inv_per_page), bb = b - pg * per_page;
+            if (bb >= per_page) { ++pg; bb -= per_page; }
+            a.chunk = i;
+            a.b = b;
+            a.bb = bb;
+            a.page = __ldg(job.x.page_table + i * job.x.pages_per_chunk + pg);
+            a.pool_buf = static_cast<const unsigned char *>(
+                job.x.kv_ptrs[(bb & 1u) * job.x.n_layers + (bb >> 1)]);
+            return a;
+        };
+        auto locate = [&](uint64_t u, const Asked &a) -> Where {
             Where w{nullptr, 0, 0u, 0u, 0u};
             if (u >= total) return w;
-            const uint64_t i = u / slabs;
-            const uint32_t b = (uint32_t)(u - i * slabs);
-            const uint32_t per_page = 2u * job.x.n_layers, pg = b / per_page, bb = b - pg * per_page;
-            const uint64_t page = __ldg(job.x.page_table + i * job.x.pages_per_chunk + pg);
-            const unsigned char *pool_buf = static_cast<const unsigned char *>(
-                job.x.kv_ptrs[(bb & 1u) * job.x.n_layers + (bb >> 1)]);
-            w.chunk = i;
-            w.first_of_page = bb == 0 ? 1u : 0u;
-            w.first_of_chunk = b == 0 ? 2u : 0u;
-            if (page >= job.x.num_pages) w.ok = 2u;                       // unusable page id
-            else if ((reinterpret_cast<uintptr_t>(pool_buf) & 15u) != 0) w.ok = 3u;   // misaligned
-            else { w.ok = 1u; w.src = pool_buf + page * (uint64_t)S::kPageBytes; }
+            w.chunk = a.chunk;
+            w.first_of_page = a.bb == 0 ? 1u : 0u;
+            w.first_of_chunk = a.b == 0 ? 2u : 0u;
+            if (a.page >= job.x.num_pages) w.ok = 2u;                     // unusable page id
+            else if ((reinterpret_cast<uintptr_t>(a.pool_buf) & 15u) != 0) w.ok = 3u;   // misaligned
+            else { w.ok = 1u; w.src = a.pool_buf + a.page * (uint64_t)S::kPageBytes; }
             return w;
         };
         bool ended = false;
-        uint64_t u_a = draw(false), u_b = draw(false), u_c = draw(false);
-        Where w_a = locate(u_a);
         uint32_t fetch_mask = 0, fetch_parity = 0;        // per stage: last arm was a fetch / its phase
-        for (uint32_t k = 0;; ++k) {
-            const uint64_t u_d = draw(ended);             // three slabs ahead
-            const Where w_b = locate(u_b);                // one slab ahead
+        uint32_t k = 0;                                   // slabs of this CTA so far
+        // One slab: draws the number three slabs ahead into `u_d`, asks for the loads of the
+        // next slab `u_b` into `q_b`, and fetches slab `u_a` whose loads `q_a` were asked for a
+        // slab ago. False when the loop is over. The caller rotates the variables by name: a
+        // copy of a value still on its way would wait for it.
+        auto step = [&](uint64_t &u_a, const uint64_t &u_b, uint64_t &u_d, const Asked &q_a,
+                        Asked &q_b) -> bool {
+            u_d = draw(ended);
+            q_b = ask(u_b);
             ended = ended || u_b >= total;
             const int s = (int)(k % R);
             const uint32_t ph = (k / R) & 1u;
-            if (!mbar_wait(raw_empty(s), ph ^ 1u, job)) { raise_abort(job, 0); break; }
+            ++k;
+            if (!mbar_wait(raw_empty(s), ph ^ 1u, job)) { raise_abort(job, 0); return false; }
+            const Where w_a = locate(u_a, q_a);
             if (u_a >= total) {                           // the stop mark
                 slot_u[s] = kEnd;
                 fetch_mask &= ~(1u << s);
                 mbar_arrive(raw_full(s));
-                break;
+                return false;
             }
             if (w_a.ok == 2u && w_a.first_of_page) st_flag(job.x.st, LSMKV_ST_BAD_PAGE, w_a.chunk);
             if (w_a.ok == 3u) st_flag(job.x.st, LSMKV_ST_MISALIGNED, w_a.chunk);
@@ -318,9 +345,15 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                 fetch_mask &= ~(1u << s);
                 mbar_arrive(raw_full(s));
             }
-            u_a = u_b; w_a = w_b;
-            u_b = u_c;
-            u_c = u_d;
+            return true;
+        };
+        uint64_t u0 = draw(false), u1 = draw(false), u2 = draw(false), u3 = 0;
+        Asked q0 = ask(u0), q1{0, nullptr, 0, 0u, 0u};
+        for (;;) {
+            if (!step(u0, u1, u3, q0, q1)) break;
+            if (!step(u1, u2, u0, q1, q0)) break;
+            if (!step(u2, u3, u1, q0, q1)) break;
+            if (!step(u3, u0, u2, q1, q0)) break;
         }
         // Do not leave while a fetch may still be writing this CTA's shared memory. A stage
         // whose last arm was a fetch is waited for here (the compute warps normally did so long
@@ -460,26 +493,29 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
                 }
             }
             asm volatile("barrier.cta.sync 1, %0;" :: "r"(WM * 32) : "memory");
-            if (gt == 0) {
-                uint32_t n_exc = 0;
-#pragma unroll
-                for (int w = 0; w < W; ++w) {             // counts become "exceptions before the part"
-                    const uint32_t c = m_wcnt[qs * W + w];
-                    m_wcnt[qs * W + w] = n_exc;
-                    n_exc += c;
+            if (warp == 0) {
+                // counts become "exceptions before the part": a scan over the W parts by lanes
+                static_assert(W <= 32, "one lane per part");
+                const uint32_t c = lane < (unsigned)W ? m_wcnt[qs * W + lane] : 0u;
+                const uint32_t incl = xpfast::warp_incl_scan(c);
+                if (lane < (unsigned)W) m_wcnt[qs * W + lane] = incl - c;
+                const uint32_t n_exc = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                __syncwarp();
+                if (lane == 0) {
+                    const bool packed = page_ok && n_exc < (uint32_t)N / 2;
+                    const uint32_t size = packed ? round16u(16u + N + N / 2 + n_exc) : 16u + 2u * N;
+                    const bool first = (slot_ok[s] & 2u) != 0u;   // the chunk's directory goes before it
+                    m_u[qs] = u;
+                    m_ok[qs] = page_ok ? 1u : 0u;
+                    m_size[qs] = size;
+                    m_info[qs] = base | (packed ? 0x100u : 0u) | (first ? 0x200u : 0u);
+                    m_nexc[qs] = n_exc;
+                    mbar_arrive(measured(qs));            // look-back and packing take it from here
+                    // (after the arrive: an arrive orders the stores before it, and would sit
+                    // out this one's trip to L2)
+                    st_state(job.state + u,
+                             kFlagAgg | ((uint64_t)size + (first ? job.x.dir_bytes : 0u)));
                 }
-                const bool packed = page_ok && n_exc < (uint32_t)N / 2;
-                const uint32_t size = packed ? round16u(16u + N + N / 2 + n_exc) : 16u + 2u * N;
-                const bool first = (slot_ok[s] & 2u) != 0u;   // the chunk's directory goes before it
-                m_u[qs] = u;
-                m_ok[qs] = page_ok ? 1u : 0u;
-                m_size[qs] = size;
-                m_info[qs] = base | (packed ? 0x100u : 0u) | (first ? 0x200u : 0u);
-                m_nexc[qs] = n_exc;
-                mbar_arrive(measured(qs));                // look-back and packing take it from here
-                // (after the arrive: an arrive orders the stores before it, and would sit out
-                // this one's trip to L2)
-                st_state(job.state + u, kFlagAgg | ((uint64_t)size + (first ? job.x.dir_bytes : 0u)));
             }
         }
         return;
