@@ -735,9 +735,21 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
     unsigned long long *next_query = reinterpret_cast<unsigned long long *>(ctx->d_dir);
     uint64_t *dir = ctx->d_dir + 2;
     uint32_t *order = ordered ? reinterpret_cast<uint32_t *>(dir + dir_entries) : nullptr;
+    const unsigned warps = (unsigned)ctx->probe_warps_per_cta;
+    const unsigned threads = warps * 32u;
+    // six CTAs of four warps per SM: with more of them every round takes longer, and the
+    // rounds of the longest query, one after another, are what the launch waits for
+    const uint64_t cap = (uint64_t)ctx->sm_count * (threads <= 768u ? 768u / threads : 1u);
+    // Few queries and no directory to fill: a CTA per query, no hand-out order, no counter,
+    // and so no launch before the probe's own.
+    const bool cta_per_query = hashed && n_query <= cap;
+    if (cta_per_query) {
+        next_query = nullptr;
+        order = nullptr;
+    }
     {
         LaunchTimer timer(ctx, s, LSMKV_K_PROBE);
-        {
+        if (!cta_per_query) {
             // blocks of 1024: the last one also orders the queries, a few per thread (without a
             // directory to fill it is the only block)
             uint64_t dgrid = (dir_entries + 1023) / 1024;
@@ -749,12 +761,7 @@ int lsmkv_probe_batch(lsmkv_ctx *ctx, void *stream, uint32_t n_query, const uint
                                                        ctx->geom.chunk_tokens, order);
             ++ctx->launches;
         }
-        const unsigned warps = (unsigned)ctx->probe_warps_per_cta;
-        const unsigned threads = warps * 32u;
         uint64_t grid = n_query;
-        // six CTAs of four warps per SM: with more of them every round takes longer, and the
-        // rounds of the longest query, one after another, are what the launch waits for
-        const uint64_t cap = (uint64_t)ctx->sm_count * (threads <= 768u ? 768u / threads : 1u);
         if (grid > cap) grid = cap;
         auto kern = !hashed ? k_probe<false, false>
                             : (wide ? k_probe<true, true> : k_probe<true, false>);

@@ -534,13 +534,17 @@ k_probe(const __grid_constant__ KeyConsts kc, const __grid_constant__ RunTable r
     const uint4 zero = make_uint4(0, 0, 0, 0);
     unsigned long long n_lookups = 0;
 
+    bool took = false;
     for (;;) {
         // queries are handed out one at a time: long and short ones balance across the CTAs
+        // (without a counter there is a CTA per query: block b takes query b and leaves)
         __syncthreads();
         if (threadIdx.x == 0) {
-            s_q = atomicAdd(next_query, 1ull);
+            s_q = next_query ? atomicAdd(next_query, 1ull)
+                             : (took ? (unsigned long long)n_query : (unsigned long long)blockIdx.x);
             s_first_miss[0] = ~0ull;
         }
+        took = true;
         key_rounds_begin(sh);
         __syncthreads();
         if (s_q >= n_query) break;
