@@ -204,6 +204,43 @@ def test_more_queries_than_the_hand_out_order_covers():
         assert ctx.last_status()["flags"] == 0
 
 
+@pytest.mark.parametrize("extra", [-1, 0, 1, 700])
+def test_as_many_queries_as_resident_ctas_and_one_more(extra):
+    """Up to six CTAs of four warps per SM a probe through hash indexes gives every query a CTA
+    of its own (no hand-out order, no counter); one query more and the queries are ordered and
+    drawn from a counter. Both sides of that edge, and well beyond it, equal the oracle."""
+    g = lsmkv.Geom(1, 1, 8, elem_bytes=2, page_tokens=4, chunk_tokens=4)
+    og = H.ogeom(g)
+    rng = np.random.default_rng(31 + extra)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n_q = 6 * sms + extra
+    stored = [rng.integers(0, 3, int(rng.integers(4, 400)), dtype=np.uint32) for _ in range(200)]
+    store = synth.make_batch(stored)
+    coff = synth.offsets(synth.chunk_counts(store.seq_off, 4))
+    qs = []
+    for i in range(n_q):
+        q = rng.integers(0, 3, int(rng.integers(0, 500)), dtype=np.uint32)
+        if i % 2 == 0:                                         # starts with a stored sequence
+            s = stored[i % len(stored)]
+            m = min(len(s), len(q))
+            q[:m] = s[:m]
+        qs.append(q)
+    query = synth.make_batch(qs)
+    qoff = synth.offsets(synth.chunk_counts(query.seq_off, 4))
+    with lsmkv.Context(g, 0) as ctx:
+        keys, vals, _, _ = H.gpu_encode(ctx, g, store, None, coff, None, None)
+        run = H.gpu_flush_run(ctx, keys, vals)
+        o_hit, o_recs, o_keys, _ = oracle.probe_batch(og, query.tokens, query.seq_off, qoff, [run],
+                                                      want_keys=True)
+        for want_keys in (False, True):
+            hit, recs, qk, _ = H.gpu_probe(ctx, query, qoff, [run], want_keys=want_keys)
+            assert np.array_equal(hit, o_hit) and np.array_equal(recs, o_recs)
+            if want_keys:
+                assert np.array_equal(qk, o_keys)
+        assert int((o_hit > 0).sum()) > n_q // 4
+        assert ctx.last_status()["flags"] == 0
+
+
 @pytest.mark.parametrize("n_runs", [5, 11, 64])
 def test_many_runs_are_searched_in_groups_newest_first(n_runs):
     """More runs than one lock-step group holds (4), up to the most a probe accepts; keys are
