@@ -541,7 +541,11 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *                       barrier of the piece with this number (pieces are numbered over the
  *                       whole launch) but starts no copy for it, so that wait runs out: the
  *                       kernel records LSMKV_ST_WAIT_EXPIRED with first_bad = the piece and
- *                       returns; the warp that owned the piece copies nothing further
+ *                       returns; the warp that owned the piece copies nothing further. The
+ *                       one-pass encoder of the compressing codec does the same with the fetch of
+ *                       the slab of this number (slabs numbered over the whole batch): the wait
+ *                       for it runs out, every role of every CTA leaves through its bounded
+ *                       waits, and the records of chunks that were not finished are zeroed
  *   "wait_cycles"       limit, in GPU clock cycles, of every bounded wait inside a kernel (the bulk
  *                       copies' completion, the one-pass encoder's hand-offs); default 2e9, about
  *                       a second; 1e5..1e11. A wait that runs out sets LSMKV_ST_WAIT_EXPIRED

@@ -456,6 +456,7 @@ int encode_xp12(lsmkv_ctx *ctx, cudaStream_t s, uint64_t n_chunks, const uint32_
         fj.abort = reinterpret_cast<unsigned int *>(scratch + 8);
         fj.state = reinterpret_cast<unsigned long long *>(scratch + 256);
         fj.wait_cycles = ctx->wait_cycles;
+        fj.test_drop_slab = ctx->test_drop_piece < 0 ? ~0ull : (uint64_t)ctx->test_drop_piece;
         CU(ctx, cudaMemsetAsync(scratch, 0, 256 + (size_t)units * 8, s));
         const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)ctx->sm_count, units);
         if (job.n_elems == 8192u)

@@ -70,6 +70,8 @@ struct Job {
     unsigned long long *state;     // [dev] one word per slab; zero before the launch
     unsigned int *abort;           // [dev] zero before the launch
     long long wait_cycles;         // limit of every wait
+    uint64_t test_drop_slab;       // test hook: the fetch of this slab is armed but never started,
+                                   // so the wait for it runs out (~0 = none)
 };
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -332,7 +334,10 @@ k_xpf_encode(const __grid_constant__ xpf::Job job)
             if (w_a.ok == 3u) st_flag(job.x.st, LSMKV_ST_MISALIGNED, w_a.chunk);
             slot_u[s] = u_a;
             slot_ok[s] = (w_a.ok == 1u ? 1u : 0u) | w_a.first_of_chunk;   // bit 1: the chunk's first slab
-            if (w_a.ok == 1u) {
+            if (w_a.ok == 1u && u_a == job.test_drop_slab) {
+                mbar_arrive_expect(raw_full(s), (uint32_t)S::kPageBytes);   // and nothing comes
+                fetch_mask &= ~(1u << s);
+            } else if (w_a.ok == 1u) {
                 mbar_arrive_expect(raw_full(s), (uint32_t)S::kPageBytes);
                 asm volatile(
                     "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes"
