@@ -1,12 +1,13 @@
 // Batched longest-cached-prefix probe.
 //
-// A CTA takes one query at a time, longest queries first. Its W warps hash 32*W consecutive
-// chunks per round (each warp one 32-chunk block; the block digests are chained through shared
-// memory; the very first round is one warp's 32 chunks), every lane
-// looks its key up in the runs newest -> oldest, a warp ballot finds each warp's first miss and
-// a shared-memory minimum gives the query's. The hit length is the number of leading chunks
-// that were all found (first-miss rule); hashing stops at the round of the first miss unless
-// the caller asked for all keys.
+// A CTA takes one query at a time, longest queries first (a batch of no more queries than CTAs fit
+// on the GPU, all runs with hash indexes: block b takes query b). Its W warps hash 32*W
+// consecutive chunks per round (each warp one 32-chunk block; the block digests are chained
+// through shared memory; the very first round is one warp's 32 chunks), every lane looks its key
+// up in the runs newest -> oldest, a warp ballot finds each warp's first miss and a shared-memory
+// minimum gives the query's. The hit length is the number of leading chunks that were all found
+// (first-miss rule); hashing stops at the round of the first miss unless the caller asked for all
+// keys.
 //
 // Lookups use fence pointers: the chunk index j is the most significant key field, so in every
 // run the keys of one j form a contiguous bucket. k_run_dir finds all bucket boundaries of all
