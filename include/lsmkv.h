@@ -397,9 +397,12 @@ int lsmkv_hindex_build(lsmkv_ctx *ctx, void *stream, const lsmkv_key_t *keys, ui
  * tensors handed over by the serving process, App. B). Same results as the device-buffer
  * calls; every pointer except `pool` and `runs[].keys/vals` is a HOST pointer (use pinned
  * memory for full transfer speed; pageable memory works). The calls stage through device
- * scratch owned by the context (grown on demand, bounded by the "host_stage_bytes" knob plus
- * the descriptors; default 1 GiB of blobs per slice), enqueue all copies and kernels on
- * `stream` and return; host outputs are valid, and host inputs may be reused, once the stream
+ * scratch owned by the context (grown on demand, bounded by twice the "host_stage_bytes" knob
+ * plus the descriptors; default 1 GiB of blobs per slice), enqueue all copies and kernels on
+ * `stream` -- the blobs of a put with the compressing codec and of a get with several slices on
+ * a second stream of the context's own, from or into two stages in turn, so that one slice
+ * travels while its neighbour is packed or scattered; that stream starts behind `stream` and
+ * `stream` waits for it, the caller sees one stream -- and return; host outputs are valid, and host inputs may be reused, once the stream
  * has reached the end of the call's work. Offsets (chunk_off / qchunk_off) are computed by
  * the library from the sequence lengths.
  *
