@@ -482,6 +482,8 @@ def main():
                       world, "identity", link)
         if not args.no_xp12_block:
             ctx_xp = lsmkv.Context(lsmkv.Geom(**dict(GEOM, flags=lsmkv.CODEC_XP12)), local_rank)
+            for k_ in ("host_stage_bytes", "host_copy_piece_bytes"):
+                ctx_xp.set_tuning(k_, ctx.get_tuning(k_))
             try:
                 e2e_xp = run_e2e(args, torch, lsmkv, ctx_xp, g, W, src_pool, dst_pool, dev, stream,
                                  barrier, world, "xp12", link)
@@ -1324,7 +1326,7 @@ def run_e2e(args, torch, lsmkv, ctx, g, W, src_pool, dst_pool, dev, stream, barr
     # never keeps the other direction of the link idle.
     import threading
     ctx_get = lsmkv.Context(ctx.geom, ctx.device)
-    for k_ in ("host_stage_bytes",):
+    for k_ in ("host_stage_bytes", "host_copy_piece_bytes"):
         ctx_get.set_tuning(k_, ctx.get_tuning(k_))
     put_done = [torch.cuda.Event() for _ in range(NS)]
     slot_free = [torch.cuda.Event() for _ in range(NS)]

@@ -540,6 +540,12 @@ uint64_t lsmkv_launch_count(const lsmkv_ctx *ctx);
  *   "host_put_device_placed"  1 = lsmkv_put_batch_host with the compressing codec never waits
  *                       (see there); "host_copy_ctas" = CTAs of the kernel that then writes the
  *                       host blob, 1..4096 (default 32: posted writes need little parallelism)
+ *   "host_copy_piece_bytes"  the host-buffer calls move blobs in copies of at most this many
+ *                       bytes, 1 MiB..64 GiB (default 128 MiB). Copies of one direction are served
+ *                       in issue order even across streams, so a smaller piece lets another
+ *                       stream's small copies in sooner and a larger one loses less at the piece
+ *                       boundaries (end to end, put and get side by side: 87 GB/s with 32 MiB,
+ *                       89 GB/s with 128 MiB on the same box)
  *   "test_drop_piece"   test hook, -1 = off (default): the bulk copy kernel arms the completion
  *                       barrier of the piece with this number (pieces are numbered over the
  *                       whole launch) but starts no copy for it, so that wait runs out: the

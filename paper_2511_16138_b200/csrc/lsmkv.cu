@@ -53,6 +53,7 @@ struct lsmkv_ctx {
     int64_t copy_mode, copy_stage_bytes, copy_stages, copy_ctas_per_sm, copy_l2_hint;
     int64_t probe_warps_per_cta, simt_ctas_per_sm, host_stage_bytes, xp_generic;
     int64_t xp_one_pass, wait_cycles, host_copy_ctas, host_put_device_placed, test_drop_piece;
+    int64_t host_copy_piece;
     uint32_t ppc;        // pages per chunk: chunk_tokens / page_tokens
     // host-buffer calls: device staging and host scratch
     void *d_io[3];
@@ -541,6 +542,7 @@ int lsmkv_create(lsmkv_ctx **out, const lsmkv_geom_t *g, int device)
     ctx->xp_one_pass = 1;
     ctx->host_copy_ctas = 32;
     ctx->test_drop_piece = -1;
+    ctx->host_copy_piece = 128ll << 20;
     ctx->wait_cycles = 2000000000ll;
 
     DeviceGuard guard(device);
@@ -1218,6 +1220,7 @@ static int64_t *tuning_slot(lsmkv_ctx *ctx, const char *name, int64_t *lo, int64
         {"host_copy_ctas", &ctx->host_copy_ctas, 1, 4096},
         {"host_put_device_placed", &ctx->host_put_device_placed, 0, 1},
         {"test_drop_piece", &ctx->test_drop_piece, -1, 1ll << 40},
+        {"host_copy_piece_bytes", &ctx->host_copy_piece, 1 << 20, 1ll << 36},
         {"wait_cycles", &ctx->wait_cycles, 100000, 100000000000ll},
     };
     for (auto &t : tab)

@@ -45,15 +45,16 @@ size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 // when they sit on different streams, so one multi-GiB copy would hold up every small copy
 // another stream issues in the same direction (and with it that stream's kernels). With
 // bounded pieces a put on one stream and a get on another keep both PCIe directions busy.
-constexpr size_t kCopyPiece = 32u << 20;
-
-cudaError_t copy_pieces(void *dst, const void *src, size_t bytes, cudaMemcpyKind kind,
-                        cudaStream_t s)
+// The piece is the context's "host_copy_piece_bytes" (every piece boundary costs the link a
+// little, every piece makes the other stream's small copies wait that much longer).
+cudaError_t copy_pieces(const lsmkv_ctx *ctx, void *dst, const void *src, size_t bytes,
+                        cudaMemcpyKind kind, cudaStream_t s)
 {
     unsigned char *d = static_cast<unsigned char *>(dst);
     const unsigned char *p = static_cast<const unsigned char *>(src);
-    for (size_t at = 0; at < bytes; at += kCopyPiece) {
-        const size_t n = std::min(kCopyPiece, bytes - at);
+    const size_t piece = (size_t)ctx->host_copy_piece;
+    for (size_t at = 0; at < bytes; at += piece) {
+        const size_t n = std::min(piece, bytes - at);
         const cudaError_t e = cudaMemcpyAsync(d + at, p + at, n, kind, s);
         if (e != cudaSuccess) return e;
     }
@@ -241,13 +242,13 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
         }
         at += (size_t)(b - a) + 1;
     }
-    if (nt) CU(ctx, copy_pieces(d_tok, tokens + t_first, nt * 4, cudaMemcpyHostToDevice, s));
+    if (nt) CU(ctx, copy_pieces(ctx, d_tok, tokens + t_first, nt * 4, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_seq, h_seq, n_rel * 8, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_coff, h_coff, n_rel * 8, cudaMemcpyHostToDevice, s));
     if (start_chunk)
         CU(ctx, cudaMemcpyAsync(d_start, start_chunk, (size_t)n_req * 4, cudaMemcpyHostToDevice, s));
     if (with_blob)
-        CU(ctx, copy_pieces(d_pages, page_table, n_chunks * ctx->ppc * 4, cudaMemcpyHostToDevice, s));
+        CU(ctx, copy_pieces(ctx, d_pages, page_table, n_chunks * ctx->ppc * 4, cudaMemcpyHostToDevice, s));
 
     // Compressing codec: how many bytes a slice produced is only known on the device. Either
     // the device places the slices in the host blob itself and nothing ever stops (on request:
@@ -317,7 +318,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
             const uint64_t used = last.offset + last.reserved - (base_offset + host_used);
             if (blob_capacity - host_used < used) return LSMKV_ECAPACITY;
             CU(ctx, cudaStreamWaitEvent(ctx->io_stream, ctx->io_ev_enc, 0));
-            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + host_used, stage, used,
+            CU(ctx, copy_pieces(ctx, static_cast<unsigned char *>(blob_out) + host_used, stage, used,
                                 cudaMemcpyDeviceToHost, ctx->io_stream));
             CU(ctx, cudaEventRecord(ctx->io_ev_free[sg], ctx->io_stream));
             stage_used[sg] = true;
@@ -325,7 +326,7 @@ extern "C" int lsmkv_put_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_req
             host_used += used;
             if (blob_bytes_out) *blob_bytes_out = host_used;
         } else if (with_blob) {
-            CU(ctx, copy_pieces(static_cast<unsigned char *>(blob_out) + coff[a] * cb, d_blob, m * cb,
+            CU(ctx, copy_pieces(ctx, static_cast<unsigned char *>(blob_out) + coff[a] * cb, d_blob, m * cb,
                                 cudaMemcpyDeviceToHost, s));
         }
     }
@@ -485,8 +486,8 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
     uint64_t *d_qoff = io.take<uint64_t>(2 * n_slices);
     uint32_t *d_hit = io.take<uint32_t>(n_slices);
     // every descriptor goes up first, so that nothing small queues behind the blob copies
-    CU(ctx, copy_pieces(d_recs, h_recs, total_hits * 16, cudaMemcpyHostToDevice, s));
-    CU(ctx, copy_pieces(d_pages, h_pages, total_hits * ppc * 4, cudaMemcpyHostToDevice, s));
+    CU(ctx, copy_pieces(ctx, d_recs, h_recs, total_hits * 16, cudaMemcpyHostToDevice, s));
+    CU(ctx, copy_pieces(ctx, d_pages, h_pages, total_hits * ppc * 4, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_qoff, h_qoff, n_slices * 16, cudaMemcpyHostToDevice, s));
     CU(ctx, cudaMemcpyAsync(d_hit, h_hit, n_slices * 4, cudaMemcpyHostToDevice, s));
     cudaStream_t up = s;                             // the stream the blobs come up on
@@ -521,7 +522,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
                 run_bytes += len;
             } else {
                 if (run_bytes)
-                    CU(ctx, copy_pieces(stage + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, up));
+                    CU(ctx, copy_pieces(ctx, stage + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, up));
                 run_dst = h_recs[k].offset;
                 run_src = src;
                 run_bytes = len;
@@ -529,7 +530,7 @@ extern "C" int lsmkv_decode_batch_host(lsmkv_ctx *ctx, void *stream, uint32_t n_
             stage_used = h_recs[k].offset + len;
         }
         if (run_bytes)
-            CU(ctx, copy_pieces(stage + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, up));
+            CU(ctx, copy_pieces(ctx, stage + run_dst, run_src, run_bytes, cudaMemcpyHostToDevice, up));
         if (staged) {
             CU(ctx, cudaEventRecord(ctx->io_ev_enc, up));
             CU(ctx, cudaStreamWaitEvent(s, ctx->io_ev_enc, 0));
